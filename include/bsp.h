@@ -1,0 +1,152 @@
+/*
+ * bsp.h -- C ABI of the weight-block-sparse linear operator Y = W*X + b on NVIDIA B200 (sm_100a).
+ *
+ * Notation is the paper's (Introduction): the kernel W is O x H x K x I, stored with the input
+ * channel innermost ([O][H][K][I], Section "Compiler and its Code generation": C_OUT x h x w x C_IN);
+ * W-bar[i][j] = W[i,*,*,j] is its O x I abstraction; a block is b_o x b_i entries of W-bar, i.e.
+ * b_o x H x K x b_i weights, with b_o x b_i one of 8x8, 4x16, 16x4; Gamma is the 0/1 mask of Eq. (1)
+ * with NB_o = O/b_o rows and NB_i = I/b_i columns.  Activations X are N x L x J x I and outputs Y are
+ * N x M x N' x O, both channel-innermost (NHWC); the batch dimension N is an addition, the paper
+ * describes one image.
+ *
+ * General rules
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller; descriptors (bsp_wdesc, bsp_xdesc,
+ *    bsp_bcsr structs) are HOST structs read during the call.  The library allocates no device memory:
+ *    scratch comes from the caller's workspace `ws` (device, 256-byte aligned), sized by the matching
+ *    *_workspace_bytes() call.  The caller zero-fills the first 256 bytes of a workspace once after
+ *    allocating it (they hold the latched status word); one workspace sized for the largest request
+ *    may serve all calls issued on one stream.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue work and
+ *    return; results are valid once the stream has been synchronised.
+ *  - Every function returns a bsp_status; nothing throws.  Argument errors are detected on the host
+ *    before anything is launched.  Device-side problems are latched in a status word inside the
+ *    workspace and read back by bsp_check().
+ *  - O and I must be multiples of b_o and b_i (Section "Experiments": a layer with fewer channels than a
+ *    block, such as a 3-channel first layer, cannot be made block sparse) and, for the product kernels,
+ *    multiples of 8.
+ */
+#ifndef BSP_H
+#define BSP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BSP_OK = 0,
+    BSP_ERR_NULL = 1,      /* a required pointer is NULL */
+    BSP_ERR_SHAPE = 2,     /* sizes <= 0, O % b_o != 0, I % b_i != 0, empty output, unsupported multiple */
+    BSP_ERR_BLOCK = 3,     /* b_o x b_i is not 8x8, 4x16 or 16x4 */
+    BSP_ERR_DTYPE = 4,     /* element type not valid for this call or combination */
+    BSP_ERR_CAPACITY = 5,  /* an output buffer or count is too small */
+    BSP_ERR_INDEX = 6,     /* compact structure inconsistent with the descriptor */
+    BSP_ERR_CUDA = 7,      /* a CUDA runtime call failed */
+    BSP_ERR_TIMEOUT = 8    /* a bounded device-side wait expired (latched in the workspace) */
+} bsp_status;
+
+typedef enum { BSP_F32 = 0, BSP_BF16 = 1, BSP_I8 = 2, BSP_I32 = 3 } bsp_dtype;
+
+/* Block importance (Section "Predetermined Sparsity ratio and Full Training Ahead"). */
+typedef enum { BSP_NORM_L2 = 0, BSP_NORM_L1 = 1 } bsp_norm;
+
+/* Which blocks compete when the lowest scores are zeroed.  LAYER: all NB_o*NB_i blocks are ranked
+ * together ("sort them in ascending order").  ROW: each row of Gamma is ranked on its own and gets
+ * n_zero zeros, the per-row reading of Eq. (2). */
+typedef enum { BSP_SCOPE_LAYER = 0, BSP_SCOPE_ROW = 1 } bsp_scope;
+
+/* Weight descriptor: W is [O][H][K][I] of `wtype` (BSP_F32, BSP_BF16 or BSP_I8). */
+typedef struct {
+    int O, I, H, K, bo, bi;
+    bsp_dtype wtype;
+} bsp_wdesc;
+
+/* Activation descriptor: X is [N][L][J][I]; output is [N][M][N'][O] with
+ * M = (L + 2 pad_h - H) / stride_h + 1 and N' = (J + 2 pad_w - K) / stride_w + 1 (integer division).
+ * Zero padding, no dilation, no groups, no kernel flip (cross-correlation). */
+typedef struct {
+    int N, L, J;
+    int stride_h, stride_w, pad_h, pad_w;
+} bsp_xdesc;
+
+/* Compacted weights (Section "Block Sparsity in a Matrix": compressed block rows).
+ *   row_ptr [NB_o+1]  first stored block of each row of Gamma; row_ptr[NB_o] = nnz
+ *   col_idx [nnz]     column of Gamma of each stored block, ascending within a row
+ *   payload [nnz][b_o][H][K][b_i]  the surviving weights in canonical order
+ *   packed            the same weights in the kernels' own tile order, written by bsp_compact and
+ *                     opaque to the caller (bsp_packed_bytes() gives its size)
+ *   nnz               number of stored blocks (host copy; used for size checks only)
+ * The product kernels read `packed`; row_ptr/col_idx/payload are the portable form. */
+typedef struct {
+    const int32_t *row_ptr;
+    const int32_t *col_idx;
+    const void *payload;
+    const void *packed;
+    int64_t nnz;
+} bsp_bcsr;
+
+/* ---- Gamma builder (Eq. (1), Eq. (2); Section "Predetermined Sparsity ratio ...") ------------------
+ * score[l][iota] = sum of w^2 (L2, ranked by its square) or sum of |w| (L1) over the b_o x H x K x b_i
+ * block; the n_zero blocks with the lowest (score, block index) pairs get Gamma = 0, all others 1.
+ * Float weights: scores are float64, each product exact, summed over (h, k, c) for each output row r of
+ * the block and then over r, always in that order, so that the mask is reproducible bit for bit.
+ * int8 weights: scores are exact int64.
+ *   W          [O][H][K][I] device, not modified
+ *   n_zero     number of blocks to zero: 0..NB (LAYER) or 0..NB_i per row (ROW)
+ *   gamma      [NB_o*NB_i] uint8 device, out
+ *   scores_opt [NB_o*NB_i] float64 (float W) or int64 (int8 W) device, out; may be NULL
+ *   ws         device scratch of bsp_mask_workspace_bytes() bytes
+ * Errors: NULL, SHAPE, BLOCK, DTYPE (wtype I32), CAPACITY (n_zero out of range), CUDA. */
+size_t bsp_mask_workspace_bytes(const bsp_wdesc *wd);
+bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
+                    uint8_t *gamma, void *scores_opt, void *ws, void *stream);
+
+/* ---- Compaction (Section "Block Sparsity in a Matrix"; Section "Subvolumes, Data Compression ...") --
+ * bsp_packed_bytes: size of the opaque `packed` buffer able to hold `nnz` stored blocks.
+ * bsp_compact_nnz : counts the ones of a device Gamma and returns the count on the host; this one call
+ *                   synchronises the stream.
+ * bsp_compact     : scans Gamma (caller supplied or from bsp_mask) row by row and writes row_ptr, col_idx,
+ *                   the canonical payload and the packed form.  `payload` may be NULL (canonical copy
+ *                   skipped); `packed` may be NULL (portable form only).  capacity_blocks is the number of
+ *                   blocks col_idx/payload/packed were sized for; if Gamma holds more, nothing beyond the
+ *                   capacity is written and BSP_ERR_CAPACITY is latched for bsp_check().
+ *                   A dense layer is the same call with Gamma == 1.
+ *   ws  device scratch of bsp_compact_workspace_bytes() bytes. */
+size_t bsp_packed_bytes(const bsp_wdesc *wd, int64_t nnz);
+size_t bsp_compact_workspace_bytes(const bsp_wdesc *wd);
+bsp_status bsp_compact_nnz(const bsp_wdesc *wd, const uint8_t *gamma, int64_t *nnz_host, void *ws,
+                           void *stream);
+bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma, int32_t *row_ptr,
+                       int32_t *col_idx, void *payload, void *packed, int64_t capacity_blocks, void *ws,
+                       void *stream);
+
+/* ---- Block-sparse products (Introduction; Section "Block Sparsity in a Matrix") ---------------------
+ * bsp_gemm  : Y[p][o] = bias[o] + sum over stored blocks (l = o / b_o, iota) sum_c W-bar[o][iota b_i + c]
+ *             X[p][iota b_i + c].  X is [P][I], Y is [P][O] (a fully connected layer is a 1x1 convolution
+ *             over P pixels); wd->H = wd->K = 1.
+ * bsp_conv2d: Y[n,y,x,o] = bias[o] + sum over stored blocks of row o / b_o, over taps (h,k) and channels c of
+ *             W[o,h,k,iota b_i + c] X[n, y s_h + h - p_h, x s_w + k - p_w, iota b_i + c], X = 0 out of bounds.
+ * Only stored blocks are read or multiplied.  Types: BF16 or F32 inputs (wtype = type of X) accumulate in
+ * float32, bias float32, ytype F32 or BF16 (round to nearest even after the bias); F32 inputs are
+ * multiplied as TF32.  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
+ *   bias may be NULL (treated as zero).  ws: device scratch of bsp_conv_workspace_bytes() bytes.
+ * Errors: NULL, SHAPE, BLOCK, DTYPE, INDEX (packed buffer does not match wd), CUDA. */
+size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd);
+bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,
+                    void *Y, bsp_dtype ytype, void *ws, void *stream);
+bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                      const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
+
+/* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
+ * (BSP_OK if none), then clears it. */
+bsp_status bsp_check(void *ws, void *stream);
+
+/* Text for a status code (static storage). */
+const char *bsp_status_string(bsp_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSP_H */

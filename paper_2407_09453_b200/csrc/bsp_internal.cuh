@@ -1,0 +1,71 @@
+// Internal declarations shared by the CUDA translation units of libbsp.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "bsp.h"
+
+namespace bsp {
+
+// The product kernels work on 8x8 tiles of W-bar: an 8x8 block is one tile, a 4x16 block covers half of
+// two tiles side by side, a 16x4 block covers half of two tiles one above the other.  A tile is stored if
+// any block overlapping it has Gamma = 1; weights of zeroed blocks inside a stored tile are written as
+// zeros.  Eight tile rows (64 output channels) form a panel; one warp owns one panel.
+constexpr int kTile = 8;                 // tile edge in channels
+constexpr int kPanelRows = 8;            // tile rows per panel
+constexpr int kPanelCh = kTile * kPanelRows;
+constexpr uint32_t kPackedMagic = 0x42535031u;   // "BSP1"
+
+// First 256 bytes of the packed buffer.
+struct PackedHeader {
+    uint32_t magic;
+    int32_t dtype, O, I, H, K, bo, bi;
+    int32_t n_panels;        // ceil(O / 64)
+    int32_t n_cols;          // I / 8 tile columns
+    int32_t tile_bytes;      // bytes of one stored tile (all taps)
+    int32_t capacity_tiles;  // tiles the payload area can hold
+    int32_t n_tiles;         // tiles stored (written on the device)
+    int32_t off_colmask;     // byte offsets from the start of the packed buffer
+    int32_t off_coloff;
+    int32_t off_panelbase;
+    int64_t off_payload;
+};
+
+struct PackedLayout {
+    int n_panels, n_cols, tile_bytes;
+    int64_t capacity_tiles;
+    size_t off_colmask, off_coloff, off_panelbase, off_payload, total_bytes;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int elem_bytes(bsp_dtype t) { return t == BSP_I8 ? 1 : (t == BSP_BF16 ? 2 : 4); }
+
+// Bytes of one stored 8x8 tile over all H*K taps, in the order the MMA fragments are read.
+inline int tile_bytes_of(bsp_dtype t, int taps)
+{
+    if (t == BSP_BF16) return 128 * taps;              // 8x8 bf16 per tap
+    if (t == BSP_I8) return 128 * ((taps + 1) / 2);    // taps paired into K=16 steps, odd tail zero padded
+    return 256 * taps;                                 // 8x8 fp32 per tap
+}
+
+PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks);
+
+// Workspace: the first 256 bytes hold the latched status word; scratch starts after it.
+constexpr size_t kWsHeader = 256;
+
+bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
+                       uint8_t *gamma, void *scores, cudaStream_t st);
+bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gamma, int32_t *row_ptr,
+                          int32_t *col_idx, void *payload, void *packed, int64_t capacity_blocks, void *ws,
+                          cudaStream_t st);
+bsp_status launch_count(const uint8_t *gamma, int64_t n, unsigned long long *out, cudaStream_t st);
+bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                       const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
+
+#define BSP_CUDA_OK(expr)                                  \
+    do {                                                   \
+        cudaError_t e_ = (expr);                           \
+        if (e_ != cudaSuccess) return BSP_ERR_CUDA;        \
+    } while (0)
+
+}  // namespace bsp
