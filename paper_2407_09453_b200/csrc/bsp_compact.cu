@@ -1,0 +1,345 @@
+// Compaction of Gamma (.) W: compressed block rows (row_ptr, col_idx, canonical payload) and the packed
+// tile form read by the product kernels.  Section "Block Sparsity in a Matrix" (compress block row) and
+// Section "Subvolumes, Data Compression, and Data Movements" of the paper.
+#include "bsp_internal.cuh"
+
+namespace bsp {
+
+PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
+{
+    PackedLayout L;
+    L.n_panels = (wd.O + kPanelCh - 1) / kPanelCh;
+    L.n_cols = wd.I / kTile;
+    L.tile_bytes = tile_bytes_of(wd.wtype, wd.H * wd.K);
+    const int64_t all_tiles = (int64_t)((wd.O + kTile - 1) / kTile) * L.n_cols;
+    // a 4x16 or 16x4 block touches two tiles; an 8x8 block is one tile
+    const int64_t per_block = (wd.bo == 8 && wd.bi == 8) ? 1 : 2;
+    int64_t cap = nnz_blocks * per_block;
+    if (cap > all_tiles) cap = all_tiles;
+    if (cap < 0) cap = 0;
+    L.capacity_tiles = cap;
+    L.off_colmask = 256;
+    L.off_coloff = align_up(L.off_colmask + (size_t)L.n_panels * L.n_cols, 256);
+    L.off_panelbase = align_up(L.off_coloff + (size_t)L.n_panels * L.n_cols * 4, 256);
+    L.off_payload = align_up(L.off_panelbase + (size_t)(L.n_panels + 1) * 4, 256);
+    L.total_bytes = align_up(L.off_payload + (size_t)cap * L.tile_bytes + 256, 256);
+    return L;
+}
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Exclusive prefix sum of v over the CTA's threads; every thread of the CTA must call it.
+__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += n;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    int before = 0, tot = 0;
+    for (int w = 0; w < kThreads / 32; ++w) {
+        const int s = warp_sums[w];
+        if (w < warp) before += s;
+        tot += s;
+    }
+    __syncthreads();
+    total = tot;
+    return before + inc - v;
+}
+
+// Launch 1.  CTAs [0, NBo): ones of one row of Gamma -> row_cnt.  CTAs [NBo, NBo + n_panels): for one panel
+// (64 output channels) the byte mask of stored tiles in every tile column, and the running count of stored
+// tiles before each column (coloff, relative to the panel).
+__global__ void __launch_bounds__(kThreads)
+count_kernel(const uint8_t *__restrict__ gamma, int NBo, int NBi, int bo, int bi, int O, int n_cols,
+             int *__restrict__ row_cnt, uint8_t *__restrict__ colmask, uint32_t *__restrict__ coloff,
+             int *__restrict__ panel_cnt)
+{
+    __shared__ int warp_sums[kThreads / 32];
+    __shared__ int s_run;
+    if ((int)blockIdx.x < NBo) {
+        const uint8_t *g = gamma + (size_t)blockIdx.x * NBi;
+        int c = 0;
+        for (int i = threadIdx.x; i < NBi; i += kThreads) c += g[i] ? 1 : 0;
+        int tot;
+        block_exclusive_scan(c, warp_sums, tot);
+        if (threadIdx.x == 0) row_cnt[blockIdx.x] = tot;
+        return;
+    }
+    const int panel = (int)blockIdx.x - NBo;
+    if (threadIdx.x == 0) s_run = 0;
+    __syncthreads();
+    for (int base = 0; base < n_cols; base += kThreads) {
+        const int col = base + threadIdx.x;
+        unsigned m = 0;
+        if (col < n_cols) {
+            for (int r = 0; r < kPanelRows; ++r) {
+                const int o0 = (panel * kPanelRows + r) * kTile;     // first channel of the tile row
+                if (o0 >= O) break;
+                // blocks overlapping the tile: rows o0/bo .. (o0+7)/bo, columns (8 col)/bi .. (8 col + 7)/bi
+                bool any = false;
+                for (int lb = o0 / bo; lb <= (o0 + kTile - 1) / bo && lb < NBo; ++lb)
+                    for (int cb = (col * kTile) / bi; cb <= (col * kTile + kTile - 1) / bi && cb < NBi; ++cb)
+                        any |= gamma[(size_t)lb * NBi + cb] != 0;
+                if (any) m |= 1u << r;
+            }
+        }
+        int tot;
+        const int before = block_exclusive_scan(__popc(m), warp_sums, tot);
+        if (col < n_cols) {
+            colmask[(size_t)panel * n_cols + col] = (uint8_t)m;
+            coloff[(size_t)panel * n_cols + col] = (uint32_t)(s_run + before);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_run += tot;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) panel_cnt[panel] = s_run;
+}
+
+// Launch 2 (one CTA): exclusive scans row_cnt -> row_ptr and panel_cnt -> panel_base, writes the packed
+// header, and latches BSP_ERR_CAPACITY if more blocks are stored than the buffers were sized for.
+__global__ void __launch_bounds__(kThreads)
+scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_ptr, const int *__restrict__ panel_cnt,
+            int n_panels, uint32_t *__restrict__ panel_base, PackedHeader *__restrict__ hdr, PackedHeader hdr_init,
+            long long capacity_blocks, long long capacity_tiles, int *__restrict__ status)
+{
+    __shared__ int warp_sums[kThreads / 32];
+    __shared__ int s_run;
+    if (threadIdx.x == 0) s_run = 0;
+    __syncthreads();
+    for (int base = 0; base < NBo; base += kThreads) {
+        const int i = base + threadIdx.x;
+        const int v = (i < NBo) ? row_cnt[i] : 0;
+        int tot;
+        const int before = block_exclusive_scan(v, warp_sums, tot);
+        if (i < NBo) row_ptr[i] = s_run + before;
+        __syncthreads();
+        if (threadIdx.x == 0) s_run += tot;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        row_ptr[NBo] = s_run;
+        if ((long long)s_run > capacity_blocks) atomicMax(status, (int)BSP_ERR_CAPACITY);
+        if (panel_base != nullptr) {
+            unsigned run = 0;
+            for (int p = 0; p < n_panels; ++p) { panel_base[p] = run; run += (unsigned)panel_cnt[p]; }
+            panel_base[n_panels] = run;
+            hdr_init.n_tiles = (int)run;
+            *hdr = hdr_init;
+            if ((long long)run > capacity_tiles) atomicMax(status, (int)BSP_ERR_CAPACITY);
+        }
+    }
+}
+
+// Launch 3a.  One CTA per row of Gamma: column indices in ascending order and the canonical payload
+// payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int NBi, int I, int HK, int bo, int bi,
+                const int32_t *__restrict__ row_ptr, int32_t *__restrict__ col_idx, T *__restrict__ payload,
+                long long capacity_blocks)
+{
+    __shared__ int warp_sums[kThreads / 32];
+    __shared__ int s_run;
+    extern __shared__ int s_cols[];      // NBi ints: columns of this row's stored blocks
+    const int l = blockIdx.x;
+    const uint8_t *g = gamma + (size_t)l * NBi;
+    const int first = row_ptr[l];
+    if (threadIdx.x == 0) s_run = 0;
+    __syncthreads();
+    for (int base = 0; base < NBi; base += kThreads) {
+        const int i = base + threadIdx.x;
+        const int v = (i < NBi && g[i]) ? 1 : 0;
+        int tot;
+        const int before = block_exclusive_scan(v, warp_sums, tot);
+        if (v) {
+            const int n = s_run + before;
+            s_cols[n] = i;
+            if ((long long)(first + n) < capacity_blocks) col_idx[first + n] = i;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_run += tot;
+        __syncthreads();
+    }
+    if (payload == nullptr) return;
+    const int cnt = s_run;
+    const int blk = bo * HK * bi;
+    const long long total = (long long)cnt * blk;
+    for (long long e = threadIdx.x; e < total; e += kThreads) {
+        const int n = (int)(e / blk);
+        const int q = (int)(e % blk);
+        int rem = q;
+        const int c = rem % bi; rem /= bi;
+        const int t = rem % HK;
+        const int r = rem / HK;
+        if ((long long)(first + n) >= capacity_blocks) continue;
+        payload[(size_t)(first + n) * blk + q] = W[((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi + c];
+    }
+}
+
+// One 32-bit word of a packed tile.  The tile at (tile row of the panel, tile column) holds, for every K-step
+// of the MMA, the B-operand fragment of all 32 lanes: lane = 4 g + t holds output channel g of the tile.
+//  bf16 : steps of two taps (m16n8k16): word 2*lane+j of step s = channels 2t, 2t+1 at tap 2s+j;
+//         an odd last tap is a step of its own (m16n8k8) with one word per lane.
+//  int8 : steps of two taps (m16n8k16): the word of lane (g,t) = channels 4(t&1)..4(t&1)+3 at tap 2s+(t>>1);
+//         a missing second tap is written as zeros.
+//  fp32 : one tap per step (m16n8k8, tf32): words 2*lane, 2*lane+1 = channel t and channel t+4.
+// o0, c0: first output and input channel of the tile.  Weights of blocks with Gamma = 0 read as zero.
+template <int DT>
+__device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, const uint8_t *__restrict__ gamma,
+                                                int word, int o0, int c0, int O, int I, int HK, int bo, int bi,
+                                                int NBi)
+{
+    auto kept = [&](int o, int ch) -> bool { return o < O && gamma[(size_t)(o / bo) * NBi + ch / bi] != 0; };
+    if constexpr (DT == BSP_BF16) {
+        const uint16_t *W = (const uint16_t *)Wv;
+        const int pairs = HK / 2;
+        int lane, tap;
+        if (word < pairs * 64) { const int s = word / 64, w = word % 64; lane = w >> 1; tap = 2 * s + (w & 1); }
+        else { lane = word - pairs * 64; tap = HK - 1; }
+        const int g = lane >> 2, t = lane & 3;
+        const int o = o0 + g, ch = c0 + 2 * t;
+        if (!kept(o, ch)) return 0u;              // both channels lie in one block (b_i is even)
+        const size_t e = ((size_t)o * HK + tap) * I + ch;
+        return (uint32_t)W[e] | ((uint32_t)W[e + 1] << 16);
+    } else if constexpr (DT == BSP_I8) {
+        const uint8_t *W = (const uint8_t *)Wv;
+        const int s = word / 32, lane = word % 32;
+        const int g = lane >> 2, t = lane & 3;
+        const int tap = 2 * s + (t >> 1);
+        const int o = o0 + g, ch = c0 + 4 * (t & 1);
+        if (tap >= HK || !kept(o, ch)) return 0u;   // four channels never straddle a block (b_i >= 4)
+        const size_t e = ((size_t)o * HK + tap) * I + ch;
+        return (uint32_t)W[e] | ((uint32_t)W[e + 1] << 8) | ((uint32_t)W[e + 2] << 16) | ((uint32_t)W[e + 3] << 24);
+    } else {
+        const uint32_t *W = (const uint32_t *)Wv;
+        const int tap = word / 64, w = word % 64;
+        const int lane = w >> 1;
+        const int g = lane >> 2, t = lane & 3;
+        const int o = o0 + g, ch = c0 + t + 4 * (w & 1);
+        if (!kept(o, ch)) return 0u;
+        return W[((size_t)o * HK + tap) * I + ch];
+    }
+}
+
+// Launch 3b.  grid (tile-column chunks, panels): every stored tile of the panel in this chunk of columns is
+// written word by word.
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+pack_kernel(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
+            int NBi, int n_cols, int cols_per_cta, int tile_bytes, const uint8_t *__restrict__ colmask,
+            const uint32_t *__restrict__ coloff, const uint32_t *__restrict__ panel_base, uint8_t *__restrict__ payload,
+            long long capacity_tiles)
+{
+    const int panel = blockIdx.y;
+    const int col_lo = blockIdx.x * cols_per_cta;
+    const int col_hi = min(n_cols, col_lo + cols_per_cta);
+    const int words = tile_bytes / 4;
+    const unsigned base = panel_base[panel];
+    for (int col = col_lo; col < col_hi; ++col) {
+        const unsigned m = colmask[(size_t)panel * n_cols + col];
+        if (!m) continue;
+        const unsigned first = base + coloff[(size_t)panel * n_cols + col];
+        const int cnt = __popc(m);
+        for (int e = threadIdx.x; e < cnt * words; e += kThreads) {
+            const int j = e / words, word = e % words;
+            unsigned mm = m;                         // j-th set bit of m = tile row
+            for (int q = 0; q < j; ++q) mm &= mm - 1;
+            const int R = __ffs(mm) - 1;
+            if ((long long)(first + j) >= capacity_tiles) continue;
+            const uint32_t v = packed_word<DT>(W, gamma, word, (panel * kPanelRows + R) * kTile, col * kTile, O, I, HK,
+                                               bo, bi, NBi);
+            ((uint32_t *)(payload + (size_t)(first + j) * tile_bytes))[word] = v;
+        }
+    }
+}
+
+__global__ void count_ones_kernel(const uint8_t *__restrict__ gamma, long long n, unsigned long long *out)
+{
+    unsigned long long c = 0;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        c += gamma[i] ? 1 : 0;
+    for (int d = 16; d > 0; d >>= 1) c += __shfl_down_sync(0xFFFFFFFFu, c, d);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(out, c);
+}
+
+}  // namespace
+
+bsp_status launch_count(const uint8_t *gamma, int64_t n, unsigned long long *out, cudaStream_t st)
+{
+    BSP_CUDA_OK(cudaMemsetAsync(out, 0, sizeof(unsigned long long), st));
+    int64_t grid = (n + 255) / 256;
+    if (grid > 296) grid = 296;
+    if (grid < 1) grid = 1;
+    count_ones_kernel<<<(unsigned)grid, 256, 0, st>>>(gamma, n, out);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gamma, int32_t *row_ptr,
+                          int32_t *col_idx, void *payload, void *packed, int64_t capacity_blocks, void *ws,
+                          cudaStream_t st)
+{
+    const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi, HK = wd.H * wd.K;
+    const PackedLayout L = packed_layout(wd, capacity_blocks);
+    int *status = (int *)ws;
+    int *row_cnt = (int *)((char *)ws + kWsHeader);
+    int *panel_cnt = row_cnt + NBo;
+    uint8_t *pk = (uint8_t *)packed;
+    uint8_t *colmask = pk ? pk + L.off_colmask : nullptr;
+    uint32_t *coloff = pk ? (uint32_t *)(pk + L.off_coloff) : nullptr;
+    uint32_t *panel_base = pk ? (uint32_t *)(pk + L.off_panelbase) : nullptr;
+
+    PackedHeader h = {};
+    h.magic = kPackedMagic; h.dtype = wd.wtype; h.O = wd.O; h.I = wd.I; h.H = wd.H; h.K = wd.K;
+    h.bo = wd.bo; h.bi = wd.bi; h.n_panels = L.n_panels; h.n_cols = L.n_cols; h.tile_bytes = L.tile_bytes;
+    h.capacity_tiles = (int32_t)L.capacity_tiles; h.n_tiles = 0;
+    h.off_colmask = (int32_t)L.off_colmask; h.off_coloff = (int32_t)L.off_coloff;
+    h.off_panelbase = (int32_t)L.off_panelbase; h.off_payload = (int64_t)L.off_payload;
+
+    count_kernel<<<NBo + (pk ? L.n_panels : 0), kThreads, 0, st>>>(gamma, NBo, NBi, wd.bo, wd.bi, wd.O, L.n_cols,
+                                                                   row_cnt, colmask, coloff, panel_cnt);
+    BSP_CUDA_OK(cudaGetLastError());
+    scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, panel_cnt, L.n_panels, panel_base, (PackedHeader *)pk, h,
+                                        (long long)capacity_blocks, (long long)L.capacity_tiles, status);
+    BSP_CUDA_OK(cudaGetLastError());
+    const size_t smem = (size_t)NBi * sizeof(int);
+    if (wd.wtype == BSP_I8)
+        csr_fill_kernel<uint8_t><<<NBo, kThreads, smem, st>>>((const uint8_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+                                                              row_ptr, col_idx, (uint8_t *)payload, capacity_blocks);
+    else if (wd.wtype == BSP_BF16)
+        csr_fill_kernel<uint16_t><<<NBo, kThreads, smem, st>>>((const uint16_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+                                                               row_ptr, col_idx, (uint16_t *)payload, capacity_blocks);
+    else
+        csr_fill_kernel<uint32_t><<<NBo, kThreads, smem, st>>>((const uint32_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+                                                               row_ptr, col_idx, (uint32_t *)payload, capacity_blocks);
+    BSP_CUDA_OK(cudaGetLastError());
+    if (pk) {
+        const int cols_per_cta = 8;
+        dim3 grid((L.n_cols + cols_per_cta - 1) / cols_per_cta, L.n_panels);
+        uint8_t *pl = pk + L.off_payload;
+        if (wd.wtype == BSP_I8)
+            pack_kernel<BSP_I8><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
+                                                           cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
+                                                           (long long)L.capacity_tiles);
+        else if (wd.wtype == BSP_BF16)
+            pack_kernel<BSP_BF16><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
+                                                             cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
+                                                             (long long)L.capacity_tiles);
+        else
+            pack_kernel<BSP_F32><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
+                                                            cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
+                                                            (long long)L.capacity_tiles);
+        BSP_CUDA_OK(cudaGetLastError());
+    }
+    return BSP_OK;
+}
+
+}  // namespace bsp

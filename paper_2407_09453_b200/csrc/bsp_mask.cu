@@ -1,0 +1,189 @@
+// Gamma builder: per-block importance and selection of the n_zero lowest blocks.
+// Eq. (1), Eq. (2) and Section "Predetermined Sparsity ratio and Full Training Ahead" of the paper.
+#include "bsp_internal.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kScoreThreads = 256;
+constexpr int kSelectThreads = 1024;
+
+// One 4-byte word of W holds 1 fp32, 2 bf16 or 4 int8 values, lowest channel in the lowest bytes.
+template <int DT> struct Acc;
+template <> struct Acc<BSP_F32> { using type = double; };
+template <> struct Acc<BSP_BF16> { using type = double; };
+template <> struct Acc<BSP_I8> { using type = long long; };
+
+template <int DT, int NORM>
+__device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc)
+{
+    if constexpr (DT == BSP_F32) {
+        const double v = (double)__uint_as_float(w);
+        acc += (NORM == BSP_NORM_L2) ? v * v : fabs(v);
+    } else if constexpr (DT == BSP_BF16) {
+        const double v0 = (double)__uint_as_float(w << 16);
+        const double v1 = (double)__uint_as_float(w & 0xFFFF0000u);
+        acc += (NORM == BSP_NORM_L2) ? v0 * v0 : fabs(v0);
+        acc += (NORM == BSP_NORM_L2) ? v1 * v1 : fabs(v1);
+    } else {
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const long long v = (long long)(int8_t)((w >> (8 * b)) & 0xFFu);
+            acc += (NORM == BSP_NORM_L2) ? v * v : (v < 0 ? -v : v);
+        }
+    }
+}
+
+// One thread sums one output row r of one block over (h, k, c) in that order; the thread with r = 0 then
+// adds the b_o row sums in order of r.  The order is part of the definition of the float score: it makes
+// the float64 result, and so Gamma, independent of the launch shape.  (Each square of a float or bf16 value
+// is exact in float64, so a fused multiply-add rounds like a multiply followed by an add.)
+// Threads are laid out with consecutive blocks of one block row on consecutive lanes, so that for a fixed
+// (r, h, k) a warp reads one contiguous stretch of input channels.
+template <int DT, int NORM>
+__global__ void __launch_bounds__(kScoreThreads)
+score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
+             typename Acc<DT>::type *__restrict__ score)
+{
+    using acc_t = typename Acc<DT>::type;
+    __shared__ acc_t part[kScoreThreads];
+    constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
+    const int blocks_per_cta = kScoreThreads / bo;
+    const int bl = threadIdx.x % blocks_per_cta;
+    const int r = threadIdx.x / blocks_per_cta;
+    const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
+    const long long NB = (long long)NBo * NBi;
+    acc_t pr = 0;
+    if (B < NB) {
+        const int l = (int)(B / NBi), iota = (int)(B % NBi);
+        const int words = bi / per_word;
+        const size_t row_words = (size_t)I / per_word;
+        const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
+        for (int t = 0; t < HK; ++t) {
+            for (int j = 0; j < words; ++j) add_word<DT, NORM>(__ldg(src + j), pr);
+            src += row_words;
+        }
+    }
+    part[threadIdx.x] = pr;
+    __syncthreads();
+    if (B < NB && r == 0) {
+        acc_t total = 0;
+        for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
+        score[B] = total;
+    }
+}
+
+// Scores are non-negative, so the bit pattern of a float64 orders like the value, as does an int64.
+// One CTA ranks one segment (the whole layer, or one row of Gamma): an 8-pass most-significant-digit
+// radix select finds the key T of the n_zero-th smallest (key, index) pair and how many keys equal to T
+// are still to be zeroed; a final pass in index order writes Gamma, zeroing the keys below T and the first
+// `ties` keys equal to T.
+__global__ void __launch_bounds__(kSelectThreads)
+select_kernel(const unsigned long long *__restrict__ key, long long seg_len, long long n_zero,
+              uint8_t *__restrict__ gamma)
+{
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ long long s_k;
+    __shared__ unsigned int warp_cnt[kSelectThreads / 32];
+    __shared__ long long s_run;
+
+    const unsigned long long *k = key + (size_t)blockIdx.x * seg_len;
+    uint8_t *g = gamma + (size_t)blockIdx.x * seg_len;
+    const int tid = threadIdx.x;
+
+    if (n_zero <= 0 || n_zero >= seg_len) {
+        const uint8_t v = (n_zero <= 0) ? 1 : 0;
+        for (long long i = tid; i < seg_len; i += kSelectThreads) g[i] = v;
+        return;
+    }
+    if (tid == 0) { s_prefix = 0ull; s_k = n_zero; }
+    for (int pass = 7; pass >= 0; --pass) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const unsigned long long prefix = s_prefix;
+        const int shift = 8 * pass;
+        for (long long i = tid; i < seg_len; i += kSelectThreads) {
+            const unsigned long long v = k[i];
+            const bool in = (pass == 7) || ((v >> (shift + 8)) == prefix);
+            if (in) atomicAdd(&hist[(unsigned)((v >> shift) & 0xFFull)], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            long long need = s_k, cum = 0;
+            int d = 0;
+            for (; d < 255; ++d) {
+                if (cum + (long long)hist[d] >= need) break;
+                cum += hist[d];
+            }
+            s_k = need - cum;
+            s_prefix = (prefix << 8) | (unsigned long long)d;
+        }
+        __syncthreads();
+    }
+    const unsigned long long T = s_prefix;
+    const long long ties = s_k;        // keys equal to T to zero, lowest indices first
+    if (tid == 0) s_run = 0;
+    __syncthreads();
+    const int lane = tid & 31, warp = tid >> 5;
+    for (long long base = 0; base < seg_len; base += kSelectThreads) {
+        const long long i = base + tid;
+        unsigned long long v = ~0ull;
+        if (i < seg_len) v = k[i];
+        const bool eq = (i < seg_len) && (v == T);
+        const unsigned ball = __ballot_sync(0xFFFFFFFFu, eq);
+        if (lane == 0) warp_cnt[warp] = __popc(ball);
+        __syncthreads();
+        long long before = s_run;
+        for (int w = 0; w < warp; ++w) before += warp_cnt[w];
+        before += __popc(ball & ((1u << lane) - 1u));
+        if (i < seg_len) g[i] = (v < T || (eq && before < ties)) ? 0 : 1;
+        __syncthreads();
+        if (tid == 0) {
+            long long tot = 0;
+            for (int w = 0; w < kSelectThreads / 32; ++w) tot += warp_cnt[w];
+            s_run += tot;
+        }
+        __syncthreads();
+    }
+}
+
+template <int DT>
+bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *scores, cudaStream_t st)
+{
+    using acc_t = typename Acc<DT>::type;
+    const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
+    const long long NB = (long long)NBo * NBi;
+    const int per_cta = kScoreThreads / wd.bo;
+    const unsigned grid = (unsigned)((NB + per_cta - 1) / per_cta);
+    if (norm == BSP_NORM_L2)
+        score_kernel<DT, BSP_NORM_L2><<<grid, kScoreThreads, 0, st>>>((const uint32_t *)W, wd.I, wd.H * wd.K, wd.bo,
+                                                                       wd.bi, NBo, NBi, (acc_t *)scores);
+    else
+        score_kernel<DT, BSP_NORM_L1><<<grid, kScoreThreads, 0, st>>>((const uint32_t *)W, wd.I, wd.H * wd.K, wd.bo,
+                                                                       wd.bi, NBo, NBi, (acc_t *)scores);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // namespace
+
+bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
+                       uint8_t *gamma, void *scores, cudaStream_t st)
+{
+    bsp_status rc;
+    if (wd.wtype == BSP_F32) rc = run_scores<BSP_F32>(wd, W, norm, scores, st);
+    else if (wd.wtype == BSP_BF16) rc = run_scores<BSP_BF16>(wd, W, norm, scores, st);
+    else rc = run_scores<BSP_I8>(wd, W, norm, scores, st);
+    if (rc != BSP_OK) return rc;
+    const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
+    const long long NB = (long long)NBo * NBi;
+    if (scope == BSP_SCOPE_LAYER)
+        select_kernel<<<1, kSelectThreads, 0, st>>>((const unsigned long long *)scores, NB, n_zero, gamma);
+    else
+        select_kernel<<<NBo, kSelectThreads, 0, st>>>((const unsigned long long *)scores, NBi, n_zero, gamma);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // namespace bsp
