@@ -1,0 +1,155 @@
+// extern "C" entry points of libbsp: argument validation on the host, then kernel launches on the caller's
+// stream.  Declarations and their contracts are in include/bsp.h.
+#include "bsp_internal.cuh"
+
+using namespace bsp;
+
+namespace {
+
+bsp_status check_wdesc(const bsp_wdesc *wd)
+{
+    if (!wd) return BSP_ERR_NULL;
+    if (wd->O <= 0 || wd->I <= 0 || wd->H <= 0 || wd->K <= 0) return BSP_ERR_SHAPE;
+    const bool ok_block = (wd->bo == 8 && wd->bi == 8) || (wd->bo == 4 && wd->bi == 16) || (wd->bo == 16 && wd->bi == 4);
+    if (!ok_block) return BSP_ERR_BLOCK;
+    if (wd->O % wd->bo != 0 || wd->I % wd->bi != 0) return BSP_ERR_SHAPE;
+    if (wd->wtype != BSP_F32 && wd->wtype != BSP_BF16 && wd->wtype != BSP_I8) return BSP_ERR_DTYPE;
+    if ((long long)wd->H * wd->K > 120) return BSP_ERR_SHAPE;
+    return BSP_OK;
+}
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char *bsp_status_string(bsp_status s)
+{
+    switch (s) {
+        case BSP_OK: return "ok";
+        case BSP_ERR_NULL: return "null pointer";
+        case BSP_ERR_SHAPE: return "bad shape";
+        case BSP_ERR_BLOCK: return "block shape is not 8x8, 4x16 or 16x4";
+        case BSP_ERR_DTYPE: return "bad element type";
+        case BSP_ERR_CAPACITY: return "buffer or count too small";
+        case BSP_ERR_INDEX: return "compact structure does not match the descriptor";
+        case BSP_ERR_CUDA: return "CUDA runtime error";
+        case BSP_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+size_t bsp_mask_workspace_bytes(const bsp_wdesc *wd)
+{
+    if (check_wdesc(wd) != BSP_OK) return 0;
+    const size_t NB = (size_t)(wd->O / wd->bo) * (wd->I / wd->bi);
+    return kWsHeader + align_up(NB * 8, 256);
+}
+
+bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
+                    uint8_t *gamma, void *scores_opt, void *ws, void *stream)
+{
+    bsp_status rc = check_wdesc(wd);
+    if (rc != BSP_OK) return rc;
+    if (!W || !gamma || !ws) return BSP_ERR_NULL;
+    if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1) return BSP_ERR_DTYPE;
+    if (scope != BSP_SCOPE_LAYER && scope != BSP_SCOPE_ROW) return BSP_ERR_DTYPE;
+    const int64_t NBi = wd->I / wd->bi, NB = (int64_t)(wd->O / wd->bo) * NBi;
+    const int64_t limit = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
+    if (n_zero < 0 || n_zero > limit) return BSP_ERR_CAPACITY;
+    void *scores = scores_opt ? scores_opt : (void *)((char *)ws + kWsHeader);
+    return launch_mask(*wd, W, norm, scope, n_zero, gamma, scores, (cudaStream_t)stream);
+}
+
+size_t bsp_packed_bytes(const bsp_wdesc *wd, int64_t nnz)
+{
+    if (check_wdesc(wd) != BSP_OK || nnz < 0) return 0;
+    return packed_layout(*wd, nnz).total_bytes;
+}
+
+size_t bsp_compact_workspace_bytes(const bsp_wdesc *wd)
+{
+    if (check_wdesc(wd) != BSP_OK) return 0;
+    const size_t n = (size_t)(wd->O / wd->bo) + (size_t)((wd->O + kPanelCh - 1) / kPanelCh) + 8;
+    return kWsHeader + align_up(n * 4, 256);
+}
+
+bsp_status bsp_compact_nnz(const bsp_wdesc *wd, const uint8_t *gamma, int64_t *nnz_host, void *ws, void *stream)
+{
+    bsp_status rc = check_wdesc(wd);
+    if (rc != BSP_OK) return rc;
+    if (!gamma || !nnz_host || !ws) return BSP_ERR_NULL;
+    const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
+    unsigned long long *cnt = (unsigned long long *)((char *)ws + kWsHeader);
+    rc = launch_count(gamma, NB, cnt, (cudaStream_t)stream);
+    if (rc != BSP_OK) return rc;
+    unsigned long long h = 0;
+    BSP_CUDA_OK(cudaMemcpyAsync(&h, cnt, sizeof(h), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    BSP_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    *nnz_host = (int64_t)h;
+    return BSP_OK;
+}
+
+bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma, int32_t *row_ptr,
+                       int32_t *col_idx, void *payload, void *packed, int64_t capacity_blocks, void *ws,
+                       void *stream)
+{
+    bsp_status rc = check_wdesc(wd);
+    if (rc != BSP_OK) return rc;
+    if (!W || !gamma || !row_ptr || !col_idx || !ws) return BSP_ERR_NULL;
+    if (capacity_blocks < 0) return BSP_ERR_CAPACITY;
+    if (packed && (wd->O % 8 != 0 || wd->I % 8 != 0)) return BSP_ERR_SHAPE;
+    if (packed && !aligned16(packed)) return BSP_ERR_SHAPE;
+    return launch_compact(*wd, W, gamma, row_ptr, col_idx, payload, packed, capacity_blocks, ws, (cudaStream_t)stream);
+}
+
+size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd)
+{
+    (void)xd;
+    if (check_wdesc(wd) != BSP_OK) return 0;
+    return kWsHeader;
+}
+
+bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                      const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
+{
+    bsp_status rc = check_wdesc(wd);
+    if (rc != BSP_OK) return rc;
+    if (!w || !xd || !X || !Y || !ws || !w->packed) return BSP_ERR_NULL;
+    if (xd->N <= 0 || xd->L <= 0 || xd->J <= 0 || xd->stride_h <= 0 || xd->stride_w <= 0 || xd->pad_h < 0 ||
+        xd->pad_w < 0)
+        return BSP_ERR_SHAPE;
+    if (xd->L + 2 * xd->pad_h < wd->H || xd->J + 2 * xd->pad_w < wd->K) return BSP_ERR_SHAPE;
+    if (wd->O % 8 != 0 || wd->I % 8 != 0) return BSP_ERR_SHAPE;
+    if (wd->wtype == BSP_I8) { if (ytype != BSP_I32) return BSP_ERR_DTYPE; }
+    else if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
+    if (!aligned16(X) || !aligned16(Y) || !aligned16(w->packed)) return BSP_ERR_SHAPE;
+    // the packed header is on the device; the host checks what it can: capacity against the descriptor
+    const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
+    if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
+    return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
+}
+
+bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,
+                    void *Y, bsp_dtype ytype, void *ws, void *stream)
+{
+    if (!wd) return BSP_ERR_NULL;
+    if (wd->H != 1 || wd->K != 1) return BSP_ERR_SHAPE;
+    if (P <= 0 || P > 0x7FFFFFFF) return BSP_ERR_SHAPE;
+    bsp_xdesc xd = {(int)P, 1, 1, 1, 1, 0, 0};
+    return bsp_conv2d(wd, w, &xd, X, bias, Y, ytype, ws, stream);
+}
+
+bsp_status bsp_check(void *ws, void *stream)
+{
+    if (!ws) return BSP_ERR_NULL;
+    int h = 0;
+    BSP_CUDA_OK(cudaMemcpyAsync(&h, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    BSP_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    if (h != 0) BSP_CUDA_OK(cudaMemsetAsync(ws, 0, sizeof(int), (cudaStream_t)stream));
+    if (h < 0 || h > (int)BSP_ERR_TIMEOUT) return BSP_ERR_CUDA;
+    return (bsp_status)h;
+}
+
+}  // extern "C"

@@ -1,0 +1,488 @@
+// Block-sparse implicit-GEMM convolution / FC product with fused bias on warp-level tensor-core MMAs.
+// Introduction (Y = W*X + b) and Section "Block Sparsity in a Matrix" of the paper: only stored 8x8 tiles of
+// W-bar are read and multiplied.
+//
+// Orientation: output pixels are the MMA M dimension, the 8 output channels of a tile row are N, input
+// channels (times taps) are K.  A CTA owns a tile of output pixels (nb images x th rows x tw columns) and
+// WN panels of 64 output channels; warp (wm, wn) accumulates 64 pixels x 64 channels in registers.
+// The input patch of the pixel tile is staged in shared memory in chunks of GC tile columns (8 channels
+// each) through a 3-stage cp.async ring, laid out [tile column][patch pixel][8 channels], so that a tap is
+// a constant byte offset and out-of-image pixels are zero filled once.  For every tile column the warp reads
+// the byte mask of stored tiles of its panel, loads the activation fragments once per K-step and issues MMAs
+// only for the tile rows whose mask bit is set; the branch is uniform across the warp.
+#include "bsp_internal.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kStages = 3;
+constexpr int kMaxTaps = 128;
+constexpr int kMT = 4;                 // 16-pixel MMA tiles per warp
+
+struct ConvParams {
+    const uint8_t *X;
+    uint8_t *Y;
+    const void *bias;
+    const uint8_t *colmask;
+    const uint32_t *coloff;
+    const uint32_t *panel_base;
+    const uint8_t *payload;
+    int N, L, J, I, O, M, Nw, H, K, sh, sw, ph, pw;
+    int nb, th, tw, PH, PW, patch_pix, tile_pix;
+    int tiles_x, tiles_y;
+    int n_cols, n_panels, tile_bytes, GC, n_chunks, stage_bytes;
+    int ytype;
+};
+
+template <int DT> struct Traits;
+template <> struct Traits<BSP_BF16> { static constexpr int CH = 16; using acc_t = float; };
+template <> struct Traits<BSP_I8> { static constexpr int CH = 8; using acc_t = int; };
+template <> struct Traits<BSP_F32> { static constexpr int CH = 32; using acc_t = float; };
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async(uint32_t dst, const void *src, int bytes, bool valid)
+{
+    const int sz = valid ? bytes : 0;
+    if (bytes == 16)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];\n" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ void mma_bf16_k16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16_k8(float (&c)[4], const uint32_t (&a)[4], uint32_t b0)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(b0));
+}
+__device__ __forceinline__ void mma_s8_k16(int (&c)[4], const uint32_t (&a)[4], uint32_t b0)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};\n"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(b0));
+}
+__device__ __forceinline__ void mma_tf32_k8(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t to_tf32(uint32_t fbits)
+{
+    uint32_t r;
+    asm volatile("cvt.rna.tf32.f32 %0, %1;\n" : "=r"(r) : "f"(__uint_as_float(fbits)));
+    return r;
+}
+
+// Byte offset, inside one tile column of the staged patch, of the top-left input pixel of output pixel q of
+// the CTA's tile (q counts images, then rows, then columns of the tile).  Pixels past the tile map to 0.
+template <int CH>
+__device__ __forceinline__ int patch_offset(const ConvParams &p, int q)
+{
+    if (q >= p.tile_pix) return 0;
+    const int ix = q % p.tw;
+    const int t = q / p.tw;
+    const int iy = t % p.th;
+    const int in = t / p.th;
+    return ((in * p.PH + iy * p.sh) * p.PW + ix * p.sw) * CH;
+}
+
+template <int DT, int WM, int WN>
+__global__ void __launch_bounds__(32 * WM * WN, 1)
+conv_mma_kernel(const __grid_constant__ ConvParams p)
+{
+    using T = Traits<DT>;
+    using acc_t = typename T::acc_t;
+    constexpr int CH = T::CH;
+    constexpr int NT = 32 * WM * WN;
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ int s_tapoff[kMaxTaps];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm = warp % WM, wn = warp / WM;
+    const int HK = p.H * p.K;
+
+    // tile origin
+    int tix = blockIdx.x;
+    const int tx = tix % p.tiles_x; tix /= p.tiles_x;
+    const int ty = tix % p.tiles_y;
+    const int tn = tix / p.tiles_y;
+    const int n0 = tn * p.nb, y0 = ty * p.th, x0 = tx * p.tw;
+    const int gy0 = y0 * p.sh - p.ph, gx0 = x0 * p.sw - p.pw;
+
+    for (int t = tid; t < kMaxTaps; t += NT) {
+        const int tt = t < HK ? t : HK - 1;
+        s_tapoff[t] = ((tt / p.K) * p.PW + (tt % p.K)) * CH;
+    }
+
+    const uint32_t smem_base = smem_u32(smem);
+
+    // ---- loader: one chunk of GC tile columns of the patch into a stage
+    auto load_chunk = [&](int c, int stage) {
+        if (c < p.n_chunks) {
+            const int col0 = c * p.GC;
+            const int ncol = min(p.GC, p.n_cols - col0);
+            const uint32_t sbase = smem_base + stage * p.stage_bytes;
+            for (int pp = tid; pp < p.patch_pix; pp += NT) {
+                const int px = pp % p.PW;
+                const int t = pp / p.PW;
+                const int py = t % p.PH;
+                const int in = t / p.PH;
+                const int n = n0 + in, gy = gy0 + py, gx = gx0 + px;
+                const bool valid = (n < p.N) && (gy >= 0) && (gy < p.L) && (gx >= 0) && (gx < p.J);
+                const uint8_t *src = p.X;
+                if (valid) src += ((((size_t)n * p.L + gy) * p.J + gx) * p.I) * (CH / 8) + (size_t)col0 * CH;
+                uint32_t dst = sbase + pp * CH;
+                for (int v = 0; v < ncol; ++v) {
+                    if constexpr (CH == 32) {
+                        cp_async(dst, src, 16, valid);
+                        cp_async(dst + 16, src + (valid ? 16 : 0), 16, valid);
+                    } else {
+                        cp_async(dst, src, CH, valid);
+                    }
+                    if (valid) src += CH;
+                    dst += p.patch_pix * CH;
+                }
+            }
+        }
+        cp_async_commit();
+    };
+
+    // ---- per-thread fragment addressing
+    int rowoff[kMT][2];
+#pragma unroll
+    for (int i = 0; i < kMT; ++i) {
+        const int qbase = (wm * kMT + i) * 16;
+        if constexpr (DT == BSP_BF16) {
+            rowoff[i][0] = patch_offset<CH>(p, qbase + (lane & 15));
+            rowoff[i][1] = 0;
+        } else {
+            rowoff[i][0] = patch_offset<CH>(p, qbase + (lane >> 2));
+            rowoff[i][1] = patch_offset<CH>(p, qbase + (lane >> 2) + 8);
+        }
+    }
+
+    acc_t acc[kMT][kPanelRows][4];
+#pragma unroll
+    for (int i = 0; i < kMT; ++i)
+#pragma unroll
+        for (int r = 0; r < kPanelRows; ++r)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][r][e] = 0;
+
+    const int panel = blockIdx.y * WN + wn;
+    const bool active = panel < p.n_panels;
+    const uint32_t pbase = active ? p.panel_base[panel] : 0u;
+    const uint8_t *cm = p.colmask + (size_t)(active ? panel : 0) * p.n_cols;
+    const uint32_t *co = p.coloff + (size_t)(active ? panel : 0) * p.n_cols;
+
+    // prefetch of the masks/offsets of one chunk: lane v holds tile column chunk*GC + v
+    auto fetch_meta = [&](int c, uint32_t &m, uint32_t &o) {
+        const int col = c * p.GC + lane;
+        m = 0; o = 0;
+        if (active && c < p.n_chunks && lane < p.GC && col < p.n_cols) { m = cm[col]; o = co[col]; }
+    };
+
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) load_chunk(s, s);
+    uint32_t meta_m, meta_o;
+    fetch_meta(0, meta_m, meta_o);
+
+    for (int c = 0; c < p.n_chunks; ++c) {
+        cp_async_wait<kStages - 2>();
+        __syncthreads();
+        load_chunk(c + kStages - 1, (c + kStages - 1) % kStages);
+        const uint32_t cur_m = meta_m, cur_o = meta_o;
+        fetch_meta(c + 1, meta_m, meta_o);
+        if (!active) continue;
+        const uint32_t stage_addr = smem_base + (c % kStages) * p.stage_bytes;
+        const int ncol = min(p.GC, p.n_cols - c * p.GC);
+        for (int v = 0; v < ncol; ++v) {
+            const uint32_t m = __shfl_sync(0xFFFFFFFFu, cur_m, v);
+            if (m == 0) continue;
+            const uint32_t off = __shfl_sync(0xFFFFFFFFu, cur_o, v);
+            const uint8_t *wt = p.payload + (size_t)(pbase + off) * p.tile_bytes;
+            const uint32_t abase = stage_addr + v * p.patch_pix * CH;
+
+            if constexpr (DT == BSP_BF16) {
+                const int n16 = HK >> 1;
+                const int sel = lane >> 4;
+                for (int s = 0; s < n16; ++s) {
+                    uint32_t a[kMT][4];
+                    const int toff = s_tapoff[2 * s + sel];
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i) ldmatrix_x4(abase + rowoff[i][0] + toff, a[i]);
+                    const uint8_t *wp = wt + s * 256 + lane * 8;
+#pragma unroll
+                    for (int r = 0; r < kPanelRows; ++r) {
+                        if (m & (1u << r)) {
+                            const uint2 b = __ldg((const uint2 *)wp);
+                            wp += p.tile_bytes;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][r], a[i], b.x, b.y);
+                        }
+                    }
+                }
+                if (HK & 1) {
+                    uint32_t a[kMT][4];
+                    const int toff = s_tapoff[HK - 1];
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i) ldmatrix_x2(abase + rowoff[i][0] + toff, a[i]);
+                    const uint8_t *wp = wt + n16 * 256 + lane * 4;
+#pragma unroll
+                    for (int r = 0; r < kPanelRows; ++r) {
+                        if (m & (1u << r)) {
+                            const uint32_t b = __ldg((const uint32_t *)wp);
+                            wp += p.tile_bytes;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][r], a[i], b);
+                        }
+                    }
+                }
+            } else if constexpr (DT == BSP_I8) {
+                const int nsteps = (HK + 1) >> 1;
+                const int t = lane & 3;
+                for (int s = 0; s < nsteps; ++s) {
+                    uint32_t a[kMT][4];
+                    const int toff = s_tapoff[2 * s + (t >> 1)] + (t & 1) * 4;
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i) {
+                        a[i][0] = lds32(abase + rowoff[i][0] + toff);
+                        a[i][1] = lds32(abase + rowoff[i][1] + toff);
+                    }
+                    const uint8_t *wp = wt + s * 128 + lane * 4;
+#pragma unroll
+                    for (int r = 0; r < kPanelRows; ++r) {
+                        if (m & (1u << r)) {
+                            const uint32_t b = __ldg((const uint32_t *)wp);
+                            wp += p.tile_bytes;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][r], a[i], b);
+                        }
+                    }
+                }
+            } else {
+                const int t = lane & 3;
+                for (int s = 0; s < HK; ++s) {
+                    uint32_t a[kMT][4];
+                    const int toff = s_tapoff[s] + t * 4;
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i) {
+                        a[i][0] = to_tf32(lds32(abase + rowoff[i][0] + toff));
+                        a[i][1] = to_tf32(lds32(abase + rowoff[i][1] + toff));
+                        a[i][2] = to_tf32(lds32(abase + rowoff[i][0] + toff + 16));
+                        a[i][3] = to_tf32(lds32(abase + rowoff[i][1] + toff + 16));
+                    }
+                    const uint8_t *wp = wt + s * 256 + lane * 8;
+#pragma unroll
+                    for (int r = 0; r < kPanelRows; ++r) {
+                        if (m & (1u << r)) {
+                            const uint2 b = __ldg((const uint2 *)wp);
+                            wp += p.tile_bytes;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) mma_tf32_k8(acc[i][r], a[i], to_tf32(b.x), to_tf32(b.y));
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- epilogue: + bias, convert, stage 16 pixels x 64 channels per warp in shared memory, store rows
+    cp_async_wait<0>();
+    __syncthreads();
+    const int oe = (p.ytype == BSP_BF16) ? 2 : 4;               // bytes per output element
+    const int pitch = kPanelCh * oe + 16;
+    uint8_t *ebuf = smem + warp * (16 * (kPanelCh * 4 + 16));
+    if (active) {
+        const int g = lane >> 2, t = lane & 3;
+        const int ch0 = panel * kPanelCh;
+        acc_t bv[kPanelRows][2];
+#pragma unroll
+        for (int r = 0; r < kPanelRows; ++r) {
+            const int o = ch0 + r * 8 + 2 * t;
+            bv[r][0] = 0; bv[r][1] = 0;
+            if (p.bias != nullptr && o < p.O) {
+                bv[r][0] = ((const acc_t *)p.bias)[o];
+                bv[r][1] = ((const acc_t *)p.bias)[o + 1];
+            }
+        }
+        const int cpr = kPanelCh * oe / 16;                      // 16-byte chunks per pixel row
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) {
+#pragma unroll
+            for (int r = 0; r < kPanelRows; ++r) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const acc_t v0 = acc[i][r][2 * hh] + bv[r][0];
+                    const acc_t v1 = acc[i][r][2 * hh + 1] + bv[r][1];
+                    uint8_t *dst = ebuf + (g + 8 * hh) * pitch + (r * 8 + 2 * t) * oe;
+                    if constexpr (DT == BSP_I8) {
+                        *(int2 *)dst = make_int2(v0, v1);
+                    } else {
+                        if (oe == 2) *(__nv_bfloat162 *)dst = __floats2bfloat162_rn(v0, v1);
+                        else *(float2 *)dst = make_float2(v0, v1);
+                    }
+                }
+            }
+            __syncwarp();
+            for (int idx = lane; idx < 16 * cpr; idx += 32) {
+                const int row = idx / cpr, chunk = idx % cpr;
+                const int q = (wm * kMT + i) * 16 + row;
+                const int o = ch0 + chunk * (16 / oe);
+                if (q < p.tile_pix && o < p.O) {
+                    const int ix = q % p.tw;
+                    const int tq = q / p.tw;
+                    const int iy = tq % p.th;
+                    const int in = tq / p.th;
+                    const int n = n0 + in, y = y0 + iy, x = x0 + ix;
+                    if (n < p.N && y < p.M && x < p.Nw) {
+                        const size_t pix = ((size_t)n * p.M + y) * p.Nw + x;
+                        *(uint4 *)(p.Y + (pix * p.O + o) * oe) = *(const uint4 *)(ebuf + row * pitch + chunk * 16);
+                    }
+                }
+            }
+            __syncwarp();
+        }
+    }
+}
+
+struct Plan {
+    int WM, WN, nb, th, tw, GC;
+    size_t smem;
+    long long tiles, ctas;
+};
+
+constexpr int kConfigs[][2] = {{2, 2}, {4, 2}, {2, 4}, {4, 1}, {8, 1}, {1, 4}};
+
+void best_tile(int tpix, int N, int M, int Nw, int &nb, int &th, int &tw, long long &tiles)
+{
+    long long best = -1;
+    long long best_area = 0;
+    for (int w = 1; w <= Nw && w <= tpix; ++w) {
+        const int hmax = tpix / w < M ? tpix / w : M;
+        for (int h = 1; h <= hmax; ++h) {
+            int b = 1;
+            if (h == M && w == Nw) { b = tpix / (h * w); if (b > N) b = N; if (b < 1) b = 1; }
+            const long long cnt = (long long)((N + b - 1) / b) * ((M + h - 1) / h) * ((Nw + w - 1) / w);
+            const long long area = (long long)b * h * w;
+            if (best < 0 || cnt < best || (cnt == best && area < best_area)) {
+                best = cnt; best_area = area; nb = b; th = h; tw = w;
+            }
+        }
+    }
+    tiles = best;
+}
+
+Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_panels, int n_cols)
+{
+    const int CH = 8 * elem_bytes(wd.wtype);
+    Plan best = {};
+    double best_cost = -1;
+    for (auto &cfg : kConfigs) {
+        Plan pl = {};
+        pl.WM = cfg[0]; pl.WN = cfg[1];
+        best_tile(pl.WM * 64, xd.N, M, Nw, pl.nb, pl.th, pl.tw, pl.tiles);
+        const int PH = (pl.th - 1) * xd.stride_h + wd.H, PW = (pl.tw - 1) * xd.stride_w + wd.K;
+        const long long patch_pix = (long long)pl.nb * PH * PW;
+        int GC = (int)(32768 / (patch_pix * CH));
+        if (GC > 32) GC = 32;
+        if (GC > n_cols) GC = n_cols;
+        if (GC < 1) GC = 1;
+        pl.GC = GC;
+        const size_t stage = align_up((size_t)GC * patch_pix * CH, 128);
+        const size_t epi = (size_t)pl.WM * pl.WN * 16 * (kPanelCh * 4 + 16);
+        pl.smem = stage * kStages > epi ? stage * kStages : epi;
+        if (pl.smem > 200 * 1024) continue;
+        pl.ctas = pl.tiles * ((n_panels + pl.WN - 1) / pl.WN);
+        const int warps = pl.WM * pl.WN;
+        // busiest SM: CTAs dealt round-robin over 148 SMs, each CTA keeping `warps` warps busy
+        const double load = (double)((pl.ctas + 147) / 148) * warps;
+        const double traffic = (double)pl.ctas * patch_pix * n_cols * CH + (double)pl.tiles * n_panels * 1.0;
+        const double cost = load * 1e15 + traffic;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = pl; }
+    }
+    return best;
+}
+
+template <int DT, int WM, int WN>
+bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
+{
+    auto kern = conv_mma_kernel<DT, WM, WN>;
+    if (pl.smem > 48 * 1024)
+        BSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+    dim3 grid((unsigned)pl.tiles, (unsigned)((p.n_panels + WN - 1) / WN));
+    kern<<<grid, 32 * WM * WN, pl.smem, st>>>(p);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+template <int DT>
+bsp_status launch_dt(const ConvParams &p, const Plan &pl, cudaStream_t st)
+{
+    if (pl.WM == 2 && pl.WN == 2) return launch_cfg<DT, 2, 2>(p, pl, st);
+    if (pl.WM == 4 && pl.WN == 2) return launch_cfg<DT, 4, 2>(p, pl, st);
+    if (pl.WM == 2 && pl.WN == 4) return launch_cfg<DT, 2, 4>(p, pl, st);
+    if (pl.WM == 4 && pl.WN == 1) return launch_cfg<DT, 4, 1>(p, pl, st);
+    if (pl.WM == 8 && pl.WN == 1) return launch_cfg<DT, 8, 1>(p, pl, st);
+    return launch_cfg<DT, 1, 4>(p, pl, st);
+}
+
+}  // namespace
+
+bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                       const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
+{
+    (void)ws;
+    const PackedLayout L = packed_layout(wd, 0);
+    const int M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1;
+    const int Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
+    const Plan pl = make_plan(wd, xd, M, Nw, L.n_panels, L.n_cols);
+    if (pl.WM == 0) return BSP_ERR_SHAPE;
+    const int CH = 8 * elem_bytes(wd.wtype);
+    const uint8_t *pk = (const uint8_t *)packed;
+    ConvParams p = {};
+    p.X = (const uint8_t *)X; p.Y = (uint8_t *)Y; p.bias = bias;
+    p.colmask = pk + L.off_colmask;
+    p.coloff = (const uint32_t *)(pk + L.off_coloff);
+    p.panel_base = (const uint32_t *)(pk + L.off_panelbase);
+    p.payload = pk + L.off_payload;
+    p.N = xd.N; p.L = xd.L; p.J = xd.J; p.I = wd.I; p.O = wd.O; p.M = M; p.Nw = Nw; p.H = wd.H; p.K = wd.K;
+    p.sh = xd.stride_h; p.sw = xd.stride_w; p.ph = xd.pad_h; p.pw = xd.pad_w;
+    p.nb = pl.nb; p.th = pl.th; p.tw = pl.tw;
+    p.PH = (pl.th - 1) * xd.stride_h + wd.H; p.PW = (pl.tw - 1) * xd.stride_w + wd.K;
+    p.patch_pix = pl.nb * p.PH * p.PW; p.tile_pix = pl.nb * pl.th * pl.tw;
+    p.tiles_x = (Nw + pl.tw - 1) / pl.tw; p.tiles_y = (M + pl.th - 1) / pl.th;
+    p.n_cols = L.n_cols; p.n_panels = L.n_panels; p.tile_bytes = L.tile_bytes; p.GC = pl.GC;
+    p.n_chunks = (L.n_cols + pl.GC - 1) / pl.GC;
+    p.stage_bytes = (int)align_up((size_t)pl.GC * p.patch_pix * CH, 128);
+    p.ytype = ytype;
+    if (wd.wtype == BSP_BF16) return launch_dt<BSP_BF16>(p, pl, st);
+    if (wd.wtype == BSP_I8) return launch_dt<BSP_I8>(p, pl, st);
+    return launch_dt<BSP_F32>(p, pl, st);
+}
+
+}  // namespace bsp
