@@ -1,0 +1,112 @@
+"""GPU parity: Gamma builder and compaction against the CPU oracle, bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2407_09453_b200 import bsp, synth
+from gpu_util import gpu_layer, gpu_mask, from_dev, make_case, to_dev, TORCH_DT
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(8, 8), (4, 16), (16, 4)]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "i8"])
+@pytest.mark.parametrize("bo,bi", SHAPES)
+@pytest.mark.parametrize("norm", [bsp.NORM_L2, bsp.NORM_L1])
+def test_scores_and_gamma_bit_exact(dtype, bo, bi, norm):
+    O, I, H, K = 96, 160, 3, 3
+    W = make_case(101, O, I, H, K, dtype)
+    NB = (O // bo) * (I // bi)
+    want_s = ref.scores(W, bo, bi, norm)
+    for n_zero in (NB // 2, 1, NB - 1):
+        g, s, _, _ = gpu_mask(W, bo, bi, dtype, n_zero, norm)
+        assert np.array_equal(s.view(np.uint64), want_s.view(np.uint64))      # identical bit patterns
+        assert np.array_equal(g, ref.mask(want_s, n_zero))
+        assert int((g == 0).sum()) == n_zero                                   # Eq. (2)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
+def test_gamma_row_scope_and_extremes(dtype):
+    bo = bi = 8
+    O, I, H, K = 64, 256, 1, 1
+    W = make_case(103, O, I, H, K, dtype)
+    want_s = ref.scores(W, bo, bi)
+    g, s, _, _ = gpu_mask(W, bo, bi, dtype, 9, scope=bsp.SCOPE_ROW)
+    assert np.array_equal(g, ref.mask(want_s, 9, ref.SCOPE_ROW)) and np.all((g == 0).sum(axis=1) == 9)
+    for n_zero in (0, 32):
+        g, _, _, _ = gpu_mask(W, bo, bi, dtype, n_zero, scope=bsp.SCOPE_ROW)
+        assert np.all(g == (1 if n_zero == 0 else 0))
+    NB = g.size
+    assert gpu_mask(W, bo, bi, dtype, 0)[0].all() and not gpu_mask(W, bo, bi, dtype, NB)[0].any()
+
+
+def test_gamma_ties_broken_by_index():
+    """int8 scores collide all the time; equal weights make every score equal."""
+    bo = bi = 8
+    W = np.full((64, 1, 1, 64), 5, dtype=np.int8)
+    g, s, _, _ = gpu_mask(W, bo, bi, "i8", 23)
+    assert np.array_equal(g.ravel(), np.r_[np.zeros(23, np.uint8), np.ones(41, np.uint8)])
+    W = synth.uniform_int(107, (128, 1, 1, 256), -3, 3).astype(np.int8)        # few distinct scores
+    want_s = ref.scores(W, bo, bi)
+    assert len(np.unique(want_s)) < want_s.size // 2
+    for n_zero in (100, 256, 301):
+        g, s, _, _ = gpu_mask(W, bo, bi, "i8", n_zero)
+        assert np.array_equal(g, ref.mask(want_s, n_zero))
+
+
+def test_gamma_large_layer_many_select_passes():
+    """More blocks than one pass of the selecting CTA covers (4096x2048 / 8x8 = 131072 blocks)."""
+    bo = bi = 8
+    W = synth.round_to_bf16(synth.normal(109, (2048, 1, 1, 1024), 1 / 32.0).astype(np.float32))
+    want_s = ref.scores(W, bo, bi)
+    g, s, _, _ = gpu_mask(W, bo, bi, "bf16", want_s.size // 2)
+    assert np.array_equal(s.view(np.uint64), want_s.view(np.uint64))
+    assert np.array_equal(g, ref.mask(want_s, want_s.size // 2))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "i8"])
+@pytest.mark.parametrize("bo,bi", SHAPES)
+def test_compact_bit_exact(dtype, bo, bi):
+    O, I, H, K = 128, 96, 3, 2
+    W = make_case(113, O, I, H, K, dtype)
+    NBo, NBi = O // bo, I // bi
+    for nz in ((NBo * NBi) // 2, 0, NBo * NBi, 5):
+        gamma = synth.random_gamma(115 + nz, NBo, NBi, nz)
+        lay = gpu_layer(W, gamma, bo, bi, dtype)
+        rp, ci, pl = ref.compact(W, gamma, bo, bi)
+        nnz = len(ci)
+        assert np.array_equal(from_dev(lay.row_ptr), rp)
+        assert np.array_equal(from_dev(lay.col_idx)[:nnz], ci)
+        got = from_dev(lay.payload)[:pl.size].reshape(pl.shape)
+        assert np.array_equal(got, pl if dtype != "bf16" else pl.astype(np.float32))
+        assert bsp.bsp_compact_nnz(lay.wd, lay.gamma, lay.ws) == nnz
+
+
+def test_compact_capacity_overflow_is_latched():
+    bo = bi = 8
+    W = make_case(117, 64, 64, 1, 1, "bf16")
+    lay = bsp.SparseLayer(64, 64, 1, 1, bo, bi, torch.bfloat16, capacity_blocks=10)
+    gamma = synth.random_gamma(119, 8, 8, 32)
+    lay.compact(to_dev(W, "bf16"), torch.from_numpy(gamma).cuda())
+    with pytest.raises(bsp.BspError) as e:
+        lay.check()
+    assert e.value.status == bsp.ERR_CAPACITY
+    lay.check()                                                                # cleared after being read
+
+
+def test_mask_then_compact_round_trip_to_masked_dense():
+    bo = bi = 8
+    O, I, H, K = 256, 256, 3, 3
+    W = make_case(121, O, I, H, K, "bf16")
+    g, s, lay, Wd = gpu_mask(W, bo, bi, "bf16", 512)
+    lay.compact(Wd)
+    lay.check()
+    rp, ci = from_dev(lay.row_ptr), from_dev(lay.col_idx)
+    pl = from_dev(lay.payload).reshape(-1, bo, H, K, bi)
+    back = np.zeros_like(W)
+    for l in range(O // bo):
+        for n in range(rp[l], rp[l + 1]):
+            back[l * bo:(l + 1) * bo, :, :, ci[n] * bi:(ci[n] + 1) * bi] = pl[n]
+    assert rp[-1] == 512 and np.array_equal(back, ref.apply_mask(W, g, bo, bi))
