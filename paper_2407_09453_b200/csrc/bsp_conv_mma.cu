@@ -18,6 +18,8 @@ namespace {
 constexpr int kStages = 3;
 constexpr int kMaxTaps = 128;
 constexpr int kMT = 4;                 // 16-pixel MMA tiles per warp
+constexpr int kMaxSmem = 200 * 1024;   // dynamic shared memory ceiling of a launch
+constexpr int kMaxDevices = 64;
 
 struct ConvParams {
     const uint8_t *X;
@@ -416,7 +418,7 @@ Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_pa
         const size_t stage = align_up((size_t)GC * patch_pix * CH, 128);
         const size_t epi = (size_t)pl.WM * pl.WN * 16 * (kPanelCh * 4 + 16);
         pl.smem = stage * kStages > epi ? stage * kStages : epi;
-        if (pl.smem > 200 * 1024) continue;
+        if (pl.smem > (size_t)kMaxSmem) continue;
         pl.ctas = pl.tiles * ((n_panels + pl.WN - 1) / pl.WN);
         const int warps = pl.WM * pl.WN;
         // busiest SM: CTAs dealt round-robin over 148 SMs, each CTA keeping `warps` warps busy
@@ -432,8 +434,16 @@ template <int DT, int WM, int WN>
 bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
 {
     auto kern = conv_mma_kernel<DT, WM, WN>;
-    if (pl.smem > 48 * 1024)
-        BSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+    // opt in to large dynamic shared memory once per device and instantiation (static shared memory counts
+    // against the default 48 KB, so the opt-in is unconditional)
+    static bool opted[kMaxDevices] = {};
+    int dev = 0;
+    BSP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BSP_ERR_CUDA;
+    if (!opted[dev]) {
+        BSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        opted[dev] = true;
+    }
     dim3 grid((unsigned)pl.tiles, (unsigned)((p.n_panels + WN - 1) / WN));
     kern<<<grid, 32 * WM * WN, pl.smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
