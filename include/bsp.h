@@ -103,6 +103,29 @@ size_t bsp_mask_workspace_bytes(const bsp_wdesc *wd);
 bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
                     uint8_t *gamma, void *scores_opt, void *ws, void *stream);
 
+/* ---- Gamma builder without caller scratch ------------------------------------------------------------
+ * (The paper has no counterpart: this entry point exists for the way the library is embedded.)
+ * Some hosts of this library may not allocate device memory at the point where a layer is masked: code that
+ * runs inside another framework's memory plan or with a fixed, pre-carved device heap, plugins that are
+ * handed only their input and output tensors, and real-time loops in which cudaMalloc (a blocking, device-
+ * wide call) is banned.  Such callers cannot size and pass the `ws` buffer that bsp_mask() needs for the
+ * block scores.  bsp_mask_static() computes exactly what bsp_mask() computes (same kernels, same bit-exact
+ * Gamma) but keeps the scores in a fixed array inside the library's device image and allocates nothing: it
+ * calls neither cudaMalloc/cudaFree nor any allocating library routine.
+ *   - Limit: NB = (O/b_o)*(I/b_i) <= BSP_MASK_STATIC_MAX_BLOCKS; a larger layer returns BSP_ERR_CAPACITY and
+ *     launches nothing.  The array (8 bytes per block, 512 KiB) is held on every GPU that loads the library,
+ *     for the life of the process.
+ *   - The first call on each device looks up the array's device address (with that device current) and
+ *     caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's scores; every entry that
+ *     is read is rewritten first, so no clearing is needed, but two calls that overlap on the GPU (different
+ *     streams, or the same layer masked concurrently) race on it.  Serialise them on one stream.
+ *   - There is no scores output and no latched status; arguments are otherwise those of bsp_mask().
+ * Errors: NULL, SHAPE, BLOCK, DTYPE, CAPACITY (n_zero out of range, or NB over the limit), CUDA. */
+#define BSP_MASK_STATIC_MAX_BLOCKS 65536
+bsp_status bsp_mask_static(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope,
+                           int64_t n_zero, uint8_t *gamma, void *stream);
+
 /* ---- Compaction (Section "Block Sparsity in a Matrix"; Section "Subvolumes, Data Compression ...") --
  * bsp_packed_bytes: size of the opaque `packed` buffer able to hold `nnz` stored blocks.
  * bsp_compact_nnz : counts the ones of a device Gamma and returns the count on the host; this one call
