@@ -23,7 +23,7 @@
  *    workspace and read back by bsp_check().
  *  - O and I must be multiples of b_o and b_i (Section "Experiments": a layer with fewer channels than a
  *    block, such as a 3-channel first layer, cannot be made block sparse) and, for the product kernels,
- *    multiples of 8.
+ *    multiples of 8 (I a multiple of 16 for int8, so that every row of X is a multiple of 16 bytes).
  */
 #ifndef BSP_H
 #define BSP_H

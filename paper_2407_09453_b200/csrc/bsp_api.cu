@@ -122,6 +122,7 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
         return BSP_ERR_SHAPE;
     if (xd->L + 2 * xd->pad_h < wd->H || xd->J + 2 * xd->pad_w < wd->K) return BSP_ERR_SHAPE;
     if (wd->O % 8 != 0 || wd->I % 8 != 0) return BSP_ERR_SHAPE;
+    if (wd->wtype == BSP_I8 && wd->I % 16 != 0) return BSP_ERR_SHAPE;   // rows of X must be 16-byte multiples
     if (wd->wtype == BSP_I8) { if (ytype != BSP_I32) return BSP_ERR_DTYPE; }
     else if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
     if (!aligned16(X) || !aligned16(Y) || !aligned16(w->packed)) return BSP_ERR_SHAPE;

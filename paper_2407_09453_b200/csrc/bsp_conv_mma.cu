@@ -1,58 +1,99 @@
-// Block-sparse implicit-GEMM convolution / FC product with fused bias on warp-level tensor-core MMAs.
-// Introduction (Y = W*X + b) and Section "Block Sparsity in a Matrix" of the paper: only stored 8x8 tiles of
-// W-bar are read and multiplied.
+// Block-sparse implicit-GEMM convolution / FC product with fused bias: TMA-fed, warp-specialised, warp-level
+// tensor-core MMAs.  Introduction (Y = W*X + b) and Section "Block Sparsity in a Matrix" of the paper: only
+// stored 8x8 tiles of W-bar are read and multiplied.
 //
 // Orientation: output pixels are the MMA M dimension, the 8 output channels of a tile row are N, input
 // channels (times taps) are K.  A CTA owns a tile of output pixels (nb images x th rows x tw columns) and
-// WN panels of 64 output channels; warp (wm, wn) accumulates 64 pixels x 64 channels in registers.
-// The input patch of the pixel tile is staged in shared memory in chunks of GC tile columns (8 channels
-// each) through a 3-stage cp.async ring, laid out [tile column][patch pixel][8 channels], so that a tap is
-// a constant byte offset and out-of-image pixels are zero filled once.  For every tile column the warp reads
-// the byte mask of stored tiles of its panel, loads the activation fragments once per K-step and issues MMAs
-// only for the tile rows whose mask bit is set; the branch is uniform across the warp.
+// WN panels of 64 output channels; consumer warp (wm, wn) accumulates 64 pixels x 64 channels in registers.
+//
+// One producer warp feeds two rings of shared-memory stages.  An activation stage holds a 128-byte slab of
+// channels (64 bf16, 128 int8 or 32 fp32 channels) of the input patch of the pixel tile: one tiled TMA load
+// with 128-byte swizzle, whose out-of-bounds fill supplies the zero padding; rows are patch pixels, so a tap
+// is a constant row offset and the swizzle keeps the 8-row fragment loads free of bank conflicts.  A weight
+// stage holds, for each of the CTA's panels, the stored tiles of GCW tile columns (8 input channels each),
+// which are one contiguous stretch of the packed payload and arrive by one bulk copy.  Loads complete on
+// "full" mbarriers; consumer warps release stages through "empty" mbarriers.  The panels' tile masks and
+// offsets are copied to shared memory once.  For every tile column a consumer warp loads the activation fragments once
+// per K-step and issues MMAs only for the tile rows whose mask bit is set (a warp-uniform branch).
+// Every mbarrier wait is bounded: on expiry the warp latches BSP_ERR_TIMEOUT in the workspace and leaves.
+#include <cuda.h>
 #include "bsp_internal.cuh"
 
 namespace bsp {
 namespace {
 
-constexpr int kStages = 3;
 constexpr int kMaxTaps = 128;
-constexpr int kMT = 4;                 // 16-pixel MMA tiles per warp
-constexpr int kMaxSmem = 200 * 1024;   // dynamic shared memory ceiling of a launch
+constexpr int kMT = 4;                    // 16-pixel MMA tiles per consumer warp
+constexpr int kMaxSmem = 200 * 1024;      // ceiling of the carved-up shared memory of a launch (+1 KB slack)
 constexpr int kMaxDevices = 64;
+constexpr int kMaxWStages = 8;            // weight ring depth
+constexpr int kMaxAStages = 3;            // activation ring depth
+constexpr int kWStageBudget = 16 * 1024;  // target bytes of one weight stage
+constexpr int kSlabBytes = 128;           // channel bytes per activation slab row (the TMA swizzle span)
+constexpr int kEpiBytes = 16 * (kPanelCh * 4 + 16);   // per-warp epilogue staging: 16 pixels x 64 channels
+constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait: try_wait attempts before giving up
 
 struct ConvParams {
-    const uint8_t *X;
+    CUtensorMap tmap;   // activations: (channel group bytes, x, y, n, group)
     uint8_t *Y;
     const void *bias;
     const uint8_t *colmask;
     const uint32_t *coloff;
     const uint32_t *panel_base;
     const uint8_t *payload;
+    int *status;
     int N, L, J, I, O, M, Nw, H, K, sh, sw, ph, pw;
     int nb, th, tw, PH, PW, patch_pix, tile_pix;
     int tiles_x, tiles_y;
-    int n_cols, n_panels, tile_bytes, GC, n_chunks, stage_bytes;
+    int n_cols, n_panels, tile_bytes;
+    int slab_cols, n_slabs, a_stages, a_stage_bytes, a_box_bytes;   // activation ring
+    int GCW, w_stages, w_stage_bytes, wseg_cap;                     // weight ring: wseg_cap bytes per panel
+    int meta_bytes, a_ring_off, w_ring_off, epi_off;                // byte offsets in dynamic shared memory
     int ytype;
 };
 
+// CB: bytes of one tile column (8 channels) inside a 128-byte slab row.
 template <int DT> struct Traits;
-template <> struct Traits<BSP_BF16> { static constexpr int CH = 16; using acc_t = float; };
-template <> struct Traits<BSP_I8> { static constexpr int CH = 8; using acc_t = int; };
-template <> struct Traits<BSP_F32> { static constexpr int CH = 32; using acc_t = float; };
+template <> struct Traits<BSP_BF16> { static constexpr int CB = 16; using acc_t = float; };
+template <> struct Traits<BSP_I8> { static constexpr int CB = 8; using acc_t = int; };
+template <> struct Traits<BSP_F32> { static constexpr int CB = 32; using acc_t = float; };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void cp_async(uint32_t dst, const void *src, int bytes, bool valid)
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    const int sz = valid ? bytes : 0;
-    if (bytes == 16)
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-    else
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+// Waits for the phase with the given parity; false if the bounded spin ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4])
 {
@@ -67,6 +108,12 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
 
@@ -99,33 +146,47 @@ __device__ __forceinline__ uint32_t to_tf32(uint32_t fbits)
     return r;
 }
 
-// Byte offset, inside one tile column of the staged patch, of the top-left input pixel of output pixel q of
-// the CTA's tile (q counts images, then rows, then columns of the tile).  Pixels past the tile map to 0.
-template <int CH>
-__device__ __forceinline__ int patch_offset(const ConvParams &p, int q)
+// Row, in the staged patch, of the top-left input pixel of output pixel q of the CTA's tile (q counts images,
+// then rows, then columns of the tile).  Pixels past the tile map to row 0.
+__device__ __forceinline__ int patch_row(const ConvParams &p, int q)
 {
     if (q >= p.tile_pix) return 0;
     const int ix = q % p.tw;
     const int t = q / p.tw;
     const int iy = t % p.th;
     const int in = t / p.th;
-    return ((in * p.PH + iy * p.sh) * p.PW + ix * p.sw) * CH;
+    return (in * p.PH + iy * p.sh) * p.PW + ix * p.sw;
 }
 
+// Shared-memory address of 16-byte chunk `chunk` of patch row `row` in a 128-byte-swizzled slab stage
+// (1024-byte aligned): the chunk index is XORed with the row index modulo 8.
+__device__ __forceinline__ uint32_t slab_addr(uint32_t stage, int row, int chunk)
+{
+    return stage + (uint32_t)row * kSlabBytes + (uint32_t)((chunk ^ (row & 7)) << 4);
+}
+
+// Threads: WM*WN consumer warps, then one producer warp.
 template <int DT, int WM, int WN>
-__global__ void __launch_bounds__(32 * WM * WN, 1)
+__global__ void __launch_bounds__(32 * (WM * WN + 1), 1)
 conv_mma_kernel(const __grid_constant__ ConvParams p)
 {
     using T = Traits<DT>;
     using acc_t = typename T::acc_t;
-    constexpr int CH = T::CH;
-    constexpr int NT = 32 * WM * WN;
-    extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ int s_tapoff[kMaxTaps];
+    constexpr int CB = T::CB;
+    constexpr int NCW = WM * WN;                 // consumer warps
+    constexpr int NT = 32 * (NCW + 1);
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    // the swizzled activation stages need 1024-byte alignment; the launch reserves the slack
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ int s_taprow[kMaxTaps];           // patch-row offset of every tap
+    __shared__ __align__(8) uint64_t s_afull[kMaxAStages];
+    __shared__ __align__(8) uint64_t s_aempty[kMaxAStages];
+    __shared__ __align__(8) uint64_t s_wfull[kMaxWStages];
+    __shared__ __align__(8) uint64_t s_wempty[kMaxWStages];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wm = warp % WM, wn = warp / WM;
     const int HK = p.H * p.K;
+    const int SA = p.a_stages, SW = p.w_stages;
 
     // tile origin
     int tix = blockIdx.x;
@@ -133,57 +194,101 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
     const int ty = tix % p.tiles_y;
     const int tn = tix / p.tiles_y;
     const int n0 = tn * p.nb, y0 = ty * p.th, x0 = tx * p.tw;
-    const int gy0 = y0 * p.sh - p.ph, gx0 = x0 * p.sw - p.pw;
 
     for (int t = tid; t < kMaxTaps; t += NT) {
         const int tt = t < HK ? t : HK - 1;
-        s_tapoff[t] = ((tt / p.K) * p.PW + (tt % p.K)) * CH;
+        s_taprow[t] = (tt / p.K) * p.PW + (tt % p.K);
     }
+    // tile offsets (with an end sentinel) and masks of the CTA's panels -> shared memory
+    uint32_t *s_coloff = (uint32_t *)smem;                                   // [WN][n_cols + 1]
+    uint8_t *s_mask = smem + (size_t)WN * (p.n_cols + 1) * 4;                // [WN][n_cols]
+    for (int i = tid; i < WN * (p.n_cols + 1); i += NT) {
+        const int pn = i / (p.n_cols + 1), col = i % (p.n_cols + 1);
+        const int pg = blockIdx.y * WN + pn;
+        uint32_t v = 0;
+        if (pg < p.n_panels)
+            v = (col < p.n_cols) ? p.coloff[(size_t)pg * p.n_cols + col] : p.panel_base[pg + 1] - p.panel_base[pg];
+        s_coloff[i] = v;
+    }
+    for (int i = tid; i < WN * p.n_cols; i += NT) {
+        const int pg = blockIdx.y * WN + i / p.n_cols;
+        s_mask[i] = (pg < p.n_panels) ? p.colmask[(size_t)pg * p.n_cols + i % p.n_cols] : (uint8_t)0;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < SA; ++s) {
+            mbar_init(smem_u32(&s_afull[s]), 1);
+            mbar_init(smem_u32(&s_aempty[s]), NCW);
+        }
+        for (int s = 0; s < SW; ++s) {
+            mbar_init(smem_u32(&s_wfull[s]), 1);
+            mbar_init(smem_u32(&s_wempty[s]), NCW);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncthreads();
 
-    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t a_ring = smem_u32(smem) + p.a_ring_off;
+    const uint32_t w_ring = smem_u32(smem) + p.w_ring_off;
 
-    // ---- loader: one chunk of GC tile columns of the patch into a stage
-    auto load_chunk = [&](int c, int stage) {
-        if (c < p.n_chunks) {
-            const int col0 = c * p.GC;
-            const int ncol = min(p.GC, p.n_cols - col0);
-            const uint32_t sbase = smem_base + stage * p.stage_bytes;
-            for (int pp = tid; pp < p.patch_pix; pp += NT) {
-                const int px = pp % p.PW;
-                const int t = pp / p.PW;
-                const int py = t % p.PH;
-                const int in = t / p.PH;
-                const int n = n0 + in, gy = gy0 + py, gx = gx0 + px;
-                const bool valid = (n < p.N) && (gy >= 0) && (gy < p.L) && (gx >= 0) && (gx < p.J);
-                const uint8_t *src = p.X;
-                if (valid) src += ((((size_t)n * p.L + gy) * p.J + gx) * p.I) * (CH / 8) + (size_t)col0 * CH;
-                uint32_t dst = sbase + pp * CH;
-                for (int v = 0; v < ncol; ++v) {
-                    if constexpr (CH == 32) {
-                        cp_async(dst, src, 16, valid);
-                        cp_async(dst + 16, src + (valid ? 16 : 0), 16, valid);
-                    } else {
-                        cp_async(dst, src, CH, valid);
+    if (warp == NCW) {
+        // ================= producer warp: one lane issues every copy =================
+        if (lane == 0) {
+            const int gx0 = x0 * p.sw - p.pw, gy0 = y0 * p.sh - p.ph;
+            bool ok = true;
+            auto issue_act = [&](int s) {
+                if (s >= p.n_slabs || !ok) return;
+                const int sa = s % SA;
+                if (s >= SA && !mbar_wait(smem_u32(&s_aempty[sa]), (uint32_t)((s / SA - 1) & 1))) { ok = false; return; }
+                const uint32_t bar = smem_u32(&s_afull[sa]);
+                mbar_expect_tx(bar, (uint32_t)p.a_box_bytes);
+                tma_load_4d(a_ring + sa * p.a_stage_bytes, &p.tmap, bar, s * kSlabBytes, gx0, gy0, n0);
+            };
+            issue_act(0);
+            int wc = 0;
+            for (int s = 0; s < p.n_slabs && ok; ++s) {
+                issue_act(s + 1);
+                const int slab_end = min(p.n_cols, (s + 1) * p.slab_cols);
+                for (int col0 = s * p.slab_cols; col0 < slab_end && ok; col0 += p.GCW, ++wc) {
+                    const int sw = wc % SW;
+                    if (wc >= SW && !mbar_wait(smem_u32(&s_wempty[sw]), (uint32_t)((wc / SW - 1) & 1))) { ok = false; break; }
+                    const int ncol = min(p.GCW, slab_end - col0);
+                    const uint32_t bar = smem_u32(&s_wfull[sw]);
+                    uint32_t tx_bytes = 0;
+                    for (int pn = 0; pn < WN; ++pn)
+                        tx_bytes += (s_coloff[pn * (p.n_cols + 1) + col0 + ncol] - s_coloff[pn * (p.n_cols + 1) + col0]) *
+                                    (uint32_t)p.tile_bytes;
+                    mbar_expect_tx(bar, tx_bytes);
+                    for (int pn = 0; pn < WN; ++pn) {
+                        const int pg = blockIdx.y * WN + pn;
+                        if (pg >= p.n_panels) break;
+                        const uint32_t first = s_coloff[pn * (p.n_cols + 1) + col0];
+                        const uint32_t bytes = (s_coloff[pn * (p.n_cols + 1) + col0 + ncol] - first) * (uint32_t)p.tile_bytes;
+                        if (bytes)
+                            bulk_load(w_ring + sw * p.w_stage_bytes + pn * p.wseg_cap,
+                                      p.payload + (size_t)(p.panel_base[pg] + first) * p.tile_bytes, bytes, bar);
                     }
-                    if (valid) src += CH;
-                    dst += p.patch_pix * CH;
                 }
             }
+            if (!ok) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
         }
-        cp_async_commit();
-    };
+        return;
+    }
 
-    // ---- per-thread fragment addressing
-    int rowoff[kMT][2];
+    // ================= consumer warps =================
+    const int wm = warp % WM, wn = warp / WM;
+    const int panel = blockIdx.y * WN + wn;
+    const bool active = panel < p.n_panels;
+
+    int rowpix[kMT][2];
 #pragma unroll
     for (int i = 0; i < kMT; ++i) {
         const int qbase = (wm * kMT + i) * 16;
         if constexpr (DT == BSP_BF16) {
-            rowoff[i][0] = patch_offset<CH>(p, qbase + (lane & 15));
-            rowoff[i][1] = 0;
+            rowpix[i][0] = patch_row(p, qbase + (lane & 15));
+            rowpix[i][1] = 0;
         } else {
-            rowoff[i][0] = patch_offset<CH>(p, qbase + (lane >> 2));
-            rowoff[i][1] = patch_offset<CH>(p, qbase + (lane >> 2) + 8);
+            rowpix[i][0] = patch_row(p, qbase + (lane >> 2));
+            rowpix[i][1] = patch_row(p, qbase + (lane >> 2) + 8);
         }
     }
 
@@ -195,200 +300,202 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[i][r][e] = 0;
 
-    const int panel = blockIdx.y * WN + wn;
-    const bool active = panel < p.n_panels;
-    const uint32_t pbase = active ? p.panel_base[panel] : 0u;
-    const uint8_t *cm = p.colmask + (size_t)(active ? panel : 0) * p.n_cols;
-    const uint32_t *co = p.coloff + (size_t)(active ? panel : 0) * p.n_cols;
+    const uint32_t *my_off = s_coloff + wn * (p.n_cols + 1);
+    const uint8_t *my_mask = s_mask + wn * p.n_cols;
+    bool ok = true;
+    int wc = 0;
 
-    // prefetch of the masks/offsets of one chunk: lane v holds tile column chunk*GC + v
-    auto fetch_meta = [&](int c, uint32_t &m, uint32_t &o) {
-        const int col = c * p.GC + lane;
-        m = 0; o = 0;
-        if (active && c < p.n_chunks && lane < p.GC && col < p.n_cols) { m = cm[col]; o = co[col]; }
-    };
+    for (int s = 0; s < p.n_slabs && ok; ++s) {
+        const int sa = s % SA;
+        if (!mbar_wait(smem_u32(&s_afull[sa]), (uint32_t)((s / SA) & 1))) { ok = false; break; }
+        const uint32_t a_stage = a_ring + sa * p.a_stage_bytes;
+        const int slab_col0 = s * p.slab_cols;
+        const int slab_end = min(p.n_cols, slab_col0 + p.slab_cols);
+        for (int col0 = slab_col0; col0 < slab_end; col0 += p.GCW, ++wc) {
+            const int sw = wc % SW;
+            if (!mbar_wait(smem_u32(&s_wfull[sw]), (uint32_t)((wc / SW) & 1))) { ok = false; break; }
+            const int ncol = min(p.GCW, slab_end - col0);
+            const uint32_t wseg = w_ring + sw * p.w_stage_bytes + wn * p.wseg_cap;
+            const uint32_t off0 = my_off[col0];
+            for (int v = 0; active && v < ncol; ++v) {
+                const uint32_t m = my_mask[col0 + v];
+                if (m == 0) continue;
+                const uint32_t wt = wseg + (my_off[col0 + v] - off0) * p.tile_bytes;
+                const int cbyte = (col0 + v - slab_col0) * CB;     // byte of the tile column inside a slab row
+                const int chunk = cbyte >> 4;
 
+                if constexpr (DT == BSP_BF16) {
+                    const int n16 = HK >> 1;
+                    const int sel = lane >> 4;
+                    for (int st = 0; st < n16; ++st) {
+                        uint32_t a[kMT][4];
+                        const int trow = s_taprow[2 * st + sel];
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) load_chunk(s, s);
-    uint32_t meta_m, meta_o;
-    fetch_meta(0, meta_m, meta_o);
-
-    for (int c = 0; c < p.n_chunks; ++c) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
-        load_chunk(c + kStages - 1, (c + kStages - 1) % kStages);
-        const uint32_t cur_m = meta_m, cur_o = meta_o;
-        fetch_meta(c + 1, meta_m, meta_o);
-        if (!active) continue;
-        const uint32_t stage_addr = smem_base + (c % kStages) * p.stage_bytes;
-        const int ncol = min(p.GC, p.n_cols - c * p.GC);
-        for (int v = 0; v < ncol; ++v) {
-            const uint32_t m = __shfl_sync(0xFFFFFFFFu, cur_m, v);
-            if (m == 0) continue;
-            const uint32_t off = __shfl_sync(0xFFFFFFFFu, cur_o, v);
-            const uint8_t *wt = p.payload + (size_t)(pbase + off) * p.tile_bytes;
-            const uint32_t abase = stage_addr + v * p.patch_pix * CH;
-
-            if constexpr (DT == BSP_BF16) {
-                const int n16 = HK >> 1;
-                const int sel = lane >> 4;
-                for (int s = 0; s < n16; ++s) {
-                    uint32_t a[kMT][4];
-                    const int toff = s_tapoff[2 * s + sel];
+                        for (int i = 0; i < kMT; ++i) ldmatrix_x4(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[i]);
+                        uint32_t wp = wt + st * 256 + lane * 8;
 #pragma unroll
-                    for (int i = 0; i < kMT; ++i) ldmatrix_x4(abase + rowoff[i][0] + toff, a[i]);
-                    const uint8_t *wp = wt + s * 256 + lane * 8;
+                        for (int r = 0; r < kPanelRows; ++r) {
+                            if (m & (1u << r)) {
+                                const uint2 b = lds64(wp);
+                                wp += p.tile_bytes;
 #pragma unroll
-                    for (int r = 0; r < kPanelRows; ++r) {
-                        if (m & (1u << r)) {
-                            const uint2 b = __ldg((const uint2 *)wp);
-                            wp += p.tile_bytes;
-#pragma unroll
-                            for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][r], a[i], b.x, b.y);
+                                for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][r], a[i], b.x, b.y);
+                            }
                         }
                     }
-                }
-                if (HK & 1) {
-                    uint32_t a[kMT][4];
-                    const int toff = s_tapoff[HK - 1];
+                    if (HK & 1) {
+                        uint32_t a[kMT][4];
+                        const int trow = s_taprow[HK - 1];
 #pragma unroll
-                    for (int i = 0; i < kMT; ++i) ldmatrix_x2(abase + rowoff[i][0] + toff, a[i]);
-                    const uint8_t *wp = wt + n16 * 256 + lane * 4;
+                        for (int i = 0; i < kMT; ++i) ldmatrix_x2(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[i]);
+                        uint32_t wp = wt + n16 * 256 + lane * 4;
 #pragma unroll
-                    for (int r = 0; r < kPanelRows; ++r) {
-                        if (m & (1u << r)) {
-                            const uint32_t b = __ldg((const uint32_t *)wp);
-                            wp += p.tile_bytes;
+                        for (int r = 0; r < kPanelRows; ++r) {
+                            if (m & (1u << r)) {
+                                const uint32_t b = lds32(wp);
+                                wp += p.tile_bytes;
 #pragma unroll
-                            for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][r], a[i], b);
+                                for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][r], a[i], b);
+                            }
                         }
                     }
-                }
-            } else if constexpr (DT == BSP_I8) {
-                const int nsteps = (HK + 1) >> 1;
-                const int t = lane & 3;
-                for (int s = 0; s < nsteps; ++s) {
-                    uint32_t a[kMT][4];
-                    const int toff = s_tapoff[2 * s + (t >> 1)] + (t & 1) * 4;
+                } else if constexpr (DT == BSP_I8) {
+                    const int nsteps = (HK + 1) >> 1;
+                    const int t = lane & 3;
+                    const int within = (cbyte & 15) + (t & 1) * 4;
+                    for (int st = 0; st < nsteps; ++st) {
+                        uint32_t a[kMT][4];
+                        const int trow = s_taprow[2 * st + (t >> 1)];
 #pragma unroll
-                    for (int i = 0; i < kMT; ++i) {
-                        a[i][0] = lds32(abase + rowoff[i][0] + toff);
-                        a[i][1] = lds32(abase + rowoff[i][1] + toff);
-                    }
-                    const uint8_t *wp = wt + s * 128 + lane * 4;
+                        for (int i = 0; i < kMT; ++i) {
+                            a[i][0] = lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk) + within);
+                            a[i][1] = lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk) + within);
+                        }
+                        uint32_t wp = wt + st * 128 + lane * 4;
 #pragma unroll
-                    for (int r = 0; r < kPanelRows; ++r) {
-                        if (m & (1u << r)) {
-                            const uint32_t b = __ldg((const uint32_t *)wp);
-                            wp += p.tile_bytes;
+                        for (int r = 0; r < kPanelRows; ++r) {
+                            if (m & (1u << r)) {
+                                const uint32_t b = lds32(wp);
+                                wp += p.tile_bytes;
 #pragma unroll
-                            for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][r], a[i], b);
+                                for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][r], a[i], b);
+                            }
                         }
                     }
-                }
-            } else {
-                const int t = lane & 3;
-                for (int s = 0; s < HK; ++s) {
-                    uint32_t a[kMT][4];
-                    const int toff = s_tapoff[s] + t * 4;
+                } else {
+                    const int t = lane & 3;
+                    for (int st = 0; st < HK; ++st) {
+                        uint32_t a[kMT][4];
+                        const int trow = s_taprow[st];
 #pragma unroll
-                    for (int i = 0; i < kMT; ++i) {
-                        a[i][0] = to_tf32(lds32(abase + rowoff[i][0] + toff));
-                        a[i][1] = to_tf32(lds32(abase + rowoff[i][1] + toff));
-                        a[i][2] = to_tf32(lds32(abase + rowoff[i][0] + toff + 16));
-                        a[i][3] = to_tf32(lds32(abase + rowoff[i][1] + toff + 16));
-                    }
-                    const uint8_t *wp = wt + s * 256 + lane * 8;
+                        for (int i = 0; i < kMT; ++i) {
+                            a[i][0] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk) + t * 4));
+                            a[i][1] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk) + t * 4));
+                            a[i][2] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk + 1) + t * 4));
+                            a[i][3] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk + 1) + t * 4));
+                        }
+                        uint32_t wp = wt + st * 256 + lane * 8;
 #pragma unroll
-                    for (int r = 0; r < kPanelRows; ++r) {
-                        if (m & (1u << r)) {
-                            const uint2 b = __ldg((const uint2 *)wp);
-                            wp += p.tile_bytes;
+                        for (int r = 0; r < kPanelRows; ++r) {
+                            if (m & (1u << r)) {
+                                const uint2 b = lds64(wp);
+                                wp += p.tile_bytes;
 #pragma unroll
-                            for (int i = 0; i < kMT; ++i) mma_tf32_k8(acc[i][r], a[i], to_tf32(b.x), to_tf32(b.y));
+                                for (int i = 0; i < kMT; ++i) mma_tf32_k8(acc[i][r], a[i], to_tf32(b.x), to_tf32(b.y));
+                            }
                         }
                     }
                 }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_wempty[sw]));
         }
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(smem_u32(&s_aempty[sa]));
     }
+    if (!ok) {
+        if (lane == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
+        return;
+    }
+    if (!active) return;
 
     // ---- epilogue: + bias, convert, stage 16 pixels x 64 channels per warp in shared memory, store rows
-    cp_async_wait<0>();
-    __syncthreads();
     const int oe = (p.ytype == BSP_BF16) ? 2 : 4;               // bytes per output element
     const int pitch = kPanelCh * oe + 16;
-    uint8_t *ebuf = smem + warp * (16 * (kPanelCh * 4 + 16));
-    if (active) {
-        const int g = lane >> 2, t = lane & 3;
-        const int ch0 = panel * kPanelCh;
-        acc_t bv[kPanelRows][2];
+    uint8_t *ebuf = smem + p.epi_off + warp * kEpiBytes;
+    const int g = lane >> 2, t = lane & 3;
+    const int ch0 = panel * kPanelCh;
+    acc_t bv[kPanelRows][2];
+#pragma unroll
+    for (int r = 0; r < kPanelRows; ++r) {
+        const int o = ch0 + r * 8 + 2 * t;
+        bv[r][0] = 0; bv[r][1] = 0;
+        if (p.bias != nullptr && o < p.O) {
+            bv[r][0] = ((const acc_t *)p.bias)[o];
+            bv[r][1] = ((const acc_t *)p.bias)[o + 1];
+        }
+    }
+    const int cpr = kPanelCh * oe / 16;                      // 16-byte chunks per pixel row
+#pragma unroll
+    for (int i = 0; i < kMT; ++i) {
 #pragma unroll
         for (int r = 0; r < kPanelRows; ++r) {
-            const int o = ch0 + r * 8 + 2 * t;
-            bv[r][0] = 0; bv[r][1] = 0;
-            if (p.bias != nullptr && o < p.O) {
-                bv[r][0] = ((const acc_t *)p.bias)[o];
-                bv[r][1] = ((const acc_t *)p.bias)[o + 1];
-            }
-        }
-        const int cpr = kPanelCh * oe / 16;                      // 16-byte chunks per pixel row
 #pragma unroll
-        for (int i = 0; i < kMT; ++i) {
-#pragma unroll
-            for (int r = 0; r < kPanelRows; ++r) {
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const acc_t v0 = acc[i][r][2 * hh] + bv[r][0];
-                    const acc_t v1 = acc[i][r][2 * hh + 1] + bv[r][1];
-                    uint8_t *dst = ebuf + (g + 8 * hh) * pitch + (r * 8 + 2 * t) * oe;
-                    if constexpr (DT == BSP_I8) {
-                        *(int2 *)dst = make_int2(v0, v1);
-                    } else {
-                        if (oe == 2) *(__nv_bfloat162 *)dst = __floats2bfloat162_rn(v0, v1);
-                        else *(float2 *)dst = make_float2(v0, v1);
-                    }
+            for (int hh = 0; hh < 2; ++hh) {
+                const acc_t v0 = acc[i][r][2 * hh] + bv[r][0];
+                const acc_t v1 = acc[i][r][2 * hh + 1] + bv[r][1];
+                uint8_t *dst = ebuf + (g + 8 * hh) * pitch + (r * 8 + 2 * t) * oe;
+                if constexpr (DT == BSP_I8) {
+                    *(int2 *)dst = make_int2(v0, v1);
+                } else {
+                    if (oe == 2) *(__nv_bfloat162 *)dst = __floats2bfloat162_rn(v0, v1);
+                    else *(float2 *)dst = make_float2(v0, v1);
                 }
             }
-            __syncwarp();
-            for (int idx = lane; idx < 16 * cpr; idx += 32) {
-                const int row = idx / cpr, chunk = idx % cpr;
-                const int q = (wm * kMT + i) * 16 + row;
-                const int o = ch0 + chunk * (16 / oe);
-                if (q < p.tile_pix && o < p.O) {
-                    const int ix = q % p.tw;
-                    const int tq = q / p.tw;
-                    const int iy = tq % p.th;
-                    const int in = tq / p.th;
-                    const int n = n0 + in, y = y0 + iy, x = x0 + ix;
-                    if (n < p.N && y < p.M && x < p.Nw) {
-                        const size_t pix = ((size_t)n * p.M + y) * p.Nw + x;
-                        *(uint4 *)(p.Y + (pix * p.O + o) * oe) = *(const uint4 *)(ebuf + row * pitch + chunk * 16);
-                    }
+        }
+        __syncwarp();
+        for (int idx = lane; idx < 16 * cpr; idx += 32) {
+            const int row = idx / cpr, chunk = idx % cpr;
+            const int q = (wm * kMT + i) * 16 + row;
+            const int o = ch0 + chunk * (16 / oe);
+            if (q < p.tile_pix && o < p.O) {
+                const int ix = q % p.tw;
+                const int tq = q / p.tw;
+                const int iy = tq % p.th;
+                const int in = tq / p.th;
+                const int n = n0 + in, y = y0 + iy, x = x0 + ix;
+                if (n < p.N && y < p.M && x < p.Nw) {
+                    const size_t pix = ((size_t)n * p.M + y) * p.Nw + x;
+                    *(uint4 *)(p.Y + (pix * p.O + o) * oe) = *(const uint4 *)(ebuf + row * pitch + chunk * 16);
                 }
             }
-            __syncwarp();
         }
+        __syncwarp();
     }
 }
 
 struct Plan {
-    int WM, WN, nb, th, tw, GC;
-    size_t smem;
+    int WM, WN, nb, th, tw;
+    int slab_cols, n_slabs, a_stages, GCW, w_stages;
+    size_t smem, a_stage_bytes, a_box_bytes, w_stage_bytes, wseg_cap, meta_bytes, a_ring_off, w_ring_off, epi_off;
     long long tiles, ctas;
 };
 
 constexpr int kConfigs[][2] = {{2, 2}, {4, 2}, {2, 4}, {4, 1}, {8, 1}, {1, 4}};
 
-void best_tile(int tpix, int N, int M, int Nw, int &nb, int &th, int &tw, long long &tiles)
+// Output-pixel tile (nb images x th x tw) of at most tpix pixels that needs the fewest tiles; box extents of
+// the TMA load are limited to 256 per dimension.
+void best_tile(int tpix, int N, int M, int Nw, int sh, int sw, int H, int K, int &nb, int &th, int &tw,
+               long long &tiles)
 {
-    long long best = -1;
-    long long best_area = 0;
+    long long best = -1, best_area = 0;
     for (int w = 1; w <= Nw && w <= tpix; ++w) {
+        if ((w - 1) * sw + K > 256) break;
         const int hmax = tpix / w < M ? tpix / w : M;
         for (int h = 1; h <= hmax; ++h) {
+            if ((h - 1) * sh + H > 256) break;
             int b = 1;
-            if (h == M && w == Nw) { b = tpix / (h * w); if (b > N) b = N; if (b < 1) b = 1; }
+            if (h == M && w == Nw) { b = tpix / (h * w); if (b > N) b = N; if (b > 256) b = 256; if (b < 1) b = 1; }
             const long long cnt = (long long)((N + b - 1) / b) * ((M + h - 1) / h) * ((Nw + w - 1) / w);
             const long long area = (long long)b * h * w;
             if (best < 0 || cnt < best || (cnt == best && area < best_area)) {
@@ -401,51 +508,91 @@ void best_tile(int tpix, int N, int M, int Nw, int &nb, int &th, int &tw, long l
 
 Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_panels, int n_cols)
 {
-    const int CH = 8 * elem_bytes(wd.wtype);
+    const int CB = 8 * elem_bytes(wd.wtype);
+    const int tile_bytes = tile_bytes_of(wd.wtype, wd.H * wd.K);
     Plan best = {};
     double best_cost = -1;
+    // Each warp layout is tried with its full pixel tile first; if the patch does not fit in shared memory
+    // (large strides or kernels) the tile is halved, leaving some MMA rows idle.
+    for (int shrink = 1; shrink <= 16 && best_cost < 0; shrink *= 2)
     for (auto &cfg : kConfigs) {
         Plan pl = {};
         pl.WM = cfg[0]; pl.WN = cfg[1];
-        best_tile(pl.WM * 64, xd.N, M, Nw, pl.nb, pl.th, pl.tw, pl.tiles);
+        pl.tiles = -1;
+        if (pl.WM * 64 / shrink < 8) continue;
+        best_tile(pl.WM * 64 / shrink, xd.N, M, Nw, xd.stride_h, xd.stride_w, wd.H, wd.K, pl.nb, pl.th, pl.tw, pl.tiles);
+        if (pl.tiles < 0) continue;
         const int PH = (pl.th - 1) * xd.stride_h + wd.H, PW = (pl.tw - 1) * xd.stride_w + wd.K;
         const long long patch_pix = (long long)pl.nb * PH * PW;
-        int GC = (int)(32768 / (patch_pix * CH));
-        if (GC > 32) GC = 32;
-        if (GC > n_cols) GC = n_cols;
-        if (GC < 1) GC = 1;
-        pl.GC = GC;
-        const size_t stage = align_up((size_t)GC * patch_pix * CH, 128);
-        const size_t epi = (size_t)pl.WM * pl.WN * 16 * (kPanelCh * 4 + 16);
-        pl.smem = stage * kStages > epi ? stage * kStages : epi;
-        if (pl.smem > (size_t)kMaxSmem) continue;
+        pl.slab_cols = kSlabBytes / CB;
+        pl.n_slabs = (n_cols + pl.slab_cols - 1) / pl.slab_cols;
+        pl.a_box_bytes = (size_t)patch_pix * kSlabBytes;
+        pl.a_stage_bytes = align_up(pl.a_box_bytes, 1024);
+        const long long per_col = (long long)pl.WN * kPanelRows * tile_bytes;
+        int GCW = (int)(kWStageBudget / per_col);
+        if (GCW > pl.slab_cols) GCW = pl.slab_cols;
+        if (GCW < 1) GCW = 1;
+        pl.GCW = GCW;
+        pl.wseg_cap = (size_t)GCW * kPanelRows * tile_bytes;
+        pl.w_stage_bytes = pl.WN * pl.wseg_cap;
+        pl.meta_bytes = align_up((size_t)pl.WN * (n_cols + 1) * 4 + (size_t)pl.WN * n_cols, 1024);
+        const size_t epi = (size_t)pl.WM * pl.WN * kEpiBytes;
+        const size_t fixed = pl.meta_bytes + epi;
+        // at least two stages in each ring; then grow the activation ring to 3 and the weight ring as far as it goes
+        if (fixed + 2 * pl.a_stage_bytes + 2 * pl.w_stage_bytes > (size_t)kMaxSmem) continue;
+        pl.a_stages = (fixed + 3 * pl.a_stage_bytes + 3 * pl.w_stage_bytes <= (size_t)kMaxSmem) ? 3 : 2;
+        if (pl.a_stages > pl.n_slabs) pl.a_stages = pl.n_slabs < 2 ? 2 : pl.n_slabs;
+        int ws = (int)(((size_t)kMaxSmem - fixed - pl.a_stages * pl.a_stage_bytes) / pl.w_stage_bytes);
+        if (ws > kMaxWStages) ws = kMaxWStages;
+        pl.w_stages = ws;
+        pl.a_ring_off = pl.meta_bytes;
+        pl.w_ring_off = pl.a_ring_off + pl.a_stages * pl.a_stage_bytes;
+        pl.epi_off = pl.w_ring_off + pl.w_stages * pl.w_stage_bytes;
+        pl.smem = pl.epi_off + epi + 1024;                  // + slack for aligning the base to 1024 bytes
         pl.ctas = pl.tiles * ((n_panels + pl.WN - 1) / pl.WN);
         const int warps = pl.WM * pl.WN;
         // busiest SM: CTAs dealt round-robin over 148 SMs, each CTA keeping `warps` warps busy
         const double load = (double)((pl.ctas + 147) / 148) * warps;
-        const double traffic = (double)pl.ctas * patch_pix * n_cols * CH + (double)pl.tiles * n_panels * 1.0;
+        const double traffic = (double)pl.ctas * patch_pix * n_cols * CB +
+                               (double)pl.tiles * n_panels * n_cols * kPanelRows * tile_bytes * 0.5;
         const double cost = load * 1e15 + traffic;
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = pl; }
     }
     return best;
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
 template <int DT, int WM, int WN>
 bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
 {
     auto kern = conv_mma_kernel<DT, WM, WN>;
-    // opt in to large dynamic shared memory once per device and instantiation (static shared memory counts
-    // against the default 48 KB, so the opt-in is unconditional)
+    // opt in to large dynamic shared memory once per device and instantiation
     static bool opted[kMaxDevices] = {};
     int dev = 0;
     BSP_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return BSP_ERR_CUDA;
     if (!opted[dev]) {
-        BSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem + 1024));
         opted[dev] = true;
     }
     dim3 grid((unsigned)pl.tiles, (unsigned)((p.n_panels + WN - 1) / WN));
-    kern<<<grid, 32 * WM * WN, pl.smem, st>>>(p);
+    kern<<<grid, 32 * (WM * WN + 1), pl.smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }
@@ -466,30 +613,48 @@ bsp_status launch_dt(const ConvParams &p, const Plan &pl, cudaStream_t st)
 bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
                        const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
 {
-    (void)ws;
     const PackedLayout L = packed_layout(wd, 0);
     const int M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1;
     const int Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
     const Plan pl = make_plan(wd, xd, M, Nw, L.n_panels, L.n_cols);
     if (pl.WM == 0) return BSP_ERR_SHAPE;
-    const int CH = 8 * elem_bytes(wd.wtype);
+    const int e = elem_bytes(wd.wtype);
     const uint8_t *pk = (const uint8_t *)packed;
     ConvParams p = {};
-    p.X = (const uint8_t *)X; p.Y = (uint8_t *)Y; p.bias = bias;
+    p.Y = (uint8_t *)Y; p.bias = bias;
     p.colmask = pk + L.off_colmask;
     p.coloff = (const uint32_t *)(pk + L.off_coloff);
     p.panel_base = (const uint32_t *)(pk + L.off_panelbase);
     p.payload = pk + L.off_payload;
+    p.status = (int *)ws;
     p.N = xd.N; p.L = xd.L; p.J = xd.J; p.I = wd.I; p.O = wd.O; p.M = M; p.Nw = Nw; p.H = wd.H; p.K = wd.K;
     p.sh = xd.stride_h; p.sw = xd.stride_w; p.ph = xd.pad_h; p.pw = xd.pad_w;
     p.nb = pl.nb; p.th = pl.th; p.tw = pl.tw;
     p.PH = (pl.th - 1) * xd.stride_h + wd.H; p.PW = (pl.tw - 1) * xd.stride_w + wd.K;
     p.patch_pix = pl.nb * p.PH * p.PW; p.tile_pix = pl.nb * pl.th * pl.tw;
     p.tiles_x = (Nw + pl.tw - 1) / pl.tw; p.tiles_y = (M + pl.th - 1) / pl.th;
-    p.n_cols = L.n_cols; p.n_panels = L.n_panels; p.tile_bytes = L.tile_bytes; p.GC = pl.GC;
-    p.n_chunks = (L.n_cols + pl.GC - 1) / pl.GC;
-    p.stage_bytes = (int)align_up((size_t)pl.GC * p.patch_pix * CH, 128);
+    p.n_cols = L.n_cols; p.n_panels = L.n_panels; p.tile_bytes = L.tile_bytes;
+    p.slab_cols = pl.slab_cols; p.n_slabs = pl.n_slabs; p.a_stages = pl.a_stages;
+    p.a_stage_bytes = (int)pl.a_stage_bytes; p.a_box_bytes = (int)pl.a_box_bytes;
+    p.GCW = pl.GCW; p.w_stages = pl.w_stages; p.w_stage_bytes = (int)pl.w_stage_bytes; p.wseg_cap = (int)pl.wseg_cap;
+    p.meta_bytes = (int)pl.meta_bytes; p.a_ring_off = (int)pl.a_ring_off; p.w_ring_off = (int)pl.w_ring_off;
+    p.epi_off = (int)pl.epi_off;
     p.ytype = ytype;
+
+    // Activations as a rank-4 byte tensor (channel bytes, x, y, n); a box is a 128-byte slab of channels of
+    // the tile's input patch, stored with the 128-byte swizzle.
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return BSP_ERR_CUDA;
+    const cuuint64_t row = (cuuint64_t)wd.I * e;
+    const cuuint64_t gdim[4] = {row, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N};
+    const cuuint64_t gstr[3] = {row, row * xd.J, row * xd.J * xd.L};
+    const cuuint32_t box[4] = {(cuuint32_t)kSlabBytes, (cuuint32_t)p.PW, (cuuint32_t)p.PH, (cuuint32_t)pl.nb};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(&p.tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(X), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return BSP_ERR_CUDA;
+
     if (wd.wtype == BSP_BF16) return launch_dt<BSP_BF16>(p, pl, st);
     if (wd.wtype == BSP_I8) return launch_dt<BSP_I8>(p, pl, st);
     return launch_dt<BSP_F32>(p, pl, st);
