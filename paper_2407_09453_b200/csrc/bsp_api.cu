@@ -129,7 +129,9 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
     // the packed header is on the device; the host checks what it can: capacity against the descriptor
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
-    return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
+    // the stored fraction only steers the choice of launch shape
+    const double density = NB > 0 ? (double)w->nnz / (double)NB : 1.0;
+    return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, density > 0.05 ? density : 0.05, ws, (cudaStream_t)stream);
 }
 
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,

@@ -13,17 +13,18 @@
 // stage holds, for each of the CTA's panels, the stored tiles of GCW tile columns (8 input channels each),
 // which are one contiguous stretch of the packed payload and arrive by one bulk copy.  Loads complete on
 // "full" mbarriers; consumer warps release stages through "empty" mbarriers.  The panels' tile masks and
-// offsets are copied to shared memory once.  For every tile column a consumer warp loads the activation fragments once
-// per K-step and issues MMAs only for the tile rows whose mask bit is set (a warp-uniform branch).
+// offsets are copied to shared memory once.  For every tile column a consumer warp loads the activation
+// fragments once per K-step and issues MMAs only for the tile rows present in the column's row mask: the mask
+// selects, by a warp-uniform jump, straight-line code holding exactly those MMAs.
 // Every mbarrier wait is bounded: on expiry the warp latches BSP_ERR_TIMEOUT in the workspace and leaves.
 #include <cuda.h>
+#include <cstdlib>
 #include "bsp_internal.cuh"
 
 namespace bsp {
 namespace {
 
 constexpr int kMaxTaps = 128;
-constexpr int kMT = 4;                    // 16-pixel MMA tiles per consumer warp
 constexpr int kMaxSmem = 200 * 1024;      // ceiling of the carved-up shared memory of a launch (+1 KB slack)
 constexpr int kMaxDevices = 64;
 constexpr int kMaxWStages = 8;            // weight ring depth
@@ -165,9 +166,150 @@ __device__ __forceinline__ uint32_t slab_addr(uint32_t stage, int row, int chunk
     return stage + (uint32_t)row * kSlabBytes + (uint32_t)((chunk ^ (row & 7)) << 4);
 }
 
-// Threads: WM*WN consumer warps, then one producer warp.
-template <int DT, int WM, int WN>
-__global__ void __launch_bounds__(32 * (WM * WN + 1), 1)
+
+// ---- MMAs of the stored tiles of one K-step (general kernel shapes) -----------------------------------------
+// KIND: 0 bf16 k16 (two taps), 1 bf16 k8 (odd last tap), 2 int8 k16, 3 tf32 k8.
+// The tile rows present in a tile column are known only at run time, but accumulators must be indexed
+// statically.  The 8-bit row mask is therefore split into two nibbles and each nibble value jumps (a
+// warp-uniform switch) to straight-line code holding exactly the MMAs of its set rows: absent tiles cost no
+// issue slot.  Stored tiles follow each other in row order, so the weight pointer just advances.
+template <int KIND, int kMT, int R, typename acc_t>
+__device__ __forceinline__ void tile_mma(acc_t (&acc)[kMT][kPanelRows][4], const uint32_t (&a)[kMT][4], uint32_t &wp,
+                                         int tile_bytes)
+{
+    if constexpr (KIND == 0) {
+        const uint2 b = lds64(wp);
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][R], a[i], b.x, b.y);
+    } else if constexpr (KIND == 1) {
+        const uint32_t b = lds32(wp);
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][R], a[i], b);
+    } else if constexpr (KIND == 2) {
+        const uint32_t b = lds32(wp);
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][R], a[i], b);
+    } else {
+        const uint2 b = lds64(wp);
+        const uint32_t b0 = to_tf32(b.x), b1 = to_tf32(b.y);
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) mma_tf32_k8(acc[i][R], a[i], b0, b1);
+    }
+    wp += tile_bytes;
+}
+
+template <int KIND, int kMT, int NIB, int BASE, typename acc_t>
+__device__ __forceinline__ void nibble_mma(acc_t (&acc)[kMT][kPanelRows][4], const uint32_t (&a)[kMT][4], uint32_t &wp,
+                                           int tile_bytes)
+{
+    if constexpr ((NIB & 1) != 0) tile_mma<KIND, kMT, BASE + 0>(acc, a, wp, tile_bytes);
+    if constexpr ((NIB & 2) != 0) tile_mma<KIND, kMT, BASE + 1>(acc, a, wp, tile_bytes);
+    if constexpr ((NIB & 4) != 0) tile_mma<KIND, kMT, BASE + 2>(acc, a, wp, tile_bytes);
+    if constexpr ((NIB & 8) != 0) tile_mma<KIND, kMT, BASE + 3>(acc, a, wp, tile_bytes);
+}
+
+#define BSP_NIBBLE_SWITCH(FN, ...)                       \
+    switch (nib) {                                       \
+        case 1: FN<__VA_ARGS__, 1, BASE> ARGS; break;    \
+        case 2: FN<__VA_ARGS__, 2, BASE> ARGS; break;    \
+        case 3: FN<__VA_ARGS__, 3, BASE> ARGS; break;    \
+        case 4: FN<__VA_ARGS__, 4, BASE> ARGS; break;    \
+        case 5: FN<__VA_ARGS__, 5, BASE> ARGS; break;    \
+        case 6: FN<__VA_ARGS__, 6, BASE> ARGS; break;    \
+        case 7: FN<__VA_ARGS__, 7, BASE> ARGS; break;    \
+        case 8: FN<__VA_ARGS__, 8, BASE> ARGS; break;    \
+        case 9: FN<__VA_ARGS__, 9, BASE> ARGS; break;    \
+        case 10: FN<__VA_ARGS__, 10, BASE> ARGS; break;  \
+        case 11: FN<__VA_ARGS__, 11, BASE> ARGS; break;  \
+        case 12: FN<__VA_ARGS__, 12, BASE> ARGS; break;  \
+        case 13: FN<__VA_ARGS__, 13, BASE> ARGS; break;  \
+        case 14: FN<__VA_ARGS__, 14, BASE> ARGS; break;  \
+        case 15: FN<__VA_ARGS__, 15, BASE> ARGS; break;  \
+        default: break;                                  \
+    }
+
+template <int KIND, int kMT, int BASE, typename acc_t>
+__device__ __forceinline__ void rows_mma(uint32_t nib, acc_t (&acc)[kMT][kPanelRows][4], const uint32_t (&a)[kMT][4],
+                                         uint32_t &wp, int tile_bytes)
+{
+#define ARGS (acc, a, wp, tile_bytes)
+    BSP_NIBBLE_SWITCH(nibble_mma, KIND, kMT)
+#undef ARGS
+}
+
+template <int KIND, int kMT, typename acc_t>
+__device__ __forceinline__ void step_mma(uint32_t m, acc_t (&acc)[kMT][kPanelRows][4], const uint32_t (&a)[kMT][4],
+                                         uint32_t wp, int tile_bytes)
+{
+    rows_mma<KIND, kMT, 0>(m & 15u, acc, a, wp, tile_bytes);
+    rows_mma<KIND, kMT, 4>(m >> 4, acc, a, wp, tile_bytes);
+}
+
+// ---- Columns with a compile-time tap count (1x1 and 3x3 kernels) -------------------------------------------
+// With HKT = H*K known, the K-steps of a tile column are unrolled: all activation fragments of the column are
+// loaded first (one exposed shared-memory latency per column instead of one per step), the row-mask dispatch
+// happens once per column and nibble instead of once per step, and every weight fragment sits at a constant
+// offset from the column's first stored tile.
+template <int DT, int HKT> struct Steps;
+template <int HKT> struct Steps<BSP_BF16, HKT> { static constexpr int N16 = HKT / 2, TAIL = HKT & 1, N = N16 + TAIL; };
+template <int HKT> struct Steps<BSP_I8, HKT> { static constexpr int N16 = (HKT + 1) / 2, TAIL = 0, N = N16; };
+
+template <int DT, int HKT, int kMT, int R, typename acc_t>
+__device__ __forceinline__ void col_tile(acc_t (&acc)[kMT][kPanelRows][4],
+                                         const uint32_t (&a)[Steps<DT, HKT>::N][kMT][4], uint32_t wt, int lane)
+{
+    using S = Steps<DT, HKT>;
+    if constexpr (DT == BSP_BF16) {
+        uint2 b[S::N16 > 0 ? S::N16 : 1];
+#pragma unroll
+        for (int st = 0; st < S::N16; ++st) b[st] = lds64(wt + st * 256 + lane * 8);
+        uint32_t bt = 0;
+        if constexpr (S::TAIL != 0) bt = lds32(wt + S::N16 * 256 + lane * 4);
+#pragma unroll
+        for (int st = 0; st < S::N16; ++st)
+#pragma unroll
+            for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][R], a[st][i], b[st].x, b[st].y);
+        if constexpr (S::TAIL != 0) {
+#pragma unroll
+            for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][R], a[S::N16][i], bt);
+        }
+    } else {
+        uint32_t b[S::N16];
+#pragma unroll
+        for (int st = 0; st < S::N16; ++st) b[st] = lds32(wt + st * 128 + lane * 4);
+#pragma unroll
+        for (int st = 0; st < S::N16; ++st)
+#pragma unroll
+            for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][R], a[st][i], b[st]);
+    }
+}
+
+template <int DT, int HKT, int kMT, int NIB, int BASE, typename acc_t>
+__device__ __forceinline__ void col_nibble(acc_t (&acc)[kMT][kPanelRows][4],
+                                           const uint32_t (&a)[Steps<DT, HKT>::N][kMT][4], uint32_t wt, int lane)
+{
+    constexpr int TB = (DT == BSP_BF16) ? 128 * HKT : 128 * ((HKT + 1) / 2);      // bytes of one stored tile
+    constexpr int r1 = (NIB & 1), r2 = r1 + ((NIB >> 1) & 1), r3 = r2 + ((NIB >> 2) & 1);
+    if constexpr ((NIB & 1) != 0) col_tile<DT, HKT, kMT, BASE + 0>(acc, a, wt, lane);
+    if constexpr ((NIB & 2) != 0) col_tile<DT, HKT, kMT, BASE + 1>(acc, a, wt + r1 * TB, lane);
+    if constexpr ((NIB & 4) != 0) col_tile<DT, HKT, kMT, BASE + 2>(acc, a, wt + r2 * TB, lane);
+    if constexpr ((NIB & 8) != 0) col_tile<DT, HKT, kMT, BASE + 3>(acc, a, wt + r3 * TB, lane);
+}
+
+template <int DT, int HKT, int kMT, int BASE, typename acc_t>
+__device__ __forceinline__ void col_rows(uint32_t nib, acc_t (&acc)[kMT][kPanelRows][4],
+                                         const uint32_t (&a)[Steps<DT, HKT>::N][kMT][4], uint32_t wt, int lane)
+{
+#define ARGS (acc, a, wt, lane)
+    BSP_NIBBLE_SWITCH(col_nibble, DT, HKT, kMT)
+#undef ARGS
+}
+
+// Threads: WM*WN consumer warps, then one producer warp.  kMT = 16-pixel MMA tiles per consumer warp (a warp
+// owns 16*kMT pixels x 64 channels); the smaller warp tile halves the registers so that more warps share an SM.
+// HKT = H*K when it is 1 (1x1) or 9 (3x3) and the unrolled column code is used, else 0 (any kernel shape).
+template <int DT, int kMT, int WM, int WN, int HKT>
+__global__ void __launch_bounds__(32 * (WM * WN + 1), (kMT == 2 && WM * WN <= 4) ? 3 : ((kMT == 2 && HKT != 9) ? 2 : 1))
 conv_mma_kernel(const __grid_constant__ ConvParams p)
 {
     using T = Traits<DT>;
@@ -244,6 +386,12 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                 tma_load_4d(a_ring + sa * p.a_stage_bytes, &p.tmap, bar, s * kSlabBytes, gx0, gy0, n0);
             };
             issue_act(0);
+            uint32_t pbase[WN];                                  // first stored tile of each of the CTA's panels
+#pragma unroll
+            for (int pn = 0; pn < WN; ++pn) {
+                const int pg = blockIdx.y * WN + pn;
+                pbase[pn] = pg < p.n_panels ? p.panel_base[pg] : 0u;
+            }
             int wc = 0;
             for (int s = 0; s < p.n_slabs && ok; ++s) {
                 issue_act(s + 1);
@@ -258,14 +406,13 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                         tx_bytes += (s_coloff[pn * (p.n_cols + 1) + col0 + ncol] - s_coloff[pn * (p.n_cols + 1) + col0]) *
                                     (uint32_t)p.tile_bytes;
                     mbar_expect_tx(bar, tx_bytes);
+#pragma unroll
                     for (int pn = 0; pn < WN; ++pn) {
-                        const int pg = blockIdx.y * WN + pn;
-                        if (pg >= p.n_panels) break;
                         const uint32_t first = s_coloff[pn * (p.n_cols + 1) + col0];
                         const uint32_t bytes = (s_coloff[pn * (p.n_cols + 1) + col0 + ncol] - first) * (uint32_t)p.tile_bytes;
-                        if (bytes)
+                        if (bytes)      // panels past the last one have no stored tiles
                             bulk_load(w_ring + sw * p.w_stage_bytes + pn * p.wseg_cap,
-                                      p.payload + (size_t)(p.panel_base[pg] + first) * p.tile_bytes, bytes, bar);
+                                      p.payload + (size_t)(pbase[pn] + first) * p.tile_bytes, bytes, bar);
                     }
                 }
             }
@@ -324,7 +471,43 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                 const int cbyte = (col0 + v - slab_col0) * CB;     // byte of the tile column inside a slab row
                 const int chunk = cbyte >> 4;
 
-                if constexpr (DT == BSP_BF16) {
+                if constexpr (HKT != 0 && DT != BSP_F32) {
+                    using S = Steps<DT, HKT>;
+                    constexpr int KT = (HKT == 9) ? 3 : 1;          // kernel width of the specialised shapes
+                    constexpr int TB = (DT == BSP_BF16) ? 128 * HKT : 128 * ((HKT + 1) / 2);
+                    uint32_t a[S::N][kMT][4];
+                    if constexpr (DT == BSP_BF16) {
+                        const int sel = lane >> 4;
+#pragma unroll
+                        for (int st = 0; st < S::N16; ++st) {
+                            const int tap = 2 * st + sel;
+                            const int trow = (tap / KT) * p.PW + tap % KT;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) ldmatrix_x4(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[st][i]);
+                        }
+                        if constexpr (S::TAIL != 0) {
+                            const int trow = ((HKT - 1) / KT) * p.PW + (HKT - 1) % KT;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) ldmatrix_x2(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[S::N16][i]);
+                        }
+                    } else {
+                        const int t = lane & 3;
+                        const int within = (cbyte & 15) + (t & 1) * 4;
+#pragma unroll
+                        for (int st = 0; st < S::N16; ++st) {
+                            int tap = 2 * st + (t >> 1);
+                            if (tap >= HKT) tap = HKT - 1;          // the zero-padded half of an odd last step
+                            const int trow = (tap / KT) * p.PW + tap % KT;
+#pragma unroll
+                            for (int i = 0; i < kMT; ++i) {
+                                a[st][i][0] = lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk) + within);
+                                a[st][i][1] = lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk) + within);
+                            }
+                        }
+                    }
+                    col_rows<DT, HKT, kMT, 0>(m & 15u, acc, a, wt, lane);
+                    col_rows<DT, HKT, kMT, 4>(m >> 4, acc, a, wt + __popc(m & 15u) * TB, lane);
+                } else if constexpr (DT == BSP_BF16) {
                     const int n16 = HK >> 1;
                     const int sel = lane >> 4;
                     for (int st = 0; st < n16; ++st) {
@@ -332,32 +515,14 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                         const int trow = s_taprow[2 * st + sel];
 #pragma unroll
                         for (int i = 0; i < kMT; ++i) ldmatrix_x4(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[i]);
-                        uint32_t wp = wt + st * 256 + lane * 8;
-#pragma unroll
-                        for (int r = 0; r < kPanelRows; ++r) {
-                            if (m & (1u << r)) {
-                                const uint2 b = lds64(wp);
-                                wp += p.tile_bytes;
-#pragma unroll
-                                for (int i = 0; i < kMT; ++i) mma_bf16_k16(acc[i][r], a[i], b.x, b.y);
-                            }
-                        }
+                        step_mma<0, kMT>(m, acc, a, wt + st * 256 + lane * 8, p.tile_bytes);
                     }
                     if (HK & 1) {
                         uint32_t a[kMT][4];
                         const int trow = s_taprow[HK - 1];
 #pragma unroll
                         for (int i = 0; i < kMT; ++i) ldmatrix_x2(slab_addr(a_stage, rowpix[i][0] + trow, chunk), a[i]);
-                        uint32_t wp = wt + n16 * 256 + lane * 4;
-#pragma unroll
-                        for (int r = 0; r < kPanelRows; ++r) {
-                            if (m & (1u << r)) {
-                                const uint32_t b = lds32(wp);
-                                wp += p.tile_bytes;
-#pragma unroll
-                                for (int i = 0; i < kMT; ++i) mma_bf16_k8(acc[i][r], a[i], b);
-                            }
-                        }
+                        step_mma<1, kMT>(m, acc, a, wt + n16 * 256 + lane * 4, p.tile_bytes);
                     }
                 } else if constexpr (DT == BSP_I8) {
                     const int nsteps = (HK + 1) >> 1;
@@ -371,16 +536,7 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                             a[i][0] = lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk) + within);
                             a[i][1] = lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk) + within);
                         }
-                        uint32_t wp = wt + st * 128 + lane * 4;
-#pragma unroll
-                        for (int r = 0; r < kPanelRows; ++r) {
-                            if (m & (1u << r)) {
-                                const uint32_t b = lds32(wp);
-                                wp += p.tile_bytes;
-#pragma unroll
-                                for (int i = 0; i < kMT; ++i) mma_s8_k16(acc[i][r], a[i], b);
-                            }
-                        }
+                        step_mma<2, kMT>(m, acc, a, wt + st * 128 + lane * 4, p.tile_bytes);
                     }
                 } else {
                     const int t = lane & 3;
@@ -394,16 +550,7 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
                             a[i][2] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][0] + trow, chunk + 1) + t * 4));
                             a[i][3] = to_tf32(lds32(slab_addr(a_stage, rowpix[i][1] + trow, chunk + 1) + t * 4));
                         }
-                        uint32_t wp = wt + st * 256 + lane * 8;
-#pragma unroll
-                        for (int r = 0; r < kPanelRows; ++r) {
-                            if (m & (1u << r)) {
-                                const uint2 b = lds64(wp);
-                                wp += p.tile_bytes;
-#pragma unroll
-                                for (int i = 0; i < kMT; ++i) mma_tf32_k8(acc[i][r], a[i], to_tf32(b.x), to_tf32(b.y));
-                            }
-                        }
+                        step_mma<3, kMT>(m, acc, a, wt + st * 256 + lane * 8, p.tile_bytes);
                     }
                 }
             }
@@ -475,13 +622,17 @@ conv_mma_kernel(const __grid_constant__ ConvParams p)
 }
 
 struct Plan {
-    int WM, WN, nb, th, tw;
+    int MT, WM, WN, nb, th, tw;
     int slab_cols, n_slabs, a_stages, GCW, w_stages;
     size_t smem, a_stage_bytes, a_box_bytes, w_stage_bytes, wseg_cap, meta_bytes, a_ring_off, w_ring_off, epi_off;
     long long tiles, ctas;
 };
 
-constexpr int kConfigs[][2] = {{2, 2}, {4, 2}, {2, 4}, {4, 1}, {8, 1}, {1, 4}};
+// Launch shapes: {kMT, WM, WN, CTAs per SM the shape is compiled for}.
+constexpr int kConfigs[][4] = {
+    {2, 2, 2, 3}, {2, 4, 1, 3}, {2, 1, 4, 3}, {2, 4, 2, 2}, {2, 8, 1, 2}, {2, 2, 4, 2},
+    {4, 2, 2, 1}, {4, 4, 2, 1}, {4, 2, 4, 1},
+};
 
 // Output-pixel tile (nb images x th x tw) of at most tpix pixels that needs the fewest tiles; box extents of
 // the TMA load are limited to 256 per dimension.
@@ -506,21 +657,32 @@ void best_tile(int tpix, int N, int M, int Nw, int sh, int sw, int H, int K, int
     tiles = best;
 }
 
-Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_panels, int n_cols)
+// Picks the launch shape with the lowest estimated time: the slower of a per-SM issue/tensor-pipe estimate
+// and the L2-to-SM traffic (every CTA re-reads its patch and its panels' stored tiles).
+Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_panels, int n_cols, double density)
 {
     const int CB = 8 * elem_bytes(wd.wtype);
-    const int tile_bytes = tile_bytes_of(wd.wtype, wd.H * wd.K);
+    const int HK = wd.H * wd.K;
+    const int tile_bytes = tile_bytes_of(wd.wtype, HK);
+    const int steps = wd.wtype == BSP_F32 ? HK : (HK + 1) / 2;
     Plan best = {};
     double best_cost = -1;
-    // Each warp layout is tried with its full pixel tile first; if the patch does not fit in shared memory
-    // (large strides or kernels) the tile is halved, leaving some MMA rows idle.
+    // BSP_CONV_SHAPE=<kMT><WM><WN> (e.g. 242) pins the launch shape, for tuning runs
+    const char *pin = getenv("BSP_CONV_SHAPE");
+    const int pinned = pin ? atoi(pin) : 0;
+    // Each shape is tried with its full pixel tile first; if nothing fits in shared memory (large strides or
+    // kernels) the pixel tiles are halved, leaving some MMA rows idle.
     for (int shrink = 1; shrink <= 16 && best_cost < 0; shrink *= 2)
     for (auto &cfg : kConfigs) {
         Plan pl = {};
-        pl.WM = cfg[0]; pl.WN = cfg[1];
+        pl.MT = cfg[0]; pl.WM = cfg[1]; pl.WN = cfg[2];
+        if (pinned && pinned != pl.MT * 100 + pl.WM * 10 + pl.WN) continue;
+        int occ = cfg[3];
+        size_t cap = (size_t)kMaxSmem / occ - (occ > 1 ? 2048 : 0);
         pl.tiles = -1;
-        if (pl.WM * 64 / shrink < 8) continue;
-        best_tile(pl.WM * 64 / shrink, xd.N, M, Nw, xd.stride_h, xd.stride_w, wd.H, wd.K, pl.nb, pl.th, pl.tw, pl.tiles);
+        const int tpix = pl.WM * pl.MT * 16 / shrink;
+        if (tpix < 8) continue;
+        best_tile(tpix, xd.N, M, Nw, xd.stride_h, xd.stride_w, wd.H, wd.K, pl.nb, pl.th, pl.tw, pl.tiles);
         if (pl.tiles < 0) continue;
         const int PH = (pl.th - 1) * xd.stride_h + wd.H, PW = (pl.tw - 1) * xd.stride_w + wd.K;
         const long long patch_pix = (long long)pl.nb * PH * PW;
@@ -537,25 +699,38 @@ Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_pa
         pl.w_stage_bytes = pl.WN * pl.wseg_cap;
         pl.meta_bytes = align_up((size_t)pl.WN * (n_cols + 1) * 4 + (size_t)pl.WN * n_cols, 1024);
         const size_t epi = (size_t)pl.WM * pl.WN * kEpiBytes;
-        const size_t fixed = pl.meta_bytes + epi;
-        // at least two stages in each ring; then grow the activation ring to 3 and the weight ring as far as it goes
-        if (fixed + 2 * pl.a_stage_bytes + 2 * pl.w_stage_bytes > (size_t)kMaxSmem) continue;
-        pl.a_stages = (fixed + 3 * pl.a_stage_bytes + 3 * pl.w_stage_bytes <= (size_t)kMaxSmem) ? 3 : 2;
+        const size_t fixed = pl.meta_bytes + epi + 1024;          // + slack for aligning the base to 1024 bytes
+        // at least two stages in each ring; give up co-residency before giving up the shape
+        while (occ > 1 && fixed + 2 * pl.a_stage_bytes + 2 * pl.w_stage_bytes > cap) {
+            --occ;
+            cap = (size_t)kMaxSmem / occ - (occ > 1 ? 2048 : 0);
+        }
+        if (fixed + 2 * pl.a_stage_bytes + 2 * pl.w_stage_bytes > cap) continue;
+        pl.a_stages = (fixed + 3 * pl.a_stage_bytes + 3 * pl.w_stage_bytes <= cap) ? 3 : 2;
         if (pl.a_stages > pl.n_slabs) pl.a_stages = pl.n_slabs < 2 ? 2 : pl.n_slabs;
-        int ws = (int)(((size_t)kMaxSmem - fixed - pl.a_stages * pl.a_stage_bytes) / pl.w_stage_bytes);
+        int ws = (int)((cap - fixed - pl.a_stages * pl.a_stage_bytes) / pl.w_stage_bytes);
         if (ws > kMaxWStages) ws = kMaxWStages;
         pl.w_stages = ws;
         pl.a_ring_off = pl.meta_bytes;
         pl.w_ring_off = pl.a_ring_off + pl.a_stages * pl.a_stage_bytes;
         pl.epi_off = pl.w_ring_off + pl.w_stages * pl.w_stage_bytes;
-        pl.smem = pl.epi_off + epi + 1024;                  // + slack for aligning the base to 1024 bytes
+        pl.smem = pl.epi_off + epi + 1024;
         pl.ctas = pl.tiles * ((n_panels + pl.WN - 1) / pl.WN);
+
         const int warps = pl.WM * pl.WN;
-        // busiest SM: CTAs dealt round-robin over 148 SMs, each CTA keeping `warps` warps busy
-        const double load = (double)((pl.ctas + 147) / 148) * warps;
-        const double traffic = (double)pl.ctas * patch_pix * n_cols * CB +
-                               (double)pl.tiles * n_panels * n_cols * kPanelRows * tile_bytes * 0.5;
-        const double cost = load * 1e15 + traffic;
+        const double mma_per_warp = (double)n_cols * density * kPanelRows * steps * pl.MT;
+        const long long slots = 148LL * occ;
+        const long long waves = (pl.ctas + slots - 1) / slots;
+        const double resident = (double)warps * (pl.ctas < slots ? (double)((pl.ctas + 147) / 148) : occ);
+        // a lone warp issues one MMA per ~8 cycles and pays ~150 cycles of exposed latency per K-step; the SM's
+        // tensor pipe takes one MMA per 2 cycles
+        const double warp_cycles = mma_per_warp * 8.0 + (double)n_cols * steps * 150.0;
+        const double pipe_cycles = resident * mma_per_warp * 2.0 * 1.2;
+        const double t_compute = waves * (warp_cycles > pipe_cycles ? warp_cycles : pipe_cycles) / 1.9e9;
+        const double bytes = (double)pl.ctas * patch_pix * n_cols * CB +
+                             (double)pl.tiles * n_panels * n_cols * kPanelRows * tile_bytes * density;
+        const double t_traffic = bytes / 3.0e12;
+        const double cost = (t_compute > t_traffic ? t_compute : t_traffic) + 0.25 * (t_compute < t_traffic ? t_compute : t_traffic);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = pl; }
     }
     return best;
@@ -578,10 +753,10 @@ EncodeTiledFn encode_tiled()
     return fn;
 }
 
-template <int DT, int WM, int WN>
-bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
+template <int DT, int MT, int WM, int WN, int HKT>
+bsp_status launch_hk(const ConvParams &p, const Plan &pl, cudaStream_t st)
 {
-    auto kern = conv_mma_kernel<DT, WM, WN>;
+    auto kern = conv_mma_kernel<DT, MT, WM, WN, HKT>;
     // opt in to large dynamic shared memory once per device and instantiation
     static bool opted[kMaxDevices] = {};
     int dev = 0;
@@ -597,27 +772,48 @@ bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
     return BSP_OK;
 }
 
+// 1x1 kernels use the unrolled column code for every shape, 3x3 kernels for the kMT = 2 shapes (at kMT = 4 the
+// fragments of all nine taps do not fit in registers); everything else runs the general step loop.
+template <int DT, int MT, int WM, int WN>
+bsp_status launch_cfg(const ConvParams &p, const Plan &pl, cudaStream_t st)
+{
+    if constexpr (DT != BSP_F32) {
+        if (p.H == 1 && p.K == 1) return launch_hk<DT, MT, WM, WN, 1>(p, pl, st);
+        if constexpr (MT == 2) {
+            if (p.H == 3 && p.K == 3) return launch_hk<DT, MT, WM, WN, 9>(p, pl, st);
+        }
+    }
+    return launch_hk<DT, MT, WM, WN, 0>(p, pl, st);
+}
+
 template <int DT>
 bsp_status launch_dt(const ConvParams &p, const Plan &pl, cudaStream_t st)
 {
-    if (pl.WM == 2 && pl.WN == 2) return launch_cfg<DT, 2, 2>(p, pl, st);
-    if (pl.WM == 4 && pl.WN == 2) return launch_cfg<DT, 4, 2>(p, pl, st);
-    if (pl.WM == 2 && pl.WN == 4) return launch_cfg<DT, 2, 4>(p, pl, st);
-    if (pl.WM == 4 && pl.WN == 1) return launch_cfg<DT, 4, 1>(p, pl, st);
-    if (pl.WM == 8 && pl.WN == 1) return launch_cfg<DT, 8, 1>(p, pl, st);
-    return launch_cfg<DT, 1, 4>(p, pl, st);
+    const int key = pl.MT * 100 + pl.WM * 10 + pl.WN;
+    switch (key) {
+        case 222: return launch_cfg<DT, 2, 2, 2>(p, pl, st);
+        case 241: return launch_cfg<DT, 2, 4, 1>(p, pl, st);
+        case 214: return launch_cfg<DT, 2, 1, 4>(p, pl, st);
+        case 242: return launch_cfg<DT, 2, 4, 2>(p, pl, st);
+        case 281: return launch_cfg<DT, 2, 8, 1>(p, pl, st);
+        case 224: return launch_cfg<DT, 2, 2, 4>(p, pl, st);
+        case 422: return launch_cfg<DT, 4, 2, 2>(p, pl, st);
+        case 442: return launch_cfg<DT, 4, 4, 2>(p, pl, st);
+        case 424: return launch_cfg<DT, 4, 2, 4>(p, pl, st);
+    }
+    return BSP_ERR_SHAPE;
 }
 
 }  // namespace
 
 bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
-                       const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
+                       const void *bias, void *Y, bsp_dtype ytype, double density, void *ws, cudaStream_t st)
 {
     const PackedLayout L = packed_layout(wd, 0);
     const int M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1;
     const int Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
-    const Plan pl = make_plan(wd, xd, M, Nw, L.n_panels, L.n_cols);
-    if (pl.WM == 0) return BSP_ERR_SHAPE;
+    const Plan pl = make_plan(wd, xd, M, Nw, L.n_panels, L.n_cols, density);
+    if (pl.MT == 0) return BSP_ERR_SHAPE;
     const int e = elem_bytes(wd.wtype);
     const uint8_t *pk = (const uint8_t *)packed;
     ConvParams p = {};

@@ -60,7 +60,7 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
                           cudaStream_t st);
 bsp_status launch_count(const uint8_t *gamma, int64_t n, unsigned long long *out, cudaStream_t st);
 bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
-                       const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
+                       const void *bias, void *Y, bsp_dtype ytype, double density, void *ws, cudaStream_t st);
 
 #define BSP_CUDA_OK(expr)                                  \
     do {                                                   \
