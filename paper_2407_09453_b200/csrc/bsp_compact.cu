@@ -138,7 +138,7 @@ scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_
     }
 }
 
-// Launch 3a.  One CTA per row of Gamma: column indices in ascending order and the canonical payload
+// Launch 3a.  gridDim.y CTAs per row of Gamma: column indices in ascending order and the canonical payload
 // payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
@@ -162,7 +162,7 @@ csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int 
         if (v) {
             const int n = s_run + before;
             s_cols[n] = i;
-            if ((long long)(first + n) < capacity_blocks) col_idx[first + n] = i;
+            if (blockIdx.y == 0 && (long long)(first + n) < capacity_blocks) col_idx[first + n] = i;
         }
         __syncthreads();
         if (threadIdx.x == 0) s_run += tot;
@@ -172,7 +172,8 @@ csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int 
     const int cnt = s_run;
     const int blk = bo * HK * bi;
     const long long total = (long long)cnt * blk;
-    for (long long e = threadIdx.x; e < total; e += kThreads) {
+    // the CTAs of one row (gridDim.y of them) all build the column list, then share the copy
+    for (long long e = (long long)blockIdx.y * kThreads + threadIdx.x; e < total; e += (long long)gridDim.y * kThreads) {
         const int n = (int)(e / blk);
         const int q = (int)(e % blk);
         int rem = q;
@@ -311,18 +312,25 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
                                         (long long)capacity_blocks, (long long)L.capacity_tiles, status);
     BSP_CUDA_OK(cudaGetLastError());
     const size_t smem = (size_t)NBi * sizeof(int);
+    // enough CTAs per row to give every SM some of the payload copy
+    int fill_y = payload ? (296 + NBo - 1) / NBo : 1;
+    if (fill_y > 16) fill_y = 16;
+    if (fill_y < 1) fill_y = 1;
+    const dim3 fill_grid((unsigned)NBo, (unsigned)fill_y);
     if (wd.wtype == BSP_I8)
-        csr_fill_kernel<uint8_t><<<NBo, kThreads, smem, st>>>((const uint8_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+        csr_fill_kernel<uint8_t><<<fill_grid, kThreads, smem, st>>>((const uint8_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
                                                               row_ptr, col_idx, (uint8_t *)payload, capacity_blocks);
     else if (wd.wtype == BSP_BF16)
-        csr_fill_kernel<uint16_t><<<NBo, kThreads, smem, st>>>((const uint16_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+        csr_fill_kernel<uint16_t><<<fill_grid, kThreads, smem, st>>>((const uint16_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
                                                                row_ptr, col_idx, (uint16_t *)payload, capacity_blocks);
     else
-        csr_fill_kernel<uint32_t><<<NBo, kThreads, smem, st>>>((const uint32_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
+        csr_fill_kernel<uint32_t><<<fill_grid, kThreads, smem, st>>>((const uint32_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
                                                                row_ptr, col_idx, (uint32_t *)payload, capacity_blocks);
     BSP_CUDA_OK(cudaGetLastError());
     if (pk) {
-        const int cols_per_cta = 8;
+        // one tile column per CTA unless that would make a needlessly large grid
+        int cols_per_cta = (int)(((long long)L.n_cols * L.n_panels + 1183) / 1184);
+        if (cols_per_cta < 1) cols_per_cta = 1;
         dim3 grid((L.n_cols + cols_per_cta - 1) / cols_per_cta, L.n_panels);
         uint8_t *pl = pk + L.off_payload;
         if (wd.wtype == BSP_I8)

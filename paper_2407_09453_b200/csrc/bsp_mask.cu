@@ -148,6 +148,29 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
     }
 }
 
+// Small segments (up to kRankMax keys): the keys sit in shared memory and every thread counts the (key, index)
+// pairs below its own, which is its rank in the ascending order; Gamma = 0 for ranks below n_zero.  Same
+// result as the radix select, in one pass instead of nine.
+constexpr int kRankMax = 2048;
+__global__ void __launch_bounds__(kSelectThreads)
+rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n_zero, uint8_t *__restrict__ gamma)
+{
+    __shared__ unsigned long long s_key[kRankMax];
+    const unsigned long long *k = key + (size_t)blockIdx.x * seg_len;
+    uint8_t *g = gamma + (size_t)blockIdx.x * seg_len;
+    for (int i = threadIdx.x; i < seg_len; i += kSelectThreads) s_key[i] = k[i];
+    __syncthreads();
+    for (int i = threadIdx.x; i < seg_len; i += kSelectThreads) {
+        const unsigned long long mine = s_key[i];
+        int rank = 0;
+        for (int j = 0; j < seg_len; ++j) {
+            const unsigned long long other = s_key[j];
+            rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
+        }
+        g[i] = ((long long)rank < n_zero) ? 0 : 1;
+    }
+}
+
 template <int DT>
 bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *scores, cudaStream_t st)
 {
@@ -178,10 +201,12 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
     if (rc != BSP_OK) return rc;
     const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
     const long long NB = (long long)NBo * NBi;
-    if (scope == BSP_SCOPE_LAYER)
-        select_kernel<<<1, kSelectThreads, 0, st>>>((const unsigned long long *)scores, NB, n_zero, gamma);
+    const long long seg = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
+    const unsigned nseg = (scope == BSP_SCOPE_LAYER) ? 1u : (unsigned)NBo;
+    if (seg <= kRankMax)
+        rank_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, (int)seg, n_zero, gamma);
     else
-        select_kernel<<<NBo, kSelectThreads, 0, st>>>((const unsigned long long *)scores, NBi, n_zero, gamma);
+        select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }
