@@ -152,23 +152,24 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
 // pairs below its own, which is its rank in the ascending order; Gamma = 0 for ranks below n_zero.  Same
 // result as the radix select, in one pass instead of nine.
 constexpr int kRankMax = 2048;
-__global__ void __launch_bounds__(kSelectThreads)
+constexpr int kRankThreads = 128;
+__global__ void __launch_bounds__(kRankThreads)
 rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n_zero, uint8_t *__restrict__ gamma)
 {
     __shared__ unsigned long long s_key[kRankMax];
     const unsigned long long *k = key + (size_t)blockIdx.x * seg_len;
     uint8_t *g = gamma + (size_t)blockIdx.x * seg_len;
-    for (int i = threadIdx.x; i < seg_len; i += kSelectThreads) s_key[i] = k[i];
+    for (int i = threadIdx.x; i < seg_len; i += kRankThreads) s_key[i] = k[i];
     __syncthreads();
-    for (int i = threadIdx.x; i < seg_len; i += kSelectThreads) {
-        const unsigned long long mine = s_key[i];
-        int rank = 0;
-        for (int j = 0; j < seg_len; ++j) {
-            const unsigned long long other = s_key[j];
-            rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
-        }
-        g[i] = ((long long)rank < n_zero) ? 0 : 1;
+    const int i = blockIdx.y * kRankThreads + threadIdx.x;          // gridDim.y CTAs share one segment
+    if (i >= seg_len) return;
+    const unsigned long long mine = s_key[i];
+    int rank = 0;
+    for (int j = 0; j < seg_len; ++j) {
+        const unsigned long long other = s_key[j];
+        rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
     }
+    g[i] = ((long long)rank < n_zero) ? 0 : 1;
 }
 
 template <int DT>
@@ -204,7 +205,8 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
     const long long seg = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
     const unsigned nseg = (scope == BSP_SCOPE_LAYER) ? 1u : (unsigned)NBo;
     if (seg <= kRankMax)
-        rank_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, (int)seg, n_zero, gamma);
+        rank_kernel<<<dim3(nseg, (unsigned)((seg + kRankThreads - 1) / kRankThreads)), kRankThreads, 0, st>>>(
+            (const unsigned long long *)scores, (int)seg, n_zero, gamma);
     else
         select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
     BSP_CUDA_OK(cudaGetLastError());
