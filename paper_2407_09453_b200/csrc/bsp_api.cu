@@ -1,6 +1,15 @@
 // extern "C" entry points of libbsp: argument validation on the host, then kernel launches on the caller's
 // stream.  Declarations and their contracts are in include/bsp.h.
+#include <cstdio>
+#include <cstdlib>
 #include "bsp_internal.cuh"
+
+namespace bsp {
+void report_cuda_error(cudaError_t e, const char *expr, const char *file, int line)
+{
+    if (getenv("BSP_DEBUG")) fprintf(stderr, "libbsp: %s failed at %s:%d: %s\n", expr, file, line, cudaGetErrorString(e));
+}
+}  // namespace bsp
 
 using namespace bsp;
 

@@ -62,10 +62,16 @@ bsp_status launch_count(const uint8_t *gamma, int64_t n, unsigned long long *out
 bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
                        const void *bias, void *Y, bsp_dtype ytype, double density, void *ws, cudaStream_t st);
 
-#define BSP_CUDA_OK(expr)                                  \
-    do {                                                   \
-        cudaError_t e_ = (expr);                           \
-        if (e_ != cudaSuccess) return BSP_ERR_CUDA;        \
+// A failed CUDA call becomes BSP_ERR_CUDA; with BSP_DEBUG set in the environment its text goes to stderr.
+void report_cuda_error(cudaError_t e, const char *expr, const char *file, int line);
+
+#define BSP_CUDA_OK(expr)                                            \
+    do {                                                             \
+        cudaError_t e_ = (expr);                                     \
+        if (e_ != cudaSuccess) {                                     \
+            bsp::report_cuda_error(e_, #expr, __FILE__, __LINE__);   \
+            return BSP_ERR_CUDA;                                     \
+        }                                                            \
     } while (0)
 
 }  // namespace bsp
