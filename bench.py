@@ -323,7 +323,7 @@ def main():
         "roofline": roof,
         "e2e": {"value": world * fl / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
-        "gpu_launches": args.steps * 7,
+        "gpu_launches": args.steps * bsp.launches_per_step(lay.wd),
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -151,6 +151,12 @@ def bsp_check(ws, stream=None):
     _raise(lib().bsp_check(_ptr(ws), _stream(stream)), "bsp_check")
 
 
+def launches_per_step(wd: WDesc) -> int:
+    """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass: score, select; count, scan,
+    fill+pack; the product kernel."""
+    return 6
+
+
 class SparseLayer:
     """Device buffers of one compacted layer plus the calls that fill and use them (marshalling only)."""
 

@@ -138,18 +138,17 @@ scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_
     }
 }
 
-// Launch 3a.  gridDim.y CTAs per row of Gamma: column indices in ascending order and the canonical payload
+// Final launch, first part.  `parts` CTAs per row of Gamma: column indices in ascending order and the canonical payload
 // payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
-csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int NBi, int I, int HK, int bo, int bi,
-                const int32_t *__restrict__ row_ptr, int32_t *__restrict__ col_idx, T *__restrict__ payload,
-                long long capacity_blocks)
+__device__ __forceinline__ void csr_fill_body(int l, int part, int parts, const T *__restrict__ W,
+                                              const uint8_t *__restrict__ gamma, int NBi, int I, int HK, int bo, int bi,
+                                              const int32_t *__restrict__ row_ptr, int32_t *__restrict__ col_idx,
+                                              T *__restrict__ payload, long long capacity_blocks)
 {
     __shared__ int warp_sums[kThreads / 32];
     __shared__ int s_run;
     extern __shared__ int s_cols[];      // NBi ints: columns of this row's stored blocks
-    const int l = blockIdx.x;
     const uint8_t *g = gamma + (size_t)l * NBi;
     const int first = row_ptr[l];
     if (threadIdx.x == 0) s_run = 0;
@@ -162,7 +161,7 @@ csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int 
         if (v) {
             const int n = s_run + before;
             s_cols[n] = i;
-            if (blockIdx.y == 0 && (long long)(first + n) < capacity_blocks) col_idx[first + n] = i;
+            if (part == 0 && (long long)(first + n) < capacity_blocks) col_idx[first + n] = i;
         }
         __syncthreads();
         if (threadIdx.x == 0) s_run += tot;
@@ -172,8 +171,8 @@ csr_fill_kernel(const T *__restrict__ W, const uint8_t *__restrict__ gamma, int 
     const int cnt = s_run;
     const int blk = bo * HK * bi;
     const long long total = (long long)cnt * blk;
-    // the CTAs of one row (gridDim.y of them) all build the column list, then share the copy
-    for (long long e = (long long)blockIdx.y * kThreads + threadIdx.x; e < total; e += (long long)gridDim.y * kThreads) {
+    // the CTAs of one row (`parts` of them) all build the column list, then share the copy
+    for (long long e = (long long)part * kThreads + threadIdx.x; e < total; e += (long long)parts * kThreads) {
         const int n = (int)(e / blk);
         const int q = (int)(e % blk);
         int rem = q;
@@ -230,17 +229,16 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
     }
 }
 
-// Launch 3b.  grid (tile-column chunks, panels): every stored tile of the panel in this chunk of columns is
+// Final launch, second part.  One CTA per (tile-column chunk, panel): every stored tile of the panel in this chunk of columns is
 // written word by word.
 template <int DT>
-__global__ void __launch_bounds__(kThreads)
-pack_kernel(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
-            int NBi, int n_cols, int cols_per_cta, int tile_bytes, const uint8_t *__restrict__ colmask,
-            const uint32_t *__restrict__ coloff, const uint32_t *__restrict__ panel_base, uint8_t *__restrict__ payload,
-            long long capacity_tiles)
+__device__ __forceinline__ void pack_body(int chunk, int panel, const void *__restrict__ W,
+                                          const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi, int NBi,
+                                          int n_cols, int cols_per_cta, int tile_bytes, const uint8_t *__restrict__ colmask,
+                                          const uint32_t *__restrict__ coloff, const uint32_t *__restrict__ panel_base,
+                                          uint8_t *__restrict__ payload, long long capacity_tiles)
 {
-    const int panel = blockIdx.y;
-    const int col_lo = blockIdx.x * cols_per_cta;
+    const int col_lo = chunk * cols_per_cta;
     const int col_hi = min(n_cols, col_lo + cols_per_cta);
     const int words = tile_bytes / 4;
     const unsigned base = panel_base[panel];
@@ -259,6 +257,38 @@ pack_kernel(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O
                                                bo, bi, NBi);
             ((uint32_t *)(payload + (size_t)(first + j) * tile_bytes))[word] = v;
         }
+    }
+}
+
+struct FillPackArgs {
+    const void *W;
+    const uint8_t *gamma;
+    int O, I, HK, bo, bi, NBo, NBi;
+    const int32_t *row_ptr;
+    int32_t *col_idx;
+    void *payload;
+    long long capacity_blocks;
+    int fill_parts;                   // CTAs per row of Gamma in the first part of the grid
+    int n_cols, n_panels, cols_per_cta, pack_chunks, tile_bytes;
+    const uint8_t *colmask;
+    const uint32_t *coloff, *panel_base;
+    uint8_t *packed_payload;          // NULL: no packed form
+    long long capacity_tiles;
+};
+
+// The last compaction launch: CTAs [0, NBo * fill_parts) write col_idx and the canonical payload, the rest write
+// the packed tiles.  T is the storage type of a weight, DT its bsp_dtype.
+template <typename T, int DT>
+__global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs a)
+{
+    const int n_fill = a.NBo * a.fill_parts;
+    if ((int)blockIdx.x < n_fill) {
+        csr_fill_body<T>((int)blockIdx.x / a.fill_parts, (int)blockIdx.x % a.fill_parts, a.fill_parts, (const T *)a.W,
+                         a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, a.row_ptr, a.col_idx, (T *)a.payload, a.capacity_blocks);
+    } else {
+        const int b = (int)blockIdx.x - n_fill;
+        pack_body<DT>(b % a.pack_chunks, b / a.pack_chunks, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.n_cols,
+                      a.cols_per_cta, a.tile_bytes, a.colmask, a.coloff, a.panel_base, a.packed_payload, a.capacity_tiles);
     }
 }
 
@@ -311,42 +341,27 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, panel_cnt, L.n_panels, panel_base, (PackedHeader *)pk, h,
                                         (long long)capacity_blocks, (long long)L.capacity_tiles, status);
     BSP_CUDA_OK(cudaGetLastError());
-    const size_t smem = (size_t)NBi * sizeof(int);
+    FillPackArgs a = {};
+    a.W = W; a.gamma = gamma; a.O = wd.O; a.I = wd.I; a.HK = HK; a.bo = wd.bo; a.bi = wd.bi; a.NBo = NBo; a.NBi = NBi;
+    a.row_ptr = row_ptr; a.col_idx = col_idx; a.payload = payload; a.capacity_blocks = capacity_blocks;
     // enough CTAs per row to give every SM some of the payload copy
-    int fill_y = payload ? (296 + NBo - 1) / NBo : 1;
-    if (fill_y > 16) fill_y = 16;
-    if (fill_y < 1) fill_y = 1;
-    const dim3 fill_grid((unsigned)NBo, (unsigned)fill_y);
-    if (wd.wtype == BSP_I8)
-        csr_fill_kernel<uint8_t><<<fill_grid, kThreads, smem, st>>>((const uint8_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
-                                                              row_ptr, col_idx, (uint8_t *)payload, capacity_blocks);
-    else if (wd.wtype == BSP_BF16)
-        csr_fill_kernel<uint16_t><<<fill_grid, kThreads, smem, st>>>((const uint16_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
-                                                               row_ptr, col_idx, (uint16_t *)payload, capacity_blocks);
-    else
-        csr_fill_kernel<uint32_t><<<fill_grid, kThreads, smem, st>>>((const uint32_t *)W, gamma, NBi, wd.I, HK, wd.bo, wd.bi,
-                                                               row_ptr, col_idx, (uint32_t *)payload, capacity_blocks);
+    a.fill_parts = payload ? (296 + NBo - 1) / NBo : 1;
+    if (a.fill_parts > 16) a.fill_parts = 16;
+    if (a.fill_parts < 1) a.fill_parts = 1;
+    a.n_cols = L.n_cols; a.n_panels = L.n_panels; a.tile_bytes = L.tile_bytes;
+    // one tile column per CTA unless that would make a needlessly large grid
+    a.cols_per_cta = (int)(((long long)L.n_cols * L.n_panels + 1183) / 1184);
+    if (a.cols_per_cta < 1) a.cols_per_cta = 1;
+    a.pack_chunks = (L.n_cols + a.cols_per_cta - 1) / a.cols_per_cta;
+    a.colmask = colmask; a.coloff = coloff; a.panel_base = panel_base;
+    a.packed_payload = pk ? pk + L.off_payload : nullptr;
+    a.capacity_tiles = (long long)L.capacity_tiles;
+    const unsigned grid = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels : 0));
+    const size_t smem = (size_t)NBi * sizeof(int);
+    if (wd.wtype == BSP_I8) fill_pack_kernel<uint8_t, BSP_I8><<<grid, kThreads, smem, st>>>(a);
+    else if (wd.wtype == BSP_BF16) fill_pack_kernel<uint16_t, BSP_BF16><<<grid, kThreads, smem, st>>>(a);
+    else fill_pack_kernel<uint32_t, BSP_F32><<<grid, kThreads, smem, st>>>(a);
     BSP_CUDA_OK(cudaGetLastError());
-    if (pk) {
-        // one tile column per CTA unless that would make a needlessly large grid
-        int cols_per_cta = (int)(((long long)L.n_cols * L.n_panels + 1183) / 1184);
-        if (cols_per_cta < 1) cols_per_cta = 1;
-        dim3 grid((L.n_cols + cols_per_cta - 1) / cols_per_cta, L.n_panels);
-        uint8_t *pl = pk + L.off_payload;
-        if (wd.wtype == BSP_I8)
-            pack_kernel<BSP_I8><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
-                                                           cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
-                                                           (long long)L.capacity_tiles);
-        else if (wd.wtype == BSP_BF16)
-            pack_kernel<BSP_BF16><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
-                                                             cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
-                                                             (long long)L.capacity_tiles);
-        else
-            pack_kernel<BSP_F32><<<grid, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, L.n_cols,
-                                                            cols_per_cta, L.tile_bytes, colmask, coloff, panel_base, pl,
-                                                            (long long)L.capacity_tiles);
-        BSP_CUDA_OK(cudaGetLastError());
-    }
     return BSP_OK;
 }
 

@@ -59,7 +59,24 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
         const int words = bi / per_word;
         const size_t row_words = (size_t)I / per_word;
         const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
-        for (int t = 0; t < HK; ++t) {
+        // loads of up to nine taps (a whole 3x3 kernel) are issued together; the adds keep the (h, k, c) order
+        constexpr int kBatch = 9, kMaxWords = 16;
+        int t = 0;
+        for (; t < HK; t += kBatch) {
+            uint32_t w[kBatch][kMaxWords];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+                for (int j = 0; j < kMaxWords; ++j)
+                    if (t + u < HK && j < words) w[u][j] = __ldg(src + (size_t)u * row_words + j);
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+                for (int j = 0; j < kMaxWords; ++j)
+                    if (t + u < HK && j < words) add_word<DT, NORM>(w[u][j], pr);
+            src += (size_t)kBatch * row_words;
+        }
+        for (; t < HK; ++t) {
             for (int j = 0; j < words; ++j) add_word<DT, NORM>(__ldg(src + j), pr);
             src += row_words;
         }
@@ -152,24 +169,45 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
 // pairs below its own, which is its rank in the ascending order; Gamma = 0 for ranks below n_zero.  Same
 // result as the radix select, in one pass instead of nine.
 constexpr int kRankMax = 2048;
-constexpr int kRankThreads = 128;
+constexpr int kRankThreads = 256;
+constexpr int kRankLanes = 8;            // lanes sharing one key; each counts an eighth of the segment
 __global__ void __launch_bounds__(kRankThreads)
 rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n_zero, uint8_t *__restrict__ gamma)
 {
     __shared__ unsigned long long s_key[kRankMax];
     const unsigned long long *k = key + (size_t)blockIdx.x * seg_len;
     uint8_t *g = gamma + (size_t)blockIdx.x * seg_len;
-    for (int i = threadIdx.x; i < seg_len; i += kRankThreads) s_key[i] = k[i];
-    __syncthreads();
-    const int i = blockIdx.y * kRankThreads + threadIdx.x;          // gridDim.y CTAs share one segment
-    if (i >= seg_len) return;
-    const unsigned long long mine = s_key[i];
-    int rank = 0;
-    for (int j = 0; j < seg_len; ++j) {
-        const unsigned long long other = s_key[j];
-        rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
+    {   // all loads of the segment are issued before the first store, so they share one trip to memory
+        unsigned long long v[kRankMax / kRankThreads];
+#pragma unroll
+        for (int u = 0; u < kRankMax / kRankThreads; ++u) {
+            const int i = u * kRankThreads + threadIdx.x;
+            v[u] = i < seg_len ? __ldg(k + i) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < kRankMax / kRankThreads; ++u) {
+            const int i = u * kRankThreads + threadIdx.x;
+            if (i < seg_len) s_key[i] = v[u];
+        }
     }
-    g[i] = ((long long)rank < n_zero) ? 0 : 1;
+    __syncthreads();
+    // gridDim.y CTAs share one segment; the keys are padded to a multiple of the CTA's share so that all
+    // lanes of a warp take part in the shuffles
+    const int i = (blockIdx.y * kRankThreads + threadIdx.x) / kRankLanes;
+    const int part = threadIdx.x % kRankLanes;
+    const bool live = i < seg_len;
+    const unsigned long long mine = live ? s_key[i] : 0ull;
+    const int per = (seg_len + kRankLanes - 1) / kRankLanes;
+    const int j0 = part * per, j1 = min(seg_len, j0 + per);
+    int rank = 0;
+    if (live)
+        for (int j = j0; j < j1; ++j) {
+            const unsigned long long other = s_key[j];
+            rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
+        }
+#pragma unroll
+    for (int d = 1; d < kRankLanes; d <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, d);
+    if (live && part == 0) g[i] = ((long long)rank < n_zero) ? 0 : 1;
 }
 
 template <int DT>
@@ -205,7 +243,7 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
     const long long seg = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
     const unsigned nseg = (scope == BSP_SCOPE_LAYER) ? 1u : (unsigned)NBo;
     if (seg <= kRankMax)
-        rank_kernel<<<dim3(nseg, (unsigned)((seg + kRankThreads - 1) / kRankThreads)), kRankThreads, 0, st>>>(
+        rank_kernel<<<dim3(nseg, (unsigned)((seg * kRankLanes + kRankThreads - 1) / kRankThreads)), kRankThreads, 0, st>>>(
             (const unsigned long long *)scores, (int)seg, n_zero, gamma);
     else
         select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
