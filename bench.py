@@ -71,6 +71,22 @@ def measured_traffic(workload: str):
     return d.get("dram_bytes_per_launch")
 
 
+def reduce_max(values, world: int, device):
+    """Per-rank timings -> their maximum over all ranks (the job's time); identity for one rank."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_tflops(flops_per_rank: float, world: int, ms: float) -> float:
+    """Whole-job throughput: every rank does flops_per_rank of useful work in the job's ms (weak scaling)."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -285,16 +301,11 @@ def main():
     lay.check()
 
     # max over ranks
-    if world > 1:
-        t = torch.tensor([ms_step, ms_e2e, float(t_conv.mean())], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, ms_e2e, ms_conv = (float(v) for v in t.cpu())
-    else:
-        ms_conv = float(t_conv.mean())
+    ms_step, ms_e2e, ms_conv = reduce_max([ms_step, ms_e2e, float(t_conv.mean())], world, "cuda")
 
     fl = useful_flops(layer, nnz, bo, bi)
     pk = peaks()
-    value = world * fl / (ms_step * 1e-3) / 1e12
+    value = job_tflops(fl, world, ms_step)
     conv_tflops = fl / (ms_conv * 1e-3) / 1e12
     abytes = algorithmic_bytes(layer, nnz, bo, bi, ex, ey)
     t_tensor = fl / (pk["bf16_tflops"] * 1e12)
@@ -321,7 +332,7 @@ def main():
         "conv_only": {"tflops": conv_tflops, "ms": ms_conv, "ms_min": float(t_conv.min()),
                       "dense_ms": ms_dense, "speedup_vs_dense": ms_dense / ms_conv},
         "roofline": roof,
-        "e2e": {"value": world * fl / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": job_tflops(fl, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": args.steps * bsp.launches_per_step(lay.wd),
         "clocks": clocks,
