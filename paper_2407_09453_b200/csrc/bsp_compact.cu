@@ -22,7 +22,30 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
     L.off_coloff = align_up(L.off_colmask + (size_t)L.n_panels * L.n_cols, 256);
     L.off_panelbase = align_up(L.off_coloff + (size_t)L.n_panels * L.n_cols * 4, 256);
     L.off_payload = align_up(L.off_panelbase + (size_t)(L.n_panels + 1) * 4, 256);
-    L.total_bytes = align_up(L.off_payload + (size_t)cap * L.tile_bytes + 256, 256);
+    size_t end = align_up(L.off_payload + (size_t)cap * L.tile_bytes + 256, 256);
+    TcLayout &T = L.tc;
+    T = TcLayout{};
+    const int HK = wd.H * wd.K;
+    T.enabled = wd.wtype == BSP_BF16 && wd.O % 8 == 0 && wd.I % (HK == 1 ? 16 : 8) == 0;
+    if (T.enabled) {
+        const int n_sr = (wd.O + kTcSuperRow - 1) / kTcSuperRow;
+        T.n_groups = (n_sr + kTcGroupRows - 1) / kTcGroupRows;
+        T.kc_ch = HK == 1 ? 16 : 8;
+        T.n_kc = wd.I / T.kc_ch;
+        T.n_units = HK == 1 ? 1 : (HK + 1) / 2;
+        T.st_bytes = T.n_units * kTcUnitBytes;
+        int64_t tcap = nnz_blocks * 2;                        // a 4x16 block can touch two super-tiles
+        if (tcap > (int64_t)n_sr * T.n_kc) tcap = (int64_t)n_sr * T.n_kc;
+        if (tcap < 0) tcap = 0;
+        T.capacity = tcap;
+        T.off_mask = end;
+        T.off_off = align_up(T.off_mask + (size_t)T.n_groups * T.n_kc, 256);
+        T.off_gcnt = align_up(T.off_off + (size_t)T.n_groups * T.n_kc * 4, 256);
+        T.off_payload = align_up(T.off_gcnt + (size_t)(T.n_groups + 1) * 4, 256);
+        T.end = align_up(T.off_payload + (size_t)tcap * T.st_bytes + 256, 256);
+        end = T.end;
+    }
+    L.total_bytes = end;
     return L;
 }
 
@@ -56,13 +79,53 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &
 // Launch 1.  CTAs [0, NBo): ones of one row of Gamma -> row_cnt.  CTAs [NBo, NBo + n_panels): for one panel
 // (64 output channels) the byte mask of stored tiles in every tile column, and the running count of stored
 // tiles before each column (coloff, relative to the panel).
+struct TcIndexArgs {
+    int n_panels, n_groups, n_kc, kc_ch;
+    uint8_t *mask;        // [n_groups][n_kc]
+    uint32_t *off;        // [n_groups][n_kc] stored super-tiles of the group before this K-group
+    uint32_t *gcnt;       // [n_groups] stored super-tiles of the group
+};
+
 __global__ void __launch_bounds__(kThreads)
 count_kernel(const uint8_t *__restrict__ gamma, int NBo, int NBi, int bo, int bi, int O, int n_cols,
              int *__restrict__ row_cnt, uint8_t *__restrict__ colmask, uint32_t *__restrict__ coloff,
-             int *__restrict__ panel_cnt)
+             int *__restrict__ panel_cnt, const TcIndexArgs tc)
 {
     __shared__ int warp_sums[kThreads / 32];
     __shared__ int s_run;
+    if ((int)blockIdx.x >= NBo + tc.n_panels) {
+        // CTAs past the panels: one group of super-rows each, for the second packed form
+        const int g = (int)blockIdx.x - NBo - tc.n_panels;
+        if (threadIdx.x == 0) s_run = 0;
+        __syncthreads();
+        for (int base = 0; base < tc.n_kc; base += kThreads) {
+            const int kc = base + threadIdx.x;
+            unsigned m = 0;
+            if (kc < tc.n_kc) {
+                for (int r = 0; r < kTcGroupRows; ++r) {
+                    const int o0 = (g * kTcGroupRows + r) * kTcSuperRow;
+                    if (o0 >= O) break;
+                    const int o1 = min(O, o0 + kTcSuperRow) - 1;
+                    const int c0 = kc * tc.kc_ch, c1 = c0 + tc.kc_ch - 1;
+                    bool any = false;
+                    for (int lb = o0 / bo; lb <= o1 / bo && lb < NBo; ++lb)
+                        for (int cb = c0 / bi; cb <= c1 / bi && cb < NBi; ++cb) any |= gamma[(size_t)lb * NBi + cb] != 0;
+                    if (any) m |= 1u << r;
+                }
+            }
+            int tot;
+            const int before = block_exclusive_scan(__popc(m), warp_sums, tot);
+            if (kc < tc.n_kc) {
+                tc.mask[(size_t)g * tc.n_kc + kc] = (uint8_t)m;
+                tc.off[(size_t)g * tc.n_kc + kc] = (uint32_t)(s_run + before);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) s_run += tot;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) tc.gcnt[g] = (uint32_t)s_run;
+        return;
+    }
     if ((int)blockIdx.x < NBo) {
         const uint8_t *g = gamma + (size_t)blockIdx.x * NBi;
         int c = 0;
@@ -260,6 +323,59 @@ __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__re
     }
 }
 
+// One 32-bit word of a stored super-tile: K-step u, then [K half h][8-row group rg][row][4 words of 2 bf16],
+// the K-major core-matrix order of a 16 x 16 tcgen05 B operand.  A convolution pairs taps 2u and 2u+1 of the
+// K-group's 8 channels (a missing odd tap reads as zero); a 1x1 layer pairs the two 8-channel halves.
+__device__ __forceinline__ uint32_t tc_word(const uint16_t *__restrict__ W, const uint8_t *__restrict__ gamma, int word,
+                                            int o_base, int kc, int O, int I, int HK, int bo, int bi, int NBi)
+{
+    const int u = word >> 7, w = word & 127;
+    const int h = w >> 6, rg = (w >> 5) & 1, row = (w >> 2) & 7, pair = w & 3;
+    const int o = o_base + rg * 8 + row;
+    int tap, ch;
+    if (HK == 1) { tap = 0; ch = (2 * kc + h) * 8 + 2 * pair; }
+    else { tap = 2 * u + h; ch = kc * 8 + 2 * pair; }
+    if (tap >= HK || o >= O || gamma[(size_t)(o / bo) * NBi + ch / bi] == 0) return 0u;
+    const size_t e = ((size_t)o * HK + tap) * I + ch;
+    return (uint32_t)W[e] | ((uint32_t)W[e + 1] << 16);
+}
+
+struct TcPackArgs {
+    int n_groups, n_kc, kc_per_cta, chunks, st_bytes;
+    const uint8_t *mask;
+    const uint32_t *off, *gcnt;
+    uint8_t *payload;
+    long long capacity;
+    int *status;
+};
+
+__device__ __forceinline__ void tc_pack_body(int chunk, int g, const TcPackArgs &t, const void *__restrict__ W,
+                                             const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
+                                             int NBi)
+{
+    unsigned base = 0;
+    for (int q = 0; q < g; ++q) base += t.gcnt[q];
+    if (chunk == 0 && threadIdx.x == 0 && (long long)(base + t.gcnt[g]) > t.capacity)
+        atomicMax(t.status, (int)BSP_ERR_CAPACITY);
+    const int kc_lo = chunk * t.kc_per_cta, kc_hi = min(t.n_kc, kc_lo + t.kc_per_cta);
+    const int words = t.st_bytes / 4;
+    for (int kc = kc_lo; kc < kc_hi; ++kc) {
+        const unsigned m = t.mask[(size_t)g * t.n_kc + kc];
+        if (!m) continue;
+        const unsigned first = base + t.off[(size_t)g * t.n_kc + kc];
+        const int cnt = __popc(m);
+        for (int e = threadIdx.x; e < cnt * words; e += kThreads) {
+            const int j = e / words, word = e % words;
+            unsigned mm = m;
+            for (int q = 0; q < j; ++q) mm &= mm - 1;
+            const int R = __ffs(mm) - 1;
+            if ((long long)(first + j) >= t.capacity) continue;
+            ((uint32_t *)(t.payload + (size_t)(first + j) * t.st_bytes))[word] =
+                tc_word((const uint16_t *)W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi);
+        }
+    }
+}
+
 struct FillPackArgs {
     const void *W;
     const uint8_t *gamma;
@@ -274,6 +390,7 @@ struct FillPackArgs {
     const uint32_t *coloff, *panel_base;
     uint8_t *packed_payload;          // NULL: no packed form
     long long capacity_tiles;
+    TcPackArgs tc;                    // tc.n_groups == 0: no second packed form
 };
 
 // The last compaction launch: CTAs [0, NBo * fill_parts) write col_idx and the canonical payload, the rest write
@@ -287,8 +404,15 @@ __global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs 
                          a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, a.row_ptr, a.col_idx, (T *)a.payload, a.capacity_blocks);
     } else {
         const int b = (int)blockIdx.x - n_fill;
-        pack_body<DT>(b % a.pack_chunks, b / a.pack_chunks, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.n_cols,
-                      a.cols_per_cta, a.tile_bytes, a.colmask, a.coloff, a.panel_base, a.packed_payload, a.capacity_tiles);
+        const int n_pack = a.packed_payload ? a.pack_chunks * a.n_panels : 0;
+        if (b < n_pack) {
+            pack_body<DT>(b % a.pack_chunks, b / a.pack_chunks, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.n_cols,
+                          a.cols_per_cta, a.tile_bytes, a.colmask, a.coloff, a.panel_base, a.packed_payload,
+                          a.capacity_tiles);
+        } else if constexpr (DT == BSP_BF16) {
+            const int c = b - n_pack;
+            tc_pack_body(c % a.tc.chunks, c / a.tc.chunks, a.tc, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi);
+        }
     }
 }
 
@@ -335,8 +459,15 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     h.off_colmask = (int32_t)L.off_colmask; h.off_coloff = (int32_t)L.off_coloff;
     h.off_panelbase = (int32_t)L.off_panelbase; h.off_payload = (int64_t)L.off_payload;
 
-    count_kernel<<<NBo + (pk ? L.n_panels : 0), kThreads, 0, st>>>(gamma, NBo, NBi, wd.bo, wd.bi, wd.O, L.n_cols,
-                                                                   row_cnt, colmask, coloff, panel_cnt);
+    const bool tc_on = pk != nullptr && L.tc.enabled;
+    TcIndexArgs ti = {};
+    ti.n_panels = pk ? L.n_panels : 0;
+    if (tc_on) {
+        ti.n_groups = L.tc.n_groups; ti.n_kc = L.tc.n_kc; ti.kc_ch = L.tc.kc_ch;
+        ti.mask = pk + L.tc.off_mask; ti.off = (uint32_t *)(pk + L.tc.off_off); ti.gcnt = (uint32_t *)(pk + L.tc.off_gcnt);
+    }
+    count_kernel<<<NBo + ti.n_panels + ti.n_groups, kThreads, 0, st>>>(gamma, NBo, NBi, wd.bo, wd.bi, wd.O, L.n_cols,
+                                                                       row_cnt, colmask, coloff, panel_cnt, ti);
     BSP_CUDA_OK(cudaGetLastError());
     scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, panel_cnt, L.n_panels, panel_base, (PackedHeader *)pk, h,
                                         (long long)capacity_blocks, (long long)L.capacity_tiles, status);
@@ -356,7 +487,16 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     a.colmask = colmask; a.coloff = coloff; a.panel_base = panel_base;
     a.packed_payload = pk ? pk + L.off_payload : nullptr;
     a.capacity_tiles = (long long)L.capacity_tiles;
-    const unsigned grid = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels : 0));
+    if (tc_on) {
+        a.tc.n_groups = L.tc.n_groups; a.tc.n_kc = L.tc.n_kc; a.tc.st_bytes = L.tc.st_bytes;
+        a.tc.kc_per_cta = (int)(((long long)L.tc.n_kc * L.tc.n_groups + 1183) / 1184);
+        if (a.tc.kc_per_cta < 1) a.tc.kc_per_cta = 1;
+        a.tc.chunks = (L.tc.n_kc + a.tc.kc_per_cta - 1) / a.tc.kc_per_cta;
+        a.tc.mask = ti.mask; a.tc.off = ti.off; a.tc.gcnt = ti.gcnt;
+        a.tc.payload = pk + L.tc.off_payload; a.tc.capacity = (long long)L.tc.capacity; a.tc.status = status;
+    }
+    const unsigned grid = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels : 0) +
+                                     (tc_on ? a.tc.chunks * a.tc.n_groups : 0));
     const size_t smem = (size_t)NBi * sizeof(int);
     if (wd.wtype == BSP_I8) fill_pack_kernel<uint8_t, BSP_I8><<<grid, kThreads, smem, st>>>(a);
     else if (wd.wtype == BSP_BF16) fill_pack_kernel<uint16_t, BSP_BF16><<<grid, kThreads, smem, st>>>(a);

@@ -31,10 +31,27 @@ struct PackedHeader {
     int64_t off_payload;
 };
 
+// Second packed form, for the tcgen05 kernel (bf16 only): W-bar is cut into super-tiles of 16 output channels
+// (a super-row) by one K-group: 8 input channels and all taps for a convolution, 16 input channels for a 1x1
+// layer.  A super-tile is stored if any 8x8 tile inside it is; it holds one 512-byte tcgen05 B operand
+// (16 x 16 bf16, K-major core matrices) per K-step of 16: a pair of taps, or the two 8-channel halves.
+// Eight super-rows (128 channels) form a group, the N range of one CTA.
+constexpr int kTcGroupRows = 8;
+constexpr int kTcSuperRow = 16;
+constexpr int kTcUnitBytes = 512;
+
+struct TcLayout {
+    bool enabled;
+    int n_groups, n_kc, kc_ch, n_units, st_bytes;   // K-groups, channels per K-group, K-steps and bytes per super-tile
+    int64_t capacity;                                // super-tiles the payload area can hold
+    size_t off_mask, off_off, off_gcnt, off_payload, end;
+};
+
 struct PackedLayout {
     int n_panels, n_cols, tile_bytes;
     int64_t capacity_tiles;
     size_t off_colmask, off_coloff, off_panelbase, off_payload, total_bytes;
+    TcLayout tc;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
