@@ -138,6 +138,10 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
     // the packed header is on the device; the host checks what it can: capacity against the descriptor
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
+    // BSP_CONV_PATH=tc runs eligible layers (bf16, stride 1) on the tcgen05 kernel; the default is the warp-MMA kernel
+    const char *path = getenv("BSP_CONV_PATH");
+    if (path && path[0] == 't' && conv_tc_eligible(*wd, *xd))
+        return launch_conv_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
     // the stored fraction only steers the choice of launch shape
     const double density = NB > 0 ? (double)w->nnz / (double)NB : 1.0;
     return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, density > 0.05 ? density : 0.05, ws, (cudaStream_t)stream);

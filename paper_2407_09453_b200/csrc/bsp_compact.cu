@@ -21,12 +21,13 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
     L.off_colmask = 256;
     L.off_coloff = align_up(L.off_colmask + (size_t)L.n_panels * L.n_cols, 256);
     L.off_panelbase = align_up(L.off_coloff + (size_t)L.n_panels * L.n_cols * 4, 256);
-    L.off_payload = align_up(L.off_panelbase + (size_t)(L.n_panels + 1) * 4, 256);
-    size_t end = align_up(L.off_payload + (size_t)cap * L.tile_bytes + 256, 256);
+    // all index arrays come first, at offsets that do not depend on the capacity; the two payloads follow
+    size_t meta_end = align_up(L.off_panelbase + (size_t)(L.n_panels + 1) * 4, 256);
     TcLayout &T = L.tc;
     T = TcLayout{};
     const int HK = wd.H * wd.K;
     T.enabled = wd.wtype == BSP_BF16 && wd.O % 8 == 0 && wd.I % (HK == 1 ? 16 : 8) == 0;
+    int64_t tcap = 0;
     if (T.enabled) {
         const int n_sr = (wd.O + kTcSuperRow - 1) / kTcSuperRow;
         T.n_groups = (n_sr + kTcGroupRows - 1) / kTcGroupRows;
@@ -34,14 +35,19 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
         T.n_kc = wd.I / T.kc_ch;
         T.n_units = HK == 1 ? 1 : (HK + 1) / 2;
         T.st_bytes = T.n_units * kTcUnitBytes;
-        int64_t tcap = nnz_blocks * 2;                        // a 4x16 block can touch two super-tiles
+        tcap = nnz_blocks * 2;                                // a 4x16 block can touch two super-tiles
         if (tcap > (int64_t)n_sr * T.n_kc) tcap = (int64_t)n_sr * T.n_kc;
         if (tcap < 0) tcap = 0;
         T.capacity = tcap;
-        T.off_mask = end;
+        T.off_mask = meta_end;
         T.off_off = align_up(T.off_mask + (size_t)T.n_groups * T.n_kc, 256);
         T.off_gcnt = align_up(T.off_off + (size_t)T.n_groups * T.n_kc * 4, 256);
-        T.off_payload = align_up(T.off_gcnt + (size_t)(T.n_groups + 1) * 4, 256);
+        meta_end = align_up(T.off_gcnt + (size_t)(T.n_groups + 1) * 4, 256);
+    }
+    L.off_payload = meta_end;
+    size_t end = align_up(L.off_payload + (size_t)cap * L.tile_bytes + 256, 256);
+    if (T.enabled) {
+        T.off_payload = end;
         T.end = align_up(T.off_payload + (size_t)tcap * T.st_bytes + 256, 256);
         end = T.end;
     }
@@ -458,6 +464,7 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     h.capacity_tiles = (int32_t)L.capacity_tiles; h.n_tiles = 0;
     h.off_colmask = (int32_t)L.off_colmask; h.off_coloff = (int32_t)L.off_coloff;
     h.off_panelbase = (int32_t)L.off_panelbase; h.off_payload = (int64_t)L.off_payload;
+    h.off_tc_payload = (int64_t)L.tc.off_payload;
 
     const bool tc_on = pk != nullptr && L.tc.enabled;
     TcIndexArgs ti = {};

@@ -1,0 +1,382 @@
+// Block-sparse implicit-GEMM convolution / FC product with fused bias on 5th-generation tensor cores
+// (tcgen05.mma, accumulators in tensor memory), bf16 inputs, stride 1.  Introduction (Y = W*X + b) and Section
+// "Block Sparsity in a Matrix" of the paper.
+//
+// One MMA is D[128 x 16] += A[128 x 16] * B[16 x 16]: 128 output positions, 16 output channels (a super-row),
+// 16 reduction elements (two taps of 8 input channels, or 16 input channels of a 1x1 layer).  That is the
+// smallest tile the instruction offers at M = 128, so the unit that can be skipped is a 16-channel x K-group
+// super-tile of W-bar; zeroed 8x8 blocks inside a stored super-tile are multiplied as zeros.
+//
+// A CTA owns 128 consecutive positions of one image and one group of 8 super-rows (128 channels, 128 fp32
+// TMEM columns).  Positions are counted over rows of the padded input width PW, so that the input of output
+// position m at tap (h, k) is the staged element m + h*PW + k: a tap is a constant offset, positions whose
+// column falls in the padding compute garbage and are not stored.  Activations are staged by tiled TMA loads
+// (out-of-bounds fill = zero padding) as planes [8-channel chunk][position][16 bytes], the no-swizzle K-major
+// core-matrix layout: 8 consecutive positions are one core matrix, the two K halves of an MMA are two planes
+// or two tap offsets (the descriptor's leading-dimension byte offset).  The stored super-tiles of the group
+// for the stage's K-groups are one contiguous stretch of the packed payload (one bulk copy).
+// Warp 0 produces, warps 1-3 issue MMAs for disjoint super-rows (accumulators in TMEM are addressed at run
+// time, so no code is specialised on the sparsity pattern), then all four warps read their TMEM lanes back,
+// add the bias and store.  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
+#include <cuda.h>
+#include <cstdlib>
+#include "bsp_internal.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kTcThreads = 128;
+constexpr int kIssuers = 3;
+constexpr int kTcMaxStages = 8;
+constexpr int kTcMaxSmem = 200 * 1024;
+constexpr int kTcMaxDevices = 64;
+constexpr int kTmemCols = 128;
+constexpr uint32_t kTcSpinLimit = 1u << 22;
+
+struct TcParams {
+    CUtensorMap tmap;        // activations as (16 bytes, x, y, n, chunk)
+    uint8_t *Y;
+    const float *bias;
+    const uint8_t *mask;
+    const uint32_t *off;
+    const uint32_t *gcnt;
+    const uint8_t *packed;     // start of the packed buffer; its header gives the super-tile payload's offset
+    int *status;
+    int N, O, M, Nw, P, H, K, ph, pw;
+    int PW, plane_bytes, tiles_per_img, is_gemm;
+    int n_kc, n_units, st_bytes, chunks_per_kc;
+    int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
+    int ytype;
+};
+
+__device__ __forceinline__ uint32_t s32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Shared-memory matrix descriptor, no swizzle, K-major: 8 rows x 16 bytes core matrices; `lbo` = bytes between
+// the two K halves, `sbo` = bytes between 8-row groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void commit_to(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_constant__ TcParams p)
+{
+    extern __shared__ __align__(16) uint8_t tc_smem_raw[];
+    uint8_t *smem = tc_smem_raw + ((128u - (s32(tc_smem_raw) & 127u)) & 127u);
+    __shared__ __align__(8) uint64_t s_full[kTcMaxStages];
+    __shared__ __align__(8) uint64_t s_empty[kTcMaxStages];
+    __shared__ __align__(8) uint64_t s_done;
+    __shared__ uint32_t s_tmem, s_touched, s_gbase, s_gcnt, s_fail;
+    __shared__ const uint8_t *s_payload;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = blockIdx.y;
+    const int S = p.stages;
+
+    // stored super-tiles of this group: masks and offsets of every K-group -> shared memory
+    uint32_t *s_off = (uint32_t *)smem;                      // [n_kc]
+    uint8_t *s_mask = smem + (size_t)p.n_kc * 4;             // [n_kc]
+    for (int i = tid; i < p.n_kc; i += kTcThreads) {
+        s_off[i] = p.off[(size_t)g * p.n_kc + i];
+        s_mask[i] = p.mask[(size_t)g * p.n_kc + i];
+    }
+    if (tid == 0) {
+        uint32_t base = 0;
+        for (int q = 0; q < g; ++q) base += p.gcnt[q];
+        s_gbase = base; s_gcnt = p.gcnt[g]; s_touched = 0; s_fail = 0;
+        s_payload = p.packed + ((const PackedHeader *)p.packed)->off_tc_payload;
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_full[s])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_empty[s])), "r"(kIssuers) : "memory");
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_done)), "r"(kIssuers) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(s32(&s_tmem)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const uint32_t tmem = s_tmem;
+
+    const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
+    const uint32_t ring = s32(smem) + meta_bytes;
+
+    // tile geometry
+    int n_img = 0, m0 = 0, y_first = 0, rowbase = 0;
+    if (p.is_gemm) { m0 = blockIdx.x * 128; }
+    else {
+        n_img = blockIdx.x / p.tiles_per_img;
+        m0 = (blockIdx.x % p.tiles_per_img) * 128;
+        y_first = m0 / p.PW;
+        rowbase = m0 - y_first * p.PW;
+    }
+
+    if (warp == 0) {
+        // ================= producer =================
+        if (lane == 0) {
+            for (int it = 0; it < p.n_stage_iters; ++it) {
+                const int slot = it % S;
+                if (it >= S && !wait_bar(s32(&s_empty[slot]), (uint32_t)((it / S - 1) & 1))) { atomicExch(&s_fail, 1u); break; }
+                const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
+                const uint32_t o_lo = s_off[kc0];
+                const uint32_t o_hi = (kc0 + nk < p.n_kc) ? s_off[kc0 + nk] : s_gcnt;
+                const uint32_t wbytes = (o_hi - o_lo) * (uint32_t)p.st_bytes;
+                const uint32_t bar = s32(&s_full[slot]);
+                const uint32_t dst = ring + slot * p.stage_bytes;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes + wbytes) : "memory");
+                const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first - p.ph, c3 = p.is_gemm ? m0 : n_img;
+                const int c4 = kc0 * p.chunks_per_kc;
+                asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+                             ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+                if (wbytes)
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                                 ::"r"(dst + p.act_bytes), "l"(s_payload + (size_t)(s_gbase + o_lo) * p.st_bytes), "r"(wbytes), "r"(bar) : "memory");
+            }
+        }
+    } else {
+        // ================= MMA issuers: warp w takes the super-rows r with r % kIssuers == w - 1 =================
+        const int me = warp - 1;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+        uint32_t touched = 0;
+        bool ok = true;
+        for (int it = 0; it < p.n_stage_iters && ok; ++it) {
+            const int slot = it % S;
+            if (!wait_bar(s32(&s_full[slot]), (uint32_t)((it / S) & 1))) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
+            const uint32_t stage = ring + slot * p.stage_bytes;
+            const uint32_t wbase = stage + p.act_bytes;
+            const uint32_t o_lo = s_off[kc0];
+            for (int kl = 0; kl < nk; ++kl) {
+                const uint32_t m = s_mask[kc0 + kl];
+                const uint32_t tile0 = s_off[kc0 + kl] - o_lo;
+                uint32_t mm = m;
+                while (mm) {
+                    const int r = __ffs(mm) - 1;
+                    mm &= mm - 1;
+                    if (r % kIssuers != me) continue;
+                    const uint32_t j = tile0 + __popc(m & ((1u << r) - 1u));
+                    for (int u = 0; u < p.n_units; ++u) {
+                        uint32_t a_addr, lbo;
+                        if (p.chunks_per_kc == 2) {       // 1x1 kernel: the K halves are two 8-channel planes
+                            a_addr = stage + (2 * kl) * p.plane_bytes + rowbase * 16;
+                            lbo = (uint32_t)p.plane_bytes;
+                        } else {
+                            const int t0 = 2 * u, t1 = 2 * u + 1;
+                            const int o0 = (t0 / p.K) * p.PW + t0 % p.K;
+                            a_addr = stage + kl * p.plane_bytes + (rowbase + o0) * 16;
+                            // a missing odd tap has zero weights; its K half reads the next position (finite data)
+                            lbo = (t1 < p.H * p.K) ? (uint32_t)(((t1 / p.K) * p.PW + t1 % p.K) - o0) * 16u : 16u;
+                        }
+                        const uint64_t adesc = smem_desc(a_addr, lbo, 128);
+                        const uint64_t bdesc = smem_desc(wbase + (j * p.n_units + u) * kTcUnitBytes, 256, 128);
+                        if (lane == 0) mma_bf16(tmem + (uint32_t)r * 16u, adesc, bdesc, idesc, (touched >> r) & 1u);
+                        touched |= 1u << r;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) commit_to(s32(&s_empty[slot]));
+        }
+        if (lane == 0) {
+            if (ok) { commit_to(s32(&s_done)); atomicOr(&s_touched, touched); }
+            else atomicExch(&s_fail, 1u);
+        }
+    }
+
+    // ================= epilogue: all four warps, TMEM lane = position =================
+    __syncwarp();
+    bool done = wait_bar(s32(&s_done), 0);
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (s_fail) done = false;
+    if (!done && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
+    if (done) {
+        const uint32_t touched = s_touched;
+        const int m = warp * 32 + lane;
+        bool valid;
+        size_t pix;
+        if (p.is_gemm) { valid = m0 + m < p.P; pix = (size_t)(m0 + m); }
+        else {
+            const int mm = m0 + m, y = mm / p.PW, x = mm % p.PW;
+            valid = y < p.M && x < p.Nw;
+            pix = ((size_t)n_img * p.M + y) * p.Nw + x;
+        }
+        const int oe = (p.ytype == BSP_BF16) ? 2 : 4;
+#pragma unroll 1
+        for (int r = 0; r < kTcGroupRows; ++r) {
+            const int ch = (g * kTcGroupRows + r) * kTcSuperRow;
+            if (ch >= p.O) break;
+            uint32_t v[16];
+            if ((touched >> r) & 1u) {
+                const uint32_t ta = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)r * 16u;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                             : "r"(ta) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0u;
+            }
+            if (!valid) continue;
+            const int nch = min(16, p.O - ch);        // 16, or 8 in a last half super-row
+            float f[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]) + ((p.bias != nullptr && e < nch) ? __ldg(p.bias + ch + e) : 0.f);
+            uint8_t *dst = p.Y + (pix * p.O + ch) * oe;
+            if (oe == 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (q * 4 < nch) *(float4 *)(dst + q * 16) = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+                    if (q * 8 < nch) {
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(f[8 * q], f[8 * q + 1]), h1 = __floats2bfloat162_rn(f[8 * q + 2], f[8 * q + 3]);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * q + 4], f[8 * q + 5]), h3 = __floats2bfloat162_rn(f[8 * q + 6], f[8 * q + 7]);
+                        *(uint4 *)(dst + q * 16) = make_uint4(*(uint32_t *)&h0, *(uint32_t *)&h1, *(uint32_t *)&h2, *(uint32_t *)&h3);
+                    }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tc_encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+}  // namespace
+
+// True if the tcgen05 kernel can run this layer: bf16, stride 1, super-tile form present, box extents in range.
+bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
+{
+    if (wd.wtype != BSP_BF16 || xd.stride_h != 1 || xd.stride_w != 1) return false;
+    const PackedLayout L = packed_layout(wd, 0);
+    if (!L.tc.enabled) return false;
+    const bool gemm = wd.H == 1 && wd.K == 1 && xd.L == 1 && xd.J == 1;
+    if (gemm) return true;
+    const int PW = xd.J + 2 * xd.pad_w;
+    const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
+    if (PW > 256 || R > 256) return false;
+    // one K-group of activations plus its dense weights must fit a stage, two stages the shared memory
+    const size_t per_kc = (size_t)R * PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + (size_t)kTcGroupRows * L.tc.st_bytes;
+    return 2 * per_kc + 16384 <= (size_t)kTcMaxSmem;
+}
+
+bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
+{
+    const PackedLayout L = packed_layout(wd, 0);
+    const TcLayout &T = L.tc;
+    const uint8_t *pk = (const uint8_t *)packed;
+    const bool gemm = wd.H == 1 && wd.K == 1 && xd.L == 1 && xd.J == 1;
+    TcParams p = {};
+    p.Y = (uint8_t *)Y; p.bias = (const float *)bias;
+    p.mask = pk + T.off_mask; p.off = (const uint32_t *)(pk + T.off_off); p.gcnt = (const uint32_t *)(pk + T.off_gcnt);
+    p.packed = pk; p.status = (int *)ws;
+    p.N = xd.N; p.O = wd.O; p.H = wd.H; p.K = wd.K; p.ph = xd.pad_h; p.pw = xd.pad_w;
+    p.M = xd.L + 2 * xd.pad_h - wd.H + 1; p.Nw = xd.J + 2 * xd.pad_w - wd.K + 1;
+    p.P = xd.N * p.M * p.Nw;
+    p.is_gemm = gemm ? 1 : 0;
+    p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch / 8;
+    int plane_pos, R = 1;
+    long long tiles;
+    if (gemm) {
+        p.PW = 1; plane_pos = 128; p.tiles_per_img = 0; tiles = ((long long)xd.N + 127) / 128;
+    } else {
+        p.PW = xd.J + 2 * xd.pad_w;
+        R = (wd.H * p.PW + 126 + wd.K - 1) / p.PW + 1;
+        plane_pos = R * p.PW;
+        p.tiles_per_img = (p.M * p.PW + 127) / 128;
+        tiles = (long long)xd.N * p.tiles_per_img;
+    }
+    p.plane_bytes = plane_pos * 16;
+    const size_t per_kc = (size_t)p.plane_bytes * p.chunks_per_kc + (size_t)kTcGroupRows * T.st_bytes;
+    int GK = (int)(49152 / per_kc);
+    if (GK < 1) GK = 1;
+    if (GK > T.n_kc) GK = T.n_kc;
+    if (GK * p.chunks_per_kc > 256) GK = 256 / p.chunks_per_kc;
+    p.GK = GK;
+    p.act_box_bytes = GK * p.chunks_per_kc * p.plane_bytes;
+    p.act_bytes = (int)align_up((size_t)p.act_box_bytes + 32, 128);      // + slack read by positions in the padding
+    p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)GK * kTcGroupRows * T.st_bytes, 128);
+    p.n_stage_iters = (T.n_kc + GK - 1) / GK;
+    const size_t meta = align_up((size_t)T.n_kc * 5, 128);
+    int stages = (int)(((size_t)kTcMaxSmem - meta - 256) / p.stage_bytes);
+    if (stages > kTcMaxStages) stages = kTcMaxStages;
+    if (stages > p.n_stage_iters) stages = p.n_stage_iters;
+    if (stages < 1) return BSP_ERR_SHAPE;
+    p.stages = stages;
+    p.ytype = ytype;
+    const size_t smem = meta + (size_t)stages * p.stage_bytes + 256;
+
+    EncodeTiledFn enc = tc_encode_tiled();
+    if (!enc) return BSP_ERR_CUDA;
+    const cuuint64_t row = (cuuint64_t)wd.I * 2;
+    const cuuint64_t gdim[5] = {16, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N, (cuuint64_t)(wd.I / 8)};
+    const cuuint64_t gstr[4] = {row, row * xd.J, row * xd.J * xd.L, 16};
+    cuuint32_t box[5];
+    if (gemm) { box[0] = 16; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
+    else { box[0] = 16; box[1] = (cuuint32_t)p.PW; box[2] = (cuuint32_t)R; box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    if (enc(&p.tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void *>(X), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return BSP_ERR_CUDA;
+
+    static bool opted[kTcMaxDevices] = {};
+    int dev = 0;
+    BSP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kTcMaxDevices) return BSP_ERR_CUDA;
+    if (!opted[dev]) {
+        BSP_CUDA_OK(cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem));
+        opted[dev] = true;
+    }
+    dim3 grid((unsigned)tiles, (unsigned)T.n_groups);
+    conv_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // namespace bsp

@@ -29,6 +29,7 @@ struct PackedHeader {
     int32_t off_coloff;
     int32_t off_panelbase;
     int64_t off_payload;
+    int64_t off_tc_payload;  // start of the super-tile payload (depends on the capacity the buffer was sized for)
 };
 
 // Second packed form, for the tcgen05 kernel (bf16 only): W-bar is cut into super-tiles of 16 output channels
@@ -81,6 +82,10 @@ bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *pac
 
 // A failed CUDA call becomes BSP_ERR_CUDA; with BSP_DEBUG set in the environment its text goes to stderr.
 void report_cuda_error(cudaError_t e, const char *expr, const char *file, int line);
+
+bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd);
+bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
 
 #define BSP_CUDA_OK(expr)                                            \
     do {                                                             \

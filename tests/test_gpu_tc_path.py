@@ -1,0 +1,81 @@
+"""GPU parity of the tcgen05 kernel (bf16, stride 1), selected with BSP_CONV_PATH=tc, against the CPU oracle."""
+import numpy as np
+import pytest
+
+from oracle import ref
+from paper_2407_09453_b200 import synth
+from gpu_util import gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_bias, make_case, make_x
+from test_gpu_product import check, run_conv_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def tc_path(monkeypatch):
+    monkeypatch.setenv("BSP_CONV_PATH", "tc")
+
+
+TC_CASES = [  # O, I, H, K, pad, spatial, batch
+    (256, 256, 3, 3, (1, 1), (14, 14), 3), (64, 64, 1, 1, (0, 0), (9, 7), 3), (128, 64, 5, 5, (2, 2), (11, 13), 2),
+    (64, 64, 1, 7, (0, 3), (17, 17), 2), (64, 64, 7, 1, (3, 0), (17, 17), 2), (64, 32, 3, 3, (0, 0), (12, 12), 2),
+    (48, 24, 3, 3, (1, 1), (6, 150), 1), (1000, 64, 1, 1, (0, 0), (3, 5), 2), (136, 128, 3, 3, (1, 1), (28, 28), 2),
+]
+
+
+@pytest.mark.parametrize("O,I,H,K,pad,sp,batch", TC_CASES)
+def test_tc_conv_shapes(O, I, H, K, pad, sp, batch):
+    run_conv_case(601 + O + H, O, I, H, K, 8, 8, "bf16", (batch, sp[0], sp[1], I), (1, 1), pad)
+
+
+@pytest.mark.parametrize("bo,bi", [(4, 16), (16, 4)])
+def test_tc_other_block_shapes(bo, bi):
+    run_conv_case(611, 96, 80, 3, 3, bo, bi, "bf16", (2, 10, 12, 80), (1, 1), (1, 1))
+
+
+@pytest.mark.parametrize("frac", [0.0, 0.25, 0.75, 1.0])
+def test_tc_sparsity_extremes_and_bf16_output(frac):
+    run_conv_case(621, 128, 128, 3, 3, 8, 8, "bf16", (2, 8, 8, 128), (1, 1), (1, 1), frac, out="bf16")
+
+
+@pytest.mark.parametrize("bo,bi", [(8, 8), (4, 16), (16, 4)])
+def test_tc_gemm_ragged(bo, bi):
+    O, I, P = 192, 256, 333
+    W = make_case(631, O, I, 1, 1, "bf16")
+    gamma = synth.random_gamma(632, O // bo, I // bi, (O // bo) * (I // bi) // 2)
+    X = make_x(633, (P, I), "bf16")
+    b = make_bias(634, O, "bf16")
+    lay = gpu_layer(W, gamma, bo, bi, "bf16")
+    got = gpu_gemm(lay, X, b, "bf16")
+    rp, ci, pl = ref.compact(W, gamma, bo, bi)
+    want = ref.gemm(O, I, bo, bi, rp, ci, pl.reshape(-1, bo, bi), X, b)
+    check(got, want, "bf16")
+
+
+def test_tc_config_resnet_conv_with_l2_gamma():
+    layer = synth.Layer("cfg2", 256, 256, 3, 3, 32, 14, 14, 1, 1, 1, 1)
+    W, X, b = synth.make_layer_tensors(layer, "bf16", config=2)
+    g, s, lay, Wd = gpu_mask(W, 8, 8, "bf16", 512)
+    lay.compact(Wd)
+    lay.check()
+    got = gpu_conv(lay, X, b, "bf16", (1, 1), (1, 1))
+    want_g = ref.mask(ref.scores(W, 8, 8), 512)
+    rp, ci, pl = ref.compact(W, want_g, 8, 8)
+    want = ref.conv2d(W.shape, 8, 8, rp, ci, pl, X, b, (1, 1), (1, 1))
+    check(got, want, "bf16")
+
+
+def test_tc_config_gemm_4096_sampled_rows():
+    O = I = 4096
+    P = 8192
+    W = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 0), (O, 1, 1, I), 1 / 64.0).astype(np.float32))
+    X = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 1), (P, I)).astype(np.float32))
+    b = synth.normal(synth.tensor_seed(3, 0, 2), (O,), 0.1).astype(np.float32)
+    NB = (O // 8) * (I // 8)
+    g, s, lay, Wd = gpu_mask(W, 8, 8, "bf16", NB // 2)
+    lay.compact(Wd)
+    lay.check()
+    got = gpu_gemm(lay, X, b, "bf16")
+    pix = np.r_[0, 127, 128, P - 1, synth.uniform_int(7, (28,), 0, P - 1)]
+    rp, ci, pl = ref.compact(W, g, 8, 8)
+    want = ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b, pix=pix)
+    check(got[pix], want, "bf16")
