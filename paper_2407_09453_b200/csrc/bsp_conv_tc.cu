@@ -89,6 +89,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     __shared__ __align__(8) uint64_t s_done;
     __shared__ uint32_t s_tmem, s_touched, s_gbase, s_gcnt, s_fail;
     __shared__ const uint8_t *s_payload;
+    __shared__ uint64_t s_ahi[64];          // per K-step of a super-tile: A descriptor without its address field
+    __shared__ uint32_t s_aoff[64];         // ... and the operand's offset from the K-group's first plane, in 16-byte units
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = blockIdx.y;
@@ -113,6 +115,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_done)), "r"(kIssuers) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
+    // tile geometry
+    int n_img = 0, m0 = 0, y_first = 0, rowbase = 0;
+    if (p.is_gemm) { m0 = blockIdx.x * 128; }
+    else {
+        n_img = blockIdx.x / p.tiles_per_img;
+        m0 = (blockIdx.x % p.tiles_per_img) * 128;
+        y_first = m0 / p.PW;
+        rowbase = m0 - y_first * p.PW;
+    }
+    for (int u = tid; u < p.n_units; u += kTcThreads) {
+        uint32_t lbo, off;
+        if (p.chunks_per_kc == 2) {                 // 1x1 kernel: the K halves are two 8-channel planes
+            off = (uint32_t)rowbase;
+            lbo = (uint32_t)p.plane_bytes;
+        } else {
+            const int t0 = 2 * u, t1 = 2 * u + 1;
+            const int o0 = (t0 / p.K) * p.PW + t0 % p.K;
+            off = (uint32_t)(rowbase + o0);
+            // a missing odd tap has zero weights; its K half reads the next position (finite data)
+            lbo = (t1 < p.H * p.K) ? (uint32_t)(((t1 / p.K) * p.PW + t1 % p.K) - o0) * 16u : 16u;
+        }
+        s_aoff[u] = off;
+        s_ahi[u] = smem_desc(0, lbo, 128);
+    }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(s32(&s_tmem)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
@@ -124,16 +150,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
 
     const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
     const uint32_t ring = s32(smem) + meta_bytes;
-
-    // tile geometry
-    int n_img = 0, m0 = 0, y_first = 0, rowbase = 0;
-    if (p.is_gemm) { m0 = blockIdx.x * 128; }
-    else {
-        n_img = blockIdx.x / p.tiles_per_img;
-        m0 = (blockIdx.x % p.tiles_per_img) * 128;
-        y_first = m0 / p.PW;
-        rowbase = m0 - y_first * p.PW;
-    }
 
     if (warp == 0) {
         // ================= producer =================
@@ -159,50 +175,68 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         }
     } else {
         // ================= MMA issuers: warp w takes the super-rows r with r % kIssuers == w - 1 =================
-        const int me = warp - 1;
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
-        uint32_t touched = 0;
-        bool ok = true;
-        for (int it = 0; it < p.n_stage_iters && ok; ++it) {
-            const int slot = it % S;
-            if (!wait_bar(s32(&s_full[slot]), (uint32_t)((it / S) & 1))) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
-            const uint32_t stage = ring + slot * p.stage_bytes;
-            const uint32_t wbase = stage + p.act_bytes;
-            const uint32_t o_lo = s_off[kc0];
-            for (int kl = 0; kl < nk; ++kl) {
-                const uint32_t m = s_mask[kc0 + kl];
-                const uint32_t tile0 = s_off[kc0 + kl] - o_lo;
-                uint32_t mm = m;
-                while (mm) {
-                    const int r = __ffs(mm) - 1;
-                    mm &= mm - 1;
-                    if (r % kIssuers != me) continue;
-                    const uint32_t j = tile0 + __popc(m & ((1u << r) - 1u));
-                    for (int u = 0; u < p.n_units; ++u) {
-                        uint32_t a_addr, lbo;
-                        if (p.chunks_per_kc == 2) {       // 1x1 kernel: the K halves are two 8-channel planes
-                            a_addr = stage + (2 * kl) * p.plane_bytes + rowbase * 16;
-                            lbo = (uint32_t)p.plane_bytes;
-                        } else {
-                            const int t0 = 2 * u, t1 = 2 * u + 1;
-                            const int o0 = (t0 / p.K) * p.PW + t0 % p.K;
-                            a_addr = stage + kl * p.plane_bytes + (rowbase + o0) * 16;
-                            // a missing odd tap has zero weights; its K half reads the next position (finite data)
-                            lbo = (t1 < p.H * p.K) ? (uint32_t)(((t1 / p.K) * p.PW + t1 % p.K) - o0) * 16u : 16u;
+        // One thread per issuing warp runs the whole issue loop: a tcgen05.mma is issued by a single thread, and
+        // keeping that thread in one long non-divergent stretch avoids a divergence region around every MMA.
+        if (lane == 0) {
+            const int me = warp - 1;
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+            // Descriptors are sums: the address field (16-byte units, low 14 bits) of an A operand is
+            // stage + plane + s_aoff[u], of a B operand weights + 32 * (tile * n_units + u); the other fields are
+            // per-unit (A: the byte offset between the K halves) or constant (B).
+            const uint64_t b_hi = smem_desc(0, 256, 128);
+            const int plane16 = (p.plane_bytes >> 4) * p.chunks_per_kc;  // 16-byte units between K-groups' planes
+            const int nu = p.n_units;
+            const uint64_t ahi0 = s_ahi[0];
+            const uint32_t aoff0 = s_aoff[0];
+            uint32_t touched = 0;
+            bool ok = true;
+            for (int it = 0; it < p.n_stage_iters && ok; ++it) {
+                const int slot = it % S;
+                if (!wait_bar(s32(&s_full[slot]), (uint32_t)((it / S) & 1))) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
+                const uint32_t stage16 = (ring + slot * p.stage_bytes) >> 4;
+                const uint32_t w16 = stage16 + (p.act_bytes >> 4);
+                const uint32_t o_lo = s_off[kc0];
+                for (int kl = 0; kl < nk; ++kl) {
+                    const uint32_t m = s_mask[kc0 + kl];
+                    uint32_t mine = m & (0x49u << me);       // this warp's rows: me, me + 3, me + 6
+                    if (mine == 0) continue;
+                    const uint32_t tile0 = s_off[kc0 + kl] - o_lo;
+                    const uint32_t a16 = stage16 + kl * plane16;
+                    if (nu == 1) {
+                        const uint64_t adesc = ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu);
+                        while (mine) {
+                            const int r = __ffs(mine) - 1;
+                            mine &= mine - 1;
+                            const uint32_t b16 = w16 + (tile0 + __popc(m & ((1u << r) - 1u))) * 32u;
+                            mma_bf16(tmem + (uint32_t)r * 16u, adesc, b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, (touched >> r) & 1u);
+                            touched |= 1u << r;
                         }
-                        const uint64_t adesc = smem_desc(a_addr, lbo, 128);
-                        const uint64_t bdesc = smem_desc(wbase + (j * p.n_units + u) * kTcUnitBytes, 256, 128);
-                        if (lane == 0) mma_bf16(tmem + (uint32_t)r * 16u, adesc, bdesc, idesc, (touched >> r) & 1u);
-                        touched |= 1u << r;
+                    } else {
+                        // up to three rows: destination, first weight tile and accumulate flag of each
+                        uint32_t d[3], b16[3], acc[3];
+                        int nr = 0;
+                        while (mine) {
+                            const int r = __ffs(mine) - 1;
+                            mine &= mine - 1;
+                            d[nr] = tmem + (uint32_t)r * 16u;
+                            b16[nr] = w16 + (tile0 + __popc(m & ((1u << r) - 1u))) * (uint32_t)nu * 32u;
+                            acc[nr] = (touched >> r) & 1u;
+                            touched |= 1u << r;
+                            ++nr;
+                        }
+                        for (int u = 0; u < nu; ++u) {
+                            const uint64_t adesc = s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu);
+                            const uint32_t bo = (uint32_t)u * 32u;
+                            if (nr > 0) mma_bf16(d[0], adesc, b_hi | (uint64_t)((b16[0] + bo) & 0x3FFFu), idesc, acc[0] | (uint32_t)(u > 0));
+                            if (nr > 1) mma_bf16(d[1], adesc, b_hi | (uint64_t)((b16[1] + bo) & 0x3FFFu), idesc, acc[1] | (uint32_t)(u > 0));
+                            if (nr > 2) mma_bf16(d[2], adesc, b_hi | (uint64_t)((b16[2] + bo) & 0x3FFFu), idesc, acc[2] | (uint32_t)(u > 0));
+                        }
                     }
                 }
+                commit_to(s32(&s_empty[slot]));
             }
-            __syncwarp();
-            if (lane == 0) commit_to(s32(&s_empty[slot]));
-        }
-        if (lane == 0) {
             if (ok) { commit_to(s32(&s_done)); atomicOr(&s_touched, touched); }
             else atomicExch(&s_fail, 1u);
         }
