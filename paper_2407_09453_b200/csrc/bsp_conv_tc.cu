@@ -15,9 +15,9 @@
 // core-matrix layout: 8 consecutive positions are one core matrix, the two K halves of an MMA are two planes
 // or two tap offsets (the descriptor's leading-dimension byte offset).  The stored super-tiles of the group
 // for the stage's K-groups are one contiguous stretch of the packed payload (one bulk copy).
-// Warp 0 produces, warps 1-3 issue MMAs for disjoint super-rows (accumulators in TMEM are addressed at run
-// time, so no code is specialised on the sparsity pattern), then all four warps read their TMEM lanes back,
-// add the bias and store.  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
+// Warps 0-7 each issue the MMAs of one super-row (an MMA this small costs more to issue than to execute, so the
+// issue is spread over eight threads; accumulators in TMEM are addressed at run time, so no code is specialised
+// on the sparsity pattern), warp 8 produces; then the eight warps read their TMEM lanes back, add the bias and store.  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
 #include <cuda.h>
 #include <cstdlib>
 #include "bsp_internal.cuh"
@@ -25,8 +25,8 @@
 namespace bsp {
 namespace {
 
-constexpr int kTcThreads = 128;
-constexpr int kIssuers = 3;
+constexpr int kIssuers = 8;                       // one issuing warp per super-row of the group
+constexpr int kTcThreads = 32 * (kIssuers + 1);   // + the producer warp
 constexpr int kTcMaxStages = 8;
 constexpr int kTcMaxSmem = 200 * 1024;
 constexpr int kTcMaxDevices = 64;
@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
     const uint32_t ring = s32(smem) + meta_bytes;
 
-    if (warp == 0) {
+    if (warp == kIssuers) {
         // ================= producer =================
         if (lane == 0) {
             for (int it = 0; it < p.n_stage_iters; ++it) {
@@ -174,11 +174,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             }
         }
     } else {
-        // ================= MMA issuers: warp w takes the super-rows r with r % kIssuers == w - 1 =================
+        // ================= MMA issuers: warp r owns super-row r =================
         // One thread per issuing warp runs the whole issue loop: a tcgen05.mma is issued by a single thread, and
         // keeping that thread in one long non-divergent stretch avoids a divergence region around every MMA.
         if (lane == 0) {
-            const int me = warp - 1;
+            const uint32_t r = (uint32_t)warp;
+            const uint32_t below = (1u << r) - 1u;
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
             // Descriptors are sums: the address field (16-byte units, low 14 bits) of an A operand is
             // stage + plane + s_aoff[u], of a B operand weights + 32 * (tile * n_units + u); the other fields are
@@ -188,9 +189,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             const int nu = p.n_units;
             const uint64_t ahi0 = s_ahi[0];
             const uint32_t aoff0 = s_aoff[0];
-            uint32_t touched = 0;
+            const uint32_t d = tmem + r * 16u;
+            uint32_t acc = 0;
             bool ok = true;
-            for (int it = 0; it < p.n_stage_iters && ok; ++it) {
+            for (int it = 0; it < p.n_stage_iters; ++it) {
                 const int slot = it % S;
                 if (!wait_bar(s32(&s_full[slot]), (uint32_t)((it / S) & 1))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -200,49 +202,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t o_lo = s_off[kc0];
                 for (int kl = 0; kl < nk; ++kl) {
                     const uint32_t m = s_mask[kc0 + kl];
-                    uint32_t mine = m & (0x49u << me);       // this warp's rows: me, me + 3, me + 6
-                    if (mine == 0) continue;
-                    const uint32_t tile0 = s_off[kc0 + kl] - o_lo;
+                    if (!((m >> r) & 1u)) continue;
+                    const uint32_t tile = s_off[kc0 + kl] - o_lo + __popc(m & below);
                     const uint32_t a16 = stage16 + kl * plane16;
                     if (nu == 1) {
-                        const uint64_t adesc = ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu);
-                        while (mine) {
-                            const int r = __ffs(mine) - 1;
-                            mine &= mine - 1;
-                            const uint32_t b16 = w16 + (tile0 + __popc(m & ((1u << r) - 1u))) * 32u;
-                            mma_bf16(tmem + (uint32_t)r * 16u, adesc, b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, (touched >> r) & 1u);
-                            touched |= 1u << r;
-                        }
+                        mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)((w16 + tile * 32u) & 0x3FFFu), idesc, acc);
                     } else {
-                        // up to three rows: destination, first weight tile and accumulate flag of each
-                        uint32_t d[3], b16[3], acc[3];
-                        int nr = 0;
-                        while (mine) {
-                            const int r = __ffs(mine) - 1;
-                            mine &= mine - 1;
-                            d[nr] = tmem + (uint32_t)r * 16u;
-                            b16[nr] = w16 + (tile0 + __popc(m & ((1u << r) - 1u))) * (uint32_t)nu * 32u;
-                            acc[nr] = (touched >> r) & 1u;
-                            touched |= 1u << r;
-                            ++nr;
-                        }
+                        uint32_t b16 = w16 + tile * (uint32_t)nu * 32u;
                         for (int u = 0; u < nu; ++u) {
-                            const uint64_t adesc = s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu);
-                            const uint32_t bo = (uint32_t)u * 32u;
-                            if (nr > 0) mma_bf16(d[0], adesc, b_hi | (uint64_t)((b16[0] + bo) & 0x3FFFu), idesc, acc[0] | (uint32_t)(u > 0));
-                            if (nr > 1) mma_bf16(d[1], adesc, b_hi | (uint64_t)((b16[1] + bo) & 0x3FFFu), idesc, acc[1] | (uint32_t)(u > 0));
-                            if (nr > 2) mma_bf16(d[2], adesc, b_hi | (uint64_t)((b16[2] + bo) & 0x3FFFu), idesc, acc[2] | (uint32_t)(u > 0));
+                            mma_bf16(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, acc | (uint32_t)(u > 0));
+                            b16 += 32u;
                         }
                     }
+                    acc = 1u;
                 }
                 commit_to(s32(&s_empty[slot]));
             }
-            if (ok) { commit_to(s32(&s_done)); atomicOr(&s_touched, touched); }
+            if (ok) { commit_to(s32(&s_done)); if (acc) atomicOr(&s_touched, 1u << r); }
             else atomicExch(&s_fail, 1u);
         }
     }
 
-    // ================= epilogue: all four warps, TMEM lane = position =================
+    // ================= epilogue: warps 0-7; warp w reads TMEM lanes 32*(w%4).. (positions) of super-rows 4*(w/4).. =================
     __syncwarp();
     bool done = wait_bar(s32(&s_done), 0);
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -251,7 +232,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     if (!done && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
     if (done) {
         const uint32_t touched = s_touched;
-        const int m = warp * 32 + lane;
+        const int lq = warp & 3;                 // a warp reaches the TMEM lanes of its quarter only
+        const int m = lq * 32 + lane;
         bool valid;
         size_t pix;
         if (p.is_gemm) { valid = m0 + m < p.P; pix = (size_t)(m0 + m); }
@@ -262,12 +244,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         }
         const int oe = (p.ytype == BSP_BF16) ? 2 : 4;
 #pragma unroll 1
-        for (int r = 0; r < kTcGroupRows; ++r) {
+        for (int r = (warp >> 2) * 4; r < (warp >> 2) * 4 + 4 && warp < kIssuers; ++r) {
             const int ch = (g * kTcGroupRows + r) * kTcSuperRow;
             if (ch >= p.O) break;
             uint32_t v[16];
             if ((touched >> r) & 1u) {
-                const uint32_t ta = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)r * 16u;
+                const uint32_t ta = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)r * 16u;
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
                              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
                                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
