@@ -14,8 +14,9 @@
  *    bsp_bcsr structs) are HOST structs read during the call.  The library allocates no device memory:
  *    scratch comes from the caller's workspace `ws` (device, 256-byte aligned), sized by the matching
  *    *_workspace_bytes() call.  The caller zero-fills the first 256 bytes of a workspace once after
- *    allocating it (they hold the latched status word); one workspace sized for the largest request
- *    may serve all calls issued on one stream.
+ *    allocating it (they hold the latched status word and the counters of the grid-wide barrier that the
+ *    single-launch kernels of small layers use); one workspace sized for the largest request may serve all
+ *    calls issued on one stream, and a workspace must not be shared by calls running on different streams.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue work and
  *    return; results are valid once the stream has been synchronised.
  *  - Every function returns a bsp_status; nothing throws.  Argument errors are detected on the host

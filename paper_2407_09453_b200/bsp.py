@@ -152,9 +152,11 @@ def bsp_check(ws, stream=None):
 
 
 def launches_per_step(wd: WDesc) -> int:
-    """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass: score, select; count, scan,
-    fill+pack; the product kernel."""
-    return 6
+    """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass.  General path: score, select;
+    count, scan, fill+pack; the product kernel.  Small layers take one launch for the mask (up to 2048 blocks) and
+    one for the compaction (up to 4096 blocks)."""
+    nb = (wd.O // wd.bo) * (wd.I // wd.bi)
+    return (1 if nb <= 2048 else 2) + (1 if nb <= 4096 else 3) + 1
 
 
 class SparseLayer:

@@ -68,7 +68,7 @@ bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope
     const int64_t limit = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
     if (n_zero < 0 || n_zero > limit) return BSP_ERR_CAPACITY;
     void *scores = scores_opt ? scores_opt : (void *)((char *)ws + kWsHeader);
-    return launch_mask(*wd, W, norm, scope, n_zero, gamma, scores, (cudaStream_t)stream);
+    return launch_mask(*wd, W, norm, scope, n_zero, gamma, scores, ws, (cudaStream_t)stream);
 }
 
 size_t bsp_packed_bytes(const bsp_wdesc *wd, int64_t nnz)

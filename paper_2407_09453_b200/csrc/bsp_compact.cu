@@ -208,18 +208,18 @@ scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_
 }
 
 // Final launch, first part.  `parts` CTAs per row of Gamma: column indices in ascending order and the canonical payload
-// payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].
+// payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].  `first` = stored blocks in the rows above; returns
+// the number of stored blocks of row l.
 template <typename T>
-__device__ __forceinline__ void csr_fill_body(int l, int part, int parts, const T *__restrict__ W,
+__device__ __forceinline__ int csr_fill_body(int l, int part, int parts, const T *__restrict__ W,
                                               const uint8_t *__restrict__ gamma, int NBi, int I, int HK, int bo, int bi,
-                                              const int32_t *__restrict__ row_ptr, int32_t *__restrict__ col_idx,
+                                              int first, int32_t *__restrict__ col_idx,
                                               T *__restrict__ payload, long long capacity_blocks)
 {
     __shared__ int warp_sums[kThreads / 32];
     __shared__ int s_run;
     extern __shared__ int s_cols[];      // NBi ints: columns of this row's stored blocks
     const uint8_t *g = gamma + (size_t)l * NBi;
-    const int first = row_ptr[l];
     if (threadIdx.x == 0) s_run = 0;
     __syncthreads();
     for (int base = 0; base < NBi; base += kThreads) {
@@ -236,21 +236,36 @@ __device__ __forceinline__ void csr_fill_body(int l, int part, int parts, const 
         if (threadIdx.x == 0) s_run += tot;
         __syncthreads();
     }
-    if (payload == nullptr) return;
+    if (payload == nullptr) return s_run;
     const int cnt = s_run;
     const int blk = bo * HK * bi;
     const long long total = (long long)cnt * blk;
-    // the CTAs of one row (`parts` of them) all build the column list, then share the copy
-    for (long long e = (long long)part * kThreads + threadIdx.x; e < total; e += (long long)parts * kThreads) {
-        const int n = (int)(e / blk);
-        const int q = (int)(e % blk);
-        int rem = q;
-        const int c = rem % bi; rem /= bi;
-        const int t = rem % HK;
-        const int r = rem / HK;
-        if ((long long)(first + n) >= capacity_blocks) continue;
-        payload[(size_t)(first + n) * blk + q] = W[((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi + c];
+    // the CTAs of one row (`parts` of them) all build the column list, then share the copy; the loads of four
+    // elements are issued before the first store
+    const long long stride = (long long)parts * kThreads;
+    for (long long e0 = (long long)part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+        T v[4];
+        size_t dst[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long e = e0 + u * stride;
+            ok[u] = e < total;
+            const int n = ok[u] ? (int)(e / blk) : 0;
+            const int q = ok[u] ? (int)(e % blk) : 0;
+            int rem = q;
+            const int c = rem % bi; rem /= bi;
+            const int t = rem % HK;
+            const int r = rem / HK;
+            ok[u] = ok[u] && (long long)(first + n) < capacity_blocks;
+            dst[u] = (size_t)(first + n) * blk + q;
+            v[u] = ok[u] ? W[((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi + c] : (T)0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (ok[u]) payload[dst[u]] = v[u];
     }
+    return cnt;
 }
 
 // One 32-bit word of a packed tile.  The tile at (tile row of the panel, tile column) holds, for every K-step
@@ -298,8 +313,40 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
     }
 }
 
-// Final launch, second part.  One CTA per (tile-column chunk, panel): every stored tile of the panel in this chunk of columns is
-// written word by word.
+// The stored tiles of one (panel, tile column), whose tile rows are the set bits of m, written word by word
+// from slot `first` on.  `parts` CTAs share the words; each thread loads four before it stores.
+template <int DT>
+__device__ __forceinline__ void pack_tiles(unsigned m, unsigned first, int panel, int col, const void *__restrict__ W,
+                                           const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi, int NBi,
+                                           int tile_bytes, uint8_t *__restrict__ payload, long long capacity_tiles,
+                                           int part, int parts)
+{
+    const int words = tile_bytes / 4;
+    const int total = __popc(m) * words;
+    const int stride = parts * kThreads;
+    for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+        uint32_t v[4];
+        uint32_t *dst[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = e0 + u * stride;
+            ok[u] = e < total;
+            const int j = ok[u] ? e / words : 0, word = ok[u] ? e % words : 0;
+            unsigned mm = m;                         // j-th set bit of m = tile row
+            for (int q = 0; q < j; ++q) mm &= mm - 1;
+            const int R = __ffs(mm) - 1;
+            ok[u] = ok[u] && (long long)(first + j) < capacity_tiles;
+            dst[u] = (uint32_t *)(payload + (size_t)(first + j) * tile_bytes) + word;
+            v[u] = ok[u] ? packed_word<DT>(W, gamma, word, (panel * kPanelRows + R) * kTile, col * kTile, O, I, HK, bo, bi, NBi) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (ok[u]) *dst[u] = v[u];
+    }
+}
+
+// Final launch, second part.  One CTA per (tile-column chunk, panel): every stored tile of the panel in this chunk of columns.
 template <int DT>
 __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__restrict__ W,
                                           const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi, int NBi,
@@ -309,23 +356,12 @@ __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__re
 {
     const int col_lo = chunk * cols_per_cta;
     const int col_hi = min(n_cols, col_lo + cols_per_cta);
-    const int words = tile_bytes / 4;
     const unsigned base = panel_base[panel];
     for (int col = col_lo; col < col_hi; ++col) {
         const unsigned m = colmask[(size_t)panel * n_cols + col];
         if (!m) continue;
-        const unsigned first = base + coloff[(size_t)panel * n_cols + col];
-        const int cnt = __popc(m);
-        for (int e = threadIdx.x; e < cnt * words; e += kThreads) {
-            const int j = e / words, word = e % words;
-            unsigned mm = m;                         // j-th set bit of m = tile row
-            for (int q = 0; q < j; ++q) mm &= mm - 1;
-            const int R = __ffs(mm) - 1;
-            if ((long long)(first + j) >= capacity_tiles) continue;
-            const uint32_t v = packed_word<DT>(W, gamma, word, (panel * kPanelRows + R) * kTile, col * kTile, O, I, HK,
-                                               bo, bi, NBi);
-            ((uint32_t *)(payload + (size_t)(first + j) * tile_bytes))[word] = v;
-        }
+        pack_tiles<DT>(m, base + coloff[(size_t)panel * n_cols + col], panel, col, W, gamma, O, I, HK, bo, bi, NBi,
+                       tile_bytes, payload, capacity_tiles, 0, 1);
     }
 }
 
@@ -355,6 +391,37 @@ struct TcPackArgs {
     int *status;
 };
 
+// The stored super-tiles of one (group, K-group), whose super-rows are the set bits of m, from slot `first` on.
+// `parts` CTAs share the words; each thread loads four before it stores.
+__device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g, int kc, const TcPackArgs &t,
+                                              const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I,
+                                              int HK, int bo, int bi, int NBi, int part, int parts)
+{
+    const int words = t.st_bytes / 4;
+    const int total = __popc(m) * words;
+    const int stride = parts * kThreads;
+    for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+        uint32_t v[4];
+        uint32_t *dst[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = e0 + u * stride;
+            ok[u] = e < total;
+            const int j = ok[u] ? e / words : 0, word = ok[u] ? e % words : 0;
+            unsigned mm = m;
+            for (int q = 0; q < j; ++q) mm &= mm - 1;
+            const int R = __ffs(mm) - 1;
+            ok[u] = ok[u] && (long long)(first + j) < t.capacity;
+            dst[u] = (uint32_t *)(t.payload + (size_t)(first + j) * t.st_bytes) + word;
+            v[u] = ok[u] ? tc_word((const uint16_t *)W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (ok[u]) *dst[u] = v[u];
+    }
+}
+
 __device__ __forceinline__ void tc_pack_body(int chunk, int g, const TcPackArgs &t, const void *__restrict__ W,
                                              const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
                                              int NBi)
@@ -364,21 +431,10 @@ __device__ __forceinline__ void tc_pack_body(int chunk, int g, const TcPackArgs 
     if (chunk == 0 && threadIdx.x == 0 && (long long)(base + t.gcnt[g]) > t.capacity)
         atomicMax(t.status, (int)BSP_ERR_CAPACITY);
     const int kc_lo = chunk * t.kc_per_cta, kc_hi = min(t.n_kc, kc_lo + t.kc_per_cta);
-    const int words = t.st_bytes / 4;
     for (int kc = kc_lo; kc < kc_hi; ++kc) {
         const unsigned m = t.mask[(size_t)g * t.n_kc + kc];
         if (!m) continue;
-        const unsigned first = base + t.off[(size_t)g * t.n_kc + kc];
-        const int cnt = __popc(m);
-        for (int e = threadIdx.x; e < cnt * words; e += kThreads) {
-            const int j = e / words, word = e % words;
-            unsigned mm = m;
-            for (int q = 0; q < j; ++q) mm &= mm - 1;
-            const int R = __ffs(mm) - 1;
-            if ((long long)(first + j) >= t.capacity) continue;
-            ((uint32_t *)(t.payload + (size_t)(first + j) * t.st_bytes))[word] =
-                tc_word((const uint16_t *)W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi);
-        }
+        tc_pack_tiles(m, base + t.off[(size_t)g * t.n_kc + kc], g, kc, t, W, gamma, O, I, HK, bo, bi, NBi, 0, 1);
     }
 }
 
@@ -397,6 +453,17 @@ struct FillPackArgs {
     uint8_t *packed_payload;          // NULL: no packed form
     long long capacity_tiles;
     TcPackArgs tc;                    // tc.n_groups == 0: no second packed form
+    // used by the single-launch kernel only, which also writes what the count and scan launches write
+    int32_t *row_ptr_out;
+    uint8_t *colmask_out;
+    uint32_t *coloff_out, *panel_base_out;
+    PackedHeader *hdr;
+    PackedHeader hdr_init;
+    uint8_t *tc_mask_out;
+    uint32_t *tc_off_out, *tc_gcnt_out;
+    int tc_kc_ch;
+    int pack_parts, tc_parts;         // CTAs sharing the words of one tile column / one K-group
+    int *status;
 };
 
 // The last compaction launch: CTAs [0, NBo * fill_parts) write col_idx and the canonical payload, the rest write
@@ -406,8 +473,9 @@ __global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs 
 {
     const int n_fill = a.NBo * a.fill_parts;
     if ((int)blockIdx.x < n_fill) {
-        csr_fill_body<T>((int)blockIdx.x / a.fill_parts, (int)blockIdx.x % a.fill_parts, a.fill_parts, (const T *)a.W,
-                         a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, a.row_ptr, a.col_idx, (T *)a.payload, a.capacity_blocks);
+        const int l = (int)blockIdx.x / a.fill_parts;
+        csr_fill_body<T>(l, (int)blockIdx.x % a.fill_parts, a.fill_parts, (const T *)a.W, a.gamma, a.NBi, a.I, a.HK, a.bo,
+                         a.bi, a.row_ptr[l], a.col_idx, (T *)a.payload, a.capacity_blocks);
     } else {
         const int b = (int)blockIdx.x - n_fill;
         const int n_pack = a.packed_payload ? a.pack_chunks * a.n_panels : 0;
@@ -418,6 +486,147 @@ __global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs 
         } else if constexpr (DT == BSP_BF16) {
             const int c = b - n_pack;
             tc_pack_body(c % a.tc.chunks, c / a.tc.chunks, a.tc, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi);
+        }
+    }
+}
+
+// Layers of up to kSmallBlocks blocks: the whole compaction in ONE launch.  Gamma fits in shared memory, so
+// every CTA counts for itself the stored blocks, tiles or super-tiles that precede its share (what the count
+// and scan launches hand over through memory in the general path) and writes its part of the index arrays.
+constexpr int kSmallBlocks = 4096;
+
+// Sum of v over the CTA's threads; every thread of the CTA must call it.
+__device__ __forceinline__ int block_sum(int v, int *warp_sums)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int tot = 0;
+    for (int w = 0; w < kThreads / 32; ++w) tot += warp_sums[w];
+    return tot;
+}
+
+// True if a block of Gamma (in shared memory) with a one overlaps output channels [o_lo, o_hi] x input channels [c_lo, c_hi].
+__device__ __forceinline__ bool any_kept(const uint8_t *g, int o_lo, int o_hi, int c_lo, int c_hi, int bo, int bi, int NBo, int NBi)
+{
+    bool any = false;
+    for (int lb = o_lo / bo; lb <= o_hi / bo && lb < NBo; ++lb)
+        for (int cb = c_lo / bi; cb <= c_hi / bi && cb < NBi; ++cb) any |= g[lb * NBi + cb] != 0;
+    return any;
+}
+
+template <typename T, int DT>
+__global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackArgs a)
+{
+    __shared__ __align__(16) uint8_t s_gamma[kSmallBlocks];
+    __shared__ int s_sum[kThreads / 32];
+    const int NB = a.NBo * a.NBi;
+    const bool word_ok = (((uintptr_t)a.gamma) & 3u) == 0;
+    for (int i = threadIdx.x * 4; i < NB; i += kThreads * 4) {
+        if (i + 4 <= NB && word_ok) *(uint32_t *)(s_gamma + i) = *(const uint32_t *)(a.gamma + i);
+        else for (int q = i; q < min(NB, i + 4); ++q) s_gamma[q] = a.gamma[q];
+    }
+    __syncthreads();
+    const int n_fill = a.NBo * a.fill_parts;
+    if ((int)blockIdx.x < n_fill) {
+        const int l = (int)blockIdx.x / a.fill_parts, part = (int)blockIdx.x % a.fill_parts;
+        int c = 0;
+        for (int i = threadIdx.x; i < l * a.NBi; i += kThreads) c += s_gamma[i] ? 1 : 0;
+        const int first = block_sum(c, s_sum);
+        const int cnt = csr_fill_body<T>(l, part, a.fill_parts, (const T *)a.W, a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, first,
+                                         a.col_idx, (T *)a.payload, a.capacity_blocks);
+        if (part == 0 && threadIdx.x == 0) {
+            a.row_ptr_out[l] = first;
+            if (l == a.NBo - 1) {
+                a.row_ptr_out[a.NBo] = first + cnt;
+                if ((long long)(first + cnt) > a.capacity_blocks) atomicMax(a.status, (int)BSP_ERR_CAPACITY);
+            }
+        }
+        return;
+    }
+    const int b = (int)blockIdx.x - n_fill;
+    const int n_pack = a.packed_payload ? a.pack_chunks * a.n_panels * a.pack_parts : 0;
+    if (b < n_pack) {
+        const int part = b % a.pack_parts, bc = b / a.pack_parts;
+        const int chunk = bc % a.pack_chunks, panel = bc / a.pack_chunks;
+        const int col_lo = chunk * a.cols_per_cta, col_hi = min(a.n_cols, col_lo + a.cols_per_cta);
+        // stored tiles of the panels above, and of this panel in the columns before col_lo
+        int c = 0;
+        const int tiles_above = panel * kPanelRows * a.n_cols;
+        for (int q = threadIdx.x; q < tiles_above; q += kThreads) {
+            const int tr = q / a.n_cols, col = q % a.n_cols;
+            c += any_kept(s_gamma, tr * kTile, tr * kTile + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi) ? 1 : 0;
+        }
+        const int base = block_sum(c, s_sum);
+        c = 0;
+        for (int q = threadIdx.x; q < kPanelRows * col_lo; q += kThreads) {
+            const int tr = panel * kPanelRows + q / col_lo, col = q % col_lo;
+            if (tr * kTile < a.O)
+                c += any_kept(s_gamma, tr * kTile, tr * kTile + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi) ? 1 : 0;
+        }
+        int before = block_sum(c, s_sum);
+        if (chunk == 0 && part == 0 && threadIdx.x == 0) a.panel_base_out[panel] = (uint32_t)base;
+        for (int col = col_lo; col < col_hi; ++col) {
+            unsigned m = 0;
+            for (int r = 0; r < kPanelRows; ++r) {
+                const int o0 = (panel * kPanelRows + r) * kTile;
+                if (o0 >= a.O) break;
+                if (any_kept(s_gamma, o0, o0 + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi)) m |= 1u << r;
+            }
+            if (part == 0 && threadIdx.x == 0) {
+                a.colmask_out[(size_t)panel * a.n_cols + col] = (uint8_t)m;
+                a.coloff_out[(size_t)panel * a.n_cols + col] = (uint32_t)before;
+            }
+            if (m) pack_tiles<DT>(m, (unsigned)(base + before), panel, col, a.W, s_gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi,
+                                  a.tile_bytes, a.packed_payload, a.capacity_tiles, part, a.pack_parts);
+            before += __popc(m);
+        }
+        if (panel == a.n_panels - 1 && chunk == a.pack_chunks - 1 && part == 0 && threadIdx.x == 0) {
+            const int total = base + before;
+            a.panel_base_out[a.n_panels] = (uint32_t)total;
+            PackedHeader h = a.hdr_init;
+            h.n_tiles = total;
+            *a.hdr = h;
+            if ((long long)total > a.capacity_tiles) atomicMax(a.status, (int)BSP_ERR_CAPACITY);
+        }
+        return;
+    }
+    if constexpr (DT == BSP_BF16) {
+        const TcPackArgs &t = a.tc;
+        const int part = (b - n_pack) % a.tc_parts, cidx = (b - n_pack) / a.tc_parts;
+        const int chunk = cidx % t.chunks, g = cidx / t.chunks;
+        const int kc_lo = chunk * t.kc_per_cta, kc_hi = min(t.n_kc, kc_lo + t.kc_per_cta);
+        auto st_kept = [&](int sr, int kc) -> bool {
+            const int o0 = sr * kTcSuperRow;
+            if (o0 >= a.O) return false;
+            return any_kept(s_gamma, o0, min(a.O, o0 + kTcSuperRow) - 1, kc * a.tc_kc_ch, kc * a.tc_kc_ch + a.tc_kc_ch - 1, a.bo,
+                            a.bi, a.NBo, a.NBi);
+        };
+        int c = 0;
+        for (int q = threadIdx.x; q < g * kTcGroupRows * t.n_kc; q += kThreads) c += st_kept(q / t.n_kc, q % t.n_kc) ? 1 : 0;
+        const int base = block_sum(c, s_sum);
+        c = 0;
+        // chunk 0 counts the whole group (it writes gcnt), the others the K-groups before their own
+        const int upto = (chunk == 0) ? t.n_kc : kc_lo;
+        for (int q = threadIdx.x; q < kTcGroupRows * upto; q += kThreads) c += st_kept(g * kTcGroupRows + q / upto, q % upto) ? 1 : 0;
+        const int counted = block_sum(c, s_sum);
+        int before = (chunk == 0) ? 0 : counted;
+        if (chunk == 0 && part == 0 && threadIdx.x == 0) {
+            a.tc_gcnt_out[g] = (uint32_t)counted;
+            if ((long long)(base + counted) > t.capacity) atomicMax(a.status, (int)BSP_ERR_CAPACITY);
+        }
+        for (int kc = kc_lo; kc < kc_hi; ++kc) {
+            unsigned m = 0;
+            for (int r = 0; r < kTcGroupRows; ++r)
+                if (st_kept(g * kTcGroupRows + r, kc)) m |= 1u << r;
+            if (part == 0 && threadIdx.x == 0) {
+                a.tc_mask_out[(size_t)g * t.n_kc + kc] = (uint8_t)m;
+                a.tc_off_out[(size_t)g * t.n_kc + kc] = (uint32_t)before;
+            }
+            if (m) tc_pack_tiles(m, (unsigned)(base + before), g, kc, t, a.W, s_gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, part, a.tc_parts);
+            before += __popc(m);
         }
     }
 }
@@ -473,12 +682,6 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
         ti.n_groups = L.tc.n_groups; ti.n_kc = L.tc.n_kc; ti.kc_ch = L.tc.kc_ch;
         ti.mask = pk + L.tc.off_mask; ti.off = (uint32_t *)(pk + L.tc.off_off); ti.gcnt = (uint32_t *)(pk + L.tc.off_gcnt);
     }
-    count_kernel<<<NBo + ti.n_panels + ti.n_groups, kThreads, 0, st>>>(gamma, NBo, NBi, wd.bo, wd.bi, wd.O, L.n_cols,
-                                                                       row_cnt, colmask, coloff, panel_cnt, ti);
-    BSP_CUDA_OK(cudaGetLastError());
-    scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, panel_cnt, L.n_panels, panel_base, (PackedHeader *)pk, h,
-                                        (long long)capacity_blocks, (long long)L.capacity_tiles, status);
-    BSP_CUDA_OK(cudaGetLastError());
     FillPackArgs a = {};
     a.W = W; a.gamma = gamma; a.O = wd.O; a.I = wd.I; a.HK = HK; a.bo = wd.bo; a.bi = wd.bi; a.NBo = NBo; a.NBi = NBi;
     a.row_ptr = row_ptr; a.col_idx = col_idx; a.payload = payload; a.capacity_blocks = capacity_blocks;
@@ -505,6 +708,32 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     const unsigned grid = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels : 0) +
                                      (tc_on ? a.tc.chunks * a.tc.n_groups : 0));
     const size_t smem = (size_t)NBi * sizeof(int);
+    if ((long long)NBo * NBi <= kSmallBlocks) {
+        // enough CTAs per tile column / K-group that a thread writes about four words
+        auto parts_for = [](int words_per_tile) {
+            const int p = (kPanelRows * words_per_tile + 4 * kThreads - 1) / (4 * kThreads);
+            return p < 1 ? 1 : (p > 8 ? 8 : p);
+        };
+        a.pack_parts = parts_for(L.tile_bytes / 4);
+        a.tc_parts = tc_on ? parts_for(L.tc.st_bytes / 4) : 1;
+        const unsigned grid_small = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels * a.pack_parts : 0) +
+                                               (tc_on ? a.tc.chunks * a.tc.n_groups * a.tc_parts : 0));
+        a.row_ptr_out = row_ptr; a.colmask_out = colmask; a.coloff_out = coloff; a.panel_base_out = panel_base;
+        a.hdr = (PackedHeader *)pk; a.hdr_init = h;
+        a.tc_mask_out = ti.mask; a.tc_off_out = ti.off; a.tc_gcnt_out = ti.gcnt; a.tc_kc_ch = ti.kc_ch;
+        a.status = status;
+        if (wd.wtype == BSP_I8) compact_small_kernel<uint8_t, BSP_I8><<<grid_small, kThreads, smem, st>>>(a);
+        else if (wd.wtype == BSP_BF16) compact_small_kernel<uint16_t, BSP_BF16><<<grid_small, kThreads, smem, st>>>(a);
+        else compact_small_kernel<uint32_t, BSP_F32><<<grid_small, kThreads, smem, st>>>(a);
+        BSP_CUDA_OK(cudaGetLastError());
+        return BSP_OK;
+    }
+    count_kernel<<<NBo + ti.n_panels + ti.n_groups, kThreads, 0, st>>>(gamma, NBo, NBi, wd.bo, wd.bi, wd.O, L.n_cols,
+                                                                       row_cnt, colmask, coloff, panel_cnt, ti);
+    BSP_CUDA_OK(cudaGetLastError());
+    scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, panel_cnt, L.n_panels, panel_base, (PackedHeader *)pk, h,
+                                        (long long)capacity_blocks, (long long)L.capacity_tiles, status);
+    BSP_CUDA_OK(cudaGetLastError());
     if (wd.wtype == BSP_I8) fill_pack_kernel<uint8_t, BSP_I8><<<grid, kThreads, smem, st>>>(a);
     else if (wd.wtype == BSP_BF16) fill_pack_kernel<uint16_t, BSP_BF16><<<grid, kThreads, smem, st>>>(a);
     else fill_pack_kernel<uint32_t, BSP_F32><<<grid, kThreads, smem, st>>>(a);

@@ -68,11 +68,13 @@ inline int tile_bytes_of(bsp_dtype t, int taps)
 
 PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks);
 
-// Workspace: the first 256 bytes hold the latched status word; scratch starts after it.
+// Workspace: the first 256 bytes hold the latched status word (word 0) and the two words of the grid-wide
+// barrier of the single-launch kernels (words kWsSyncWord, kWsSyncWord + 1); scratch starts after them.
 constexpr size_t kWsHeader = 256;
+constexpr int kWsSyncWord = 2;
 
 bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
-                       uint8_t *gamma, void *scores, cudaStream_t st);
+                       uint8_t *gamma, void *scores, void *ws, cudaStream_t st);
 bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gamma, int32_t *row_ptr,
                           int32_t *col_idx, void *payload, void *packed, int64_t capacity_blocks, void *ws,
                           cudaStream_t st);

@@ -41,47 +41,48 @@ __device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc
 // Threads are laid out with consecutive blocks of one block row on consecutive lanes, so that for a fixed
 // (r, h, k) a warp reads one contiguous stretch of input channels.
 template <int DT, int NORM>
+__device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
+                                                          int NBi, long long B, int r)
+{
+    using acc_t = typename Acc<DT>::type;
+    constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
+    acc_t pr = 0;
+    const int l = (int)(B / NBi), iota = (int)(B % NBi);
+    const int words = bi / per_word;
+    const size_t row_words = (size_t)I / per_word;
+    const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
+    // loads of up to nine taps (a whole 3x3 kernel) are issued together; the adds keep the (h, k, c) order
+    constexpr int kBatch = 9, kMaxWords = 16;
+    for (int t = 0; t < HK; t += kBatch) {
+        uint32_t w[kBatch][kMaxWords];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+            for (int j = 0; j < kMaxWords; ++j)
+                if (t + u < HK && j < words) w[u][j] = __ldg(src + (size_t)u * row_words + j);
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+            for (int j = 0; j < kMaxWords; ++j)
+                if (t + u < HK && j < words) add_word<DT, NORM>(w[u][j], pr);
+        src += (size_t)kBatch * row_words;
+    }
+    return pr;
+}
+
+template <int DT, int NORM>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
              typename Acc<DT>::type *__restrict__ score)
 {
     using acc_t = typename Acc<DT>::type;
     __shared__ acc_t part[kScoreThreads];
-    constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
     const int blocks_per_cta = kScoreThreads / bo;
     const int bl = threadIdx.x % blocks_per_cta;
     const int r = threadIdx.x / blocks_per_cta;
     const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
     const long long NB = (long long)NBo * NBi;
-    acc_t pr = 0;
-    if (B < NB) {
-        const int l = (int)(B / NBi), iota = (int)(B % NBi);
-        const int words = bi / per_word;
-        const size_t row_words = (size_t)I / per_word;
-        const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
-        // loads of up to nine taps (a whole 3x3 kernel) are issued together; the adds keep the (h, k, c) order
-        constexpr int kBatch = 9, kMaxWords = 16;
-        int t = 0;
-        for (; t < HK; t += kBatch) {
-            uint32_t w[kBatch][kMaxWords];
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u)
-#pragma unroll
-                for (int j = 0; j < kMaxWords; ++j)
-                    if (t + u < HK && j < words) w[u][j] = __ldg(src + (size_t)u * row_words + j);
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u)
-#pragma unroll
-                for (int j = 0; j < kMaxWords; ++j)
-                    if (t + u < HK && j < words) add_word<DT, NORM>(w[u][j], pr);
-            src += (size_t)kBatch * row_words;
-        }
-        for (; t < HK; ++t) {
-            for (int j = 0; j < words; ++j) add_word<DT, NORM>(__ldg(src + j), pr);
-            src += row_words;
-        }
-    }
-    part[threadIdx.x] = pr;
+    part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
     __syncthreads();
     if (B < NB && r == 0) {
         acc_t total = 0;
@@ -210,6 +211,106 @@ rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n
     if (live && part == 0) g[i] = ((long long)rank < n_zero) ? 0 : 1;
 }
 
+// Layers of up to kRankMax blocks: scores and ranks in ONE cooperative launch.  Every CTA scores its blocks,
+// the CTAs meet at a grid-wide barrier, then every CTA ranks its own blocks against the keys of their segment
+// (b_o lanes per key).  The barrier is two words: arrivals (reset by the last arriver, so the next launch starts
+// from zero whatever its grid) and a generation that the last arriver bumps; the wait on the generation is
+// bounded and latches BSP_ERR_TIMEOUT.
+constexpr unsigned kGridSpinLimit = 1u << 24;
+
+template <int DT, int NORM>
+__global__ void __launch_bounds__(kScoreThreads)
+mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
+                  typename Acc<DT>::type *score, int seg_len, long long n_zero, uint8_t *__restrict__ gamma,
+                  unsigned *sync, int *status)
+{
+    using acc_t = typename Acc<DT>::type;
+    __shared__ acc_t part[kScoreThreads];
+    __shared__ unsigned long long s_key[kRankMax];
+    __shared__ int s_ok;
+    const int blocks_per_cta = kScoreThreads / bo;
+    const int NB = NBo * NBi;
+    {
+        const int bl = threadIdx.x % blocks_per_cta, r = threadIdx.x / blocks_per_cta;
+        const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
+        part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+        __syncthreads();
+        if (B < NB && r == 0) {
+            acc_t total = 0;
+            for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
+            score[B] = total;
+        }
+    }
+    // grid-wide barrier
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        volatile unsigned *gen = sync + 1;
+        const unsigned g0 = *gen;
+        int ok = 1;
+        __threadfence();
+        if (atomicAdd(sync, 1u) == gridDim.x - 1) {
+            atomicExch(sync, 0u);
+            __threadfence();
+            atomicAdd(sync + 1, 1u);
+        } else {
+            unsigned spin = 0;
+            while (*gen == g0 && ++spin < kGridSpinLimit) __nanosleep(20);
+            if (*gen == g0) { ok = 0; atomicMax(status, (int)BSP_ERR_TIMEOUT); }
+        }
+        __threadfence();
+        s_ok = ok;
+    }
+    __syncthreads();
+    if (!s_ok) return;
+    // every key of the layer -> shared memory (written by other CTAs of this launch: read through L2)
+    {
+        const unsigned long long *k = (const unsigned long long *)score;
+        unsigned long long v[kRankMax / kScoreThreads];
+#pragma unroll
+        for (int u = 0; u < kRankMax / kScoreThreads; ++u) {
+            const int i = u * kScoreThreads + threadIdx.x;
+            v[u] = i < NB ? __ldcg(k + i) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < kRankMax / kScoreThreads; ++u) {
+            const int i = u * kScoreThreads + threadIdx.x;
+            if (i < NB) s_key[i] = v[u];
+        }
+    }
+    __syncthreads();
+    const int i = blockIdx.x * blocks_per_cta + threadIdx.x / bo;    // b_o lanes share one key
+    const int lane_part = threadIdx.x % bo;
+    const bool live = i < NB;
+    const int seg0 = live ? (i / seg_len) * seg_len : 0;
+    const unsigned long long mine = live ? s_key[i] : 0ull;
+    const int per = (seg_len + bo - 1) / bo;
+    const int j0 = seg0 + lane_part * per, j1 = min(seg0 + seg_len, j0 + per);
+    int rank = 0;
+    if (live)
+        for (int j = j0; j < j1; ++j) {
+            const unsigned long long other = s_key[j];
+            rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
+        }
+    for (int d = 1; d < bo; d <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, d);
+    if (live && lane_part == 0) gamma[i] = ((long long)rank < n_zero) ? 0 : 1;
+}
+
+template <int DT, int NORM>
+bsp_status run_mask_small(const bsp_wdesc &wd, const void *W, int seg_len, long long n_zero, uint8_t *gamma, void *scores,
+                          unsigned *sync, int *status, cudaStream_t st)
+{
+    using acc_t = typename Acc<DT>::type;
+    const uint32_t *Wp = (const uint32_t *)W;
+    int I = wd.I, HK = wd.H * wd.K, bo = wd.bo, bi = wd.bi, NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
+    acc_t *sc = (acc_t *)scores;
+    const int per_cta = kScoreThreads / wd.bo;
+    const unsigned grid = (unsigned)((NBo * NBi + per_cta - 1) / per_cta);
+    void *args[] = {&Wp, &I, &HK, &bo, &bi, &NBo, &NBi, &sc, &seg_len, &n_zero, &gamma, &sync, &status};
+    BSP_CUDA_OK(cudaLaunchCooperativeKernel((const void *)mask_small_kernel<DT, NORM>, dim3(grid), dim3(kScoreThreads), args, 0, st));
+    return BSP_OK;
+}
+
 template <int DT>
 bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *scores, cudaStream_t st)
 {
@@ -231,9 +332,26 @@ bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *s
 }  // namespace
 
 bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
-                       uint8_t *gamma, void *scores, cudaStream_t st)
+                       uint8_t *gamma, void *scores, void *ws, cudaStream_t st)
 {
     bsp_status rc;
+    {
+        const long long NB = (long long)(wd.O / wd.bo) * (wd.I / wd.bi);
+        if (ws != nullptr && NB <= kRankMax) {
+            const int seg_len = (int)((scope == BSP_SCOPE_LAYER) ? NB : wd.I / wd.bi);
+            int *status = (int *)ws;
+            unsigned *sync = (unsigned *)ws + kWsSyncWord;
+            const bool l2 = norm == BSP_NORM_L2;
+            if (wd.wtype == BSP_F32)
+                return l2 ? run_mask_small<BSP_F32, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                          : run_mask_small<BSP_F32, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+            if (wd.wtype == BSP_BF16)
+                return l2 ? run_mask_small<BSP_BF16, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                          : run_mask_small<BSP_BF16, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+            return l2 ? run_mask_small<BSP_I8, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                      : run_mask_small<BSP_I8, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+        }
+    }
     if (wd.wtype == BSP_F32) rc = run_scores<BSP_F32>(wd, W, norm, scores, st);
     else if (wd.wtype == BSP_BF16) rc = run_scores<BSP_BF16>(wd, W, norm, scores, st);
     else rc = run_scores<BSP_I8>(wd, W, norm, scores, st);

@@ -41,5 +41,5 @@ extern "C" bsp_status bsp_mask_static(const bsp_wdesc *wd, const void *W, bsp_no
         g_scores_ptr[dev] = p;
     }
     // every score the selection reads is rewritten by the score kernel first, so nothing needs clearing
-    return bsp::launch_mask(*wd, W, norm, scope, n_zero, gamma, g_scores_ptr[dev], (cudaStream_t)stream);
+    return bsp::launch_mask(*wd, W, norm, scope, n_zero, gamma, g_scores_ptr[dev], nullptr, (cudaStream_t)stream);
 }

@@ -84,6 +84,23 @@ def test_compact_bit_exact(dtype, bo, bi):
         assert bsp.bsp_compact_nnz(lay.wd, lay.gamma, lay.ws) == nnz
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
+@pytest.mark.parametrize("bo,bi", SHAPES)
+def test_compact_more_blocks_than_the_single_launch_path_takes(dtype, bo, bi):
+    """8192 blocks: the count / scan / fill launches instead of the one-launch kernel of small layers."""
+    O, I, H, K = 512, 1024, 1, 1
+    W = make_case(123, O, I, H, K, dtype)
+    NBo, NBi = O // bo, I // bi
+    assert NBo * NBi > 4096
+    gamma = synth.random_gamma(125, NBo, NBi, (NBo * NBi) // 3)
+    lay = gpu_layer(W, gamma, bo, bi, dtype)
+    rp, ci, pl = ref.compact(W, gamma, bo, bi)
+    assert np.array_equal(from_dev(lay.row_ptr), rp)
+    assert np.array_equal(from_dev(lay.col_idx)[:len(ci)], ci)
+    got = from_dev(lay.payload)[:pl.size].reshape(pl.shape)
+    assert np.array_equal(got, pl if dtype != "bf16" else pl.astype(np.float32))
+
+
 def test_compact_capacity_overflow_is_latched():
     bo = bi = 8
     W = make_case(117, 64, 64, 1, 1, "bf16")

@@ -83,6 +83,22 @@ def test_conv_taps_strides_padding(dtype, H, K, stride, pad, sp):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "i8"])
+@pytest.mark.parametrize("path", ["mma", "tc"])
+def test_gemm_packed_forms_of_the_multi_launch_compaction(dtype, path, monkeypatch):
+    """8192 blocks: both packed forms come from the count / scan / fill launches, not the one-launch kernel."""
+    monkeypatch.setenv("BSP_CONV_PATH", path)
+    O, I, P = 512, 1024, 200
+    W = make_case(451, O, I, 1, 1, dtype)
+    gamma = synth.random_gamma(452, O // 8, I // 8, (O // 8) * (I // 8) // 2)
+    X = make_x(453, (P, I), dtype)
+    b = make_bias(454, O, dtype)
+    lay = gpu_layer(W, gamma, 8, 8, dtype)
+    got = gpu_gemm(lay, X, b, dtype)
+    rp, ci, pl = ref.compact(W, gamma, 8, 8)
+    check(got, ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b), dtype)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
 @pytest.mark.parametrize("bo,bi", [(4, 16), (16, 4)])
 def test_conv_other_block_shapes(dtype, bo, bi):
     run_conv_case(401, 96, 80, 3, 3, bo, bi, dtype, (2, 10, 12, 80), (1, 1), (1, 1))
