@@ -57,12 +57,14 @@ def algorithmic_bytes(layer, nnz, bo, bi, ex, ey):
             + nnz * bo * bi * layer.H * layer.K * ex + 4 * (nnz + NBo + 1) + 4 * layer.O)
 
 
-def measured_traffic(workload: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None when the kernel
-    source has changed since the counters were taken (or no capture exists for this workload)."""
+def measured_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch of the dominant kernel (conv_mma_kernel or conv_tc_kernel) from the committed ncu
+    summary, or None when the kernel source has changed since the counters were taken (or no capture exists
+    for this workload)."""
     import hashlib
-    path = os.path.join(ROOT, "profiles", f"traffic_conv_mma_{workload}.json")
-    src = os.path.join(ROOT, "paper_2407_09453_b200", "csrc", "bsp_conv_mma.cu")
+    stem = kernel[:-len("_kernel")]
+    path = os.path.join(ROOT, "profiles", f"traffic_{stem}_{workload}.json")
+    src = os.path.join(ROOT, "paper_2407_09453_b200", "csrc", f"bsp_{stem}.cu")
     if not (os.path.exists(path) and os.path.exists(src)):
         return None
     d = json.load(open(path))
@@ -317,8 +319,9 @@ def main():
         gbs = abytes / (ms_conv * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / pk["hbm_gbs"], "traffic": None}
-    roof["traffic"] = measured_traffic(layer.name)
-    roof.update({"kernel": "conv_mma_kernel", "algorithmic_bytes": abytes, "peak_source": pk["source"] + " (burst)",
+    kernel = bsp.conv_kernel_name(lay.wd, bsp.XDesc(layer.N, layer.L, layer.J, stride[0], stride[1], pad[0], pad[1]))
+    roof["traffic"] = measured_traffic(layer.name, kernel)
+    roof.update({"kernel": kernel, "algorithmic_bytes": abytes, "peak_source": pk["source"] + " (burst)",
                  "kernel_ms": ms_conv, "roofline_ms": max(t_tensor, t_hbm) * 1e3})
 
     out = {

@@ -156,12 +156,18 @@ bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma,
  * float32, bias float32, ytype F32 or BF16 (round to nearest even after the bias); F32 inputs are
  * multiplied as TF32.  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
  *   bias may be NULL (treated as zero).  ws: device scratch of bsp_conv_workspace_bytes() bytes.
+ * Two kernels implement the products.  BF16 layers with stride 1 run on the tensor-memory kernel
+ * ("conv_tc_kernel": tcgen05 MMAs on 16-channel super-tiles of the second packed form); everything else, and
+ * every layer when the environment variable BSP_CONV_PATH starts with 'm', runs on the warp-MMA kernel
+ * ("conv_mma_kernel", 8x8 tiles).  bsp_conv_kernel_name() says which one a call with these descriptors takes
+ * (static storage; NULL for invalid descriptors).
  * Errors: NULL, SHAPE, BLOCK, DTYPE, INDEX (packed buffer does not match wd), CUDA. */
 size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd);
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,
                     void *Y, bsp_dtype ytype, void *ws, void *stream);
 bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
+const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd);
 
 /* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
  * (BSP_OK if none), then clears it. */

@@ -22,7 +22,7 @@ SCOPE_LAYER, SCOPE_ROW = 0, 1
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_packed_bytes", "bsp_compact_workspace_bytes",
            "bsp_compact_nnz", "bsp_compact", "bsp_conv_workspace_bytes", "bsp_gemm", "bsp_conv2d",
-           "bsp_check", "bsp_status_string"]
+           "bsp_conv_kernel_name", "bsp_check", "bsp_status_string"]
 
 
 class BspError(RuntimeError):
@@ -60,6 +60,7 @@ def lib():
                   "bsp_conv_workspace_bytes"):
             getattr(L, n).restype = C.c_size_t
         L.bsp_status_string.restype = C.c_char_p
+        L.bsp_conv_kernel_name.restype = C.c_char_p
         for n in ("bsp_mask", "bsp_compact_nnz", "bsp_compact", "bsp_gemm", "bsp_conv2d", "bsp_check"):
             getattr(L, n).restype = C.c_int
         _lib = L
@@ -149,6 +150,14 @@ def bsp_conv2d(wd: WDesc, w: Bcsr, xd: XDesc, X, bias, Y, ytype, ws, stream=None
 
 def bsp_check(ws, stream=None):
     _raise(lib().bsp_check(_ptr(ws), _stream(stream)), "bsp_check")
+
+
+def conv_kernel_name(wd: WDesc, xd: XDesc) -> str:
+    """Name of the product kernel that bsp_conv2d / bsp_gemm launch for these descriptors."""
+    r = lib().bsp_conv_kernel_name(C.byref(wd), C.byref(xd))
+    if r is None:
+        raise BspError(ERR_SHAPE, "bsp_conv_kernel_name")
+    return r.decode()
 
 
 def launches_per_step(wd: WDesc) -> int:

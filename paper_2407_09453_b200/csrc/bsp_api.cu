@@ -29,6 +29,14 @@ bsp_status check_wdesc(const bsp_wdesc *wd)
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
+// The tensor-memory kernel takes every layer it can run unless BSP_CONV_PATH asks for the warp-MMA kernel.
+bool use_tc(const bsp_wdesc &wd, const bsp_xdesc &xd)
+{
+    const char *path = getenv("BSP_CONV_PATH");
+    if (path && path[0] == 'm') return false;
+    return conv_tc_eligible(wd, xd);
+}
+
 }  // namespace
 
 extern "C" {
@@ -138,13 +146,17 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
     // the packed header is on the device; the host checks what it can: capacity against the descriptor
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
-    // BSP_CONV_PATH=tc runs eligible layers (bf16, stride 1) on the tcgen05 kernel; the default is the warp-MMA kernel
-    const char *path = getenv("BSP_CONV_PATH");
-    if (path && path[0] == 't' && conv_tc_eligible(*wd, *xd))
+    if (use_tc(*wd, *xd))
         return launch_conv_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
     // the stored fraction only steers the choice of launch shape
     const double density = NB > 0 ? (double)w->nnz / (double)NB : 1.0;
     return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, density > 0.05 ? density : 0.05, ws, (cudaStream_t)stream);
+}
+
+const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd)
+{
+    if (check_wdesc(wd) != BSP_OK || !xd) return nullptr;
+    return use_tc(*wd, *xd) ? "conv_tc_kernel" : "conv_mma_kernel";
 }
 
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,

@@ -310,8 +310,9 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
     if (wd.wtype != BSP_BF16 || xd.stride_h != 1 || xd.stride_w != 1) return false;
     const PackedLayout L = packed_layout(wd, 0);
     if (!L.tc.enabled) return false;
-    const bool gemm = wd.H == 1 && wd.K == 1 && xd.L == 1 && xd.J == 1;
-    if (gemm) return true;
+    // a 1x1 kernel without padding is a matrix product over all N*L*J positions
+    const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
+    if (gemm) return (long long)xd.N * xd.L * xd.J <= 0x7FFFFFFF;
     const int PW = xd.J + 2 * xd.pad_w;
     const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
     if (PW > 256 || R > 256) return false;
@@ -326,7 +327,8 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const PackedLayout L = packed_layout(wd, 0);
     const TcLayout &T = L.tc;
     const uint8_t *pk = (const uint8_t *)packed;
-    const bool gemm = wd.H == 1 && wd.K == 1 && xd.L == 1 && xd.J == 1;
+    const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
+    const long long n_pos = (long long)xd.N * xd.L * xd.J;      // positions of a 1x1 layer, taken as one long row
     TcParams p = {};
     p.Y = (uint8_t *)Y; p.bias = (const float *)bias;
     p.mask = pk + T.off_mask; p.off = (const uint32_t *)(pk + T.off_off); p.gcnt = (const uint32_t *)(pk + T.off_gcnt);
@@ -339,7 +341,7 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     int plane_pos, R = 1;
     long long tiles;
     if (gemm) {
-        p.PW = 1; plane_pos = 128; p.tiles_per_img = 0; tiles = ((long long)xd.N + 127) / 128;
+        p.PW = 1; plane_pos = 128; p.tiles_per_img = 0; tiles = (n_pos + 127) / 128;
     } else {
         p.PW = xd.J + 2 * xd.pad_w;
         R = (wd.H * p.PW + 126 + wd.K - 1) / p.PW + 1;
@@ -370,8 +372,9 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     EncodeTiledFn enc = tc_encode_tiled();
     if (!enc) return BSP_ERR_CUDA;
     const cuuint64_t row = (cuuint64_t)wd.I * 2;
-    const cuuint64_t gdim[5] = {16, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N, (cuuint64_t)(wd.I / 8)};
-    const cuuint64_t gstr[4] = {row, row * xd.J, row * xd.J * xd.L, 16};
+    const cuuint64_t gJ = gemm ? 1 : (cuuint64_t)xd.J, gL = gemm ? 1 : (cuuint64_t)xd.L, gN = gemm ? (cuuint64_t)n_pos : (cuuint64_t)xd.N;
+    const cuuint64_t gdim[5] = {16, gJ, gL, gN, (cuuint64_t)(wd.I / 8)};
+    const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, 16};
     cuuint32_t box[5];
     if (gemm) { box[0] = 16; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
     else { box[0] = 16; box[1] = (cuuint32_t)p.PW; box[2] = (cuuint32_t)R; box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }

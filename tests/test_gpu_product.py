@@ -13,6 +13,18 @@ from gpu_util import (TIGHT, TOL, gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_
 
 pytestmark = pytest.mark.gpu
 
+
+@pytest.fixture(autouse=True, params=["auto", "mma"])
+def conv_path(request, monkeypatch):
+    """Every case runs twice: with the library's own choice of product kernel (the tensor-memory kernel for bf16,
+    stride 1) and with the warp-MMA kernel forced, so that both kernels see every bf16 shape."""
+    if request.param == "mma":
+        monkeypatch.setenv("BSP_CONV_PATH", "mma")
+    else:
+        monkeypatch.delenv("BSP_CONV_PATH", raising=False)
+    return request.param
+
+
 SHAPES = [(8, 8), (4, 16), (16, 4)]
 
 

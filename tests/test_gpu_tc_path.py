@@ -1,4 +1,4 @@
-"""GPU parity of the tcgen05 kernel (bf16, stride 1), selected with BSP_CONV_PATH=tc, against the CPU oracle."""
+"""GPU parity of the tcgen05 kernel (bf16, stride 1; BSP_CONV_PATH=tc rules out an override from outside) against the CPU oracle."""
 import numpy as np
 import pytest
 
