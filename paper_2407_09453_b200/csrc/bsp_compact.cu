@@ -59,6 +59,9 @@ namespace {
 
 constexpr int kThreads = 256;
 
+// b_o and b_i are 4, 8 or 16: divisions by them are shifts by lg().
+__device__ __forceinline__ int lg(int b) { return 31 - __clz(b); }
+
 // Exclusive prefix sum of v over the CTA's threads; every thread of the CTA must call it.
 __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &total)
 {
@@ -114,8 +117,8 @@ count_kernel(const uint8_t *__restrict__ gamma, int NBo, int NBi, int bo, int bi
                     const int o1 = min(O, o0 + kTcSuperRow) - 1;
                     const int c0 = kc * tc.kc_ch, c1 = c0 + tc.kc_ch - 1;
                     bool any = false;
-                    for (int lb = o0 / bo; lb <= o1 / bo && lb < NBo; ++lb)
-                        for (int cb = c0 / bi; cb <= c1 / bi && cb < NBi; ++cb) any |= gamma[(size_t)lb * NBi + cb] != 0;
+                    for (int lb = o0 >> lg(bo); lb <= (o1 >> lg(bo)) && lb < NBo; ++lb)
+                        for (int cb = c0 >> lg(bi); cb <= (c1 >> lg(bi)) && cb < NBi; ++cb) any |= gamma[(size_t)lb * NBi + cb] != 0;
                     if (any) m |= 1u << r;
                 }
             }
@@ -153,8 +156,8 @@ count_kernel(const uint8_t *__restrict__ gamma, int NBo, int NBi, int bo, int bi
                 if (o0 >= O) break;
                 // blocks overlapping the tile: rows o0/bo .. (o0+7)/bo, columns (8 col)/bi .. (8 col + 7)/bi
                 bool any = false;
-                for (int lb = o0 / bo; lb <= (o0 + kTile - 1) / bo && lb < NBo; ++lb)
-                    for (int cb = (col * kTile) / bi; cb <= (col * kTile + kTile - 1) / bi && cb < NBi; ++cb)
+                for (int lb = o0 >> lg(bo); lb <= ((o0 + kTile - 1) >> lg(bo)) && lb < NBo; ++lb)
+                    for (int cb = (col * kTile) >> lg(bi); cb <= ((col * kTile + kTile - 1) >> lg(bi)) && cb < NBi; ++cb)
                         any |= gamma[(size_t)lb * NBi + cb] != 0;
                 if (any) m |= 1u << r;
             }
@@ -239,24 +242,24 @@ __device__ __forceinline__ int csr_fill_body(int l, int part, int parts, const T
     if (payload == nullptr) return s_run;
     const int cnt = s_run;
     const int blk = bo * HK * bi;
-    const long long total = (long long)cnt * blk;
+    const long long total = (long long)cnt * blk;      // at most I * b_o * H * K elements: fits 32 bits
     // the CTAs of one row (`parts` of them) all build the column list, then share the copy; the loads of four
     // elements are issued before the first store
-    const long long stride = (long long)parts * kThreads;
-    for (long long e0 = (long long)part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+    const unsigned stride = (unsigned)parts * kThreads, utotal = (unsigned)total, ublk = (unsigned)blk;
+    for (unsigned e0 = (unsigned)part * kThreads + threadIdx.x; e0 < utotal; e0 += 4 * stride) {
         T v[4];
         size_t dst[4];
         bool ok[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const long long e = e0 + u * stride;
-            ok[u] = e < total;
-            const int n = ok[u] ? (int)(e / blk) : 0;
-            const int q = ok[u] ? (int)(e % blk) : 0;
+            const unsigned e = e0 + u * stride;
+            ok[u] = e < utotal;
+            const int n = ok[u] ? (int)(e / ublk) : 0;
+            const int q = ok[u] ? (int)(e - (unsigned)n * ublk) : 0;
             int rem = q;
-            const int c = rem % bi; rem /= bi;
-            const int t = rem % HK;
+            const int c = rem & (bi - 1); rem >>= lg(bi);
             const int r = rem / HK;
+            const int t = rem - r * HK;
             ok[u] = ok[u] && (long long)(first + n) < capacity_blocks;
             dst[u] = (size_t)(first + n) * blk + q;
             v[u] = ok[u] ? W[((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi + c] : (T)0;
@@ -281,7 +284,7 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
                                                 int word, int o0, int c0, int O, int I, int HK, int bo, int bi,
                                                 int NBi)
 {
-    auto kept = [&](int o, int ch) -> bool { return o < O && gamma[(size_t)(o / bo) * NBi + ch / bi] != 0; };
+    auto kept = [&](int o, int ch) -> bool { return o < O && gamma[(size_t)(o >> lg(bo)) * NBi + (ch >> lg(bi))] != 0; };
     if constexpr (DT == BSP_BF16) {
         const uint16_t *W = (const uint16_t *)Wv;
         const int pairs = HK / 2;
@@ -332,7 +335,7 @@ __device__ __forceinline__ void pack_tiles(unsigned m, unsigned first, int panel
         for (int u = 0; u < 4; ++u) {
             const int e = e0 + u * stride;
             ok[u] = e < total;
-            const int j = ok[u] ? e / words : 0, word = ok[u] ? e % words : 0;
+            const int j = ok[u] ? (int)((unsigned)e / (unsigned)words) : 0, word = ok[u] ? e - j * words : 0;
             unsigned mm = m;                         // j-th set bit of m = tile row
             for (int q = 0; q < j; ++q) mm &= mm - 1;
             const int R = __ffs(mm) - 1;
@@ -377,7 +380,7 @@ __device__ __forceinline__ uint32_t tc_word(const uint16_t *__restrict__ W, cons
     int tap, ch;
     if (HK == 1) { tap = 0; ch = (2 * kc + h) * 8 + 2 * pair; }
     else { tap = 2 * u + h; ch = kc * 8 + 2 * pair; }
-    if (tap >= HK || o >= O || gamma[(size_t)(o / bo) * NBi + ch / bi] == 0) return 0u;
+    if (tap >= HK || o >= O || gamma[(size_t)(o >> lg(bo)) * NBi + (ch >> lg(bi))] == 0) return 0u;
     const size_t e = ((size_t)o * HK + tap) * I + ch;
     return (uint32_t)W[e] | ((uint32_t)W[e + 1] << 16);
 }
@@ -408,7 +411,7 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
         for (int u = 0; u < 4; ++u) {
             const int e = e0 + u * stride;
             ok[u] = e < total;
-            const int j = ok[u] ? e / words : 0, word = ok[u] ? e % words : 0;
+            const int j = ok[u] ? (int)((unsigned)e / (unsigned)words) : 0, word = ok[u] ? e - j * words : 0;
             unsigned mm = m;
             for (int q = 0; q < j; ++q) mm &= mm - 1;
             const int R = __ffs(mm) - 1;
@@ -512,8 +515,8 @@ __device__ __forceinline__ int block_sum(int v, int *warp_sums)
 __device__ __forceinline__ bool any_kept(const uint8_t *g, int o_lo, int o_hi, int c_lo, int c_hi, int bo, int bi, int NBo, int NBi)
 {
     bool any = false;
-    for (int lb = o_lo / bo; lb <= o_hi / bo && lb < NBo; ++lb)
-        for (int cb = c_lo / bi; cb <= c_hi / bi && cb < NBi; ++cb) any |= g[lb * NBi + cb] != 0;
+    for (int lb = o_lo >> lg(bo); lb <= (o_hi >> lg(bo)) && lb < NBo; ++lb)
+        for (int cb = c_lo >> lg(bi); cb <= (c_hi >> lg(bi)) && cb < NBi; ++cb) any |= g[lb * NBi + cb] != 0;
     return any;
 }
 

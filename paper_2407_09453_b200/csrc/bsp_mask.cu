@@ -40,34 +40,68 @@ __device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc
 // is exact in float64, so a fused multiply-add rounds like a multiply followed by an add.)
 // Threads are laid out with consecutive blocks of one block row on consecutive lanes, so that for a fixed
 // (r, h, k) a warp reads one contiguous stretch of input channels.
+// Sum of one output row r of block B over (h, k, c) in that order, for a block of WORDS 32-bit words per tap.
+// Loads of up to nine taps (a whole 3x3 kernel) are issued together, as 16-byte loads when `vec` says that the
+// rows are 16-byte aligned; the adds keep the (h, k, c) order.
+template <int DT, int NORM, int WORDS>
+__device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__restrict__ src, size_t row_words, int HK, bool vec)
+{
+    using acc_t = typename Acc<DT>::type;
+    constexpr int kBatch = 9;
+    acc_t pr = 0;
+    for (int t = 0; t < HK; t += kBatch) {
+        uint32_t w[kBatch][WORDS];
+        if constexpr (WORDS % 4 == 0) {
+            if (vec) {
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+                    for (int j = 0; j < WORDS; j += 4)
+                        if (t + u < HK) {
+                            const uint4 q = __ldg((const uint4 *)(src + (size_t)u * row_words + j));
+                            w[u][j] = q.x; w[u][j + 1] = q.y; w[u][j + 2] = q.z; w[u][j + 3] = q.w;
+                        }
+            } else {
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+                    for (int j = 0; j < WORDS; ++j)
+                        if (t + u < HK) w[u][j] = __ldg(src + (size_t)u * row_words + j);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+                for (int j = 0; j < WORDS; ++j)
+                    if (t + u < HK) w[u][j] = __ldg(src + (size_t)u * row_words + j);
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u)
+#pragma unroll
+            for (int j = 0; j < WORDS; ++j)
+                if (t + u < HK) add_word<DT, NORM>(w[u][j], pr);
+        src += (size_t)kBatch * row_words;
+    }
+    return pr;
+}
+
 template <int DT, int NORM>
 __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
                                                           int NBi, long long B, int r)
 {
-    using acc_t = typename Acc<DT>::type;
     constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
-    acc_t pr = 0;
     const int l = (int)(B / NBi), iota = (int)(B % NBi);
     const int words = bi / per_word;
     const size_t row_words = (size_t)I / per_word;
     const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
-    // loads of up to nine taps (a whole 3x3 kernel) are issued together; the adds keep the (h, k, c) order
-    constexpr int kBatch = 9, kMaxWords = 16;
-    for (int t = 0; t < HK; t += kBatch) {
-        uint32_t w[kBatch][kMaxWords];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-#pragma unroll
-            for (int j = 0; j < kMaxWords; ++j)
-                if (t + u < HK && j < words) w[u][j] = __ldg(src + (size_t)u * row_words + j);
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-#pragma unroll
-            for (int j = 0; j < kMaxWords; ++j)
-                if (t + u < HK && j < words) add_word<DT, NORM>(w[u][j], pr);
-        src += (size_t)kBatch * row_words;
+    const bool vec = (((uintptr_t)W) & 15u) == 0 && row_words % 4 == 0;
+    switch (words) {
+        case 1: return row_sum_w<DT, NORM, 1>(src, row_words, HK, vec);
+        case 2: return row_sum_w<DT, NORM, 2>(src, row_words, HK, vec);
+        case 4: return row_sum_w<DT, NORM, 4>(src, row_words, HK, vec);
+        case 8: return row_sum_w<DT, NORM, 8>(src, row_words, HK, vec);
+        default: return row_sum_w<DT, NORM, 16>(src, row_words, HK, vec);
     }
-    return pr;
 }
 
 template <int DT, int NORM>
@@ -220,7 +254,7 @@ constexpr unsigned kGridSpinLimit = 1u << 24;
 
 template <int DT, int NORM>
 __global__ void __launch_bounds__(kScoreThreads)
-mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
+mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi, int BC,
                   typename Acc<DT>::type *score, int seg_len, long long n_zero, uint8_t *__restrict__ gamma,
                   unsigned *sync, int *status)
 {
@@ -228,16 +262,17 @@ mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
     __shared__ acc_t part[kScoreThreads];
     __shared__ unsigned long long s_key[kRankMax];
     __shared__ int s_ok;
-    const int blocks_per_cta = kScoreThreads / bo;
     const int NB = NBo * NBi;
+    // BC blocks per CTA: b_o threads score one block, then 256 / BC lanes rank one key
     {
-        const int bl = threadIdx.x % blocks_per_cta, r = threadIdx.x / blocks_per_cta;
-        const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
-        part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+        const int bl = threadIdx.x % BC, r = threadIdx.x / BC;
+        const long long B = (long long)blockIdx.x * BC + bl;
+        const bool mine = r < bo && B < NB;
+        part[threadIdx.x] = mine ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
         __syncthreads();
-        if (B < NB && r == 0) {
+        if (mine && r == 0) {
             acc_t total = 0;
-            for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
+            for (int q = 0; q < bo; ++q) total += part[q * BC + bl];
             score[B] = total;
         }
     }
@@ -279,20 +314,19 @@ mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
         }
     }
     __syncthreads();
-    const int i = blockIdx.x * blocks_per_cta + threadIdx.x / bo;    // b_o lanes share one key
-    const int lane_part = threadIdx.x % bo;
+    const int LK = kScoreThreads / BC;                          // lanes per key, at most 32
+    const int i = blockIdx.x * BC + threadIdx.x / LK;
+    const int lane_part = threadIdx.x % LK;
     const bool live = i < NB;
     const int seg0 = live ? (i / seg_len) * seg_len : 0;
     const unsigned long long mine = live ? s_key[i] : 0ull;
-    const int per = (seg_len + bo - 1) / bo;
-    const int j0 = seg0 + lane_part * per, j1 = min(seg0 + seg_len, j0 + per);
     int rank = 0;
     if (live)
-        for (int j = j0; j < j1; ++j) {
+        for (int j = seg0 + lane_part; j < seg0 + seg_len; j += LK) {   // consecutive lanes, consecutive keys
             const unsigned long long other = s_key[j];
             rank += (other < mine || (other == mine && j < i)) ? 1 : 0;
         }
-    for (int d = 1; d < bo; d <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, d);
+    for (int d = 1; d < LK; d <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, d);
     if (live && lane_part == 0) gamma[i] = ((long long)rank < n_zero) ? 0 : 1;
 }
 
@@ -304,9 +338,11 @@ bsp_status run_mask_small(const bsp_wdesc &wd, const void *W, int seg_len, long 
     const uint32_t *Wp = (const uint32_t *)W;
     int I = wd.I, HK = wd.H * wd.K, bo = wd.bo, bi = wd.bi, NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
     acc_t *sc = (acc_t *)scores;
-    const int per_cta = kScoreThreads / wd.bo;
-    const unsigned grid = (unsigned)((NBo * NBi + per_cta - 1) / per_cta);
-    void *args[] = {&Wp, &I, &HK, &bo, &bi, &NBo, &NBi, &sc, &seg_len, &n_zero, &gamma, &sync, &status};
+    // few blocks per CTA spread the layer over the SMs; the grid stays small enough to be co-resident
+    int BC = 8;
+    while ((NBo * NBi + BC - 1) / BC > 128 && BC * 2 * wd.bo <= kScoreThreads) BC *= 2;
+    const unsigned grid = (unsigned)((NBo * NBi + BC - 1) / BC);
+    void *args[] = {&Wp, &I, &HK, &bo, &bi, &NBo, &NBi, &BC, &sc, &seg_len, &n_zero, &gamma, &sync, &status};
     BSP_CUDA_OK(cudaLaunchCooperativeKernel((const void *)mask_small_kernel<DT, NORM>, dim3(grid), dim3(kScoreThreads), args, 0, st));
     return BSP_OK;
 }
