@@ -61,7 +61,7 @@ size_t bsp_mask_workspace_bytes(const bsp_wdesc *wd)
 {
     if (check_wdesc(wd) != BSP_OK) return 0;
     const size_t NB = (size_t)(wd->O / wd->bo) * (wd->I / wd->bi);
-    return kWsHeader + align_up(NB * 8, 256);
+    return kWsHeader + align_up(NB * 8, 256) + align_up(kSelectScratch, 256);
 }
 
 bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,

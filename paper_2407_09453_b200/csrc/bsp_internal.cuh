@@ -72,6 +72,10 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks);
 // barrier of the single-launch kernels (words kWsSyncWord, kWsSyncWord + 1); scratch starts after them.
 constexpr size_t kWsHeader = 256;
 constexpr int kWsSyncWord = 2;
+// Scratch of the cooperative select after the scores in the mask workspace: 8 x 256 histogram words and one
+// word per CTA.
+constexpr int kSelectMaxCtas = 1024;
+constexpr size_t kSelectScratch = (8 * 256 + kSelectMaxCtas) * 4;
 
 bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
                        uint8_t *gamma, void *scores, void *ws, cudaStream_t st);

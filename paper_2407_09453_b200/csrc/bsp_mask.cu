@@ -200,6 +200,127 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
     }
 }
 
+// Grid-wide barrier of a cooperative launch (all CTAs co-resident), reusable within the launch: `sync[0]`
+// counts arrivals and is reset by the last arriver, `sync[1]` is a generation that the last arriver bumps.
+// Thread 0 of each CTA takes part; the wait is bounded.  Returns false if it expired.
+constexpr unsigned kGridSpinLimit = 1u << 24;
+__device__ __forceinline__ bool grid_barrier(unsigned *sync)
+{
+    __shared__ int s_bar_ok;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        volatile unsigned *gen = sync + 1;
+        const unsigned g0 = *gen;
+        int ok = 1;
+        __threadfence();
+        if (atomicAdd(sync, 1u) == gridDim.x - 1) {
+            atomicExch(sync, 0u);
+            __threadfence();
+            atomicAdd(sync + 1, 1u);
+        } else {
+            unsigned spin = 0;
+            while (*gen == g0 && ++spin < kGridSpinLimit) __nanosleep(20);
+            if (*gen == g0) ok = 0;
+        }
+        __threadfence();
+        s_bar_ok = ok;
+    }
+    __syncthreads();
+    return s_bar_ok != 0;
+}
+
+// The radix select of select_kernel for one large segment (the whole layer), spread over a cooperative grid:
+// CTA c owns a contiguous slice of the keys.  Each of the eight passes adds the CTAs' digit histograms into
+// ghist[pass][256] (zeroed by the host before the launch), the CTAs meet at the grid barrier, and every CTA
+// derives the digit for itself.  Keys equal to the threshold T are zeroed lowest index first: the CTAs publish
+// how many such keys their slices hold (geq[c]), meet again, and each counts those in the slices before its own.
+constexpr int kCoopThreads = 512;
+__global__ void __launch_bounds__(kCoopThreads)
+select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long long n_zero, uint8_t *__restrict__ gamma,
+                   unsigned *ghist, unsigned *geq, unsigned *sync, int *status)
+{
+    __shared__ unsigned hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ long long s_k;
+    __shared__ unsigned warp_cnt[kCoopThreads / 32];
+    __shared__ long long s_run;
+    const int tid = threadIdx.x;
+    const long long slice = (n + gridDim.x - 1) / gridDim.x;
+    const long long lo = (long long)blockIdx.x * slice, hi = min(n, lo + slice);
+    if (tid == 0) { s_prefix = 0ull; s_k = n_zero; }
+    for (int pass = 7; pass >= 0; --pass) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const unsigned long long prefix = s_prefix;
+        const int shift = 8 * pass;
+        for (long long i = lo + tid; i < hi; i += kCoopThreads) {
+            const unsigned long long v = key[i];
+            const bool in = (pass == 7) || ((v >> (shift + 8)) == prefix);
+            if (in) atomicAdd(&hist[(unsigned)((v >> shift) & 0xFFull)], 1u);
+        }
+        __syncthreads();
+        if (tid < 256 && hist[tid]) atomicAdd(&ghist[pass * 256 + tid], hist[tid]);
+        if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
+        if (tid < 256) hist[tid] = __ldcg(&ghist[pass * 256 + tid]);
+        __syncthreads();
+        if (tid == 0) {
+            long long need = s_k, cum = 0;
+            int d = 0;
+            for (; d < 255; ++d) {
+                if (cum + (long long)hist[d] >= need) break;
+                cum += hist[d];
+            }
+            s_k = need - cum;
+            s_prefix = (prefix << 8) | (unsigned long long)d;
+        }
+        __syncthreads();
+    }
+    const unsigned long long T = s_prefix;
+    const long long ties = s_k;        // keys equal to T to zero, lowest indices first
+    // keys equal to T in this slice
+    {
+        unsigned c = 0;
+        for (long long i = lo + tid; i < hi; i += kCoopThreads) c += key[i] == T ? 1u : 0u;
+        for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, d);
+        if ((tid & 31) == 0) warp_cnt[tid >> 5] = c;
+        __syncthreads();
+        if (tid == 0) {
+            unsigned tot = 0;
+            for (int w = 0; w < kCoopThreads / 32; ++w) tot += warp_cnt[w];
+            geq[blockIdx.x] = tot;
+        }
+    }
+    if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
+    if (tid == 0) {
+        long long before = 0;
+        for (unsigned c = 0; c < blockIdx.x; ++c) before += __ldcg(&geq[c]);
+        s_run = before;
+    }
+    __syncthreads();
+    const int lane = tid & 31, warp = tid >> 5;
+    for (long long base = lo; base < hi; base += kCoopThreads) {
+        const long long i = base + tid;
+        unsigned long long v = ~0ull;
+        if (i < hi) v = key[i];
+        const bool eq = (i < hi) && (v == T);
+        const unsigned ball = __ballot_sync(0xFFFFFFFFu, eq);
+        if (lane == 0) warp_cnt[warp] = __popc(ball);
+        __syncthreads();
+        long long before = s_run;
+        for (int w = 0; w < warp; ++w) before += warp_cnt[w];
+        before += __popc(ball & ((1u << lane) - 1u));
+        if (i < hi) gamma[i] = (v < T || (eq && before < ties)) ? 0 : 1;
+        __syncthreads();
+        if (tid == 0) {
+            long long tot = 0;
+            for (int w = 0; w < kCoopThreads / 32; ++w) tot += warp_cnt[w];
+            s_run += tot;
+        }
+        __syncthreads();
+    }
+}
+
 // Small segments (up to kRankMax keys): the keys sit in shared memory and every thread counts the (key, index)
 // pairs below its own, which is its rank in the ascending order; Gamma = 0 for ranks below n_zero.  Same
 // result as the radix select, in one pass instead of nine.
@@ -250,7 +371,6 @@ rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n
 // (b_o lanes per key).  The barrier is two words: arrivals (reset by the last arriver, so the next launch starts
 // from zero whatever its grid) and a generation that the last arriver bumps; the wait on the generation is
 // bounded and latches BSP_ERR_TIMEOUT.
-constexpr unsigned kGridSpinLimit = 1u << 24;
 
 template <int DT, int NORM>
 __global__ void __launch_bounds__(kScoreThreads)
@@ -261,7 +381,6 @@ mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
     using acc_t = typename Acc<DT>::type;
     __shared__ acc_t part[kScoreThreads];
     __shared__ unsigned long long s_key[kRankMax];
-    __shared__ int s_ok;
     const int NB = NBo * NBi;
     // BC blocks per CTA: b_o threads score one block, then 256 / BC lanes rank one key
     {
@@ -276,28 +395,10 @@ mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
             score[B] = total;
         }
     }
-    // grid-wide barrier
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        volatile unsigned *gen = sync + 1;
-        const unsigned g0 = *gen;
-        int ok = 1;
-        __threadfence();
-        if (atomicAdd(sync, 1u) == gridDim.x - 1) {
-            atomicExch(sync, 0u);
-            __threadfence();
-            atomicAdd(sync + 1, 1u);
-        } else {
-            unsigned spin = 0;
-            while (*gen == g0 && ++spin < kGridSpinLimit) __nanosleep(20);
-            if (*gen == g0) { ok = 0; atomicMax(status, (int)BSP_ERR_TIMEOUT); }
-        }
-        __threadfence();
-        s_ok = ok;
+    if (!grid_barrier(sync)) {
+        if (threadIdx.x == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT);
+        return;
     }
-    __syncthreads();
-    if (!s_ok) return;
     // every key of the layer -> shared memory (written by other CTAs of this launch: read through L2)
     {
         const unsigned long long *k = (const unsigned long long *)score;
@@ -399,7 +500,27 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
     if (seg <= kRankMax)
         rank_kernel<<<dim3(nseg, (unsigned)((seg * kRankLanes + kRankThreads - 1) / kRankThreads)), kRankThreads, 0, st>>>(
             (const unsigned long long *)scores, (int)seg, n_zero, gamma);
-    else
+    else if (ws != nullptr && nseg == 1 && n_zero > 0 && n_zero < seg) {
+        // one large segment: the select runs on a cooperative grid of at most one CTA per SM
+        static int sm_count[64] = {};
+        int dev = 0;
+        BSP_CUDA_OK(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return BSP_ERR_CUDA;
+        if (sm_count[dev] == 0) BSP_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        long long grid = (seg + 2 * kCoopThreads - 1) / (2 * kCoopThreads);
+        if (grid > sm_count[dev]) grid = sm_count[dev];
+        if (grid > kSelectMaxCtas) grid = kSelectMaxCtas;
+        unsigned *ghist = (unsigned *)((char *)ws + kWsHeader + align_up((size_t)NB * 8, 256));
+        unsigned *geq = ghist + 8 * 256;
+        BSP_CUDA_OK(cudaMemsetAsync(ghist, 0, 8 * 256 * sizeof(unsigned), st));
+        const unsigned long long *keys = (const unsigned long long *)scores;
+        long long n = seg, nz = n_zero;
+        unsigned *sync = (unsigned *)ws + kWsSyncWord;
+        int *status = (int *)ws;
+        void *args[] = {&keys, &n, &nz, &gamma, &ghist, &geq, &sync, &status};
+        BSP_CUDA_OK(cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, 0, st));
+        return BSP_OK;
+    } else
         select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;

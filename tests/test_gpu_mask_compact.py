@@ -56,6 +56,20 @@ def test_gamma_ties_broken_by_index():
         assert np.array_equal(g, ref.mask(want_s, n_zero))
 
 
+def test_gamma_ties_in_a_layer_of_many_blocks():
+    """8192 blocks with few distinct int8 scores: the multi-CTA select must zero equal keys lowest index first,
+    across the slices of different CTAs."""
+    bo = bi = 8
+    W = synth.uniform_int(131, (512, 1, 1, 1024), -3, 3).astype(np.int8)
+    want_s = ref.scores(W, bo, bi)
+    assert len(np.unique(want_s)) < want_s.size // 8
+    for n_zero in (1, 4097, want_s.size - 1):
+        g, s, _, _ = gpu_mask(W, bo, bi, "i8", n_zero)
+        assert np.array_equal(g, ref.mask(want_s, n_zero))
+    g, _, _, _ = gpu_mask(W, bo, bi, "i8", 40, scope=bsp.SCOPE_ROW)
+    assert np.array_equal(g, ref.mask(want_s, 40, ref.SCOPE_ROW))
+
+
 def test_gamma_large_layer_many_select_passes():
     """More blocks than one pass of the selecting CTA covers (4096x2048 / 8x8 = 131072 blocks)."""
     bo = bi = 8
