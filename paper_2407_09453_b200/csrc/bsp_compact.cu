@@ -368,14 +368,18 @@ __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__re
     }
 }
 
-// One 32-bit word of a stored super-tile: K-step u, then [K half h][8-row group rg][row][4 words of 2 bf16],
-// the K-major core-matrix order of a 16 x 16 tcgen05 B operand.  A convolution pairs taps 2u and 2u+1 of the
-// K-group's 8 channels (a missing odd tap reads as zero); a 1x1 layer pairs the two 8-channel halves.
+// One 32-bit word of a stored super-tile: K-step u, then [8-row group rg][K half h][row][4 words of 2 bf16]:
+// 8 rows x 16 bytes are one core matrix of a K-major tcgen05 B operand without swizzle, the K halves are 128
+// bytes apart and the row groups 256.  The stored super-tiles of one (group, K-group) are laid out K-step
+// major, [u][stored tile][512 bytes], so that for one K-step the tiles of consecutive stored super-rows form ONE
+// B operand of 16 x (number of tiles) rows with a uniform 256-byte row-group stride.
+// A convolution pairs taps 2u and 2u+1 of the K-group's 8 channels (a missing odd tap reads as zero); a 1x1
+// layer pairs the two 8-channel halves.
 __device__ __forceinline__ uint32_t tc_word(const uint16_t *__restrict__ W, const uint8_t *__restrict__ gamma, int word,
                                             int o_base, int kc, int O, int I, int HK, int bo, int bi, int NBi)
 {
     const int u = word >> 7, w = word & 127;
-    const int h = w >> 6, rg = (w >> 5) & 1, row = (w >> 2) & 7, pair = w & 3;
+    const int rg = w >> 6, h = (w >> 5) & 1, row = (w >> 2) & 7, pair = w & 3;
     const int o = o_base + rg * 8 + row;
     int tap, ch;
     if (HK == 1) { tap = 0; ch = (2 * kc + h) * 8 + 2 * pair; }
@@ -401,7 +405,8 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
                                               int HK, int bo, int bi, int NBi, int part, int parts)
 {
     const int words = t.st_bytes / 4;
-    const int total = __popc(m) * words;
+    const int cnt = __popc(m);
+    const int total = cnt * words;
     const int stride = parts * kThreads;
     for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
         uint32_t v[4];
@@ -415,8 +420,9 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
             unsigned mm = m;
             for (int q = 0; q < j; ++q) mm &= mm - 1;
             const int R = __ffs(mm) - 1;
-            ok[u] = ok[u] && (long long)(first + j) < t.capacity;
-            dst[u] = (uint32_t *)(t.payload + (size_t)(first + j) * t.st_bytes) + word;
+            ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
+            // K-step (word >> 7) major within the K-group, then the stored tile, then the word of the 512-byte unit
+            dst[u] = (uint32_t *)(t.payload + (size_t)first * t.st_bytes) + ((size_t)((word >> 7) * cnt + j) << 7) + (word & 127);
             v[u] = ok[u] ? tc_word((const uint16_t *)W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
         }
 #pragma unroll

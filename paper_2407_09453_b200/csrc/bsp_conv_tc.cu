@@ -2,22 +2,26 @@
 // (tcgen05.mma, accumulators in tensor memory), bf16 inputs, stride 1.  Introduction (Y = W*X + b) and Section
 // "Block Sparsity in a Matrix" of the paper.
 //
-// One MMA is D[128 x 16] += A[128 x 16] * B[16 x 16]: 128 output positions, 16 output channels (a super-row),
-// 16 reduction elements (two taps of 8 input channels, or 16 input channels of a 1x1 layer).  That is the
-// smallest tile the instruction offers at M = 128, so the unit that can be skipped is a 16-channel x K-group
-// super-tile of W-bar; zeroed 8x8 blocks inside a stored super-tile are multiplied as zeros.
+// One MMA is D[128 x 16n] += A[128 x 16] * B[16 x 16n]: 128 output positions, n consecutive stored super-rows
+// of 16 output channels, 16 reduction elements (two taps of 8 input channels, or 16 input channels of a 1x1
+// layer).  The unit that can be skipped is a 16-channel x K-group super-tile of W-bar; zeroed 8x8 blocks inside
+// a stored super-tile are multiplied as zeros.  The stored super-tiles of a run of consecutive super-rows lie
+// side by side in the packed payload and in tensor memory, so a run is ONE MMA with N = 16 x (run length): a
+// dense layer issues N = 128 MMAs, a sparse one an MMA per run of its mask.
 //
-// A CTA owns 128 consecutive positions of one image and one group of 8 super-rows (128 channels, 128 fp32
-// TMEM columns).  Positions are counted over rows of the padded input width PW, so that the input of output
-// position m at tap (h, k) is the staged element m + h*PW + k: a tap is a constant offset, positions whose
-// column falls in the padding compute garbage and are not stored.  Activations are staged by tiled TMA loads
-// (out-of-bounds fill = zero padding) as planes [8-channel chunk][position][16 bytes], the no-swizzle K-major
-// core-matrix layout: 8 consecutive positions are one core matrix, the two K halves of an MMA are two planes
-// or two tap offsets (the descriptor's leading-dimension byte offset).  The stored super-tiles of the group
-// for the stage's K-groups are one contiguous stretch of the packed payload (one bulk copy).
-// Warps 0-7 each issue the MMAs of one super-row (an MMA this small costs more to issue than to execute, so the
-// issue is spread over eight threads; accumulators in TMEM are addressed at run time, so no code is specialised
-// on the sparsity pattern), warp 8 produces; then the eight warps read their TMEM lanes back, add the bias and store.  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
+// A CTA owns 128 consecutive positions of one image and one group of 8 super-rows (128 channels).  Positions
+// are counted over rows of the padded input width PW, so that the input of output position m at tap (h, k) is
+// the staged element m + h*PW + k: a tap is a constant offset, positions whose column falls in the padding
+// compute garbage and are not stored.  Activations are staged by tiled TMA loads (out-of-bounds fill = zero
+// padding) as planes [8-channel chunk][position][16 bytes], the no-swizzle K-major core-matrix layout: 8
+// consecutive positions are one core matrix, the two K halves of an MMA are two planes or two tap offsets (the
+// descriptor's leading-dimension byte offset).  The stored super-tiles of the group for the stage's K-groups are
+// one contiguous stretch of the packed payload (one bulk copy).
+// Warps 0-3 issue: issuer s takes the K-groups kc with kc % 4 == s and accumulates them in its own 128 columns
+// of tensor memory (an MMA this small costs more to issue than to execute, and MMAs of different threads on one
+// accumulator are not ordered, hence four accumulator sets, zeroed at the start and summed at the end).  Warp 4
+// produces.  Then all eight warps read their TMEM lanes back, add the four sets and the bias, and store.
+// Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
 #include <cuda.h>
 #include <cstdlib>
 #include "bsp_internal.cuh"
@@ -25,12 +29,12 @@
 namespace bsp {
 namespace {
 
-constexpr int kIssuers = 8;                       // one issuing warp per super-row of the group
-constexpr int kTcThreads = 32 * (kIssuers + 1);   // + the producer warp
+constexpr int kIssuers = 4;                       // issuing warps = accumulator sets (K-groups interleaved over them)
+constexpr int kTcThreads = 256;                   // warps 0-3 issue, warp 4 produces, all eight run the epilogue
 constexpr int kTcMaxStages = 8;
 constexpr int kTcMaxSmem = 200 * 1024;
 constexpr int kTcMaxDevices = 64;
-constexpr int kTmemCols = 128;
+constexpr int kTmemCols = 128 * kIssuers;
 constexpr uint32_t kTcSpinLimit = 1u << 22;
 
 struct TcParams {
@@ -87,7 +91,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     __shared__ __align__(8) uint64_t s_full[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_empty[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_done;
-    __shared__ uint32_t s_tmem, s_touched, s_gbase, s_gcnt, s_fail;
+    __shared__ uint32_t s_tmem, s_gbase, s_gcnt, s_fail;
     __shared__ const uint8_t *s_payload;
     __shared__ uint64_t s_ahi[64];          // per K-step of a super-tile: A descriptor without its address field
     __shared__ uint32_t s_aoff[64];         // ... and the operand's offset from the K-group's first plane, in 16-byte units
@@ -106,7 +110,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     if (tid == 0) {
         uint32_t base = 0;
         for (int q = 0; q < g; ++q) base += p.gcnt[q];
-        s_gbase = base; s_gcnt = p.gcnt[g]; s_touched = 0; s_fail = 0;
+        s_gbase = base; s_gcnt = p.gcnt[g]; s_fail = 0;
         s_payload = p.packed + ((const PackedHeader *)p.packed)->off_tc_payload;
         for (int s = 0; s < S; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_full[s])), "r"(1) : "memory");
@@ -147,12 +151,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem = s_tmem;
+    // every accumulator starts at zero, so that every MMA accumulates and super-rows without a stored tile read as
+    // zero: warps 0-3 clear the 32 TMEM lanes they can reach, all columns
+    if (warp < 4) {
+        const uint32_t z = 0u;
+        for (int c = 0; c < kTmemCols; c += 16)
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};\n"
+                         ::"r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c), "r"(z) : "memory");
+        asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
 
     const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
     const uint32_t ring = s32(smem) + meta_bytes;
 
     if (warp == kIssuers) {
-        // ================= producer =================
+        // ================= producer (warp 4) =================
         if (lane == 0) {
             for (int it = 0; it < p.n_stage_iters; ++it) {
                 const int slot = it % S;
@@ -173,24 +189,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                                  ::"r"(dst + p.act_bytes), "l"(s_payload + (size_t)(s_gbase + o_lo) * p.st_bytes), "r"(wbytes), "r"(bar) : "memory");
             }
         }
-    } else {
-        // ================= MMA issuers: warp r owns super-row r =================
+    } else if (warp < kIssuers) {
+        // ================= MMA issuers: warp s takes the K-groups kc with kc % kIssuers == s =================
         // One thread per issuing warp runs the whole issue loop: a tcgen05.mma is issued by a single thread, and
         // keeping that thread in one long non-divergent stretch avoids a divergence region around every MMA.
         if (lane == 0) {
-            const uint32_t r = (uint32_t)warp;
-            const uint32_t below = (1u << r) - 1u;
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // + (N >> 3) << 17
             // Descriptors are sums: the address field (16-byte units, low 14 bits) of an A operand is
-            // stage + plane + s_aoff[u], of a B operand weights + 32 * (tile * n_units + u); the other fields are
-            // per-unit (A: the byte offset between the K halves) or constant (B).
-            const uint64_t b_hi = smem_desc(0, 256, 128);
+            // stage + plane + s_aoff[u]; of a B operand weights + 32 * (tiles before the K-group * n_units
+            // + u * tiles of the K-group + tiles before the run).  B: K halves 128 bytes apart, row groups 256.
+            const uint64_t b_hi = smem_desc(0, 128, 256);
             const int plane16 = (p.plane_bytes >> 4) * p.chunks_per_kc;  // 16-byte units between K-groups' planes
-            const int nu = p.n_units;
+            const uint32_t nu = (uint32_t)p.n_units;
             const uint64_t ahi0 = s_ahi[0];
             const uint32_t aoff0 = s_aoff[0];
-            const uint32_t d = tmem + r * 16u;
-            uint32_t acc = 0;
+            const uint32_t dset = tmem + (uint32_t)warp * 128u;
             bool ok = true;
             for (int it = 0; it < p.n_stage_iters; ++it) {
                 const int slot = it % S;
@@ -200,30 +213,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t stage16 = (ring + slot * p.stage_bytes) >> 4;
                 const uint32_t w16 = stage16 + (p.act_bytes >> 4);
                 const uint32_t o_lo = s_off[kc0];
-                for (int kl = 0; kl < nk; ++kl) {
-                    const uint32_t m = s_mask[kc0 + kl];
-                    if (!((m >> r) & 1u)) continue;
-                    const uint32_t tile = s_off[kc0 + kl] - o_lo + __popc(m & below);
+                int kl = (warp - kc0) & (kIssuers - 1);           // first K-group of the stage that is mine
+                for (; kl < nk; kl += kIssuers) {
+                    uint32_t m = s_mask[kc0 + kl];
+                    if (m == 0) continue;
+                    const uint32_t cnt = __popc(m);
                     const uint32_t a16 = stage16 + kl * plane16;
-                    if (nu == 1) {
-                        mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)((w16 + tile * 32u) & 0x3FFFu), idesc, acc);
-                    } else {
-                        uint32_t b16 = w16 + tile * (uint32_t)nu * 32u;
-                        for (int u = 0; u < nu; ++u) {
-                            mma_bf16(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, acc | (uint32_t)(u > 0));
-                            b16 += 32u;
+                    uint32_t b16 = w16 + (s_off[kc0 + kl] - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
+                    while (m) {
+                        const int r0 = __ffs(m) - 1;
+                        const int len = __ffs(~(m >> r0)) - 1;                  // run of stored super-rows r0 .. r0 + len - 1
+                        m &= ~(((1u << len) - 1u) << r0);
+                        const uint32_t idesc = idesc0 | ((uint32_t)(len * 16 >> 3) << 17);
+                        const uint32_t d = dset + (uint32_t)r0 * 16u;
+                        if (nu == 1) {
+                            mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
+                        } else {
+                            uint32_t bu = b16;
+                            for (uint32_t u = 0; u < nu; ++u) {
+                                mma_bf16(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(bu & 0x3FFFu), idesc, 1u);
+                                bu += cnt * 32u;
+                            }
                         }
+                        b16 += (uint32_t)len * 32u;
                     }
-                    acc = 1u;
                 }
                 commit_to(s32(&s_empty[slot]));
             }
-            if (ok) { commit_to(s32(&s_done)); if (acc) atomicOr(&s_touched, 1u << r); }
+            if (ok) commit_to(s32(&s_done));
             else atomicExch(&s_fail, 1u);
         }
     }
 
-    // ================= epilogue: warps 0-7; warp w reads TMEM lanes 32*(w%4).. (positions) of super-rows 4*(w/4).. =================
+    // ================= epilogue: all eight warps; warp w reads TMEM lanes 32*(w%4).. (positions) of super-rows 4*(w/4).. =================
     __syncwarp();
     bool done = wait_bar(s32(&s_done), 0);
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -231,7 +253,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     if (s_fail) done = false;
     if (!done && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
     if (done) {
-        const uint32_t touched = s_touched;
         const int lq = warp & 3;                 // a warp reaches the TMEM lanes of its quarter only
         const int m = lq * 32 + lane;
         bool valid;
@@ -244,26 +265,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         }
         const int oe = (p.ytype == BSP_BF16) ? 2 : 4;
 #pragma unroll 1
-        for (int r = (warp >> 2) * 4; r < (warp >> 2) * 4 + 4 && warp < kIssuers; ++r) {
+        for (int r = (warp >> 2) * 4; r < (warp >> 2) * 4 + 4; ++r) {
             const int ch = (g * kTcGroupRows + r) * kTcSuperRow;
             if (ch >= p.O) break;
-            uint32_t v[16];
-            if ((touched >> r) & 1u) {
-                const uint32_t ta = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)r * 16u;
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
-                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                             : "r"(ta) : "memory");
-                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-            } else {
+            // the four accumulator sets of this super-row
+            uint32_t v[kIssuers][16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = 0u;
+            for (int s = 0; s < kIssuers; ++s) {
+                const uint32_t ta = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)(s * 128 + r * 16);
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+                             : "=r"(v[s][0]), "=r"(v[s][1]), "=r"(v[s][2]), "=r"(v[s][3]), "=r"(v[s][4]), "=r"(v[s][5]), "=r"(v[s][6]), "=r"(v[s][7]),
+                               "=r"(v[s][8]), "=r"(v[s][9]), "=r"(v[s][10]), "=r"(v[s][11]), "=r"(v[s][12]), "=r"(v[s][13]), "=r"(v[s][14]), "=r"(v[s][15])
+                             : "r"(ta) : "memory");
             }
+            asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
             if (!valid) continue;
             const int nch = min(16, p.O - ch);        // 16, or 8 in a last half super-row
             float f[16];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]) + ((p.bias != nullptr && e < nch) ? __ldg(p.bias + ch + e) : 0.f);
+            for (int e = 0; e < 16; ++e)
+                f[e] = ((__uint_as_float(v[0][e]) + __uint_as_float(v[1][e])) + (__uint_as_float(v[2][e]) + __uint_as_float(v[3][e]))) +
+                       ((p.bias != nullptr && e < nch) ? __ldg(p.bias + ch + e) : 0.f);
             uint8_t *dst = p.Y + (pix * p.O + ch) * oe;
             if (oe == 4) {
 #pragma unroll
