@@ -334,13 +334,20 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
     if (!L.tc.enabled) return false;
     // a 1x1 kernel without padding is a matrix product over all N*L*J positions
     const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
-    if (gemm) return (long long)xd.N * xd.L * xd.J <= 0x7FFFFFFF;
-    const int PW = xd.J + 2 * xd.pad_w;
-    const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
-    if (PW > 256 || R > 256) return false;
-    // one K-group of activations plus its dense weights must fit a stage, two stages the shared memory
-    const size_t per_kc = (size_t)R * PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + (size_t)kTcGroupRows * L.tc.st_bytes;
-    return 2 * per_kc + 16384 <= (size_t)kTcMaxSmem;
+    // the per-K-group index of the group plus two stages (one K-group of activations and its dense weights
+    // each) must fit the shared memory
+    const size_t meta = align_up((size_t)L.tc.n_kc * 5, 128);
+    size_t per_kc;
+    if (gemm) {
+        if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
+        per_kc = (size_t)128 * 32 + (size_t)kTcGroupRows * L.tc.st_bytes;
+    } else {
+        const int PW = xd.J + 2 * xd.pad_w;
+        const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
+        if (PW > 256 || R > 256) return false;
+        per_kc = (size_t)R * PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + (size_t)kTcGroupRows * L.tc.st_bytes;
+    }
+    return 2 * (per_kc + 256) + meta + 256 <= (size_t)kTcMaxSmem;
 }
 
 bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
