@@ -578,12 +578,12 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
         int before = block_sum(c, s_sum);
         if (chunk == 0 && part == 0 && threadIdx.x == 0) a.panel_base_out[panel] = (uint32_t)base;
         for (int col = col_lo; col < col_hi; ++col) {
-            unsigned m = 0;
-            for (int r = 0; r < kPanelRows; ++r) {
-                const int o0 = (panel * kPanelRows + r) * kTile;
-                if (o0 >= a.O) break;
-                if (any_kept(s_gamma, o0, o0 + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi)) m |= 1u << r;
-            }
+            // lane r of every warp looks at tile row r; the ballot is the column's mask
+            const int lane = threadIdx.x & 31;
+            const int o0 = (panel * kPanelRows + lane) * kTile;
+            const bool bit = lane < kPanelRows && o0 < a.O &&
+                             any_kept(s_gamma, o0, o0 + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi);
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, bit);
             if (part == 0 && threadIdx.x == 0) {
                 a.colmask_out[(size_t)panel * a.n_cols + col] = (uint8_t)m;
                 a.coloff_out[(size_t)panel * a.n_cols + col] = (uint32_t)before;
@@ -627,9 +627,8 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
             if ((long long)(base + counted) > t.capacity) atomicMax(a.status, (int)BSP_ERR_CAPACITY);
         }
         for (int kc = kc_lo; kc < kc_hi; ++kc) {
-            unsigned m = 0;
-            for (int r = 0; r < kTcGroupRows; ++r)
-                if (st_kept(g * kTcGroupRows + r, kc)) m |= 1u << r;
+            const int lane = threadIdx.x & 31;           // lane r of every warp looks at super-row r
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, lane < kTcGroupRows && st_kept(g * kTcGroupRows + lane, kc));
             if (part == 0 && threadIdx.x == 0) {
                 a.tc_mask_out[(size_t)g * t.n_kc + kc] = (uint8_t)m;
                 a.tc_off_out[(size_t)g * t.n_kc + kc] = (uint32_t)before;
