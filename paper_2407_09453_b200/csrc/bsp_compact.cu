@@ -517,6 +517,17 @@ __device__ __forceinline__ int block_sum(int v, int *warp_sums)
     return tot;
 }
 
+// Non-zero bytes among the first n bytes of Gamma in shared memory (the array is 16-byte aligned), four per load:
+// this thread's share; the caller adds the shares with block_sum().
+__device__ __forceinline__ int ones_share(const uint8_t *g, int n)
+{
+    int c = 0;
+    const int nw = n >> 2;
+    for (int i = threadIdx.x; i < nw; i += kThreads) c += __popc(__vsetne4(((const uint32_t *)g)[i], 0u));
+    if ((int)threadIdx.x < (n & 3)) c += g[(nw << 2) + threadIdx.x] ? 1 : 0;
+    return c;
+}
+
 // True if a block of Gamma (in shared memory) with a one overlaps output channels [o_lo, o_hi] x input channels [c_lo, c_hi].
 __device__ __forceinline__ bool any_kept(const uint8_t *g, int o_lo, int o_hi, int c_lo, int c_hi, int bo, int bi, int NBo, int NBi)
 {
@@ -541,9 +552,7 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
     const int n_fill = a.NBo * a.fill_parts;
     if ((int)blockIdx.x < n_fill) {
         const int l = (int)blockIdx.x / a.fill_parts, part = (int)blockIdx.x % a.fill_parts;
-        int c = 0;
-        for (int i = threadIdx.x; i < l * a.NBi; i += kThreads) c += s_gamma[i] ? 1 : 0;
-        const int first = block_sum(c, s_sum);
+        const int first = block_sum(ones_share(s_gamma, l * a.NBi), s_sum);
         const int cnt = csr_fill_body<T>(l, part, a.fill_parts, (const T *)a.W, a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, first,
                                          a.col_idx, (T *)a.payload, a.capacity_blocks);
         if (part == 0 && threadIdx.x == 0) {
@@ -564,9 +573,13 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
         // stored tiles of the panels above, and of this panel in the columns before col_lo
         int c = 0;
         const int tiles_above = panel * kPanelRows * a.n_cols;
-        for (int q = threadIdx.x; q < tiles_above; q += kThreads) {
-            const int tr = q / a.n_cols, col = q % a.n_cols;
-            c += any_kept(s_gamma, tr * kTile, tr * kTile + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi) ? 1 : 0;
+        if (a.bo == kTile && a.bi == kTile) {
+            c = ones_share(s_gamma, tiles_above);             // an 8x8 block is a tile
+        } else {
+            for (int q = threadIdx.x; q < tiles_above; q += kThreads) {
+                const int tr = q / a.n_cols, col = q % a.n_cols;
+                c += any_kept(s_gamma, tr * kTile, tr * kTile + kTile - 1, col * kTile, col * kTile + kTile - 1, a.bo, a.bi, a.NBo, a.NBi) ? 1 : 0;
+            }
         }
         const int base = block_sum(c, s_sum);
         c = 0;

@@ -112,12 +112,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         for (int q = 0; q < g; ++q) base += p.gcnt[q];
         s_gbase = base; s_gcnt = p.gcnt[g]; s_fail = 0;
         s_payload = p.packed + ((const PackedHeader *)p.packed)->off_tc_payload;
-        for (int s = 0; s < S; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_full[s])), "r"(1) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_empty[s])), "r"(kIssuers) : "memory");
-        }
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_done)), "r"(kIssuers) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     // tile geometry
     int n_img = 0, m0 = 0, y_first = 0, rowbase = 0;
@@ -143,6 +137,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         s_aoff[u] = off;
         s_ahi[u] = smem_desc(0, lbo, 128);
     }
+    // The producer thread sets the barriers up and starts the activation loads of the first stages at once: they
+    // need nothing of the index arrays that the other threads are still fetching.  A full barrier takes two
+    // arrivals per phase, one with the activation bytes and one with the weight bytes.
+    const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
+    const uint32_t ring = s32(smem) + meta_bytes;
+    const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first - p.ph, c3 = p.is_gemm ? m0 : n_img;
+    if (warp == kIssuers && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmap) : "memory");
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_full[s])), "r"(2) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_empty[s])), "r"(kIssuers) : "memory");
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(s32(&s_done)), "r"(kIssuers) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        for (int it = 0; it < min(S, p.n_stage_iters); ++it) {
+            const uint32_t bar = s32(&s_full[it]);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
+            asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+                         ::"r"(ring + it * p.stage_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(it * p.GK * p.chunks_per_kc) : "memory");
+        }
+    }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(s32(&s_tmem)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
@@ -164,9 +179,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
 
-    const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
-    const uint32_t ring = s32(smem) + meta_bytes;
-
     if (warp == kIssuers) {
         // ================= producer (warp 4) =================
         if (lane == 0) {
@@ -179,11 +191,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t wbytes = (o_hi - o_lo) * (uint32_t)p.st_bytes;
                 const uint32_t bar = s32(&s_full[slot]);
                 const uint32_t dst = ring + slot * p.stage_bytes;
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes + wbytes) : "memory");
-                const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first - p.ph, c3 = p.is_gemm ? m0 : n_img;
-                const int c4 = kc0 * p.chunks_per_kc;
-                asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
-                             ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+                if (it >= S) {          // the first S activation loads were issued before the index arrays arrived
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
+                    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+                                 ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(kc0 * p.chunks_per_kc) : "memory");
+                }
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(wbytes) : "memory");
                 if (wbytes)
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
                                  ::"r"(dst + p.act_bytes), "l"(s_payload + (size_t)(s_gbase + o_lo) * p.st_bytes), "r"(wbytes), "r"(bar) : "memory");
