@@ -49,6 +49,7 @@ struct TcParams {
     int N, O, M, Nw, P, H, K, ph, pw;
     int PW, plane_bytes, tiles_per_img, is_gemm;
     int n_kc, n_units, st_bytes, chunks_per_kc;
+    int coords_per_kc;        // steps of the tensor map's last coordinate per K-group
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
     int ytype;
 };
@@ -87,7 +88,7 @@ __device__ __forceinline__ void commit_to(uint32_t bar)
 __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_constant__ TcParams p)
 {
     extern __shared__ __align__(16) uint8_t tc_smem_raw[];
-    uint8_t *smem = tc_smem_raw + ((128u - (s32(tc_smem_raw) & 127u)) & 127u);
+    uint8_t *smem = tc_smem_raw + ((1024u - (s32(tc_smem_raw) & 1023u)) & 1023u);   // stages of swizzled planes start on 1 KB
     __shared__ __align__(8) uint64_t s_full[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_empty[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_done;
@@ -124,7 +125,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     }
     for (int u = tid; u < p.n_units; u += kTcThreads) {
         uint32_t lbo, off;
-        if (p.chunks_per_kc == 2) {                 // 1x1 kernel: the K halves are two 8-channel planes
+        if (p.is_gemm) {
+            // matrix product: a K-group's plane is [position][32 bytes = 16 channels] under the 32-byte swizzle,
+            // 8 positions (256 bytes) per row group; the leading-dimension offset is not used
+            s_aoff[u] = 0;
+            s_ahi[u] = smem_desc(0, 16, 256) | (6ull << 61);
+            continue;
+        }
+        if (p.chunks_per_kc == 2) {                 // 1x1 kernel with padding: the K halves are two 8-channel planes
             off = (uint32_t)rowbase;
             lbo = (uint32_t)p.plane_bytes;
         } else {
@@ -140,7 +148,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     // The producer thread sets the barriers up and starts the activation loads of the first stages at once: they
     // need nothing of the index arrays that the other threads are still fetching.  A full barrier takes two
     // arrivals per phase, one with the activation bytes and one with the weight bytes.
-    const int meta_bytes = ((p.n_kc * 5 + 127) / 128) * 128;
+    const int meta_bytes = ((p.n_kc * 5 + 1023) / 1024) * 1024;
     const uint32_t ring = s32(smem) + meta_bytes;
     const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first - p.ph, c3 = p.is_gemm ? m0 : n_img;
     if (warp == kIssuers && lane == 0) {
@@ -155,7 +163,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             const uint32_t bar = s32(&s_full[it]);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
             asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
-                         ::"r"(ring + it * p.stage_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(it * p.GK * p.chunks_per_kc) : "memory");
+                         ::"r"(ring + it * p.stage_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(it * p.GK * p.coords_per_kc) : "memory");
         }
     }
     if (warp == 0) {
@@ -194,7 +202,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 if (it >= S) {          // the first S activation loads were issued before the index arrays arrived
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
                     asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
-                                 ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(kc0 * p.chunks_per_kc) : "memory");
+                                 ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(kc0 * p.coords_per_kc) : "memory");
                 }
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(wbytes) : "memory");
                 if (wbytes)
@@ -349,7 +357,7 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
     const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
     // the per-K-group index of the group plus two stages (one K-group of activations and its dense weights
     // each) must fit the shared memory
-    const size_t meta = align_up((size_t)L.tc.n_kc * 5, 128);
+    const size_t meta = align_up((size_t)L.tc.n_kc * 5, 1024);
     size_t per_kc;
     if (gemm) {
         if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
@@ -360,7 +368,7 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
         if (PW > 256 || R > 256) return false;
         per_kc = (size_t)R * PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + (size_t)kTcGroupRows * L.tc.st_bytes;
     }
-    return 2 * (per_kc + 256) + meta + 256 <= (size_t)kTcMaxSmem;
+    return 2 * (per_kc + 1024) + meta + 1024 <= (size_t)kTcMaxSmem;
 }
 
 bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
@@ -380,6 +388,7 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     p.P = xd.N * p.M * p.Nw;
     p.is_gemm = gemm ? 1 : 0;
     p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch / 8;
+    p.coords_per_kc = gemm ? 1 : p.chunks_per_kc;
     int plane_pos, R = 1;
     long long tiles;
     if (gemm) {
@@ -400,29 +409,31 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     p.GK = GK;
     p.act_box_bytes = GK * p.chunks_per_kc * p.plane_bytes;
     p.act_bytes = (int)align_up((size_t)p.act_box_bytes + 32, 128);      // + slack read by positions in the padding
-    p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)GK * kTcGroupRows * T.st_bytes, 128);
+    p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)GK * kTcGroupRows * T.st_bytes, 1024);
     p.n_stage_iters = (T.n_kc + GK - 1) / GK;
-    const size_t meta = align_up((size_t)T.n_kc * 5, 128);
-    int stages = (int)(((size_t)kTcMaxSmem - meta - 256) / p.stage_bytes);
+    const size_t meta = align_up((size_t)T.n_kc * 5, 1024);
+    int stages = (int)(((size_t)kTcMaxSmem - meta - 1024) / p.stage_bytes);
     if (stages > kTcMaxStages) stages = kTcMaxStages;
     if (stages > p.n_stage_iters) stages = p.n_stage_iters;
     if (stages < 1) return BSP_ERR_SHAPE;
     p.stages = stages;
     p.ytype = ytype;
-    const size_t smem = meta + (size_t)stages * p.stage_bytes + 256;
+    const size_t smem = meta + (size_t)stages * p.stage_bytes + 1024;
 
     EncodeTiledFn enc = tc_encode_tiled();
     if (!enc) return BSP_ERR_CUDA;
     const cuuint64_t row = (cuuint64_t)wd.I * 2;
     const cuuint64_t gJ = gemm ? 1 : (cuuint64_t)xd.J, gL = gemm ? 1 : (cuuint64_t)xd.L, gN = gemm ? (cuuint64_t)n_pos : (cuuint64_t)xd.N;
-    const cuuint64_t gdim[5] = {16, gJ, gL, gN, (cuuint64_t)(wd.I / 8)};
-    const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, 16};
+    // innermost extent: one 8-channel chunk (16 bytes), or for a matrix product a whole K-group (32 bytes, swizzled)
+    const cuuint64_t inner = gemm ? 32 : 16;
+    const cuuint64_t gdim[5] = {inner, gJ, gL, gN, (cuuint64_t)(wd.I * 2 / inner)};
+    const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, inner};
     cuuint32_t box[5];
-    if (gemm) { box[0] = 16; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
+    if (gemm) { box[0] = 32; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)GK; }
     else { box[0] = 16; box[1] = (cuuint32_t)p.PW; box[2] = (cuuint32_t)R; box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     if (enc(&p.tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void *>(X), gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, gemm ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return BSP_ERR_CUDA;
 
