@@ -43,11 +43,10 @@ __device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc
 // Sum of one output row r of block B over (h, k, c) in that order, for a block of WORDS 32-bit words per tap.
 // Loads of up to nine taps (a whole 3x3 kernel) are issued together, as 16-byte loads when `vec` says that the
 // rows are 16-byte aligned; the adds keep the (h, k, c) order.
-template <int DT, int NORM, int WORDS>
+template <int DT, int NORM, int WORDS, int kBatch>
 __device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__restrict__ src, size_t row_words, int HK, bool vec)
 {
     using acc_t = typename Acc<DT>::type;
-    constexpr int kBatch = 9;
     acc_t pr = 0;
     for (int t = 0; t < HK; t += kBatch) {
         uint32_t w[kBatch][WORDS];
@@ -85,7 +84,9 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__re
     return pr;
 }
 
-template <int DT, int NORM>
+// kBatch = taps whose loads are in flight together: 9 (a 3x3 kernel at once), or 1 in the kernels compiled for
+// one-tap layers, which then need few registers and keep many CTAs resident.
+template <int DT, int NORM, int kBatch>
 __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
                                                           int NBi, long long B, int r)
 {
@@ -96,15 +97,15 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__rest
     const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
     const bool vec = (((uintptr_t)W) & 15u) == 0 && row_words % 4 == 0;
     switch (words) {
-        case 1: return row_sum_w<DT, NORM, 1>(src, row_words, HK, vec);
-        case 2: return row_sum_w<DT, NORM, 2>(src, row_words, HK, vec);
-        case 4: return row_sum_w<DT, NORM, 4>(src, row_words, HK, vec);
-        case 8: return row_sum_w<DT, NORM, 8>(src, row_words, HK, vec);
-        default: return row_sum_w<DT, NORM, 16>(src, row_words, HK, vec);
+        case 1: return row_sum_w<DT, NORM, 1, kBatch>(src, row_words, HK, vec);
+        case 2: return row_sum_w<DT, NORM, 2, kBatch>(src, row_words, HK, vec);
+        case 4: return row_sum_w<DT, NORM, 4, kBatch>(src, row_words, HK, vec);
+        case 8: return row_sum_w<DT, NORM, 8, kBatch>(src, row_words, HK, vec);
+        default: return row_sum_w<DT, NORM, 16, kBatch>(src, row_words, HK, vec);
     }
 }
 
-template <int DT, int NORM>
+template <int DT, int NORM, int kBatch>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
              typename Acc<DT>::type *__restrict__ score)
@@ -116,7 +117,7 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
     const int r = threadIdx.x / blocks_per_cta;
     const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
     const long long NB = (long long)NBo * NBi;
-    part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+    part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
     __syncthreads();
     if (B < NB && r == 0) {
         acc_t total = 0;
@@ -254,10 +255,18 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
         __syncthreads();
         const unsigned long long prefix = s_prefix;
         const int shift = 8 * pass;
-        for (long long i = lo + tid; i < hi; i += kCoopThreads) {
-            const unsigned long long v = key[i];
-            const bool in = (pass == 7) || ((v >> (shift + 8)) == prefix);
-            if (in) atomicAdd(&hist[(unsigned)((v >> shift) & 0xFFull)], 1u);
+        // lanes with the same digit add once (the leading digits of float keys are nearly all alike)
+        for (long long base = lo; base < hi; base += kCoopThreads) {
+            const long long i = base + tid;
+            unsigned long long v = 0ull;
+            bool in = false;
+            if (i < hi) {
+                v = key[i];
+                in = (pass == 7) || ((v >> (shift + 8)) == prefix);
+            }
+            const unsigned digit = in ? (unsigned)((v >> shift) & 0xFFull) : 256u;
+            const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+            if (in && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
         }
         __syncthreads();
         if (tid < 256 && hist[tid]) atomicAdd(&ghist[pass * 256 + tid], hist[tid]);
@@ -372,7 +381,7 @@ rank_kernel(const unsigned long long *__restrict__ key, int seg_len, long long n
 // from zero whatever its grid) and a generation that the last arriver bumps; the wait on the generation is
 // bounded and latches BSP_ERR_TIMEOUT.
 
-template <int DT, int NORM>
+template <int DT, int NORM, int kBatch>
 __global__ void __launch_bounds__(kScoreThreads)
 mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi, int BC,
                   typename Acc<DT>::type *score, int seg_len, long long n_zero, uint8_t *__restrict__ gamma,
@@ -387,7 +396,7 @@ mask_small_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
         const int bl = threadIdx.x % BC, r = threadIdx.x / BC;
         const long long B = (long long)blockIdx.x * BC + bl;
         const bool mine = r < bo && B < NB;
-        part[threadIdx.x] = mine ? row_sum<DT, NORM>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+        part[threadIdx.x] = mine ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
         __syncthreads();
         if (mine && r == 0) {
             acc_t total = 0;
@@ -444,7 +453,8 @@ bsp_status run_mask_small(const bsp_wdesc &wd, const void *W, int seg_len, long 
     while ((NBo * NBi + BC - 1) / BC > 128 && BC * 2 * wd.bo <= kScoreThreads) BC *= 2;
     const unsigned grid = (unsigned)((NBo * NBi + BC - 1) / BC);
     void *args[] = {&Wp, &I, &HK, &bo, &bi, &NBo, &NBi, &BC, &sc, &seg_len, &n_zero, &gamma, &sync, &status};
-    BSP_CUDA_OK(cudaLaunchCooperativeKernel((const void *)mask_small_kernel<DT, NORM>, dim3(grid), dim3(kScoreThreads), args, 0, st));
+    const void *kern = HK == 1 ? (const void *)mask_small_kernel<DT, NORM, 1> : (const void *)mask_small_kernel<DT, NORM, 9>;
+    BSP_CUDA_OK(cudaLaunchCooperativeKernel(kern, dim3(grid), dim3(kScoreThreads), args, 0, st));
     return BSP_OK;
 }
 
@@ -456,12 +466,16 @@ bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *s
     const long long NB = (long long)NBo * NBi;
     const int per_cta = kScoreThreads / wd.bo;
     const unsigned grid = (unsigned)((NB + per_cta - 1) / per_cta);
-    if (norm == BSP_NORM_L2)
-        score_kernel<DT, BSP_NORM_L2><<<grid, kScoreThreads, 0, st>>>((const uint32_t *)W, wd.I, wd.H * wd.K, wd.bo,
-                                                                       wd.bi, NBo, NBi, (acc_t *)scores);
-    else
-        score_kernel<DT, BSP_NORM_L1><<<grid, kScoreThreads, 0, st>>>((const uint32_t *)W, wd.I, wd.H * wd.K, wd.bo,
-                                                                       wd.bi, NBo, NBi, (acc_t *)scores);
+    const int HK = wd.H * wd.K;
+    const uint32_t *Wp = (const uint32_t *)W;
+    acc_t *sc = (acc_t *)scores;
+    if (norm == BSP_NORM_L2) {
+        if (HK == 1) score_kernel<DT, BSP_NORM_L2, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+        else score_kernel<DT, BSP_NORM_L2, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+    } else {
+        if (HK == 1) score_kernel<DT, BSP_NORM_L1, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+        else score_kernel<DT, BSP_NORM_L1, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+    }
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }
