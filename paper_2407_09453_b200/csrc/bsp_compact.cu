@@ -210,6 +210,42 @@ scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_
     }
 }
 
+// Copies the cnt stored blocks of row l (columns s_cols[]) into the canonical payload in pieces of type V (one or
+// several elements; a block row of b_i elements is contiguous in W and in the payload).  Each thread loads four
+// pieces before it stores them.
+template <typename T, typename V>
+__device__ __forceinline__ void fill_copy(int l, int part, int parts, const T *__restrict__ W, int I, int HK, int bo, int bi,
+                                          int first, int cnt, const int *s_cols, T *__restrict__ payload,
+                                          long long capacity_blocks)
+{
+    constexpr int per = (int)(sizeof(V) / sizeof(T));
+    const int bi_v = bi / per;                          // pieces per block row, a power of two
+    const int blk = bo * HK * bi;
+    const unsigned blk_v = (unsigned)(bo * HK * bi_v);
+    const unsigned total = (unsigned)cnt * blk_v;       // at most I * b_o * H * K: fits 32 bits
+    const unsigned stride = (unsigned)parts * kThreads;
+    for (unsigned e0 = (unsigned)part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+        V v[4];
+        V *dst[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned e = e0 + u * stride;
+            ok[u] = e < total;
+            const int n = ok[u] ? (int)(e / blk_v) : 0;
+            const int q = ok[u] ? (int)(e - (unsigned)n * blk_v) : 0;
+            const int c = q & (bi_v - 1), rt = q >> lg(bi_v);
+            const int r = rt / HK, t = rt - r * HK;
+            ok[u] = ok[u] && (long long)(first + n) < capacity_blocks;
+            dst[u] = (V *)(payload + (size_t)(first + n) * blk + (size_t)rt * bi) + c;
+            if (ok[u]) v[u] = *((const V *)(W + ((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi) + c);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (ok[u]) *dst[u] = v[u];
+    }
+}
+
 // Final launch, first part.  `parts` CTAs per row of Gamma: column indices in ascending order and the canonical payload
 // payload[n][r][h][k][c] = W[l b_o + r][h][k][iota b_i + c].  `first` = stored blocks in the rows above; returns
 // the number of stored blocks of row l.
@@ -241,33 +277,16 @@ __device__ __forceinline__ int csr_fill_body(int l, int part, int parts, const T
     }
     if (payload == nullptr) return s_run;
     const int cnt = s_run;
-    const int blk = bo * HK * bi;
-    const long long total = (long long)cnt * blk;      // at most I * b_o * H * K elements: fits 32 bits
-    // the CTAs of one row (`parts` of them) all build the column list, then share the copy; the loads of four
-    // elements are issued before the first store
-    const unsigned stride = (unsigned)parts * kThreads, utotal = (unsigned)total, ublk = (unsigned)blk;
-    for (unsigned e0 = (unsigned)part * kThreads + threadIdx.x; e0 < utotal; e0 += 4 * stride) {
-        T v[4];
-        size_t dst[4];
-        bool ok[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const unsigned e = e0 + u * stride;
-            ok[u] = e < utotal;
-            const int n = ok[u] ? (int)(e / ublk) : 0;
-            const int q = ok[u] ? (int)(e - (unsigned)n * ublk) : 0;
-            int rem = q;
-            const int c = rem & (bi - 1); rem >>= lg(bi);
-            const int r = rem / HK;
-            const int t = rem - r * HK;
-            ok[u] = ok[u] && (long long)(first + n) < capacity_blocks;
-            dst[u] = (size_t)(first + n) * blk + q;
-            v[u] = ok[u] ? W[((size_t)(l * bo + r) * HK + t) * I + (size_t)s_cols[n] * bi + c] : (T)0;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (ok[u]) payload[dst[u]] = v[u];
-    }
+    // the CTAs of one row (`parts` of them) all build the column list, then share the copy, in the widest pieces
+    // (up to 16 bytes) that the block width, the row pitch of W and the two base addresses allow
+    const size_t row_bytes = (size_t)bi * sizeof(T), pitch = (size_t)I * sizeof(T);
+    const uintptr_t bases = (uintptr_t)W | (uintptr_t)payload;
+    size_t vb = 16;
+    while (vb > sizeof(T) && (row_bytes % vb || pitch % vb || bases % vb)) vb >>= 1;
+    if (vb == 16) fill_copy<T, uint4>(l, part, parts, W, I, HK, bo, bi, first, cnt, s_cols, payload, capacity_blocks);
+    else if (vb == 8) fill_copy<T, uint2>(l, part, parts, W, I, HK, bo, bi, first, cnt, s_cols, payload, capacity_blocks);
+    else if (vb == 4 && sizeof(T) < 4) fill_copy<T, uint32_t>(l, part, parts, W, I, HK, bo, bi, first, cnt, s_cols, payload, capacity_blocks);
+    else fill_copy<T, T>(l, part, parts, W, I, HK, bo, bi, first, cnt, s_cols, payload, capacity_blocks);
     return cnt;
 }
 
@@ -316,6 +335,72 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
     }
 }
 
+// Eight consecutive input channels (16 bytes) of W[o][tap][ch0 ..] in bf16, with the channels of zeroed blocks
+// cleared; rows past O and taps past HK read as zero.  Needs I % 8 == 0 and a 16-byte aligned W.
+__device__ __forceinline__ uint4 bf16_chunk(const uint16_t *__restrict__ W, const uint8_t *gamma, int o, int tap, int ch0,
+                                            int O, int I, int HK, int bo, int bi, int NBi)
+{
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (o >= O || tap >= HK) return v;
+    const uint8_t *grow = gamma + (size_t)(o >> lg(bo)) * NBi;
+    if (bi >= 8) {
+        if (grow[ch0 >> lg(bi)] == 0) return v;
+        return __ldg((const uint4 *)(W + ((size_t)o * HK + tap) * I + ch0));
+    }
+    const bool k0 = grow[ch0 >> 2] != 0, k1 = grow[(ch0 >> 2) + 1] != 0;    // b_i = 4: two blocks per chunk
+    if (!k0 && !k1) return v;
+    v = __ldg((const uint4 *)(W + ((size_t)o * HK + tap) * I + ch0));
+    if (!k0) v.x = v.y = 0u;
+    if (!k1) v.z = v.w = 0u;
+    return v;
+}
+
+// bf16 tiles of one (panel, tile column) in 16-byte chunks: the 32 bytes of tile row g in a two-tap step are the
+// words of its two chunks interleaved (w0 v0 w1 v1 ...), the 16 bytes of an odd last tap are its chunk.
+__device__ __forceinline__ void pack_tiles_bf16(unsigned m, unsigned first, int panel, int col, const uint16_t *__restrict__ W,
+                                                const uint8_t *gamma, int O, int I, int HK, int bo, int bi, int NBi,
+                                                int tile_bytes, uint8_t *__restrict__ payload, long long capacity_tiles,
+                                                int part, int parts)
+{
+    const int pairs = HK >> 1;
+    const int ipt = (pairs + (HK & 1)) * 8;             // items per tile: (step, tile row)
+    const int total = __popc(m) * ipt;
+    const int stride = parts * kThreads;
+    for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 2 * stride) {
+        uint4 a[2], b[2];
+        uint8_t *dst[2];
+        bool ok[2], two[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int e = e0 + u * stride;
+            ok[u] = e < total;
+            const int j = ok[u] ? (int)((unsigned)e / (unsigned)ipt) : 0, rem = ok[u] ? e - j * ipt : 0;
+            const int s = rem >> 3, g = rem & 7;
+            unsigned mm = m;
+            for (int q = 0; q < j; ++q) mm &= mm - 1;
+            const int o = (panel * kPanelRows + (__ffs(mm) - 1)) * kTile + g;
+            ok[u] = ok[u] && (long long)(first + j) < capacity_tiles;
+            two[u] = s < pairs;
+            dst[u] = payload + (size_t)(first + j) * tile_bytes + (two[u] ? s * 256 + g * 32 : pairs * 256 + g * 16);
+            a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (ok[u]) {
+                a[u] = bf16_chunk(W, gamma, o, two[u] ? 2 * s : HK - 1, col * kTile, O, I, HK, bo, bi, NBi);
+                if (two[u]) b[u] = bf16_chunk(W, gamma, o, 2 * s + 1, col * kTile, O, I, HK, bo, bi, NBi);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (!ok[u]) continue;
+            if (two[u]) {
+                ((uint4 *)dst[u])[0] = make_uint4(a[u].x, b[u].x, a[u].y, b[u].y);
+                ((uint4 *)dst[u])[1] = make_uint4(a[u].z, b[u].z, a[u].w, b[u].w);
+            } else {
+                *(uint4 *)dst[u] = a[u];
+            }
+        }
+    }
+}
+
 // The stored tiles of one (panel, tile column), whose tile rows are the set bits of m, written word by word
 // from slot `first` on.  `parts` CTAs share the words; each thread loads four before it stores.
 template <int DT>
@@ -324,6 +409,13 @@ __device__ __forceinline__ void pack_tiles(unsigned m, unsigned first, int panel
                                            int tile_bytes, uint8_t *__restrict__ payload, long long capacity_tiles,
                                            int part, int parts)
 {
+    if constexpr (DT == BSP_BF16) {
+        if ((I & 7) == 0 && (((uintptr_t)W) & 15u) == 0) {
+            pack_tiles_bf16(m, first, panel, col, (const uint16_t *)W, gamma, O, I, HK, bo, bi, NBi, tile_bytes, payload,
+                            capacity_tiles, part, parts);
+            return;
+        }
+    }
     const int words = tile_bytes / 4;
     const int total = __popc(m) * words;
     const int stride = parts * kThreads;
@@ -404,8 +496,38 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
                                               const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I,
                                               int HK, int bo, int bi, int NBi, int part, int parts)
 {
-    const int words = t.st_bytes / 4;
     const int cnt = __popc(m);
+    if ((I & 7) == 0 && (((uintptr_t)W) & 15u) == 0) {
+        // 16-byte chunks: one (row group, K half, row) slot of a K-step is eight channels of one weight row and tap
+        const int nu = t.st_bytes >> 9;
+        const int total = cnt * nu * 32;
+        const int stride = parts * kThreads;
+        for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
+            uint4 v[4];
+            uint4 *dst[4];
+            bool ok[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = e0 + u * stride;
+                ok[u] = e < total;
+                const int j = ok[u] ? (int)((unsigned)e / (unsigned)(nu * 32)) : 0, rem = ok[u] ? e - j * nu * 32 : 0;
+                const int ks = rem >> 5, slot = rem & 31;
+                const int rg = slot >> 4, h = (slot >> 3) & 1, row = slot & 7;
+                unsigned mm = m;
+                for (int q = 0; q < j; ++q) mm &= mm - 1;
+                const int o = (g * kTcGroupRows + (__ffs(mm) - 1)) * kTcSuperRow + rg * 8 + row;
+                const int tap = HK == 1 ? 0 : 2 * ks + h, ch0 = HK == 1 ? (2 * kc + h) * 8 : kc * 8;
+                ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
+                dst[u] = (uint4 *)(t.payload + (size_t)first * t.st_bytes + ((size_t)(ks * cnt + j) << 9)) + slot;
+                v[u] = ok[u] ? bf16_chunk((const uint16_t *)W, gamma, o, tap, ch0, O, I, HK, bo, bi, NBi) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (ok[u]) *dst[u] = v[u];
+        }
+        return;
+    }
+    const int words = t.st_bytes / 4;
     const int total = cnt * words;
     const int stride = parts * kThreads;
     for (int e0 = part * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
@@ -730,13 +852,20 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
                                      (tc_on ? a.tc.chunks * a.tc.n_groups : 0));
     const size_t smem = (size_t)NBi * sizeof(int);
     if ((long long)NBo * NBi <= kSmallBlocks) {
-        // enough CTAs per tile column / K-group that a thread writes about four words
-        auto parts_for = [](int words_per_tile) {
-            const int p = (kPanelRows * words_per_tile + 4 * kThreads - 1) / (4 * kThreads);
-            return p < 1 ? 1 : (p > 8 ? 8 : p);
+        // enough CTAs per row, tile column and K-group that a thread moves about four pieces: 16-byte chunks for
+        // bf16 (two per item in the first packed form), 32-bit words otherwise
+        auto parts_for = [](long long items, int per_thread) {
+            const long long p = (items + (long long)per_thread * kThreads - 1) / ((long long)per_thread * kThreads);
+            return (int)(p < 1 ? 1 : (p > 8 ? 8 : p));
         };
-        a.pack_parts = parts_for(L.tile_bytes / 4);
-        a.tc_parts = tc_on ? parts_for(L.tc.st_bytes / 4) : 1;
+        const bool chunks = wd.wtype == BSP_BF16 && wd.I % 8 == 0 && ((uintptr_t)W & 15u) == 0;
+        a.pack_parts = chunks ? parts_for((long long)kPanelRows * ((HK + 1) / 2) * 8, 2) : parts_for((long long)kPanelRows * L.tile_bytes / 4, 4);
+        a.tc_parts = !tc_on ? 1 : chunks ? parts_for((long long)kTcGroupRows * L.tc.n_units * 32, 4) : parts_for((long long)kTcGroupRows * L.tc.st_bytes / 4, 4);
+        if (payload) {
+            const size_t esz = wd.wtype == BSP_F32 ? 4 : (wd.wtype == BSP_BF16 ? 2 : 1);
+            const long long row_pieces = (long long)NBi * wd.bo * HK * ((wd.bi * esz + 15) / 16);   // a row with every block stored
+            a.fill_parts = parts_for(row_pieces / 2, 4);
+        }
         const unsigned grid_small = (unsigned)(NBo * a.fill_parts + (pk ? a.pack_chunks * L.n_panels * a.pack_parts : 0) +
                                                (tc_on ? a.tc.chunks * a.tc.n_groups * a.tc_parts : 0));
         a.row_ptr_out = row_ptr; a.colmask_out = colmask; a.coloff_out = coloff; a.panel_base_out = panel_base;
