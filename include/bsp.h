@@ -17,6 +17,9 @@
  *    allocating it (they hold the latched status word and the counters of the grid-wide barrier that the
  *    single-launch kernels of small layers use); one workspace sized for the largest request may serve all
  *    calls issued on one stream, and a workspace must not be shared by calls running on different streams.
+ *  - Alignment: W and the canonical payload must be 4-byte aligned (the set-up kernels read
+ *    32-bit words and use 16-byte accesses when the addresses allow it); X, Y and the packed buffer 16-byte
+ *    aligned.  A misaligned pointer is BSP_ERR_SHAPE.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue work and
  *    return; results are valid once the stream has been synchronised.
  *  - Every function returns a bsp_status; nothing throws.  Argument errors are detected on the host

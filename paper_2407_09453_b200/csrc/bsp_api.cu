@@ -28,6 +28,7 @@ bsp_status check_wdesc(const bsp_wdesc *wd)
 }
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+bool aligned4(const void *p) { return ((uintptr_t)p & 3u) == 0; }
 
 // The tensor-memory kernel takes every layer it can run unless BSP_CONV_PATH asks for the warp-MMA kernel.
 bool use_tc(const bsp_wdesc &wd, const bsp_xdesc &xd)
@@ -70,6 +71,7 @@ bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope
     bsp_status rc = check_wdesc(wd);
     if (rc != BSP_OK) return rc;
     if (!W || !gamma || !ws) return BSP_ERR_NULL;
+    if (!aligned4(W)) return BSP_ERR_SHAPE;
     if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1) return BSP_ERR_DTYPE;
     if (scope != BSP_SCOPE_LAYER && scope != BSP_SCOPE_ROW) return BSP_ERR_DTYPE;
     const int64_t NBi = wd->I / wd->bi, NB = (int64_t)(wd->O / wd->bo) * NBi;
@@ -118,6 +120,7 @@ bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma,
     if (capacity_blocks < 0) return BSP_ERR_CAPACITY;
     if (packed && (wd->O % 8 != 0 || wd->I % 8 != 0)) return BSP_ERR_SHAPE;
     if (packed && !aligned16(packed)) return BSP_ERR_SHAPE;
+    if (!aligned4(W) || (payload && !aligned4(payload))) return BSP_ERR_SHAPE;
     return launch_compact(*wd, W, gamma, row_ptr, col_idx, payload, packed, capacity_blocks, ws, (cudaStream_t)stream);
 }
 
@@ -175,7 +178,9 @@ bsp_status bsp_check(void *ws, void *stream)
     int h = 0;
     BSP_CUDA_OK(cudaMemcpyAsync(&h, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     BSP_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
-    if (h != 0) BSP_CUDA_OK(cudaMemsetAsync(ws, 0, sizeof(int), (cudaStream_t)stream));
+    // a latched status is cleared once read; after a timeout the grid-barrier words are cleared with it, since a
+    // launch that gave up may have left arrivals behind
+    if (h != 0) BSP_CUDA_OK(cudaMemsetAsync(ws, 0, h == (int)BSP_ERR_TIMEOUT ? (kWsSyncWord + 2) * sizeof(int) : sizeof(int), (cudaStream_t)stream));
     if (h < 0 || h > (int)BSP_ERR_TIMEOUT) return BSP_ERR_CUDA;
     return (bsp_status)h;
 }

@@ -454,7 +454,12 @@ bsp_status run_mask_small(const bsp_wdesc &wd, const void *W, int seg_len, long 
     const unsigned grid = (unsigned)((NBo * NBi + BC - 1) / BC);
     void *args[] = {&Wp, &I, &HK, &bo, &bi, &NBo, &NBi, &BC, &sc, &seg_len, &n_zero, &gamma, &sync, &status};
     const void *kern = HK == 1 ? (const void *)mask_small_kernel<DT, NORM, 1> : (const void *)mask_small_kernel<DT, NORM, 9>;
-    BSP_CUDA_OK(cudaLaunchCooperativeKernel(kern, dim3(grid), dim3(kScoreThreads), args, 0, st));
+    const cudaError_t e = cudaLaunchCooperativeKernel(kern, dim3(grid), dim3(kScoreThreads), args, 0, st);
+    if (e == cudaErrorCooperativeLaunchTooLarge) {      // fewer SMs than CTAs (a partitioned GPU): the caller takes the multi-launch path
+        (void)cudaGetLastError();
+        return BSP_ERR_CAPACITY;
+    }
+    BSP_CUDA_OK(e);
     return BSP_OK;
 }
 
@@ -493,14 +498,17 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
             int *status = (int *)ws;
             unsigned *sync = (unsigned *)ws + kWsSyncWord;
             const bool l2 = norm == BSP_NORM_L2;
+            bsp_status small;
             if (wd.wtype == BSP_F32)
-                return l2 ? run_mask_small<BSP_F32, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
-                          : run_mask_small<BSP_F32, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
-            if (wd.wtype == BSP_BF16)
-                return l2 ? run_mask_small<BSP_BF16, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
-                          : run_mask_small<BSP_BF16, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
-            return l2 ? run_mask_small<BSP_I8, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
-                      : run_mask_small<BSP_I8, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+                small = l2 ? run_mask_small<BSP_F32, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                           : run_mask_small<BSP_F32, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+            else if (wd.wtype == BSP_BF16)
+                small = l2 ? run_mask_small<BSP_BF16, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                           : run_mask_small<BSP_BF16, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+            else
+                small = l2 ? run_mask_small<BSP_I8, BSP_NORM_L2>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st)
+                           : run_mask_small<BSP_I8, BSP_NORM_L1>(wd, W, seg_len, n_zero, gamma, scores, sync, status, st);
+            if (small != BSP_ERR_CAPACITY) return small;
         }
     }
     if (wd.wtype == BSP_F32) rc = run_scores<BSP_F32>(wd, W, norm, scores, st);
@@ -532,7 +540,14 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
         unsigned *sync = (unsigned *)ws + kWsSyncWord;
         int *status = (int *)ws;
         void *args[] = {&keys, &n, &nz, &gamma, &ghist, &geq, &sync, &status};
-        BSP_CUDA_OK(cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, 0, st));
+        const cudaError_t e = cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, 0, st);
+        if (e == cudaErrorCooperativeLaunchTooLarge) {
+            (void)cudaGetLastError();
+            select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
+            BSP_CUDA_OK(cudaGetLastError());
+            return BSP_OK;
+        }
+        BSP_CUDA_OK(e);
         return BSP_OK;
     } else
         select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);

@@ -24,6 +24,7 @@ extern "C" bsp_status bsp_mask_static(const bsp_wdesc *wd, const void *W, bsp_no
     if (wd->O % wd->bo != 0 || wd->I % wd->bi != 0) return BSP_ERR_SHAPE;
     if (wd->wtype != BSP_F32 && wd->wtype != BSP_BF16 && wd->wtype != BSP_I8) return BSP_ERR_DTYPE;
     if (!W || !gamma) return BSP_ERR_NULL;
+    if (((uintptr_t)W & 3u) != 0) return BSP_ERR_SHAPE;
     if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1) return BSP_ERR_DTYPE;
     if (scope != BSP_SCOPE_LAYER && scope != BSP_SCOPE_ROW) return BSP_ERR_DTYPE;
     const int64_t NBi = wd->I / wd->bi, NB = (int64_t)(wd->O / wd->bo) * NBi;

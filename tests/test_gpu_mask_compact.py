@@ -115,6 +115,39 @@ def test_compact_more_blocks_than_the_single_launch_path_takes(dtype, bo, bi):
     assert np.array_equal(got, pl if dtype != "bf16" else pl.astype(np.float32))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "i8", "f32"])
+def test_mask_and_compact_of_weights_at_an_odd_address(dtype):
+    """W starting four bytes into an allocation: the 16-byte loads of the score and copy loops must give way to
+    narrower ones, with the same bits out; an address that is not a multiple of four is refused."""
+    bo = bi = 8
+    O, I, H, K = 64, 72, 3, 3
+    W = make_case(127, O, I, H, K, dtype)
+    skip = {"bf16": 2, "i8": 4, "f32": 1}[dtype]
+    big = torch.empty(W.size + 16, dtype=TORCH_DT[dtype], device="cuda")
+    Wd = big[skip:skip + W.size].view(O, H, K, I)
+    Wd.copy_(to_dev(W, dtype))
+    assert Wd.data_ptr() % 16 == 4
+    lay = bsp.SparseLayer(O, I, H, K, bo, bi, TORCH_DT[dtype])
+    if dtype != "f32":
+        odd = big[1:1 + W.size].view(O, H, K, I)
+        with pytest.raises(bsp.BspError) as e:
+            lay.mask(odd, 1)
+        assert e.value.status == bsp.ERR_SHAPE
+    sc = torch.empty(lay.NBo * lay.NBi, dtype=torch.int64 if dtype == "i8" else torch.float64, device="cuda")
+    n_zero = lay.NBo * lay.NBi // 2
+    lay.mask(Wd, n_zero, scores=sc)
+    lay.compact(Wd)
+    lay.check()
+    want_s = ref.scores(W, bo, bi)
+    assert np.array_equal(from_dev(sc).view(np.uint64), want_s.reshape(-1).view(np.uint64))
+    g = ref.mask(want_s, n_zero)
+    assert np.array_equal(from_dev(lay.gamma).reshape(g.shape), g)
+    rp, ci, pl = ref.compact(W, g, bo, bi)
+    assert np.array_equal(from_dev(lay.row_ptr), rp) and np.array_equal(from_dev(lay.col_idx)[:len(ci)], ci)
+    got = from_dev(lay.payload)[:pl.size].reshape(pl.shape)
+    assert np.array_equal(got, pl if dtype != "bf16" else pl.astype(np.float32))
+
+
 def test_compact_capacity_overflow_is_latched():
     bo = bi = 8
     W = make_case(117, 64, 64, 1, 1, "bf16")
