@@ -26,12 +26,14 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
     TcLayout &T = L.tc;
     T = TcLayout{};
     const int HK = wd.H * wd.K;
-    T.enabled = wd.wtype == BSP_BF16 && wd.O % 8 == 0 && wd.I % (HK == 1 ? 16 : 8) == 0;
+    // a K-step of the tensor-memory kernel is 32 bytes of input channels: 16 bf16 or 32 int8
+    const int cpc = wd.wtype == BSP_I8 ? 16 : 8;          // channels per 16-byte chunk
+    T.enabled = (wd.wtype == BSP_BF16 || wd.wtype == BSP_I8) && wd.O % 8 == 0 && wd.I % (HK == 1 ? 2 * cpc : cpc) == 0;
     int64_t tcap = 0;
     if (T.enabled) {
         const int n_sr = (wd.O + kTcSuperRow - 1) / kTcSuperRow;
         T.n_groups = (n_sr + kTcGroupRows - 1) / kTcGroupRows;
-        T.kc_ch = HK == 1 ? 16 : 8;
+        T.kc_ch = HK == 1 ? 2 * cpc : cpc;
         T.n_kc = wd.I / T.kc_ch;
         T.n_units = HK == 1 ? 1 : (HK + 1) / 2;
         T.st_bytes = T.n_units * kTcUnitBytes;
@@ -335,24 +337,39 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
     }
 }
 
-// Eight consecutive input channels (16 bytes) of W[o][tap][ch0 ..] in bf16, with the channels of zeroed blocks
-// cleared; rows past O and taps past HK read as zero.  Needs I % 8 == 0 and a 16-byte aligned W.
-__device__ __forceinline__ uint4 bf16_chunk(const uint16_t *__restrict__ W, const uint8_t *gamma, int o, int tap, int ch0,
-                                            int O, int I, int HK, int bo, int bi, int NBi)
+// Sixteen bytes of W[o][tap][ch0 ..] (16 / esz consecutive input channels of esz bytes each), with the channels of
+// zeroed blocks cleared; rows past O and taps past HK read as zero.  Needs 16-byte aligned rows of W.
+__device__ __forceinline__ uint4 w_chunk(const void *__restrict__ W, const uint8_t *gamma, int esz, int o, int tap, int ch0,
+                                         int O, int I, int HK, int bo, int bi, int NBi)
 {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (o >= O || tap >= HK) return v;
     const uint8_t *grow = gamma + (size_t)(o >> lg(bo)) * NBi;
-    if (bi >= 8) {
-        if (grow[ch0 >> lg(bi)] == 0) return v;
-        return __ldg((const uint4 *)(W + ((size_t)o * HK + tap) * I + ch0));
+    const uint4 *src = (const uint4 *)((const uint8_t *)W + (((size_t)o * HK + tap) * I + ch0) * esz);
+    const int cpc = 16 / esz;
+    const int b0 = ch0 >> lg(bi);
+    if (bi >= cpc) return grow[b0] ? __ldg(src) : v;
+    if (cpc / bi == 2) {                                   // two blocks per chunk
+        const bool k0 = grow[b0] != 0, k1 = grow[b0 + 1] != 0;
+        if (!k0 && !k1) return v;
+        v = __ldg(src);
+        if (!k0) v.x = v.y = 0u;
+        if (!k1) v.z = v.w = 0u;
+        return v;
     }
-    const bool k0 = grow[ch0 >> 2] != 0, k1 = grow[(ch0 >> 2) + 1] != 0;    // b_i = 4: two blocks per chunk
-    if (!k0 && !k1) return v;
-    v = __ldg((const uint4 *)(W + ((size_t)o * HK + tap) * I + ch0));
-    if (!k0) v.x = v.y = 0u;
-    if (!k1) v.z = v.w = 0u;
+    const bool k0 = grow[b0] != 0, k1 = grow[b0 + 1] != 0, k2 = grow[b0 + 2] != 0, k3 = grow[b0 + 3] != 0;   // four
+    if (!k0 && !k1 && !k2 && !k3) return v;
+    v = __ldg(src);
+    if (!k0) v.x = 0u;
+    if (!k1) v.y = 0u;
+    if (!k2) v.z = 0u;
+    if (!k3) v.w = 0u;
     return v;
+}
+__device__ __forceinline__ uint4 bf16_chunk(const uint16_t *__restrict__ W, const uint8_t *gamma, int o, int tap, int ch0,
+                                            int O, int I, int HK, int bo, int bi, int NBi)
+{
+    return w_chunk(W, gamma, 2, o, tap, ch0, O, I, HK, bo, bi, NBi);
 }
 
 // bf16 tiles of one (panel, tile column) in 16-byte chunks: the 32 bytes of tile row g in a two-tap step are the
@@ -467,22 +484,24 @@ __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__re
 // B operand of 16 x (number of tiles) rows with a uniform 256-byte row-group stride.
 // A convolution pairs taps 2u and 2u+1 of the K-group's 8 channels (a missing odd tap reads as zero); a 1x1
 // layer pairs the two 8-channel halves.
-__device__ __forceinline__ uint32_t tc_word(const uint16_t *__restrict__ W, const uint8_t *__restrict__ gamma, int word,
+__device__ __forceinline__ uint32_t tc_word(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int esz, int word,
                                             int o_base, int kc, int O, int I, int HK, int bo, int bi, int NBi)
 {
     const int u = word >> 7, w = word & 127;
     const int rg = w >> 6, h = (w >> 5) & 1, row = (w >> 2) & 7, pair = w & 3;
     const int o = o_base + rg * 8 + row;
+    const int cpc = 16 / esz, cpw = 4 / esz;              // channels per 16-byte chunk and per 32-bit word
     int tap, ch;
-    if (HK == 1) { tap = 0; ch = (2 * kc + h) * 8 + 2 * pair; }
-    else { tap = 2 * u + h; ch = kc * 8 + 2 * pair; }
+    if (HK == 1) { tap = 0; ch = (2 * kc + h) * cpc + pair * cpw; }
+    else { tap = 2 * u + h; ch = kc * cpc + pair * cpw; }
+    // the channels of a word lie in one block (b_i is a multiple of 4)
     if (tap >= HK || o >= O || gamma[(size_t)(o >> lg(bo)) * NBi + (ch >> lg(bi))] == 0) return 0u;
-    const size_t e = ((size_t)o * HK + tap) * I + ch;
-    return (uint32_t)W[e] | ((uint32_t)W[e + 1] << 16);
+    return *(const uint32_t *)((const uint8_t *)W + (((size_t)o * HK + tap) * I + ch) * esz);
 }
 
 struct TcPackArgs {
     int n_groups, n_kc, kc_per_cta, chunks, st_bytes;
+    int esz;                          // bytes per weight: 2 (bf16) or 1 (int8)
     const uint8_t *mask;
     const uint32_t *off, *gcnt;
     uint8_t *payload;
@@ -497,8 +516,9 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
                                               int HK, int bo, int bi, int NBi, int part, int parts)
 {
     const int cnt = __popc(m);
-    if ((I & 7) == 0 && (((uintptr_t)W) & 15u) == 0) {
-        // 16-byte chunks: one (row group, K half, row) slot of a K-step is eight channels of one weight row and tap
+    const int cpc = 16 / t.esz;
+    if (((I * t.esz) & 15) == 0 && (((uintptr_t)W) & 15u) == 0) {
+        // 16-byte chunks: one (row group, K half, row) slot of a K-step is one chunk of one weight row and tap
         const int nu = t.st_bytes >> 9;
         const int total = cnt * nu * 32;
         const int stride = parts * kThreads;
@@ -516,10 +536,10 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
                 unsigned mm = m;
                 for (int q = 0; q < j; ++q) mm &= mm - 1;
                 const int o = (g * kTcGroupRows + (__ffs(mm) - 1)) * kTcSuperRow + rg * 8 + row;
-                const int tap = HK == 1 ? 0 : 2 * ks + h, ch0 = HK == 1 ? (2 * kc + h) * 8 : kc * 8;
+                const int tap = HK == 1 ? 0 : 2 * ks + h, ch0 = HK == 1 ? (2 * kc + h) * cpc : kc * cpc;
                 ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
                 dst[u] = (uint4 *)(t.payload + (size_t)first * t.st_bytes + ((size_t)(ks * cnt + j) << 9)) + slot;
-                v[u] = ok[u] ? bf16_chunk((const uint16_t *)W, gamma, o, tap, ch0, O, I, HK, bo, bi, NBi) : make_uint4(0u, 0u, 0u, 0u);
+                v[u] = ok[u] ? w_chunk(W, gamma, t.esz, o, tap, ch0, O, I, HK, bo, bi, NBi) : make_uint4(0u, 0u, 0u, 0u);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u)
@@ -545,7 +565,7 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
             ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
             // K-step (word >> 7) major within the K-group, then the stored tile, then the word of the 512-byte unit
             dst[u] = (uint32_t *)(t.payload + (size_t)first * t.st_bytes) + ((size_t)((word >> 7) * cnt + j) << 7) + (word & 127);
-            v[u] = ok[u] ? tc_word((const uint16_t *)W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
+            v[u] = ok[u] ? tc_word(W, gamma, t.esz, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
@@ -614,7 +634,7 @@ __global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs 
             pack_body<DT>(b % a.pack_chunks, b / a.pack_chunks, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.n_cols,
                           a.cols_per_cta, a.tile_bytes, a.colmask, a.coloff, a.panel_base, a.packed_payload,
                           a.capacity_tiles);
-        } else if constexpr (DT == BSP_BF16) {
+        } else if constexpr (DT != BSP_F32) {
             const int c = b - n_pack;
             tc_pack_body(c % a.tc.chunks, c / a.tc.chunks, a.tc, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi);
         }
@@ -737,7 +757,7 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
         }
         return;
     }
-    if constexpr (DT == BSP_BF16) {
+    if constexpr (DT != BSP_F32) {
         const TcPackArgs &t = a.tc;
         const int part = (b - n_pack) % a.tc_parts, cidx = (b - n_pack) / a.tc_parts;
         const int chunk = cidx % t.chunks, g = cidx / t.chunks;
@@ -842,6 +862,7 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     a.capacity_tiles = (long long)L.capacity_tiles;
     if (tc_on) {
         a.tc.n_groups = L.tc.n_groups; a.tc.n_kc = L.tc.n_kc; a.tc.st_bytes = L.tc.st_bytes;
+        a.tc.esz = wd.wtype == BSP_I8 ? 1 : 2;
         a.tc.kc_per_cta = (int)(((long long)L.tc.n_kc * L.tc.n_groups + 1183) / 1184);
         if (a.tc.kc_per_cta < 1) a.tc.kc_per_cta = 1;
         a.tc.chunks = (L.tc.n_kc + a.tc.kc_per_cta - 1) / a.tc.kc_per_cta;
@@ -859,8 +880,9 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
             return (int)(p < 1 ? 1 : (p > 8 ? 8 : p));
         };
         const bool chunks = wd.wtype == BSP_BF16 && wd.I % 8 == 0 && ((uintptr_t)W & 15u) == 0;
+        const bool tc_chunks = wd.wtype != BSP_F32 && (wd.I * (wd.wtype == BSP_I8 ? 1 : 2)) % 16 == 0 && ((uintptr_t)W & 15u) == 0;
         a.pack_parts = chunks ? parts_for((long long)kPanelRows * ((HK + 1) / 2) * 8, 2) : parts_for((long long)kPanelRows * L.tile_bytes / 4, 4);
-        a.tc_parts = !tc_on ? 1 : chunks ? parts_for((long long)kTcGroupRows * L.tc.n_units * 32, 4) : parts_for((long long)kTcGroupRows * L.tc.st_bytes / 4, 4);
+        a.tc_parts = !tc_on ? 1 : tc_chunks ? parts_for((long long)kTcGroupRows * L.tc.n_units * 32, 4) : parts_for((long long)kTcGroupRows * L.tc.st_bytes / 4, 4);
         if (payload) {
             const size_t esz = wd.wtype == BSP_F32 ? 4 : (wd.wtype == BSP_BF16 ? 2 : 1);
             const long long row_pieces = (long long)NBi * wd.bo * HK * ((wd.bi * esz + 15) / 16);   // a row with every block stored

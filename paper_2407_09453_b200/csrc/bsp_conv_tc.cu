@@ -52,6 +52,7 @@ struct TcParams {
     int coords_per_kc;        // steps of the tensor map's last coordinate per K-group
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
     int ytype;
+    int is_i8;                // int8 inputs, int32 accumulators and bias (kind::i8); otherwise bf16 -> fp32 (kind::f16)
 };
 
 __device__ __forceinline__ uint32_t s32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -78,6 +79,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
                  ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void commit_to(uint32_t bar)
@@ -215,7 +221,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         // One thread per issuing warp runs the whole issue loop: a tcgen05.mma is issued by a single thread, and
         // keeping that thread in one long non-divergent stretch avoids a divergence region around every MMA.
         if (lane == 0) {
-            const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // + (N >> 3) << 17
+            // instruction descriptor: D fp32, A and B bf16 (or D int32, A and B signed 8-bit), M = 128; + (N >> 3) << 17
+            const bool i8 = p.is_i8 != 0;
+            const uint32_t idesc0 = ((i8 ? 2u : 1u) << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
             // Descriptors are sums: the address field (16-byte units, low 14 bits) of an A operand is
             // stage + plane + s_aoff[u]; of a B operand weights + 32 * (tiles before the K-group * n_units
             // + u * tiles of the K-group + tiles before the run).  B: K halves 128 bytes apart, row groups 256.
@@ -248,11 +256,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                         const uint32_t idesc = idesc0 | ((uint32_t)(len * 16 >> 3) << 17);
                         const uint32_t d = dset + (uint32_t)r0 * 16u;
                         if (nu == 1) {
-                            mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
+                            if (i8) mma_i8(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
+                            else mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
                         } else {
                             uint32_t bu = b16;
                             for (uint32_t u = 0; u < nu; ++u) {
-                                mma_bf16(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(bu & 0x3FFFu), idesc, 1u);
+                                if (i8) mma_i8(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(bu & 0x3FFFu), idesc, 1u);
+                                else mma_bf16(d, s_ahi[u] | (uint64_t)((a16 + s_aoff[u]) & 0x3FFFu), b_hi | (uint64_t)(bu & 0x3FFFu), idesc, 1u);
                                 bu += cnt * 32u;
                             }
                         }
@@ -302,6 +312,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
             if (!valid) continue;
             const int nch = min(16, p.O - ch);        // 16, or 8 in a last half super-row
+            if (p.is_i8) {                            // exact: int32 sums of the four sets + int32 bias, int32 out
+                int iv[16];
+                const int *ib = (const int *)p.bias;
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    iv[e] = (int)v[0][e] + (int)v[1][e] + (int)v[2][e] + (int)v[3][e] + ((ib != nullptr && e < nch) ? __ldg(ib + ch + e) : 0);
+                uint8_t *dsti = p.Y + (pix * p.O + ch) * 4;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (q * 4 < nch) *(int4 *)(dsti + q * 16) = make_int4(iv[4 * q], iv[4 * q + 1], iv[4 * q + 2], iv[4 * q + 3]);
+                continue;
+            }
             float f[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e)
@@ -350,7 +372,7 @@ EncodeTiledFn tc_encode_tiled()
 // True if the tcgen05 kernel can run this layer: bf16, stride 1, super-tile form present, box extents in range.
 bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
 {
-    if (wd.wtype != BSP_BF16 || xd.stride_h != 1 || xd.stride_w != 1) return false;
+    if ((wd.wtype != BSP_BF16 && wd.wtype != BSP_I8) || xd.stride_h != 1 || xd.stride_w != 1) return false;
     const PackedLayout L = packed_layout(wd, 0);
     if (!L.tc.enabled) return false;
     // a 1x1 kernel without padding is a matrix product over all N*L*J positions
@@ -387,7 +409,9 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     p.M = xd.L + 2 * xd.pad_h - wd.H + 1; p.Nw = xd.J + 2 * xd.pad_w - wd.K + 1;
     p.P = xd.N * p.M * p.Nw;
     p.is_gemm = gemm ? 1 : 0;
-    p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch / 8;
+    const int esz = wd.wtype == BSP_I8 ? 1 : 2;
+    p.is_i8 = wd.wtype == BSP_I8 ? 1 : 0;
+    p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch * esz / 16;
     p.coords_per_kc = gemm ? 1 : p.chunks_per_kc;
     int plane_pos, R = 1;
     long long tiles;
@@ -422,11 +446,11 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
 
     EncodeTiledFn enc = tc_encode_tiled();
     if (!enc) return BSP_ERR_CUDA;
-    const cuuint64_t row = (cuuint64_t)wd.I * 2;
+    const cuuint64_t row = (cuuint64_t)wd.I * esz;
     const cuuint64_t gJ = gemm ? 1 : (cuuint64_t)xd.J, gL = gemm ? 1 : (cuuint64_t)xd.L, gN = gemm ? (cuuint64_t)n_pos : (cuuint64_t)xd.N;
     // innermost extent: one 8-channel chunk (16 bytes), or for a matrix product a whole K-group (32 bytes, swizzled)
     const cuuint64_t inner = gemm ? 32 : 16;
-    const cuuint64_t gdim[5] = {inner, gJ, gL, gN, (cuuint64_t)(wd.I * 2 / inner)};
+    const cuuint64_t gdim[5] = {inner, gJ, gL, gN, (cuuint64_t)(row / inner)};
     const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, inner};
     cuuint32_t box[5];
     if (gemm) { box[0] = 32; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)GK; }
