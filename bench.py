@@ -310,18 +310,22 @@ def main():
     value = job_tflops(fl, world, ms_step)
     conv_tflops = fl / (ms_conv * 1e-3) / 1e12
     abytes = algorithmic_bytes(layer, nnz, bo, bi, ex, ey)
-    t_tensor = fl / (pk["bf16_tflops"] * 1e12)
+    # the tensor peak of the path's own input type: the measured bf16 peak times the nominal ratio of the dense peaks
+    # (int8 4.5 : bf16 2.25 : tf32 1.1 PFLOP/s)
+    ratio = {"bf16": 1.0, "i8": 2.0, "f32": 1.1 / 2.25}[dtype]
+    tensor_peak = pk["bf16_tflops"] * ratio
+    t_tensor = fl / (tensor_peak * 1e12)
     t_hbm = abytes / (pk["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm:
-        roof = {"bound": "tensor", "achieved": conv_tflops, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": conv_tflops / pk["bf16_tflops"], "traffic": None}
+        roof = {"bound": "tensor", "achieved": conv_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
+                "frac": conv_tflops / tensor_peak, "traffic": None}
     else:
         gbs = abytes / (ms_conv * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / pk["hbm_gbs"], "traffic": None}
     kernel = bsp.conv_kernel_name(lay.wd, bsp.XDesc(layer.N, layer.L, layer.J, stride[0], stride[1], pad[0], pad[1]))
     roof["traffic"] = measured_traffic(layer.name, kernel)
-    roof.update({"kernel": kernel, "algorithmic_bytes": abytes, "peak_source": pk["source"] + " (burst)",
+    roof.update({"kernel": kernel, "algorithmic_bytes": abytes, "peak_source": pk["source"] + " (burst)" + ("" if dtype == "bf16" else f" bf16 x {ratio:.3g} nominal ratio"),
                  "kernel_ms": ms_conv, "roofline_ms": max(t_tensor, t_hbm) * 1e3})
 
     out = {

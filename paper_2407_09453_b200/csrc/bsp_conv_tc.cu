@@ -1,10 +1,10 @@
 // Block-sparse implicit-GEMM convolution / FC product with fused bias on 5th-generation tensor cores
-// (tcgen05.mma, accumulators in tensor memory), bf16 inputs, stride 1.  Introduction (Y = W*X + b) and Section
+// (tcgen05.mma, accumulators in tensor memory), bf16 (fp32 accumulators) or int8 (int32, exact) inputs, stride 1.  Introduction (Y = W*X + b) and Section
 // "Block Sparsity in a Matrix" of the paper.
 //
 // One MMA is D[128 x 16n] += A[128 x 16] * B[16 x 16n]: 128 output positions, n consecutive stored super-rows
-// of 16 output channels, 16 reduction elements (two taps of 8 input channels, or 16 input channels of a 1x1
-// layer).  The unit that can be skipped is a 16-channel x K-group super-tile of W-bar; zeroed 8x8 blocks inside
+// of 16 output channels, 32 bytes of reduction elements (two taps of 8 bf16 / 16 int8 input channels, or 16 / 32
+// input channels of a 1x1 layer).  The unit that can be skipped is a 16-channel x K-group super-tile of W-bar; zeroed 8x8 blocks inside
 // a stored super-tile are multiplied as zeros.  The stored super-tiles of a run of consecutive super-rows lie
 // side by side in the packed payload and in tensor memory, so a run is ONE MMA with N = 16 x (run length): a
 // dense layer issues N = 128 MMAs, a sparse one an MMA per run of its mask.
@@ -369,7 +369,7 @@ EncodeTiledFn tc_encode_tiled()
 
 }  // namespace
 
-// True if the tcgen05 kernel can run this layer: bf16, stride 1, super-tile form present, box extents in range.
+// True if the tcgen05 kernel can run this layer: bf16 or int8, stride 1, super-tile form present, box extents in range.
 bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
 {
     if ((wd.wtype != BSP_BF16 && wd.wtype != BSP_I8) || xd.stride_h != 1 || xd.stride_w != 1) return false;

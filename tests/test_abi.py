@@ -64,3 +64,20 @@ def test_host_validation_without_gpu(lib):
     assert lib.bsp_gemm(C.byref(good), C.byref(h), one, C.c_int64(4), None, one, bsp.F32, one, None) == bsp.ERR_SHAPE
     assert lib.bsp_compact(C.byref(good), one, one, one, one, None, None, C.c_int64(-1), one, None) == bsp.ERR_CAPACITY
     assert lib.bsp_check(None, None) == bsp.ERR_NULL
+
+
+def test_product_kernel_choice(monkeypatch):
+    """bf16 and int8 layers with stride 1 take the tensor-memory kernel; fp32, strided layers and BSP_CONV_PATH=mma
+    take the warp-MMA kernel (a host-side decision: no GPU needed)."""
+    import torch
+    monkeypatch.delenv("BSP_CONV_PATH", raising=False)
+    s1 = bsp.XDesc(2, 14, 14, 1, 1, 1, 1)
+    s2 = bsp.XDesc(2, 14, 14, 2, 2, 1, 1)
+    for dt, want in ((torch.bfloat16, "conv_tc_kernel"), (torch.int8, "conv_tc_kernel"), (torch.float32, "conv_mma_kernel")):
+        wd = bsp.wdesc(64, 64, 3, 3, 8, 8, dt)
+        assert bsp.conv_kernel_name(wd, s1) == want
+        assert bsp.conv_kernel_name(wd, s2) == "conv_mma_kernel"
+    # a 1x1 int8 layer needs 32 input channels per K-step
+    assert bsp.conv_kernel_name(bsp.wdesc(64, 48, 1, 1, 8, 8, torch.int8), bsp.XDesc(2, 7, 7, 1, 1, 0, 0)) == "conv_mma_kernel"
+    monkeypatch.setenv("BSP_CONV_PATH", "mma")
+    assert bsp.conv_kernel_name(bsp.wdesc(64, 64, 3, 3, 8, 8, torch.bfloat16), s1) == "conv_mma_kernel"
