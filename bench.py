@@ -180,6 +180,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50_conv3x3_256_b32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the three calls of a step one by one instead of replaying a CUDA graph of them")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     layer, dtype, (bo, bi), sparsity, cfg = workload(args.workload)
@@ -242,21 +243,56 @@ def main():
         step()
     lay.check()
 
+    # ---- one step (the three calls) as a CUDA graph, captured on a side stream through the same C ABI
+    graph, how = None, "three calls per step, launched one by one"
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+            torch.cuda.synchronize()
+            graph.replay()
+            lay.check()
+            how = "CUDA graph of the three calls, one replay per step"
+        except Exception as e:          # capture not available: time the plain calls
+            graph, how = None, f"three calls per step, launched one by one (graph capture failed: {type(e).__name__})"
+            torch.cuda.synchronize()
+
     # ---- device-timed steps, inputs resident in HBM, L2 flushed between steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    ev_step = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
     sampler = ClockSampler(local)
     sampler.start()
     barrier()
     for k in range(args.steps):
         flush.zero_()
-        step(evs[k])
+        ev_step[k][0].record(stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            step()
+        ev_step[k][1].record(stream)
     barrier()
     clocks = sampler.stop()
+    lay.check()
+    t_step = np.array([e[0].elapsed_time(e[1]) for e in ev_step])
+    ms_step = float(t_step.mean())
+
+    # ---- the phases of a step, each call bracketed by events (launched one by one; the events and launch gaps make
+    # their sum larger than a graph replay of the step)
+    n_ph = max(10, min(args.steps, 50))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_ph)]
+    for k in range(n_ph):
+        flush.zero_()
+        step(evs[k])
+    torch.cuda.synchronize()
     t_mask = np.array([e[0].elapsed_time(e[1]) for e in evs])
     t_comp = np.array([e[1].elapsed_time(e[2]) for e in evs])
     t_conv = np.array([e[2].elapsed_time(e[3]) for e in evs])
-    t_step = np.array([e[0].elapsed_time(e[3]) for e in evs])
-    ms_step = float(t_step.mean())
 
     # ---- the same layer dense (Gamma == 1) through the same kernel, for the speedup
     ones = torch.ones(NB, dtype=torch.uint8, device="cuda")
@@ -333,9 +369,11 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": {"bf16": "bf16", "f32": "tf32", "i8": "int8"}[dtype], "data": "synthetic",
         "config": {"workload": layer.name, "block": f"{bo}x{bi}", "sparsity": sparsity, "nnz_blocks": nnz,
-                   "step": "bsp_mask + bsp_compact + bsp_conv2d", "l2": "flushed between steps (384 MB write)",
+                   "step": "bsp_mask + bsp_compact + bsp_conv2d", "launch": how,
+                   "l2": "flushed between steps (384 MB write)",
                    "per_gpu_batch": layer.N},
-        "phases_ms": {"mask": float(t_mask.mean()), "compact": float(t_comp.mean()), "conv": ms_conv},
+        "phases_ms": {"mask": float(t_mask.mean()), "compact": float(t_comp.mean()), "conv": ms_conv,
+                      "note": "each call between its own events, launched one by one"},
         "conv_only": {"tflops": conv_tflops, "ms": ms_conv, "ms_min": float(t_conv.min()),
                       "dense_ms": ms_dense, "speedup_vs_dense": ms_dense / ms_conv},
         "roofline": roof,
