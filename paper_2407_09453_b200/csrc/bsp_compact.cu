@@ -339,17 +339,21 @@ __device__ __forceinline__ uint32_t packed_word(const void *__restrict__ Wv, con
 
 // Sixteen bytes of W[o][tap][ch0 ..] (16 / esz consecutive input channels of esz bytes each), with the channels of
 // zeroed blocks cleared; rows past O and taps past HK read as zero.  Needs 16-byte aligned rows of W.
-__device__ __forceinline__ uint4 w_chunk(const void *__restrict__ W, const uint8_t *gamma, int esz, int o, int tap, int ch0,
+template <int esz>
+__device__ __forceinline__ uint4 w_chunk(const void *__restrict__ W, const uint8_t *gamma, int o, int tap, int ch0,
                                          int O, int I, int HK, int bo, int bi, int NBi)
 {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (o >= O || tap >= HK) return v;
     const uint8_t *grow = gamma + (size_t)(o >> lg(bo)) * NBi;
-    const uint4 *src = (const uint4 *)((const uint8_t *)W + (((size_t)o * HK + tap) * I + ch0) * esz);
-    const int cpc = 16 / esz;
+    constexpr int cpc = 16 / esz;
     const int b0 = ch0 >> lg(bi);
-    if (bi >= cpc) return grow[b0] ? __ldg(src) : v;
-    if (cpc / bi == 2) {                                   // two blocks per chunk
+    if (bi >= cpc) {
+        if (grow[b0] == 0) return v;
+        return __ldg((const uint4 *)((const uint8_t *)W + (((size_t)o * HK + tap) * I + ch0) * esz));
+    }
+    const uint4 *src = (const uint4 *)((const uint8_t *)W + (((size_t)o * HK + tap) * I + ch0) * esz);
+    if (cpc == 8 || cpc / bi == 2) {                       // two blocks per chunk (always, for 8-channel chunks and b_i = 4)
         const bool k0 = grow[b0] != 0, k1 = grow[b0 + 1] != 0;
         if (!k0 && !k1) return v;
         v = __ldg(src);
@@ -369,7 +373,7 @@ __device__ __forceinline__ uint4 w_chunk(const void *__restrict__ W, const uint8
 __device__ __forceinline__ uint4 bf16_chunk(const uint16_t *__restrict__ W, const uint8_t *gamma, int o, int tap, int ch0,
                                             int O, int I, int HK, int bo, int bi, int NBi)
 {
-    return w_chunk(W, gamma, 2, o, tap, ch0, O, I, HK, bo, bi, NBi);
+    return w_chunk<2>(W, gamma, o, tap, ch0, O, I, HK, bo, bi, NBi);
 }
 
 // bf16 tiles of one (panel, tile column) in 16-byte chunks: the 32 bytes of tile row g in a two-tap step are the
@@ -484,13 +488,14 @@ __device__ __forceinline__ void pack_body(int chunk, int panel, const void *__re
 // B operand of 16 x (number of tiles) rows with a uniform 256-byte row-group stride.
 // A convolution pairs taps 2u and 2u+1 of the K-group's 8 channels (a missing odd tap reads as zero); a 1x1
 // layer pairs the two 8-channel halves.
-__device__ __forceinline__ uint32_t tc_word(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int esz, int word,
+template <int esz>
+__device__ __forceinline__ uint32_t tc_word(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int word,
                                             int o_base, int kc, int O, int I, int HK, int bo, int bi, int NBi)
 {
     const int u = word >> 7, w = word & 127;
     const int rg = w >> 6, h = (w >> 5) & 1, row = (w >> 2) & 7, pair = w & 3;
     const int o = o_base + rg * 8 + row;
-    const int cpc = 16 / esz, cpw = 4 / esz;              // channels per 16-byte chunk and per 32-bit word
+    constexpr int cpc = 16 / esz, cpw = 4 / esz;          // channels per 16-byte chunk and per 32-bit word
     int tap, ch;
     if (HK == 1) { tap = 0; ch = (2 * kc + h) * cpc + pair * cpw; }
     else { tap = 2 * u + h; ch = kc * cpc + pair * cpw; }
@@ -501,7 +506,6 @@ __device__ __forceinline__ uint32_t tc_word(const void *__restrict__ W, const ui
 
 struct TcPackArgs {
     int n_groups, n_kc, kc_per_cta, chunks, st_bytes;
-    int esz;                          // bytes per weight: 2 (bf16) or 1 (int8)
     const uint8_t *mask;
     const uint32_t *off, *gcnt;
     uint8_t *payload;
@@ -511,13 +515,14 @@ struct TcPackArgs {
 
 // The stored super-tiles of one (group, K-group), whose super-rows are the set bits of m, from slot `first` on.
 // `parts` CTAs share the words; each thread loads four before it stores.
+template <int esz>      // bytes per weight: 2 (bf16) or 1 (int8)
 __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g, int kc, const TcPackArgs &t,
                                               const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I,
                                               int HK, int bo, int bi, int NBi, int part, int parts)
 {
     const int cnt = __popc(m);
-    const int cpc = 16 / t.esz;
-    if (((I * t.esz) & 15) == 0 && (((uintptr_t)W) & 15u) == 0) {
+    constexpr int cpc = 16 / esz;
+    if (((I * esz) & 15) == 0 && (((uintptr_t)W) & 15u) == 0) {
         // 16-byte chunks: one (row group, K half, row) slot of a K-step is one chunk of one weight row and tap
         const int nu = t.st_bytes >> 9;
         const int total = cnt * nu * 32;
@@ -539,7 +544,7 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
                 const int tap = HK == 1 ? 0 : 2 * ks + h, ch0 = HK == 1 ? (2 * kc + h) * cpc : kc * cpc;
                 ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
                 dst[u] = (uint4 *)(t.payload + (size_t)first * t.st_bytes + ((size_t)(ks * cnt + j) << 9)) + slot;
-                v[u] = ok[u] ? w_chunk(W, gamma, t.esz, o, tap, ch0, O, I, HK, bo, bi, NBi) : make_uint4(0u, 0u, 0u, 0u);
+                v[u] = ok[u] ? w_chunk<esz>(W, gamma, o, tap, ch0, O, I, HK, bo, bi, NBi) : make_uint4(0u, 0u, 0u, 0u);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u)
@@ -565,7 +570,7 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
             ok[u] = ok[u] && (long long)(first + cnt) <= t.capacity;
             // K-step (word >> 7) major within the K-group, then the stored tile, then the word of the 512-byte unit
             dst[u] = (uint32_t *)(t.payload + (size_t)first * t.st_bytes) + ((size_t)((word >> 7) * cnt + j) << 7) + (word & 127);
-            v[u] = ok[u] ? tc_word(W, gamma, t.esz, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
+            v[u] = ok[u] ? tc_word<esz>(W, gamma, word, (g * kTcGroupRows + R) * kTcSuperRow, kc, O, I, HK, bo, bi, NBi) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
@@ -573,6 +578,7 @@ __device__ __forceinline__ void tc_pack_tiles(unsigned m, unsigned first, int g,
     }
 }
 
+template <int esz>
 __device__ __forceinline__ void tc_pack_body(int chunk, int g, const TcPackArgs &t, const void *__restrict__ W,
                                              const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
                                              int NBi)
@@ -585,7 +591,7 @@ __device__ __forceinline__ void tc_pack_body(int chunk, int g, const TcPackArgs 
     for (int kc = kc_lo; kc < kc_hi; ++kc) {
         const unsigned m = t.mask[(size_t)g * t.n_kc + kc];
         if (!m) continue;
-        tc_pack_tiles(m, base + t.off[(size_t)g * t.n_kc + kc], g, kc, t, W, gamma, O, I, HK, bo, bi, NBi, 0, 1);
+        tc_pack_tiles<esz>(m, base + t.off[(size_t)g * t.n_kc + kc], g, kc, t, W, gamma, O, I, HK, bo, bi, NBi, 0, 1);
     }
 }
 
@@ -636,7 +642,7 @@ __global__ void __launch_bounds__(kThreads) fill_pack_kernel(const FillPackArgs 
                           a.capacity_tiles);
         } else if constexpr (DT != BSP_F32) {
             const int c = b - n_pack;
-            tc_pack_body(c % a.tc.chunks, c / a.tc.chunks, a.tc, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi);
+            tc_pack_body<DT == BSP_I8 ? 1 : 2>(c % a.tc.chunks, c / a.tc.chunks, a.tc, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi);
         }
     }
 }
@@ -788,7 +794,7 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
                 a.tc_mask_out[(size_t)g * t.n_kc + kc] = (uint8_t)m;
                 a.tc_off_out[(size_t)g * t.n_kc + kc] = (uint32_t)before;
             }
-            if (m) tc_pack_tiles(m, (unsigned)(base + before), g, kc, t, a.W, s_gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, part, a.tc_parts);
+            if (m) tc_pack_tiles<DT == BSP_I8 ? 1 : 2>(m, (unsigned)(base + before), g, kc, t, a.W, s_gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, part, a.tc_parts);
             before += __popc(m);
         }
     }
@@ -862,7 +868,6 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     a.capacity_tiles = (long long)L.capacity_tiles;
     if (tc_on) {
         a.tc.n_groups = L.tc.n_groups; a.tc.n_kc = L.tc.n_kc; a.tc.st_bytes = L.tc.st_bytes;
-        a.tc.esz = wd.wtype == BSP_I8 ? 1 : 2;
         a.tc.kc_per_cta = (int)(((long long)L.tc.n_kc * L.tc.n_groups + 1183) / 1184);
         if (a.tc.kc_per_cta < 1) a.tc.kc_per_cta = 1;
         a.tc.chunks = (L.tc.n_kc + a.tc.kc_per_cta - 1) / a.tc.kc_per_cta;

@@ -52,7 +52,6 @@ struct TcParams {
     int coords_per_kc;        // steps of the tensor map's last coordinate per K-group
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
     int ytype;
-    int is_i8;                // int8 inputs, int32 accumulators and bias (kind::i8); otherwise bf16 -> fp32 (kind::f16)
 };
 
 __device__ __forceinline__ uint32_t s32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -91,6 +90,8 @@ __device__ __forceinline__ void commit_to(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 
+// kI8: int8 inputs with int32 accumulators, bias and output (kind::i8); otherwise bf16 with fp32 (kind::f16).
+template <bool kI8>
 __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_constant__ TcParams p)
 {
     extern __shared__ __align__(16) uint8_t tc_smem_raw[];
@@ -222,7 +223,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         // keeping that thread in one long non-divergent stretch avoids a divergence region around every MMA.
         if (lane == 0) {
             // instruction descriptor: D fp32, A and B bf16 (or D int32, A and B signed 8-bit), M = 128; + (N >> 3) << 17
-            const bool i8 = p.is_i8 != 0;
+            constexpr bool i8 = kI8;
             const uint32_t idesc0 = ((i8 ? 2u : 1u) << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
             // Descriptors are sums: the address field (16-byte units, low 14 bits) of an A operand is
             // stage + plane + s_aoff[u]; of a B operand weights + 32 * (tiles before the K-group * n_units
@@ -312,7 +313,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
             if (!valid) continue;
             const int nch = min(16, p.O - ch);        // 16, or 8 in a last half super-row
-            if (p.is_i8) {                            // exact: int32 sums of the four sets + int32 bias, int32 out
+            if constexpr (kI8) {                      // exact: int32 sums of the four sets + int32 bias, int32 out
                 int iv[16];
                 const int *ib = (const int *)p.bias;
 #pragma unroll
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 for (int q = 0; q < 4; ++q)
                     if (q * 4 < nch) *(int4 *)(dsti + q * 16) = make_int4(iv[4 * q], iv[4 * q + 1], iv[4 * q + 2], iv[4 * q + 3]);
                 continue;
-            }
+            } else {
             float f[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e)
@@ -342,6 +343,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                         __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * q + 4], f[8 * q + 5]), h3 = __floats2bfloat162_rn(f[8 * q + 6], f[8 * q + 7]);
                         *(uint4 *)(dst + q * 16) = make_uint4(*(uint32_t *)&h0, *(uint32_t *)&h1, *(uint32_t *)&h2, *(uint32_t *)&h3);
                     }
+            }
             }
         }
     }
@@ -410,7 +412,6 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     p.P = xd.N * p.M * p.Nw;
     p.is_gemm = gemm ? 1 : 0;
     const int esz = wd.wtype == BSP_I8 ? 1 : 2;
-    p.is_i8 = wd.wtype == BSP_I8 ? 1 : 0;
     p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch * esz / 16;
     p.coords_per_kc = gemm ? 1 : p.chunks_per_kc;
     int plane_pos, R = 1;
@@ -466,11 +467,13 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     BSP_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kTcMaxDevices) return BSP_ERR_CUDA;
     if (!opted[dev]) {
-        BSP_CUDA_OK(cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem));
         opted[dev] = true;
     }
     dim3 grid((unsigned)tiles, (unsigned)T.n_groups);
-    conv_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
+    if (wd.wtype == BSP_I8) conv_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(p);
+    else conv_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }

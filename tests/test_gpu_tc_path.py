@@ -1,9 +1,12 @@
-"""GPU parity of the tcgen05 kernel (bf16, stride 1; BSP_CONV_PATH=tc rules out an override from outside) against the CPU oracle."""
+"""GPU parity of the tcgen05 kernel (bf16 and int8, stride 1; BSP_CONV_PATH=tc rules out an override from outside)
+against the CPU oracle: within tolerance for bf16, bit for bit for int8."""
 import numpy as np
 import pytest
 
 from oracle import ref
-from paper_2407_09453_b200 import synth
+import torch
+
+from paper_2407_09453_b200 import bsp, synth
 from gpu_util import gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_bias, make_case, make_x
 from test_gpu_product import check, run_conv_case
 
@@ -25,6 +28,27 @@ TC_CASES = [  # O, I, H, K, pad, spatial, batch
 @pytest.mark.parametrize("O,I,H,K,pad,sp,batch", TC_CASES)
 def test_tc_conv_shapes(O, I, H, K, pad, sp, batch):
     run_conv_case(601 + O + H, O, I, H, K, 8, 8, "bf16", (batch, sp[0], sp[1], I), (1, 1), pad)
+
+
+I8_CASES = [  # O, I, H, K, pad, spatial, batch: I a multiple of 16 (conv) or 32 (1x1) so that the kernel applies
+    (128, 128, 3, 3, (1, 1), (14, 14), 3), (64, 64, 1, 1, (0, 0), (9, 7), 3), (72, 48, 5, 5, (2, 2), (11, 13), 2),
+    (64, 32, 1, 7, (0, 3), (17, 17), 2), (1000, 64, 1, 1, (0, 0), (3, 5), 2), (136, 16, 3, 3, (1, 1), (28, 28), 2),
+]
+
+
+@pytest.mark.parametrize("O,I,H,K,pad,sp,batch", I8_CASES)
+@pytest.mark.parametrize("bo,bi", [(8, 8), (4, 16), (16, 4)])
+def test_tc_int8_bit_exact(O, I, H, K, pad, sp, batch, bo, bi):
+    if O % bo or I % bi:
+        pytest.skip("channels are not a multiple of the block")
+    xd = bsp.XDesc(batch, sp[0], sp[1], 1, 1, pad[0], pad[1])
+    assert bsp.conv_kernel_name(bsp.wdesc(O, I, H, K, bo, bi, torch.int8), xd) == "conv_tc_kernel"
+    run_conv_case(641 + O + H, O, I, H, K, bo, bi, "i8", (batch, sp[0], sp[1], I), (1, 1), pad)
+
+
+@pytest.mark.parametrize("frac", [0.0, 0.75, 1.0])
+def test_tc_int8_sparsity_extremes(frac):
+    run_conv_case(651, 128, 128, 3, 3, 8, 8, "i8", (2, 8, 8, 128), (1, 1), (1, 1), frac)
 
 
 @pytest.mark.parametrize("bo,bi", [(4, 16), (16, 4)])
