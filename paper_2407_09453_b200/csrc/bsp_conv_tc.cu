@@ -50,6 +50,8 @@ struct TcParams {
     int PW, plane_bytes, tiles_per_img, is_gemm;
     int n_kc, n_units, st_bytes, chunks_per_kc;
     int coords_per_kc;        // steps of the tensor map's last coordinate per K-group
+    int mt;                   // 128-position tiles per CTA: 1, or 2 for large matrix products (the weights are then
+                              // fetched once for 256 positions); the four issuers split into mt halves x 4/mt K phases
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
     int ytype;
 };
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     }
     // tile geometry
     int n_img = 0, m0 = 0, y_first = 0, rowbase = 0;
-    if (p.is_gemm) { m0 = blockIdx.x * 128; }
+    if (p.is_gemm) { m0 = blockIdx.x * 128 * p.mt; }
     else {
         n_img = blockIdx.x / p.tiles_per_img;
         m0 = (blockIdx.x % p.tiles_per_img) * 128;
@@ -234,6 +236,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             const uint64_t ahi0 = s_ahi[0];
             const uint32_t aoff0 = s_aoff[0];
             const uint32_t dset = tmem + (uint32_t)warp * 128u;
+            const int kphases = kIssuers / p.mt, kphase = warp % kphases;      // K-groups kc with kc % kphases == kphase
+            const uint32_t ahalf = (uint32_t)(warp / kphases) * 256u;          // second 128 positions: 4096 bytes into the plane
             bool ok = true;
             for (int it = 0; it < p.n_stage_iters; ++it) {
                 const int slot = it % S;
@@ -243,12 +247,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t stage16 = (ring + slot * p.stage_bytes) >> 4;
                 const uint32_t w16 = stage16 + (p.act_bytes >> 4);
                 const uint32_t o_lo = s_off[kc0];
-                int kl = (warp - kc0) & (kIssuers - 1);           // first K-group of the stage that is mine
-                for (; kl < nk; kl += kIssuers) {
+                int kl = (kphase - kc0) & (kphases - 1);          // first K-group of the stage that is mine
+                for (; kl < nk; kl += kphases) {
                     uint32_t m = s_mask[kc0 + kl];
                     if (m == 0) continue;
                     const uint32_t cnt = __popc(m);
-                    const uint32_t a16 = stage16 + kl * plane16;
+                    const uint32_t a16 = stage16 + kl * plane16 + ahalf;
                     uint32_t b16 = w16 + (s_off[kc0 + kl] - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
                     while (m) {
                         const int r0 = __ffs(m) - 1;
@@ -286,7 +290,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     if (!done && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
     if (done) {
         const int lq = warp & 3;                 // a warp reaches the TMEM lanes of its quarter only
-        const int m = lq * 32 + lane;
+        // one position tile: warps 0-3 take super-rows 0-3, warps 4-7 rows 4-7, four accumulator sets each;
+        // two tiles: warps 0-3 take the first 128 positions (sets 0, 1), warps 4-7 the second (sets 2, 3), all rows
+        const int half = p.mt == 2 ? (warp >> 2) : 0;
+        const int set0 = p.mt == 2 ? 2 * half : 0, nsets = kIssuers / p.mt;
+        const int r_lo = p.mt == 2 ? 0 : (warp >> 2) * 4, r_hi = p.mt == 2 ? kTcGroupRows : r_lo + 4;
+        const int m = half * 128 + lq * 32 + lane;
         bool valid;
         size_t pix;
         if (p.is_gemm) { valid = m0 + m < p.P; pix = (size_t)(m0 + m); }
@@ -297,18 +306,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         }
         const int oe = (p.ytype == BSP_BF16) ? 2 : 4;
 #pragma unroll 1
-        for (int r = (warp >> 2) * 4; r < (warp >> 2) * 4 + 4; ++r) {
+        for (int r = r_lo; r < r_hi; ++r) {
             const int ch = (g * kTcGroupRows + r) * kTcSuperRow;
             if (ch >= p.O) break;
             // the four accumulator sets of this super-row
             uint32_t v[kIssuers][16];
 #pragma unroll
             for (int s = 0; s < kIssuers; ++s) {
-                const uint32_t ta = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)(s * 128 + r * 16);
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
-                             : "=r"(v[s][0]), "=r"(v[s][1]), "=r"(v[s][2]), "=r"(v[s][3]), "=r"(v[s][4]), "=r"(v[s][5]), "=r"(v[s][6]), "=r"(v[s][7]),
-                               "=r"(v[s][8]), "=r"(v[s][9]), "=r"(v[s][10]), "=r"(v[s][11]), "=r"(v[s][12]), "=r"(v[s][13]), "=r"(v[s][14]), "=r"(v[s][15])
-                             : "r"(ta) : "memory");
+                if (s < nsets) {
+                    const uint32_t ta = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)((set0 + s) * 128 + r * 16);
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+                                 : "=r"(v[s][0]), "=r"(v[s][1]), "=r"(v[s][2]), "=r"(v[s][3]), "=r"(v[s][4]), "=r"(v[s][5]), "=r"(v[s][6]), "=r"(v[s][7]),
+                                   "=r"(v[s][8]), "=r"(v[s][9]), "=r"(v[s][10]), "=r"(v[s][11]), "=r"(v[s][12]), "=r"(v[s][13]), "=r"(v[s][14]), "=r"(v[s][15])
+                                 : "r"(ta) : "memory");
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[s][e] = 0u;
+                }
             }
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
             if (!valid) continue;
@@ -385,7 +399,7 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
     size_t per_kc;
     if (gemm) {
         if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
-        per_kc = (size_t)128 * 32 + (size_t)kTcGroupRows * L.tc.st_bytes;
+        per_kc = (size_t)256 * 32 + (size_t)kTcGroupRows * L.tc.st_bytes;       // up to 256 positions per CTA
     } else {
         const int PW = xd.J + 2 * xd.pad_w;
         const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
@@ -414,10 +428,13 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const int esz = wd.wtype == BSP_I8 ? 1 : 2;
     p.n_kc = T.n_kc; p.n_units = T.n_units; p.st_bytes = T.st_bytes; p.chunks_per_kc = T.kc_ch * esz / 16;
     p.coords_per_kc = gemm ? 1 : p.chunks_per_kc;
+    p.mt = 1;
     int plane_pos, R = 1;
     long long tiles;
     if (gemm) {
-        p.PW = 1; plane_pos = 128; p.tiles_per_img = 0; tiles = (n_pos + 127) / 128;
+        // large products take 256 positions per CTA when that still leaves two waves of CTAs
+        p.mt = ((n_pos + 255) / 256) * T.n_groups >= 2 * 148 ? 2 : 1;
+        p.PW = 1; plane_pos = 128 * p.mt; p.tiles_per_img = 0; tiles = (n_pos + plane_pos - 1) / plane_pos;
     } else {
         p.PW = xd.J + 2 * xd.pad_w;
         R = (wd.H * p.PW + 126 + wd.K - 1) / p.PW + 1;
@@ -454,7 +471,7 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const cuuint64_t gdim[5] = {inner, gJ, gL, gN, (cuuint64_t)(row / inner)};
     const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, inner};
     cuuint32_t box[5];
-    if (gemm) { box[0] = 32; box[1] = 1; box[2] = 1; box[3] = 128; box[4] = (cuuint32_t)GK; }
+    if (gemm) { box[0] = 32; box[1] = 1; box[2] = 1; box[3] = (cuuint32_t)(128 * p.mt); box[4] = (cuuint32_t)GK; }
     else { box[0] = 16; box[1] = (cuuint32_t)p.PW; box[2] = (cuuint32_t)R; box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     if (enc(&p.tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void *>(X), gdim, gstr, box, estr,

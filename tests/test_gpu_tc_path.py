@@ -75,6 +75,20 @@ def test_tc_gemm_ragged(bo, bi):
     check(got, want, "bf16")
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
+def test_tc_gemm_two_position_tiles_per_cta(dtype):
+    """Enough CTAs that a matrix product takes 256 positions per CTA (two accumulator halves); ragged last tile."""
+    O, I, P = 1024, 64, 9500
+    W = make_case(661, O, I, 1, 1, dtype)
+    gamma = synth.random_gamma(662, O // 8, I // 8, (O // 8) * (I // 8) // 2)
+    X = make_x(663, (P, I), dtype)
+    b = make_bias(664, O, dtype)
+    lay = gpu_layer(W, gamma, 8, 8, dtype)
+    got = gpu_gemm(lay, X, b, dtype)
+    rp, ci, pl = ref.compact(W, gamma, 8, 8)
+    check(got, ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b), dtype)
+
+
 def test_tc_config_resnet_conv_with_l2_gamma():
     layer = synth.Layer("cfg2", 256, 256, 3, 3, 32, 14, 14, 1, 1, 1, 1)
     W, X, b = synth.make_layer_tensors(layer, "bf16", config=2)
