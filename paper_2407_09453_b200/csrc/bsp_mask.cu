@@ -273,15 +273,31 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
         if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
         if (tid < 256) hist[tid] = __ldcg(&ghist[pass * 256 + tid]);
         __syncthreads();
-        if (tid == 0) {
-            long long need = s_k, cum = 0;
-            int d = 0;
-            for (; d < 255; ++d) {
-                if (cum + (long long)hist[d] >= need) break;
-                cum += hist[d];
+        if (tid < 32) {
+            // the digit d with cum(d - 1) < need <= cum(d): each lane sums eight bins, a warp scan finds the lane, the
+            // lane walks its bins
+            const long long need = s_k;
+            long long mine = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) mine += hist[tid * 8 + q];
+            long long inc = mine;
+#pragma unroll
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                const long long n = __shfl_up_sync(0xFFFFFFFFu, inc, dd);
+                if (tid >= dd) inc += n;
             }
-            s_k = need - cum;
-            s_prefix = (prefix << 8) | (unsigned long long)d;
+            const unsigned reach = __ballot_sync(0xFFFFFFFFu, inc >= need);
+            const int owner = reach ? __ffs(reach) - 1 : 31;        // need <= total, so some lane reaches it
+            if (tid == owner) {
+                long long cum = inc - mine;
+                int d = tid * 8;
+                for (; d < tid * 8 + 7; ++d) {
+                    if (cum + (long long)hist[d] >= need) break;
+                    cum += hist[d];
+                }
+                s_k = need - cum;
+                s_prefix = (prefix << 8) | (unsigned long long)d;
+            }
         }
         __syncthreads();
     }
