@@ -159,7 +159,7 @@ def run_reference(args, layer, dtype, bo, bi, sparsity, cfg):
     nnz = NB - n_zero
     for _ in range(min(args.warmup, 1)):
         time_oracle(layer, dtype, bo, bi, n_zero, W, X, b, 0, 1)
-    t, cores, reps = time_oracle(layer, dtype, bo, bi, n_zero, W, X, b, 0, args.steps)
+    t, cores, reps = time_oracle(layer, dtype, bo, bi, n_zero, W, X, b, float("inf"), max(args.steps, 1))   # exactly K passes
     val = useful_flops(layer, nnz, bo, bi) / t / 1e12
     sample = f"all {layer.P} output pixels of the workload, {reps} passes"
     print(json.dumps({
