@@ -50,6 +50,11 @@ struct TcParams {
     int PW, plane_bytes, tiles_per_img, is_gemm;
     int n_kc, n_units, st_bytes, chunks_per_kc;
     int coords_per_kc;        // steps of the tensor map's last coordinate per K-group
+    // Strides: the padded input splits into s_h x s_w phase images (rows = a mod s_h, columns = b mod s_w); tap (h, k)
+    // reads phase (h mod s_h, k mod s_w) at the constant offset (h / s_h, k / s_w), so every phase in use is staged as a
+    // stride-1 plane set of its own (one tiled load each, through the tensor map's element strides).
+    int sh, sw, n_phase, phase_bytes;      // phase_bytes: bytes of one phase's planes in a stage
+    int ph_a[4], ph_b[4];                  // the phases in use, in the order they lie in a stage
     int mt;                   // 128-position tiles per CTA: 1, or 2 for large matrix products (the weights are then
                               // fetched once for 256 positions); the four issuers split into mt halves x 4/mt K phases
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
@@ -145,11 +150,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             off = (uint32_t)rowbase;
             lbo = (uint32_t)p.plane_bytes;
         } else {
+            // position offset (16-byte units from the stage's first plane) of a tap: its phase's planes, then (h / s_h) rows
+            // and k / s_w columns
+            auto tap_off = [&](int t) -> int {
+                const int h = t / p.K, k = t % p.K;
+                int ph = 0;
+                for (int i = 0; i < p.n_phase; ++i)
+                    if (p.ph_a[i] == h % p.sh && p.ph_b[i] == k % p.sw) ph = i;
+                return ph * (p.phase_bytes >> 4) + (h / p.sh) * p.PW + k / p.sw;
+            };
             const int t0 = 2 * u, t1 = 2 * u + 1;
-            const int o0 = (t0 / p.K) * p.PW + t0 % p.K;
+            const int o0 = tap_off(t0);
             off = (uint32_t)(rowbase + o0);
-            // a missing odd tap has zero weights; its K half reads the next position (finite data)
-            lbo = (t1 < p.H * p.K) ? (uint32_t)(((t1 / p.K) * p.PW + t1 % p.K) - o0) * 16u : 16u;
+            // a missing odd tap has zero weights; its K half reads the next position (finite data).  The host orders
+            // the phases so that the second tap of a pair lies after the first.
+            lbo = (t1 < p.H * p.K) ? (uint32_t)(tap_off(t1) - o0) * 16u : 16u;
         }
         s_aoff[u] = off;
         s_ahi[u] = smem_desc(0, lbo, 128);
@@ -159,7 +174,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     // arrivals per phase, one with the activation bytes and one with the weight bytes.
     const int meta_bytes = ((p.n_kc * 5 + 1023) / 1024) * 1024;
     const uint32_t ring = s32(smem) + meta_bytes;
-    const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first - p.ph, c3 = p.is_gemm ? m0 : n_img;
+    // first input column and row of the tile's phase (0, 0); phase (a, b) starts a rows and b columns further
+    const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first * p.sh - p.ph, c3 = p.is_gemm ? m0 : n_img;
     if (warp == kIssuers && lane == 0) {
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmap) : "memory");
         for (int s = 0; s < S; ++s) {
@@ -170,9 +186,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         for (int it = 0; it < min(S, p.n_stage_iters); ++it) {
             const uint32_t bar = s32(&s_full[it]);
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
-            asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
-                         ::"r"(ring + it * p.stage_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(it * p.GK * p.coords_per_kc) : "memory");
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)(p.n_phase * p.act_box_bytes)) : "memory");
+            for (int ph = 0; ph < p.n_phase; ++ph)
+                asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+                             ::"r"(ring + it * p.stage_bytes + ph * p.phase_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1 + p.ph_b[ph]),
+                               "r"(c2 + p.ph_a[ph]), "r"(c3), "r"(it * p.GK * p.coords_per_kc) : "memory");
         }
     }
     if (warp == 0) {
@@ -209,9 +227,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t bar = s32(&s_full[slot]);
                 const uint32_t dst = ring + slot * p.stage_bytes;
                 if (it >= S) {          // the first S activation loads were issued before the index arrays arrived
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)p.act_box_bytes) : "memory");
-                    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
-                                 ::"r"(dst), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(kc0 * p.coords_per_kc) : "memory");
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)(p.n_phase * p.act_box_bytes)) : "memory");
+                    for (int ph = 0; ph < p.n_phase; ++ph)
+                        asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+                                     ::"r"(dst + ph * p.phase_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1 + p.ph_b[ph]), "r"(c2 + p.ph_a[ph]),
+                                       "r"(c3), "r"(kc0 * p.coords_per_kc) : "memory");
                 }
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(wbytes) : "memory");
                 if (wbytes)
@@ -385,26 +405,91 @@ EncodeTiledFn tc_encode_tiled()
 
 }  // namespace
 
+namespace {
+// Position geometry of a layer for the tensor-memory kernel.  Output positions are counted over rows of PW = N' + (K-1)/s_w
+// positions; a CTA's 128 positions need R rows of every phase image in use.
+struct TcGeo {
+    bool gemm;
+    int M, Nw, PW, R, n_phase, ph_a[4], ph_b[4];
+};
+
+bool tc_geometry(const bsp_wdesc &wd, const bsp_xdesc &xd, TcGeo &g)
+{
+    g = TcGeo{};
+    g.gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0 && xd.stride_h == 1 && xd.stride_w == 1;
+    g.M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1;
+    g.Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
+    g.n_phase = 1; g.PW = 1; g.R = 1;
+    if (g.gemm) return true;
+    const int sh = xd.stride_h, sw = xd.stride_w;
+    const int Hq = (wd.H - 1) / sh, Kq = (wd.K - 1) / sw;
+    g.PW = g.Nw + Kq;
+    g.R = (g.PW - 1 + 127 + Hq * g.PW + Kq) / g.PW + 1;
+    if (g.PW * sw > 256 || g.R * sh > 256) return false;          // extents of a tiled load
+    // phases (h mod s_h, k mod s_w) that some tap reads
+    int n = 0, pa[4], pb[4];
+    for (int h = 0; h < wd.H; ++h)
+        for (int k = 0; k < wd.K; ++k) {
+            bool seen = false;
+            for (int i = 0; i < n; ++i) seen |= pa[i] == h % sh && pb[i] == k % sw;
+            if (seen) continue;
+            if (n == 4) return false;
+            pa[n] = h % sh; pb[n] = k % sw; ++n;
+        }
+    // an MMA multiplies taps 2u and 2u+1, the second at a non-negative byte offset from the first: find an order of
+    // the phases in shared memory in which the second tap's phase never lies before the first's
+    int perm[4] = {0, 1, 2, 3};
+    const int HK = wd.H * wd.K;
+    for (int trial = 0; trial < 24; ++trial) {
+        int pos[4];                                       // pos[i]: place of phase i in this order
+        {   // the trial-th permutation of 0..3 (factorial number system), restricted to the first n entries
+            int pool[4] = {0, 1, 2, 3}, t = trial;
+            const int f[4] = {6, 2, 1, 1};
+            for (int i = 0; i < 4; ++i) {
+                const int q = t / f[i]; t %= f[i];
+                perm[i] = pool[q];
+                for (int j = q; j < 3; ++j) pool[j] = pool[j + 1];
+            }
+        }
+        bool uses_only = true;
+        for (int i = 0; i < n; ++i) uses_only &= perm[i] < n;     // the first n places hold the n phases
+        if (!uses_only) continue;
+        for (int i = 0; i < n; ++i) pos[perm[i]] = i;
+        bool ok = true;
+        for (int t0 = 0; t0 + 1 < HK && ok; t0 += 2) {
+            int i0 = 0, i1 = 0;
+            for (int i = 0; i < n; ++i) {
+                if (pa[i] == (t0 / wd.K) % sh && pb[i] == (t0 % wd.K) % sw) i0 = i;
+                if (pa[i] == ((t0 + 1) / wd.K) % sh && pb[i] == ((t0 + 1) % wd.K) % sw) i1 = i;
+            }
+            ok = pos[i0] <= pos[i1];
+        }
+        if (!ok) continue;
+        g.n_phase = n;
+        for (int i = 0; i < n; ++i) { g.ph_a[i] = pa[perm[i]]; g.ph_b[i] = pb[perm[i]]; }
+        return true;
+    }
+    return false;
+}
+}  // namespace
+
 // True if the tcgen05 kernel can run this layer: bf16 or int8, stride 1, super-tile form present, box extents in range.
 bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
 {
-    if ((wd.wtype != BSP_BF16 && wd.wtype != BSP_I8) || xd.stride_h != 1 || xd.stride_w != 1) return false;
+    if (wd.wtype != BSP_BF16 && wd.wtype != BSP_I8) return false;
     const PackedLayout L = packed_layout(wd, 0);
     if (!L.tc.enabled) return false;
-    // a 1x1 kernel without padding is a matrix product over all N*L*J positions
-    const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
+    TcGeo g;
+    if (!tc_geometry(wd, xd, g)) return false;
     // the per-K-group index of the group plus two stages (one K-group of activations and its dense weights
     // each) must fit the shared memory
     const size_t meta = align_up((size_t)L.tc.n_kc * 5, 1024);
     size_t per_kc;
-    if (gemm) {
+    if (g.gemm) {
         if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
         per_kc = (size_t)256 * 32 + (size_t)kTcGroupRows * L.tc.st_bytes;       // up to 256 positions per CTA
     } else {
-        const int PW = xd.J + 2 * xd.pad_w;
-        const int R = (wd.H * PW + 126 + wd.K - 1) / PW + 1;
-        if (PW > 256 || R > 256) return false;
-        per_kc = (size_t)R * PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + (size_t)kTcGroupRows * L.tc.st_bytes;
+        per_kc = (size_t)g.n_phase * ((size_t)g.R * g.PW * 16 * (wd.H * wd.K == 1 ? 2 : 1) + 128) + (size_t)kTcGroupRows * L.tc.st_bytes;
     }
     return 2 * (per_kc + 1024) + meta + 1024 <= (size_t)kTcMaxSmem;
 }
@@ -415,14 +500,18 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const PackedLayout L = packed_layout(wd, 0);
     const TcLayout &T = L.tc;
     const uint8_t *pk = (const uint8_t *)packed;
-    const bool gemm = wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0;
+    TcGeo geo;
+    if (!tc_geometry(wd, xd, geo)) return BSP_ERR_SHAPE;
+    const bool gemm = geo.gemm;
     const long long n_pos = (long long)xd.N * xd.L * xd.J;      // positions of a 1x1 layer, taken as one long row
     TcParams p = {};
     p.Y = (uint8_t *)Y; p.bias = (const float *)bias;
     p.mask = pk + T.off_mask; p.off = (const uint32_t *)(pk + T.off_off); p.gcnt = (const uint32_t *)(pk + T.off_gcnt);
     p.packed = pk; p.status = (int *)ws;
     p.N = xd.N; p.O = wd.O; p.H = wd.H; p.K = wd.K; p.ph = xd.pad_h; p.pw = xd.pad_w;
-    p.M = xd.L + 2 * xd.pad_h - wd.H + 1; p.Nw = xd.J + 2 * xd.pad_w - wd.K + 1;
+    p.M = geo.M; p.Nw = geo.Nw;
+    p.sh = xd.stride_h; p.sw = xd.stride_w; p.n_phase = geo.n_phase;
+    for (int i = 0; i < 4; ++i) { p.ph_a[i] = geo.ph_a[i]; p.ph_b[i] = geo.ph_b[i]; }
     p.P = xd.N * p.M * p.Nw;
     p.is_gemm = gemm ? 1 : 0;
     const int esz = wd.wtype == BSP_I8 ? 1 : 2;
@@ -436,21 +525,23 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         p.mt = ((n_pos + 255) / 256) * T.n_groups >= 2 * 148 ? 2 : 1;
         p.PW = 1; plane_pos = 128 * p.mt; p.tiles_per_img = 0; tiles = (n_pos + plane_pos - 1) / plane_pos;
     } else {
-        p.PW = xd.J + 2 * xd.pad_w;
-        R = (wd.H * p.PW + 126 + wd.K - 1) / p.PW + 1;
+        p.PW = geo.PW;
+        R = geo.R;
         plane_pos = R * p.PW;
         p.tiles_per_img = (p.M * p.PW + 127) / 128;
         tiles = (long long)xd.N * p.tiles_per_img;
     }
     p.plane_bytes = plane_pos * 16;
-    const size_t per_kc = (size_t)p.plane_bytes * p.chunks_per_kc + (size_t)kTcGroupRows * T.st_bytes;
+    const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + 128) + (size_t)kTcGroupRows * T.st_bytes;
     int GK = (int)(49152 / per_kc);
     if (GK < 1) GK = 1;
     if (GK > T.n_kc) GK = T.n_kc;
     if (GK * p.chunks_per_kc > 256) GK = 256 / p.chunks_per_kc;
     p.GK = GK;
     p.act_box_bytes = GK * p.chunks_per_kc * p.plane_bytes;
-    p.act_bytes = (int)align_up((size_t)p.act_box_bytes + 32, 128);      // + slack read by positions in the padding
+    // every tiled load must land on a 128-byte boundary of shared memory: the phases' plane sets are padded to that
+    p.phase_bytes = (int)align_up((size_t)p.act_box_bytes, 128);
+    p.act_bytes = (int)align_up((size_t)p.n_phase * p.phase_bytes + 32, 128);        // + slack read by positions in the padding
     p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)GK * kTcGroupRows * T.st_bytes, 1024);
     p.n_stage_iters = (T.n_kc + GK - 1) / GK;
     const size_t meta = align_up((size_t)T.n_kc * 5, 1024);
@@ -472,8 +563,9 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const cuuint64_t gstr[4] = {row, row * gJ, row * gJ * gL, inner};
     cuuint32_t box[5];
     if (gemm) { box[0] = 32; box[1] = 1; box[2] = 1; box[3] = (cuuint32_t)(128 * p.mt); box[4] = (cuuint32_t)GK; }
-    else { box[0] = 16; box[1] = (cuuint32_t)p.PW; box[2] = (cuuint32_t)R; box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
-    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    // a box traverses PW * s_w columns and R * s_h rows in steps of the strides: PW x R positions arrive
+    else { box[0] = 16; box[1] = (cuuint32_t)(p.PW * p.sw); box[2] = (cuuint32_t)(R * p.sh); box[3] = 1; box[4] = (cuuint32_t)(GK * p.chunks_per_kc); }
+    const cuuint32_t estr[5] = {1, gemm ? 1u : (cuuint32_t)p.sw, gemm ? 1u : (cuuint32_t)p.sh, 1, 1};
     if (enc(&p.tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void *>(X), gdim, gstr, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, gemm ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)

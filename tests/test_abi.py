@@ -67,8 +67,8 @@ def test_host_validation_without_gpu(lib):
 
 
 def test_product_kernel_choice(monkeypatch):
-    """bf16 and int8 layers with stride 1 take the tensor-memory kernel; fp32, strided layers and BSP_CONV_PATH=mma
-    take the warp-MMA kernel (a host-side decision: no GPU needed)."""
+    """bf16 and int8 layers take the tensor-memory kernel, strided ones included; fp32 and BSP_CONV_PATH=mma take the
+    warp-MMA kernel (a host-side decision: no GPU needed)."""
     import torch
     monkeypatch.delenv("BSP_CONV_PATH", raising=False)
     s1 = bsp.XDesc(2, 14, 14, 1, 1, 1, 1)
@@ -76,7 +76,9 @@ def test_product_kernel_choice(monkeypatch):
     for dt, want in ((torch.bfloat16, "conv_tc_kernel"), (torch.int8, "conv_tc_kernel"), (torch.float32, "conv_mma_kernel")):
         wd = bsp.wdesc(64, 64, 3, 3, 8, 8, dt)
         assert bsp.conv_kernel_name(wd, s1) == want
-        assert bsp.conv_kernel_name(wd, s2) == "conv_mma_kernel"
+        assert bsp.conv_kernel_name(wd, s2) == want
+    # a stride of 3 over a 5x5 kernel would need nine phase images: more than the kernel stages
+    assert bsp.conv_kernel_name(bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16), bsp.XDesc(2, 20, 20, 3, 3, 2, 2)) == "conv_mma_kernel"
     # a 1x1 int8 layer needs 32 input channels per K-step
     assert bsp.conv_kernel_name(bsp.wdesc(64, 48, 1, 1, 8, 8, torch.int8), bsp.XDesc(2, 7, 7, 1, 1, 0, 0)) == "conv_mma_kernel"
     monkeypatch.setenv("BSP_CONV_PATH", "mma")

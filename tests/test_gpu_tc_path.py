@@ -30,6 +30,27 @@ def test_tc_conv_shapes(O, I, H, K, pad, sp, batch):
     run_conv_case(601 + O + H, O, I, H, K, 8, 8, "bf16", (batch, sp[0], sp[1], I), (1, 1), pad)
 
 
+STRIDED = [  # O, I, H, K, stride, pad, spatial, batch, runs on the tensor-memory kernel
+    (128, 64, 3, 3, (2, 2), (1, 1), (15, 15), 3, True), (64, 64, 1, 1, (2, 2), (0, 0), (14, 14), 3, True),
+    (64, 32, 3, 3, (2, 2), (0, 0), (17, 17), 2, True), (64, 64, 3, 3, (2, 1), (1, 1), (28, 9), 2, True),
+    (256, 128, 3, 3, (2, 2), (1, 1), (56, 56), 1, True), (64, 32, 5, 5, (2, 2), (2, 2), (30, 30), 1, True),
+    # 49 taps: two stages of one K-group's weights (25 K-steps x 8 super-rows) do not fit the shared memory
+    (64, 32, 7, 7, (2, 2), (3, 3), (30, 30), 1, False),
+    # 5 taps per row at a column stride of 2: tap pairs (A, B) and (B, A) of the two phases cannot both lie in
+    # ascending order in shared memory, so this one stays on the warp-MMA kernel
+    (72, 48, 5, 5, (1, 2), (2, 1), (11, 13), 2, False),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
+@pytest.mark.parametrize("O,I,H,K,stride,pad,sp,batch,on_tc", STRIDED)
+def test_tc_strided(dtype, O, I, H, K, stride, pad, sp, batch, on_tc):
+    xd = bsp.XDesc(batch, sp[0], sp[1], stride[0], stride[1], pad[0], pad[1])
+    tdt = torch.int8 if dtype == "i8" else torch.bfloat16
+    assert bsp.conv_kernel_name(bsp.wdesc(O, I, H, K, 8, 8, tdt), xd) == ("conv_tc_kernel" if on_tc else "conv_mma_kernel")
+    run_conv_case(671 + O + H, O, I, H, K, 8, 8, dtype, (batch, sp[0], sp[1], I), stride, pad)
+
+
 I8_CASES = [  # O, I, H, K, pad, spatial, batch: I a multiple of 16 (conv) or 32 (1x1) so that the kernel applies
     (128, 128, 3, 3, (1, 1), (14, 14), 3), (64, 64, 1, 1, (0, 0), (9, 7), 3), (72, 48, 5, 5, (2, 2), (11, 13), 2),
     (64, 32, 1, 7, (0, 3), (17, 17), 2), (1000, 64, 1, 1, (0, 0), (3, 5), 2), (136, 16, 3, 3, (1, 1), (28, 28), 2),
