@@ -159,8 +159,9 @@ bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma,
  * float32, bias float32, ytype F32 or BF16 (round to nearest even after the bias); F32 inputs are
  * multiplied as TF32.  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
  *   bias may be NULL (treated as zero).  ws: device scratch of bsp_conv_workspace_bytes() bytes.
- * Two kernels implement the products.  BF16 and I8 layers with stride 1 run on the tensor-memory kernel
- * ("conv_tc_kernel": tcgen05 MMAs on 16-channel super-tiles of the second packed form); everything else, and
+ * Two kernels implement the products.  BF16 and I8 layers run on the tensor-memory kernel ("conv_tc_kernel":
+ * tcgen05 MMAs on 16-channel super-tiles of the second packed form) unless their shape rules it out (more than
+ * four stride residues in use, a tile that does not fit shared memory, I not a multiple of the K-step); those, F32, and
  * every layer when the environment variable BSP_CONV_PATH starts with 'm', runs on the warp-MMA kernel
  * ("conv_mma_kernel", 8x8 tiles).  bsp_conv_kernel_name() says which one a call with these descriptors takes
  * (static storage; NULL for invalid descriptors).

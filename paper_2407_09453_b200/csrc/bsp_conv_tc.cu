@@ -1,5 +1,6 @@
 // Block-sparse implicit-GEMM convolution / FC product with fused bias on 5th-generation tensor cores
-// (tcgen05.mma, accumulators in tensor memory), bf16 (fp32 accumulators) or int8 (int32, exact) inputs, stride 1.  Introduction (Y = W*X + b) and Section
+// (tcgen05.mma, accumulators in tensor memory), bf16 (fp32 accumulators) or int8 (int32, exact) inputs, any stride
+// whose residues in use number at most four.  Introduction (Y = W*X + b) and Section
 // "Block Sparsity in a Matrix" of the paper.
 //
 // One MMA is D[128 x 16n] += A[128 x 16] * B[16 x 16n]: 128 output positions, n consecutive stored super-rows
@@ -473,7 +474,7 @@ bool tc_geometry(const bsp_wdesc &wd, const bsp_xdesc &xd, TcGeo &g)
 }
 }  // namespace
 
-// True if the tcgen05 kernel can run this layer: bf16 or int8, stride 1, super-tile form present, box extents in range.
+// True if the tcgen05 kernel can run this layer: bf16 or int8, super-tile form present, box extents in range.
 bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
 {
     if (wd.wtype != BSP_BF16 && wd.wtype != BSP_I8) return false;
