@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             // and k / s_w columns
             auto tap_off = [&](int t) -> int {
                 const int h = t / p.K, k = t % p.K;
+                if (p.n_phase == 1 && p.sh == 1 && p.sw == 1) return h * p.PW + k;       // stride 1: the tap's row and column
                 int ph = 0;
                 for (int i = 0; i < p.n_phase; ++i)
                     if (p.ph_a[i] == h % p.sh && p.ph_b[i] == k % p.sw) ph = i;
@@ -533,7 +534,8 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         tiles = (long long)xd.N * p.tiles_per_img;
     }
     p.plane_bytes = plane_pos * 16;
-    const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + 128) + (size_t)kTcGroupRows * T.st_bytes;
+    // (several phases: each plane set is padded to 128 bytes)
+    const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + (p.n_phase > 1 ? 128 : 0)) + (size_t)kTcGroupRows * T.st_bytes;
     int GK = (int)(49152 / per_kc);
     if (GK < 1) GK = 1;
     if (GK > T.n_kc) GK = T.n_kc;
