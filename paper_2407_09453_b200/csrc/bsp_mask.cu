@@ -203,28 +203,28 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
 
 // Grid-wide barrier of a cooperative launch (all CTAs co-resident), reusable within the launch: `sync[0]`
 // counts arrivals and is reset by the last arriver, `sync[1]` is a generation that the last arriver bumps.
-// Thread 0 of each CTA takes part; the wait is bounded.  Returns false if it expired.
+// Thread 0 of each CTA takes part (release on arrival, acquire on the generation; the CTA barriers around it
+// extend both to the other threads); the wait is bounded.  Returns false if it expired.
 constexpr unsigned kGridSpinLimit = 1u << 24;
 __device__ __forceinline__ bool grid_barrier(unsigned *sync)
 {
     __shared__ int s_bar_ok;
-    __threadfence();
-    __syncthreads();
+    __syncthreads();                         // the CTA's writes are ordered before thread 0's release below
     if (threadIdx.x == 0) {
-        volatile unsigned *gen = sync + 1;
-        const unsigned g0 = *gen;
+        unsigned g0, old, g;
         int ok = 1;
-        __threadfence();
-        if (atomicAdd(sync, 1u) == gridDim.x - 1) {
-            atomicExch(sync, 0u);
-            __threadfence();
-            atomicAdd(sync + 1, 1u);
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];\n" : "=r"(g0) : "l"(sync + 1) : "memory");
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;\n" : "=r"(old) : "l"(sync) : "memory");
+        if (old == gridDim.x - 1) {
+            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;\n" ::"l"(sync), "r"(0u) : "memory");
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;\n" ::"l"(sync + 1) : "memory");
         } else {
             unsigned spin = 0;
-            while (*gen == g0 && ++spin < kGridSpinLimit) __nanosleep(20);
-            if (*gen == g0) ok = 0;
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(g) : "l"(sync + 1) : "memory");
+            } while (g == g0 && ++spin < kGridSpinLimit);
+            if (g == g0) ok = 0;
         }
-        __threadfence();
         s_bar_ok = ok;
     }
     __syncthreads();
