@@ -37,7 +37,7 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
         T.n_kc = wd.I / T.kc_ch;
         T.n_units = HK == 1 ? 1 : (HK + 1) / 2;
         T.st_bytes = T.n_units * kTcUnitBytes;
-        tcap = nnz_blocks * 2;                                // a 4x16 block can touch two super-tiles
+        tcap = nnz_blocks * 4;                                // a 4x16 block can touch two super-tiles; gap fillers at most double them
         if (tcap > (int64_t)n_sr * T.n_kc) tcap = (int64_t)n_sr * T.n_kc;
         if (tcap < 0) tcap = 0;
         T.capacity = tcap;
@@ -60,6 +60,11 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
 namespace {
 
 constexpr int kThreads = 256;
+
+// The super-tiles stored for one (group, K-group), given the mask of those that hold a kept block: a missing
+// super-row between two present ones is stored too (as zeros), because one MMA over the joined run costs less than
+// two MMAs around the gap (every MMA fetches the 128 x 32-byte activation tile again).
+__device__ __forceinline__ unsigned tc_fill_gaps(unsigned m) { return (m | ((m << 1) & (m >> 1))) & 0xFFu; }
 
 // b_o and b_i are 4, 8 or 16: divisions by them are shifts by lg().
 __device__ __forceinline__ int lg(int b) { return 31 - __clz(b); }
@@ -124,6 +129,7 @@ count_kernel(const uint8_t *__restrict__ gamma, int NBo, int NBi, int bo, int bi
                     if (any) m |= 1u << r;
                 }
             }
+            m = tc_fill_gaps(m);
             int tot;
             const int before = block_exclusive_scan(__popc(m), warp_sums, tot);
             if (kc < tc.n_kc) {
@@ -774,13 +780,23 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
             return any_kept(s_gamma, o0, min(a.O, o0 + kTcSuperRow) - 1, kc * a.tc_kc_ch, kc * a.tc_kc_ch + a.tc_kc_ch - 1, a.bo,
                             a.bi, a.NBo, a.NBi);
         };
-        int c = 0;
-        for (int q = threadIdx.x; q < g * kTcGroupRows * t.n_kc; q += kThreads) c += st_kept(q / t.n_kc, q % t.n_kc) ? 1 : 0;
-        const int base = block_sum(c, s_sum);
-        c = 0;
+        // Stored super-tiles (gap fillers included) of n_masks (group, K-group) pairs, pair i being (g0 + i / n_kc,
+        // i % n_kc): eight consecutive lanes look at the eight super-rows of one pair, a ballot assembles its mask.
+        auto count_stored = [&](int g0, int n_masks) -> int {
+            int cnt = 0;
+            const int lane = threadIdx.x & 31;
+            for (int q0 = 0; q0 < n_masks * kTcGroupRows; q0 += kThreads) {
+                const int q = q0 + threadIdx.x, i = q >> 3;
+                const bool bit = i < n_masks && st_kept((g0 + i / t.n_kc) * kTcGroupRows + (q & 7), i % t.n_kc);
+                const unsigned m = (__ballot_sync(0xFFFFFFFFu, bit) >> (lane & 24)) & 0xFFu;
+                if ((lane & 7) == 0) cnt += __popc(tc_fill_gaps(m));
+            }
+            return cnt;
+        };
+        const int base = block_sum(count_stored(0, g * t.n_kc), s_sum);
         // chunk 0 counts the whole group (it writes gcnt), the others the K-groups before their own
         const int upto = (chunk == 0) ? t.n_kc : kc_lo;
-        for (int q = threadIdx.x; q < kTcGroupRows * upto; q += kThreads) c += st_kept(g * kTcGroupRows + q / upto, q % upto) ? 1 : 0;
+        const int c = count_stored(g, upto);
         const int counted = block_sum(c, s_sum);
         int before = (chunk == 0) ? 0 : counted;
         if (chunk == 0 && part == 0 && threadIdx.x == 0) {
@@ -789,7 +805,7 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
         }
         for (int kc = kc_lo; kc < kc_hi; ++kc) {
             const int lane = threadIdx.x & 31;           // lane r of every warp looks at super-row r
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, lane < kTcGroupRows && st_kept(g * kTcGroupRows + lane, kc));
+            const unsigned m = tc_fill_gaps(__ballot_sync(0xFFFFFFFFu, lane < kTcGroupRows && st_kept(g * kTcGroupRows + lane, kc)));
             if (part == 0 && threadIdx.x == 0) {
                 a.tc_mask_out[(size_t)g * t.n_kc + kc] = (uint8_t)m;
                 a.tc_off_out[(size_t)g * t.n_kc + kc] = (uint32_t)before;
