@@ -155,7 +155,9 @@ bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma,
  *             over P pixels); wd->H = wd->K = 1.
  * bsp_conv2d: Y[n,y,x,o] = bias[o] + sum over stored blocks of row o / b_o, over taps (h,k) and channels c of
  *             W[o,h,k,iota b_i + c] X[n, y s_h + h - p_h, x s_w + k - p_w, iota b_i + c], X = 0 out of bounds.
- * Only stored blocks are read or multiplied.  Types: BF16 or F32 inputs (wtype = type of X) accumulate in
+ * Only stored blocks are read or multiplied (the tensor-memory kernel works on 16-channel super-tiles: zeroed
+ * blocks that share a super-tile with a stored block, and a missing super-row between two present ones, are
+ * multiplied as zeros).  Types: BF16 or F32 inputs (wtype = type of X) accumulate in
  * float32, bias float32, ytype F32 or BF16 (round to nearest even after the bias); F32 inputs are
  * multiplied as TF32.  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
  *   bias may be NULL (treated as zero).  ws: device scratch of bsp_conv_workspace_bytes() bytes.
