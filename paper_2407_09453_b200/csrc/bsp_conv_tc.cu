@@ -11,17 +11,21 @@
 // dense layer issues N = 128 MMAs, a sparse one an MMA per run of its mask.
 //
 // A CTA owns 128 consecutive positions of one image and one group of 8 super-rows (128 channels).  Positions
-// are counted over rows of the padded input width PW, so that the input of output position m at tap (h, k) is
-// the staged element m + h*PW + k: a tap is a constant offset, positions whose column falls in the padding
-// compute garbage and are not stored.  Activations are staged by tiled TMA loads (out-of-bounds fill = zero
-// padding) as planes [8-channel chunk][position][16 bytes], the no-swizzle K-major core-matrix layout: 8
+// are counted over rows of PW = N' + (K-1)/s_w positions (the padded input width at stride 1), so that the input
+// of output position m at tap (h, k) is a staged element at a constant offset from m: positions whose column falls
+// beyond N' compute garbage and are not stored.  Activations are staged by tiled TMA loads (out-of-bounds fill =
+// zero padding) as planes [16-byte chunk][position][16 bytes], the no-swizzle K-major core-matrix layout: 8
 // consecutive positions are one core matrix, the two K halves of an MMA are two planes or two tap offsets (the
-// descriptor's leading-dimension byte offset).  The stored super-tiles of the group for the stage's K-groups are
-// one contiguous stretch of the packed payload (one bulk copy).
+// descriptor's leading-dimension byte offset).  With strides, each residue (h mod s_h, k mod s_w) in use is staged
+// as a stride-1 image of its own through the tensor map's element strides.  An unpadded stride-1 1x1 layer is a
+// matrix product over all N*L*J positions: its K-groups are staged as [position][32 bytes] planes under the 32-byte
+// swizzle, 256 positions per CTA when the grid stays large.  The stored super-tiles of the group for the stage's
+// K-groups are one contiguous stretch of the packed payload (one bulk copy).
 // Warps 0-3 issue: issuer s takes the K-groups kc with kc % 4 == s and accumulates them in its own 128 columns
 // of tensor memory (an MMA this small costs more to issue than to execute, and MMAs of different threads on one
-// accumulator are not ordered, hence four accumulator sets, zeroed at the start and summed at the end).  Warp 4
-// produces.  Then all eight warps read their TMEM lanes back, add the four sets and the bias, and store.
+// accumulator are not ordered, hence four accumulator sets, zeroed at the start and summed at the end; with 256
+// positions the issuers split into two position halves x two K phases).  Warp 4 produces.  Then all eight warps
+// read their TMEM lanes back, add the sets and the bias, and store.
 // Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
 #include <cuda.h>
 #include <cstdlib>
