@@ -62,6 +62,9 @@ struct TcParams {
     int ph_a[4], ph_b[4];                  // the phases in use, in the order they lie in a stage
     int mt;                   // 128-position tiles per CTA: 1, or 2 for large matrix products (the weights are then
                               // fetched once for 256 positions); the four issuers split into mt halves x 4/mt K phases
+    int ng;                   // channel groups per CTA: 1, or 2 for the largest matrix products (mt == 2 only: the
+                              // activations are then fetched once for 256 channels); issuer = (half, group), all K-groups
+    int n_groups, w_stride;   // groups of the layer; bytes between the two groups' weights in a stage
     int GK, n_stage_iters, stages, stage_bytes, act_bytes, act_box_bytes;
     int ytype;
 };
@@ -111,26 +114,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     __shared__ __align__(8) uint64_t s_full[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_empty[kTcMaxStages];
     __shared__ __align__(8) uint64_t s_done;
-    __shared__ uint32_t s_tmem, s_gbase, s_gcnt, s_fail;
+    __shared__ uint32_t s_tmem, s_gbase[2], s_gcnt[2], s_fail;
     __shared__ const uint8_t *s_payload;
     __shared__ uint64_t s_ahi[64];          // per K-step of a super-tile: A descriptor without its address field
     __shared__ uint32_t s_aoff[64];         // ... and the operand's offset from the K-group's first plane, in 16-byte units
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int g = blockIdx.y;
+    const int g = blockIdx.y * p.ng;
     const int S = p.stages;
 
     // stored super-tiles of this group: masks and offsets of every K-group -> shared memory
-    uint32_t *s_off = (uint32_t *)smem;                      // [n_kc]
-    uint8_t *s_mask = smem + (size_t)p.n_kc * 4;             // [n_kc]
-    for (int i = tid; i < p.n_kc; i += kTcThreads) {
-        s_off[i] = p.off[(size_t)g * p.n_kc + i];
-        s_mask[i] = p.mask[(size_t)g * p.n_kc + i];
+    // (a second group beyond the layer's last reads as empty)
+    uint32_t *s_off = (uint32_t *)smem;                             // [ng][n_kc]
+    uint8_t *s_mask = smem + (size_t)p.ng * p.n_kc * 4;             // [ng][n_kc]
+    const int n_meta = (g + p.ng <= p.n_groups ? p.ng : 1) * p.n_kc;
+    for (int i = tid; i < p.ng * p.n_kc; i += kTcThreads) {
+        s_off[i] = i < n_meta ? p.off[(size_t)g * p.n_kc + i] : 0u;
+        s_mask[i] = i < n_meta ? p.mask[(size_t)g * p.n_kc + i] : (uint8_t)0;
     }
     if (tid == 0) {
         uint32_t base = 0;
         for (int q = 0; q < g; ++q) base += p.gcnt[q];
-        s_gbase = base; s_gcnt = p.gcnt[g]; s_fail = 0;
+        s_gbase[0] = base; s_gcnt[0] = p.gcnt[g];
+        const bool second = p.ng == 2 && g + 1 < p.n_groups;
+        s_gbase[1] = base + p.gcnt[g]; s_gcnt[1] = second ? p.gcnt[g + 1] : 0u;
+        s_fail = 0;
         s_payload = p.packed + ((const PackedHeader *)p.packed)->off_tc_payload;
     }
     // tile geometry
@@ -178,7 +186,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     // The producer thread sets the barriers up and starts the activation loads of the first stages at once: they
     // need nothing of the index arrays that the other threads are still fetching.  A full barrier takes two
     // arrivals per phase, one with the activation bytes and one with the weight bytes.
-    const int meta_bytes = ((p.n_kc * 5 + 1023) / 1024) * 1024;
+    const int meta_bytes = ((p.ng * p.n_kc * 5 + 1023) / 1024) * 1024;
     const uint32_t ring = s32(smem) + meta_bytes;
     // first input column and row of the tile's phase (0, 0); phase (a, b) starts a rows and b columns further
     const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first * p.sh - p.ph, c3 = p.is_gemm ? m0 : n_img;
@@ -222,27 +230,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
 
     if (warp == kIssuers) {
         // ================= producer (warp 4) =================
+        // (one thread runs the whole loop, so its instruction count per stage is on the critical path: the slot, the
+        // barrier parity and the addresses advance by additions, loop invariants sit in registers)
         if (lane == 0) {
-            for (int it = 0; it < p.n_stage_iters; ++it) {
-                const int slot = it % S;
-                if (it >= S && !wait_bar(s32(&s_empty[slot]), (uint32_t)((it / S - 1) & 1))) { atomicExch(&s_fail, 1u); break; }
-                const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
-                const uint32_t o_lo = s_off[kc0];
-                const uint32_t o_hi = (kc0 + nk < p.n_kc) ? s_off[kc0 + nk] : s_gcnt;
-                const uint32_t wbytes = (o_hi - o_lo) * (uint32_t)p.st_bytes;
-                const uint32_t bar = s32(&s_full[slot]);
-                const uint32_t dst = ring + slot * p.stage_bytes;
-                if (it >= S) {          // the first S activation loads were issued before the index arrays arrived
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"((uint32_t)(p.n_phase * p.act_box_bytes)) : "memory");
-                    for (int ph = 0; ph < p.n_phase; ++ph)
+            const int GK = p.GK, n_kc = p.n_kc, n_it = p.n_stage_iters, n_phase = p.n_phase, ng = p.ng;
+            const uint32_t st_bytes = (uint32_t)p.st_bytes, act_tx = (uint32_t)(p.n_phase * p.act_box_bytes);
+            const uint32_t stage_bytes = (uint32_t)p.stage_bytes, w_first = (uint32_t)p.act_bytes, w_stride = (uint32_t)p.w_stride;
+            const uint32_t full0 = s32(&s_full[0]), empty0 = s32(&s_empty[0]);
+            const uint8_t *const pay0 = s_payload + (size_t)s_gbase[0] * st_bytes;
+            const uint8_t *const pay1 = s_payload + (size_t)s_gbase[1] * st_bytes;
+            const uint32_t gcnt0 = s_gcnt[0], gcnt1 = s_gcnt[1];
+            uint32_t slot = 0, wrapped = 0, dst = ring;       // wrapped: times the ring has been filled
+            int kc0 = 0, kcoord = 0;
+            for (int it = 0; it < n_it; ++it) {
+                const uint32_t bar = full0 + slot * 8u;
+                if (wrapped && !wait_bar(empty0 + slot * 8u, (wrapped - 1u) & 1u)) { atomicExch(&s_fail, 1u); break; }
+                const int kc1 = kc0 + GK;
+                const uint32_t lo0 = s_off[kc0], hi0 = kc1 < n_kc ? s_off[kc1] : gcnt0;
+                uint32_t lo1 = 0u, hi1 = 0u;
+                if (ng == 2) { lo1 = s_off[n_kc + kc0]; hi1 = kc1 < n_kc ? s_off[n_kc + kc1] : gcnt1; }
+                const uint32_t wb0 = (hi0 - lo0) * st_bytes, wb1 = (hi1 - lo1) * st_bytes;
+                if (wrapped) {          // the first S activation loads were issued before the index arrays arrived
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(act_tx) : "memory");
+                    for (int ph = 0; ph < n_phase; ++ph)
                         asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
                                      ::"r"(dst + ph * p.phase_bytes), "l"(&p.tmap), "r"(bar), "r"(0), "r"(c1 + p.ph_b[ph]), "r"(c2 + p.ph_a[ph]),
-                                       "r"(c3), "r"(kc0 * p.coords_per_kc) : "memory");
+                                       "r"(c3), "r"(kcoord) : "memory");
                 }
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(wbytes) : "memory");
-                if (wbytes)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(wb0 + wb1) : "memory");
+                if (wb0)
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
-                                 ::"r"(dst + p.act_bytes), "l"(s_payload + (size_t)(s_gbase + o_lo) * p.st_bytes), "r"(wbytes), "r"(bar) : "memory");
+                                 ::"r"(dst + w_first), "l"(pay0 + (size_t)lo0 * st_bytes), "r"(wb0), "r"(bar) : "memory");
+                if (wb1)
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                                 ::"r"(dst + w_first + w_stride), "l"(pay1 + (size_t)lo1 * st_bytes), "r"(wb1), "r"(bar) : "memory");
+                kc0 = kc1; kcoord += GK * p.coords_per_kc;
+                if (++slot == (uint32_t)S) { slot = 0; ++wrapped; dst = ring; } else dst += stage_bytes;
             }
         }
     } else if (warp < kIssuers) {
@@ -257,29 +280,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             // stage + plane + s_aoff[u]; of a B operand weights + 32 * (tiles before the K-group * n_units
             // + u * tiles of the K-group + tiles before the run).  B: K halves 128 bytes apart, row groups 256.
             const uint64_t b_hi = smem_desc(0, 128, 256);
-            const int plane16 = (p.plane_bytes >> 4) * p.chunks_per_kc;  // 16-byte units between K-groups' planes
+            const uint32_t plane16 = (uint32_t)((p.plane_bytes >> 4) * p.chunks_per_kc);  // 16-byte units between K-groups' planes
             const uint32_t nu = (uint32_t)p.n_units;
             const uint64_t ahi0 = s_ahi[0];
             const uint32_t aoff0 = s_aoff[0];
             const uint32_t dset = tmem + (uint32_t)warp * 128u;
-            const int kphases = kIssuers / p.mt, kphase = warp % kphases;      // K-groups kc with kc % kphases == kphase
-            const uint32_t ahalf = (uint32_t)(warp / kphases) * 256u;          // second 128 positions: 4096 bytes into the plane
+            // two groups per CTA: issuer = (position half, group), every K-group; its accumulator is its own 128 columns
+            const int gq = p.ng == 2 ? (warp & 1) : 0;
+            const int kphases = p.ng == 2 ? 1 : kIssuers / p.mt;
+            const int kphase = warp % kphases;                                  // K-groups kc with kc % kphases == kphase
+            const uint32_t ahalf = (uint32_t)(p.mt == 2 ? warp >> 1 : 0) * 256u;  // second 128 positions: 4096 bytes into the plane
+            const uint32_t *my_off = s_off + gq * p.n_kc;
+            const uint8_t *my_mask = s_mask + gq * p.n_kc;
+            // (as in the producer: running slot, parity and addresses, invariants in registers)
+            const int GK = p.GK, n_kc = p.n_kc, n_it = p.n_stage_iters;
+            const uint32_t ring16 = ring >> 4, stage_step16 = (uint32_t)p.stage_bytes >> 4;
+            const uint32_t wofs16 = (uint32_t)(p.act_bytes + gq * p.w_stride) >> 4;
+            const uint32_t full0 = s32(&s_full[0]), empty0 = s32(&s_empty[0]);
+            uint32_t slot = 0, par = 0, stage16 = ring16;
+            int kc0 = 0;
             bool ok = true;
-            for (int it = 0; it < p.n_stage_iters; ++it) {
-                const int slot = it % S;
-                if (!wait_bar(s32(&s_full[slot]), (uint32_t)((it / S) & 1))) { ok = false; break; }
+            for (int it = 0; it < n_it; ++it, kc0 += GK) {
+                if (!wait_bar(full0 + slot * 8u, par)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const int kc0 = it * p.GK, nk = min(p.GK, p.n_kc - kc0);
-                const uint32_t stage16 = (ring + slot * p.stage_bytes) >> 4;
-                const uint32_t w16 = stage16 + (p.act_bytes >> 4);
-                const uint32_t o_lo = s_off[kc0];
+                const int nk = min(GK, n_kc - kc0);
+                const uint32_t w16 = stage16 + wofs16;
+                const uint32_t o_lo = my_off[kc0];
                 int kl = (kphase - kc0) & (kphases - 1);          // first K-group of the stage that is mine
                 for (; kl < nk; kl += kphases) {
-                    uint32_t m = s_mask[kc0 + kl];
+                    uint32_t m = my_mask[kc0 + kl];
                     if (m == 0) continue;
                     const uint32_t cnt = __popc(m);
-                    const uint32_t a16 = stage16 + kl * plane16 + ahalf;
-                    uint32_t b16 = w16 + (s_off[kc0 + kl] - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
+                    const uint32_t a16 = stage16 + (uint32_t)kl * plane16 + ahalf;
+                    uint32_t b16 = w16 + (my_off[kc0 + kl] - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
                     while (m) {
                         const int r0 = __ffs(m) - 1;
                         const int len = __ffs(~(m >> r0)) - 1;                  // run of stored super-rows r0 .. r0 + len - 1
@@ -300,7 +333,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                         b16 += (uint32_t)len * 32u;
                     }
                 }
-                commit_to(s32(&s_empty[slot]));
+                commit_to(empty0 + slot * 8u);
+                if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; stage16 = ring16; } else stage16 += stage_step16;
             }
             if (ok) commit_to(s32(&s_done));
             else atomicExch(&s_fail, 1u);
@@ -319,7 +353,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         // one position tile: warps 0-3 take super-rows 0-3, warps 4-7 rows 4-7, four accumulator sets each;
         // two tiles: warps 0-3 take the first 128 positions (sets 0, 1), warps 4-7 the second (sets 2, 3), all rows
         const int half = p.mt == 2 ? (warp >> 2) : 0;
-        const int set0 = p.mt == 2 ? 2 * half : 0, nsets = kIssuers / p.mt;
+        // (two groups: one accumulator set per (half, group), nothing to add)
+        const int nsets = p.ng == 2 ? 1 : kIssuers / p.mt;
         const int r_lo = p.mt == 2 ? 0 : (warp >> 2) * 4, r_hi = p.mt == 2 ? kTcGroupRows : r_lo + 4;
         const int m = half * 128 + lq * 32 + lane;
         bool valid;
@@ -332,8 +367,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
         }
         const int oe = (p.ytype == BSP_BF16) ? 2 : 4;
 #pragma unroll 1
-        for (int r = r_lo; r < r_hi; ++r) {
-            const int ch = (g * kTcGroupRows + r) * kTcSuperRow;
+        for (int rr = r_lo; rr < r_hi + (p.ng - 1) * kTcGroupRows; ++rr) {
+            const int gq = rr / kTcGroupRows, r = rr % kTcGroupRows;          // group of the CTA, super-row in it
+            const int set0 = p.ng == 2 ? 2 * half + gq : (p.mt == 2 ? 2 * half : 0);
+            const int ch = ((g + gq) * kTcGroupRows + r) * kTcSuperRow;
             if (ch >= p.O) break;
             // the four accumulator sets of this super-row
             uint32_t v[kIssuers][16];
@@ -538,8 +575,16 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         tiles = (long long)xd.N * p.tiles_per_img;
     }
     p.plane_bytes = plane_pos * 16;
+    // The largest matrix products take two channel groups per CTA as well (256 positions x 256 channels: every
+    // activation byte fetched from L2 then feeds twice the arithmetic), while the grid still fills the SMs twice.
+    p.ng = 1; p.n_groups = T.n_groups;
+    if (gemm && p.mt == 2 && T.n_groups >= 2 && tiles * ((T.n_groups + 1) / 2) >= 2 * 148) p.ng = 2;
+    if (const char *e = getenv("BSP_TC_GROUPS")) {                 // tuning: pin the groups per CTA
+        if (e[0] == '1') p.ng = 1;
+        if (e[0] == '2' && gemm && p.mt == 2 && T.n_groups >= 2) p.ng = 2;
+    }
     // (several phases: each plane set is padded to 128 bytes)
-    const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + (p.n_phase > 1 ? 128 : 0)) + (size_t)kTcGroupRows * T.st_bytes;
+    const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + (p.n_phase > 1 ? 128 : 0)) + (size_t)p.ng * kTcGroupRows * T.st_bytes;
     int GK = (int)(49152 / per_kc);
     if (GK < 1) GK = 1;
     if (GK > T.n_kc) GK = T.n_kc;
@@ -549,9 +594,10 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     // every tiled load must land on a 128-byte boundary of shared memory: the phases' plane sets are padded to that
     p.phase_bytes = (int)align_up((size_t)p.act_box_bytes, 128);
     p.act_bytes = (int)align_up((size_t)p.n_phase * p.phase_bytes + 32, 128);        // + slack read by positions in the padding
-    p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)GK * kTcGroupRows * T.st_bytes, 1024);
+    p.w_stride = GK * kTcGroupRows * T.st_bytes;
+    p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)p.ng * p.w_stride, 1024);
     p.n_stage_iters = (T.n_kc + GK - 1) / GK;
-    const size_t meta = align_up((size_t)T.n_kc * 5, 1024);
+    const size_t meta = align_up((size_t)p.ng * T.n_kc * 5, 1024);
     int stages = (int)(((size_t)kTcMaxSmem - meta - 1024) / p.stage_bytes);
     if (stages > kTcMaxStages) stages = kTcMaxStages;
     if (stages > p.n_stage_iters) stages = p.n_stage_iters;
@@ -587,7 +633,7 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         BSP_CUDA_OK(cudaFuncSetAttribute(conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem));
         opted[dev] = true;
     }
-    dim3 grid((unsigned)tiles, (unsigned)T.n_groups);
+    dim3 grid((unsigned)tiles, (unsigned)((T.n_groups + p.ng - 1) / p.ng));
     if (wd.wtype == BSP_I8) conv_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(p);
     else conv_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());

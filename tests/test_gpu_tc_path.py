@@ -110,6 +110,23 @@ def test_tc_gemm_two_position_tiles_per_cta(dtype):
     check(got, ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b), dtype)
 
 
+@pytest.mark.parametrize("dtype,frac", [("bf16", 0.5), ("i8", 0.75), ("bf16", 0.0)])
+def test_tc_gemm_two_channel_groups_per_cta(dtype, frac, monkeypatch):
+    """256 positions x 256 channels per CTA (BSP_TC_GROUPS=2 pins what only the largest products choose): nine
+    channel groups, so the last CTA row has no second group; a last half super-row; ragged last position tile."""
+    monkeypatch.setenv("BSP_TC_GROUPS", "2")
+    O, I, P = 1144, 96, 8500
+    W = make_case(681, O, I, 1, 1, dtype)
+    NB = (O // 8) * (I // 8)
+    gamma = synth.random_gamma(682, O // 8, I // 8, int(NB * frac))
+    X = make_x(683, (P, I), dtype)
+    b = make_bias(684, O, dtype)
+    lay = gpu_layer(W, gamma, 8, 8, dtype)
+    got = gpu_gemm(lay, X, b, dtype)
+    rp, ci, pl = ref.compact(W, gamma, 8, 8)
+    check(got, ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b), dtype)
+
+
 def test_tc_config_resnet_conv_with_l2_gamma():
     layer = synth.Layer("cfg2", 256, 256, 3, 3, 32, 14, 14, 1, 1, 1, 1)
     W, X, b = synth.make_layer_tensors(layer, "bf16", config=2)
