@@ -41,6 +41,7 @@ constexpr int kTcMaxSmem = 200 * 1024;
 constexpr int kTcMaxDevices = 64;
 constexpr int kTmemCols = 128 * kIssuers;
 constexpr uint32_t kTcSpinLimit = 1u << 22;
+constexpr uint32_t kOffMask = 0x0FFFFFFFu;          // low bits of a K-group entry's first word: super-tiles before it
 
 struct TcParams {
     CUtensorMap tmap;        // activations as (16 bytes, x, y, n, chunk)
@@ -125,12 +126,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
 
     // stored super-tiles of this group: masks and offsets of every K-group -> shared memory
     // (a second group beyond the layer's last reads as empty)
-    uint32_t *s_off = (uint32_t *)smem;                             // [ng][n_kc]
-    uint8_t *s_mask = smem + (size_t)p.ng * p.n_kc * 4;             // [ng][n_kc]
+    // One entry per K-group, decoded here by all threads so that the issuing threads need not: .x = stored super-tiles
+    // of the group before the K-group (28 bits) and in it (4 bits); .y = its runs of consecutive stored super-rows, a
+    // byte each, first run lowest: 0x80 | first row << 3 | (length - 1); a zero byte ends the list.
+    uint2 *s_ent = (uint2 *)smem;                                   // [ng][n_kc]
     const int n_meta = (g + p.ng <= p.n_groups ? p.ng : 1) * p.n_kc;
     for (int i = tid; i < p.ng * p.n_kc; i += kTcThreads) {
-        s_off[i] = i < n_meta ? p.off[(size_t)g * p.n_kc + i] : 0u;
-        s_mask[i] = i < n_meta ? p.mask[(size_t)g * p.n_kc + i] : (uint8_t)0;
+        uint32_t off = 0u, m = 0u;
+        if (i < n_meta) { off = p.off[(size_t)g * p.n_kc + i]; m = p.mask[(size_t)g * p.n_kc + i]; }
+        uint32_t runs = 0u, sh = 0u;
+        for (uint32_t mm = m; mm;) {
+            const uint32_t r0 = (uint32_t)__ffs(mm) - 1u, len = (uint32_t)__ffs(~(mm >> r0)) - 1u;
+            mm &= ~(((1u << len) - 1u) << r0);
+            runs |= (0x80u | (r0 << 3) | (len - 1u)) << sh;
+            sh += 8u;
+        }
+        s_ent[i] = make_uint2(off | ((uint32_t)__popc(m) << 28), runs);
     }
     if (tid == 0) {
         uint32_t base = 0;
@@ -186,7 +197,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     // The producer thread sets the barriers up and starts the activation loads of the first stages at once: they
     // need nothing of the index arrays that the other threads are still fetching.  A full barrier takes two
     // arrivals per phase, one with the activation bytes and one with the weight bytes.
-    const int meta_bytes = ((p.ng * p.n_kc * 5 + 1023) / 1024) * 1024;
+    const int meta_bytes = ((p.ng * p.n_kc * 8 + 1023) / 1024) * 1024;
     const uint32_t ring = s32(smem) + meta_bytes;
     // first input column and row of the tile's phase (0, 0); phase (a, b) starts a rows and b columns further
     const int c1 = p.is_gemm ? 0 : -p.pw, c2 = p.is_gemm ? 0 : y_first * p.sh - p.ph, c3 = p.is_gemm ? m0 : n_img;
@@ -246,9 +257,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 const uint32_t bar = full0 + slot * 8u;
                 if (wrapped && !wait_bar(empty0 + slot * 8u, (wrapped - 1u) & 1u)) { atomicExch(&s_fail, 1u); break; }
                 const int kc1 = kc0 + GK;
-                const uint32_t lo0 = s_off[kc0], hi0 = kc1 < n_kc ? s_off[kc1] : gcnt0;
+                const uint32_t lo0 = s_ent[kc0].x & kOffMask, hi0 = kc1 < n_kc ? s_ent[kc1].x & kOffMask : gcnt0;
                 uint32_t lo1 = 0u, hi1 = 0u;
-                if (ng == 2) { lo1 = s_off[n_kc + kc0]; hi1 = kc1 < n_kc ? s_off[n_kc + kc1] : gcnt1; }
+                if (ng == 2) { lo1 = s_ent[n_kc + kc0].x & kOffMask; hi1 = kc1 < n_kc ? s_ent[n_kc + kc1].x & kOffMask : gcnt1; }
                 const uint32_t wb0 = (hi0 - lo0) * st_bytes, wb1 = (hi1 - lo1) * st_bytes;
                 if (wrapped) {          // the first S activation loads were issued before the index arrays arrived
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(act_tx) : "memory");
@@ -290,8 +301,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             const int kphases = p.ng == 2 ? 1 : kIssuers / p.mt;
             const int kphase = warp % kphases;                                  // K-groups kc with kc % kphases == kphase
             const uint32_t ahalf = (uint32_t)(p.mt == 2 ? warp >> 1 : 0) * 256u;  // second 128 positions: 4096 bytes into the plane
-            const uint32_t *my_off = s_off + gq * p.n_kc;
-            const uint8_t *my_mask = s_mask + gq * p.n_kc;
+            const uint2 *my_ent = s_ent + gq * p.n_kc;
             // (as in the producer: running slot, parity and addresses, invariants in registers)
             const int GK = p.GK, n_kc = p.n_kc, n_it = p.n_stage_iters;
             const uint32_t ring16 = ring >> 4, stage_step16 = (uint32_t)p.stage_bytes >> 4;
@@ -305,23 +315,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const int nk = min(GK, n_kc - kc0);
                 const uint32_t w16 = stage16 + wofs16;
-                const uint32_t o_lo = my_off[kc0];
+                const uint32_t o_lo = my_ent[kc0].x & kOffMask;
                 int kl = (kphase - kc0) & (kphases - 1);          // first K-group of the stage that is mine
                 for (; kl < nk; kl += kphases) {
-                    uint32_t m = my_mask[kc0 + kl];
-                    if (m == 0) continue;
-                    const uint32_t cnt = __popc(m);
+                    const uint2 ent = my_ent[kc0 + kl];
+                    uint32_t runs = ent.y;
+                    if (runs == 0u) continue;
+                    const uint32_t cnt = ent.x >> 28;
                     const uint32_t a16 = stage16 + (uint32_t)kl * plane16 + ahalf;
-                    uint32_t b16 = w16 + (my_off[kc0 + kl] - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
-                    while (m) {
-                        const int r0 = __ffs(m) - 1;
-                        const int len = __ffs(~(m >> r0)) - 1;                  // run of stored super-rows r0 .. r0 + len - 1
-                        m &= ~(((1u << len) - 1u) << r0);
-                        const uint32_t idesc = idesc0 | ((uint32_t)(len * 16 >> 3) << 17);
-                        const uint32_t d = dset + (uint32_t)r0 * 16u;
+                    const uint64_t a0 = ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu);
+                    uint32_t b16 = w16 + ((ent.x & kOffMask) - o_lo) * nu * 32u;   // first tile of the K-group, K-step 0
+                    for (; runs; runs >>= 8) {
+                        const uint32_t r0 = (runs >> 3) & 7u, len = (runs & 7u) + 1u;   // stored super-rows r0 .. r0 + len - 1
+                        const uint32_t idesc = idesc0 | (len << 18);                   // N = 16 len, the field holds N / 8
+                        const uint32_t d = dset + r0 * 16u;
                         if (nu == 1) {
-                            if (i8) mma_i8(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
-                            else mma_bf16(d, ahi0 | (uint64_t)((a16 + aoff0) & 0x3FFFu), b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
+                            if (i8) mma_i8(d, a0, b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
+                            else mma_bf16(d, a0, b_hi | (uint64_t)(b16 & 0x3FFFu), idesc, 1u);
                         } else {
                             uint32_t bu = b16;
                             for (uint32_t u = 0; u < nu; ++u) {
@@ -330,7 +340,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                                 bu += cnt * 32u;
                             }
                         }
-                        b16 += (uint32_t)len * 32u;
+                        b16 += len * 32u;
                     }
                 }
                 commit_to(empty0 + slot * 8u);
@@ -526,7 +536,7 @@ bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd)
     if (!tc_geometry(wd, xd, g)) return false;
     // the per-K-group index of the group plus two stages (one K-group of activations and its dense weights
     // each) must fit the shared memory
-    const size_t meta = align_up((size_t)L.tc.n_kc * 5, 1024);
+    const size_t meta = align_up((size_t)L.tc.n_kc * 8, 1024);
     size_t per_kc;
     if (g.gemm) {
         if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
@@ -597,7 +607,7 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     p.w_stride = GK * kTcGroupRows * T.st_bytes;
     p.stage_bytes = (int)align_up((size_t)p.act_bytes + (size_t)p.ng * p.w_stride, 1024);
     p.n_stage_iters = (T.n_kc + GK - 1) / GK;
-    const size_t meta = align_up((size_t)p.ng * T.n_kc * 5, 1024);
+    const size_t meta = align_up((size_t)p.ng * T.n_kc * 8, 1024);
     int stages = (int)(((size_t)kTcMaxSmem - meta - 1024) / p.stage_bytes);
     if (stages > kTcMaxStages) stages = kTcMaxStages;
     if (stages > p.n_stage_iters) stages = p.n_stage_iters;
