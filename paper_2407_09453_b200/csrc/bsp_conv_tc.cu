@@ -83,6 +83,20 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
     return false;
 }
 
+// The same wait by polling: mbarrier.test_wait does not suspend the thread, and on a phase that is already
+// complete it answers in a fraction of the ~200 cycles that try_wait takes.  For the single threads that run the
+// producer and issue loops, where every cycle of a wait is on the critical path.
+__device__ __forceinline__ bool poll_bar(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
 // Shared-memory matrix descriptor, no swizzle, K-major: 8 rows x 16 bytes core matrices; `lbo` = bytes between
 // the two K halves, `sbo` = bytes between 8-row groups.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
@@ -255,7 +269,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             int kc0 = 0, kcoord = 0;
             for (int it = 0; it < n_it; ++it) {
                 const uint32_t bar = full0 + slot * 8u;
-                if (wrapped && !wait_bar(empty0 + slot * 8u, (wrapped - 1u) & 1u)) { atomicExch(&s_fail, 1u); break; }
+                if (wrapped && !poll_bar(empty0 + slot * 8u, (wrapped - 1u) & 1u)) { atomicExch(&s_fail, 1u); break; }
                 const int kc1 = kc0 + GK;
                 const uint32_t lo0 = s_ent[kc0].x & kOffMask, hi0 = kc1 < n_kc ? s_ent[kc1].x & kOffMask : gcnt0;
                 uint32_t lo1 = 0u, hi1 = 0u;
@@ -311,7 +325,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
             int kc0 = 0;
             bool ok = true;
             for (int it = 0; it < n_it; ++it, kc0 += GK) {
-                if (!wait_bar(full0 + slot * 8u, par)) { ok = false; break; }
+                if (!poll_bar(full0 + slot * 8u, par)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const int nk = min(GK, n_kc - kc0);
                 const uint32_t w16 = stage16 + wofs16;
@@ -352,7 +366,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
     }
 
     // ================= epilogue: all eight warps; warp w reads TMEM lanes 32*(w%4).. (positions) of super-rows 4*(w/4).. =================
+    // (threads without a loop of their own park at the block barrier, not in a polling loop, until the loops end)
     __syncwarp();
+    __syncthreads();
     bool done = wait_bar(s32(&s_done), 0);
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     __syncthreads();
