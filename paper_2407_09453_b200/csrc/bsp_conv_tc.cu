@@ -120,6 +120,42 @@ __device__ __forceinline__ void commit_to(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 
+// Transposes 4x4 blocks of 16-byte chunks inside every group of four lanes: on entry a lane holds the four chunks
+// (v[4c .. 4c+3], c = 0..3) of its own row, on exit chunk (lane % 4) of the four rows of its group (v[4j .. 4j+3] =
+// row j of the group).  All 32 lanes take part.
+__device__ __forceinline__ void transpose_chunks(uint32_t (&v)[16], int lane)
+{
+    const bool hi2 = (lane & 2) != 0, hi1 = (lane & 1) != 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {          // the 2x2 blocks off the diagonal change places (partner: lane ^ 2)
+        const uint32_t s0 = hi2 ? v[k] : v[8 + k], s1 = hi2 ? v[4 + k] : v[12 + k];
+        const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, s0, 2), r1 = __shfl_xor_sync(0xFFFFFFFFu, s1, 2);
+        if (hi2) { v[k] = r0; v[4 + k] = r1; } else { v[8 + k] = r0; v[12 + k] = r1; }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {          // then the off-diagonal chunks inside every 2x2 block (partner: lane ^ 1)
+        const uint32_t s0 = hi1 ? v[k] : v[4 + k], s1 = hi1 ? v[8 + k] : v[12 + k];
+        const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, s0, 1), r1 = __shfl_xor_sync(0xFFFFFFFFu, s1, 1);
+        if (hi1) { v[k] = r0; v[8 + k] = r1; } else { v[4 + k] = r0; v[12 + k] = r1; }
+    }
+}
+
+// Stores 16 32-bit outputs per lane (one row of Y each: `dst`, used if `valid`) so that a warp instruction writes whole
+// 64-byte pieces of eight rows instead of 16 bytes of thirty-two: the chunks are transposed inside groups of four
+// lanes, lane 4q + c then writes chunk c of the rows of lanes 4q .. 4q + 3.  nch: channels present (8 or 16).
+__device__ __forceinline__ void store_rows32(uint32_t (&v)[16], uint8_t *dst, bool valid, int nch, int lane)
+{
+    transpose_chunks(v, lane);
+    const int c = lane & 3, first = lane & ~3;
+    const unsigned long long d = (unsigned long long)dst;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int ok = __shfl_sync(0xFFFFFFFFu, (int)valid, first + j);
+        const unsigned long long dj = __shfl_sync(0xFFFFFFFFu, d, first + j);
+        if (ok && 4 * c < nch) *(uint4 *)(dj + 16u * c) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    }
+}
+
 // kI8: int8 inputs with int32 accumulators, bias and output (kind::i8); otherwise bf16 with fp32 (kind::f16).
 template <bool kI8>
 __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_constant__ TcParams p)
@@ -414,18 +450,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                 }
             }
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-            if (!valid) continue;
             const int nch = min(16, p.O - ch);        // 16, or 8 in a last half super-row
             if constexpr (kI8) {                      // exact: int32 sums of the four sets + int32 bias, int32 out
-                int iv[16];
+                uint32_t iv[16];
                 const int *ib = (const int *)p.bias;
 #pragma unroll
                 for (int e = 0; e < 16; ++e)
-                    iv[e] = (int)v[0][e] + (int)v[1][e] + (int)v[2][e] + (int)v[3][e] + ((ib != nullptr && e < nch) ? __ldg(ib + ch + e) : 0);
-                uint8_t *dsti = p.Y + (pix * p.O + ch) * 4;
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (q * 4 < nch) *(int4 *)(dsti + q * 16) = make_int4(iv[4 * q], iv[4 * q + 1], iv[4 * q + 2], iv[4 * q + 3]);
+                    iv[e] = (uint32_t)((int)v[0][e] + (int)v[1][e] + (int)v[2][e] + (int)v[3][e] + ((ib != nullptr && e < nch) ? __ldg(ib + ch + e) : 0));
+                store_rows32(iv, p.Y + (pix * p.O + ch) * 4, valid, nch, lane);
                 continue;
             } else {
             float f[16];
@@ -435,13 +467,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) conv_tc_kernel(const __grid_con
                        ((p.bias != nullptr && e < nch) ? __ldg(p.bias + ch + e) : 0.f);
             uint8_t *dst = p.Y + (pix * p.O + ch) * oe;
             if (oe == 4) {
+                uint32_t fv[16];
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (q * 4 < nch) *(float4 *)(dst + q * 16) = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+                for (int e = 0; e < 16; ++e) fv[e] = __float_as_uint(f[e]);
+                store_rows32(fv, dst, valid, nch, lane);
             } else {
 #pragma unroll
                 for (int q = 0; q < 2; ++q)
-                    if (q * 8 < nch) {
+                    if (valid && q * 8 < nch) {
                         __nv_bfloat162 h0 = __floats2bfloat162_rn(f[8 * q], f[8 * q + 1]), h1 = __floats2bfloat162_rn(f[8 * q + 2], f[8 * q + 3]);
                         __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * q + 4], f[8 * q + 5]), h3 = __floats2bfloat162_rn(f[8 * q + 6], f[8 * q + 7]);
                         *(uint4 *)(dst + q * 16) = make_uint4(*(uint32_t *)&h0, *(uint32_t *)&h1, *(uint32_t *)&h2, *(uint32_t *)&h3);
