@@ -24,8 +24,13 @@
 // Warps 0-3 issue: issuer s takes the K-groups kc with kc % 4 == s and accumulates them in its own 128 columns
 // of tensor memory (an MMA this small costs more to issue than to execute, and MMAs of different threads on one
 // accumulator are not ordered, hence four accumulator sets, zeroed at the start and summed at the end; with 256
-// positions the issuers split into two position halves x two K phases).  Warp 4 produces.  Then all eight warps
-// read their TMEM lanes back, add the sets and the bias, and store.
+// positions the issuers split into two position halves x two K phases; the largest products take two channel
+// groups per CTA as well, 256 positions x 256 channels, and every issuer then owns one (half, group) quadrant over
+// all K-groups).  Warp 4 produces.  The producer and the issuers are single threads whose instruction count per stage
+// is on the critical path: the runs of every K-group are decoded once, by all threads, into 8-byte entries in shared
+// memory, and the loops advance slot, parity and addresses by additions and poll their barriers.  Then all eight warps
+// read their TMEM lanes back, add the sets and the bias, transpose 16-byte chunks inside groups of four lanes and
+// store 64-byte pieces of rows.
 // Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
 #include <cuda.h>
 #include <cstdlib>
