@@ -175,6 +175,15 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd);
 
+/* The same product on a named kernel, for validation and tuning: every kernel must give the result of the
+ * definition above, so the tests run each layer on every kernel that can take it.  BSP_KERNEL_AUTO is bsp_conv2d();
+ * a kernel that cannot take the layer returns BSP_ERR_SHAPE and launches nothing. */
+typedef enum { BSP_KERNEL_AUTO = 0, BSP_KERNEL_GEMM_TC = 1, BSP_KERNEL_CONV_TC = 2, BSP_KERNEL_CONV_MMA = 3 } bsp_kernel;
+bsp_status bsp_conv2d_on(bsp_kernel which, const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                         const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
+/* 1 if the named kernel can run a layer with these descriptors and output type, else 0 (host-side decision). */
+int bsp_conv_kernel_takes(bsp_kernel which, const bsp_wdesc *wd, const bsp_xdesc *xd, bsp_dtype ytype);
+
 /* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
  * (BSP_OK if none), then clears it. */
 bsp_status bsp_check(void *ws, void *stream);

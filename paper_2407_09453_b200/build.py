@@ -1,14 +1,20 @@
-"""Builds libbsp.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Builds libbsp.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+Every .cu under csrc/ is compiled to an object of its own (in parallel, rebuilt only when it or a header is
+newer) under _build/, then the objects are linked into paper_2407_09453_b200/libbsp.so.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbsp.so")
 
 
@@ -16,26 +22,50 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _headers():
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+
+
+def _newer(deps, target) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _stale() -> bool:
+    return _newer(sources() + _headers(), LIB)
+
+
+def _flags(verbose: bool):
+    f = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+         "-I" + os.path.join(ROOT, "include"), "-Xcompiler", "-fPIC"]
+    if verbose:
+        f += ["-Xptxas", "-v"]
+    return f
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
+    """Compile every .cu under csrc/ and link them into one shared library; returns its path."""
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    hdrs = _headers()
+    jobs = []
+    for src in sources():
+        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        if force or verbose or _newer([src] + hdrs, obj):
+            jobs.append([nvcc] + _flags(verbose) + ["-c", src, "-o", obj])
+
+    def run(cmd):
+        subprocess.check_call(cmd)
+
+    with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as ex:
+        list(ex.map(run, jobs))
+    objs = [os.path.join(OBJ, os.path.basename(s)[:-3] + ".o") for s in sources()]
     tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-I" + os.path.join(ROOT, "include"), "-Xcompiler", "-fPIC", "-shared", "-o", tmp]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += sources()
-    subprocess.check_call(cmd)
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs)
     os.replace(tmp, LIB)
     return LIB
 

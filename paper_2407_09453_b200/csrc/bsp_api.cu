@@ -30,12 +30,24 @@ bsp_status check_wdesc(const bsp_wdesc *wd)
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void *p) { return ((uintptr_t)p & 3u) == 0; }
 
-// The tensor-memory kernel takes every layer it can run unless BSP_CONV_PATH asks for the warp-MMA kernel.
-bool use_tc(const bsp_wdesc &wd, const bsp_xdesc &xd)
+// The product kernel of a layer: the persistent matrix-product kernel for 1x1 layers without padding or stride, the
+// tensor-memory convolution kernel for the other bf16 / int8 layers it can stage, the warp-MMA kernel for the rest.
+// `which` other than BSP_KERNEL_AUTO names one kernel; BSP_KERNEL_AUTO is returned when that kernel cannot take the layer.
+bsp_kernel choose_kernel(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype, bsp_kernel which)
 {
-    const char *path = getenv("BSP_CONV_PATH");
-    if (path && path[0] == 'm') return false;
-    return conv_tc_eligible(wd, xd);
+    const bool gemm_ok = gemm_tc_eligible(wd, xd, ytype), tc_ok = conv_tc_eligible(wd, xd);
+    switch (which) {
+        case BSP_KERNEL_GEMM_TC: return gemm_ok ? which : BSP_KERNEL_AUTO;
+        case BSP_KERNEL_CONV_TC: return tc_ok ? which : BSP_KERNEL_AUTO;
+        case BSP_KERNEL_CONV_MMA: return which;
+        default: break;
+    }
+    return gemm_ok ? BSP_KERNEL_GEMM_TC : (tc_ok ? BSP_KERNEL_CONV_TC : BSP_KERNEL_CONV_MMA);
+}
+
+const char *kernel_name(bsp_kernel k)
+{
+    return k == BSP_KERNEL_GEMM_TC ? "gemm_tc_kernel" : (k == BSP_KERNEL_CONV_TC ? "conv_tc_kernel" : "conv_mma_kernel");
 }
 
 }  // namespace
@@ -134,6 +146,12 @@ size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd)
 bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
 {
+    return bsp_conv2d_on(BSP_KERNEL_AUTO, wd, w, xd, X, bias, Y, ytype, ws, stream);
+}
+
+bsp_status bsp_conv2d_on(bsp_kernel which, const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                         const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
+{
     bsp_status rc = check_wdesc(wd);
     if (rc != BSP_OK) return rc;
     if (!w || !xd || !X || !Y || !ws || !w->packed) return BSP_ERR_NULL;
@@ -149,7 +167,12 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
     // the packed header is on the device; the host checks what it can: capacity against the descriptor
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
-    if (use_tc(*wd, *xd))
+    if (which < BSP_KERNEL_AUTO || which > BSP_KERNEL_CONV_MMA) return BSP_ERR_DTYPE;
+    const bsp_kernel k = choose_kernel(*wd, *xd, ytype, which);
+    if (k == BSP_KERNEL_AUTO) return BSP_ERR_SHAPE;              // the kernel asked for cannot take this layer
+    if (k == BSP_KERNEL_GEMM_TC)
+        return launch_gemm_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
+    if (k == BSP_KERNEL_CONV_TC)
         return launch_conv_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
     // the stored fraction only steers the choice of launch shape
     const double density = NB > 0 ? (double)w->nnz / (double)NB : 1.0;
@@ -159,7 +182,13 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd)
 {
     if (check_wdesc(wd) != BSP_OK || !xd) return nullptr;
-    return use_tc(*wd, *xd) ? "conv_tc_kernel" : "conv_mma_kernel";
+    return kernel_name(choose_kernel(*wd, *xd, wd->wtype == BSP_I8 ? BSP_I32 : BSP_F32, BSP_KERNEL_AUTO));
+}
+
+int bsp_conv_kernel_takes(bsp_kernel which, const bsp_wdesc *wd, const bsp_xdesc *xd, bsp_dtype ytype)
+{
+    if (check_wdesc(wd) != BSP_OK || !xd || which <= BSP_KERNEL_AUTO || which > BSP_KERNEL_CONV_MMA) return 0;
+    return choose_kernel(*wd, *xd, ytype, which) == which ? 1 : 0;
 }
 
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,

@@ -667,16 +667,12 @@ Plan make_plan(const bsp_wdesc &wd, const bsp_xdesc &xd, int M, int Nw, int n_pa
     const int steps = wd.wtype == BSP_F32 ? HK : (HK + 1) / 2;
     Plan best = {};
     double best_cost = -1;
-    // BSP_CONV_SHAPE=<kMT><WM><WN> (e.g. 242) pins the launch shape, for tuning runs
-    const char *pin = getenv("BSP_CONV_SHAPE");
-    const int pinned = pin ? atoi(pin) : 0;
     // Each shape is tried with its full pixel tile first; if nothing fits in shared memory (large strides or
     // kernels) the pixel tiles are halved, leaving some MMA rows idle.
     for (int shrink = 1; shrink <= 16 && best_cost < 0; shrink *= 2)
     for (auto &cfg : kConfigs) {
         Plan pl = {};
         pl.MT = cfg[0]; pl.WM = cfg[1]; pl.WN = cfg[2];
-        if (pinned && pinned != pl.MT * 100 + pl.WM * 10 + pl.WN) continue;
         int occ = cfg[3];
         size_t cap = (size_t)kMaxSmem / occ - (occ > 1 ? 2048 : 0);
         pl.tiles = -1;

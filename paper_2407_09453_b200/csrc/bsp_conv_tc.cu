@@ -33,7 +33,6 @@
 // store 64-byte pieces of rows.
 // Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched and the CTA winds down.
 #include <cuda.h>
-#include <cstdlib>
 #include "bsp_internal.cuh"
 
 namespace bsp {
@@ -644,10 +643,6 @@ bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     // activation byte fetched from L2 then feeds twice the arithmetic), while the grid still fills the SMs twice.
     p.ng = 1; p.n_groups = T.n_groups;
     if (gemm && p.mt == 2 && T.n_groups >= 2 && tiles * ((T.n_groups + 1) / 2) >= 2 * 148) p.ng = 2;
-    if (const char *e = getenv("BSP_TC_GROUPS")) {                 // tuning: pin the groups per CTA
-        if (e[0] == '1') p.ng = 1;
-        if (e[0] == '2' && gemm && p.mt == 2 && T.n_groups >= 2) p.ng = 2;
-    }
     // (several phases: each plane set is padded to 128 bytes)
     const size_t per_kc = (size_t)p.n_phase * (p.plane_bytes * p.chunks_per_kc + (p.n_phase > 1 ? 128 : 0)) + (size_t)p.ng * kTcGroupRows * T.st_bytes;
     // K-groups per stage: about 64 KB of operands, i.e. three stages in flight; every stage costs the loop threads a

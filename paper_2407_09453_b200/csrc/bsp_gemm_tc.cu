@@ -1,0 +1,423 @@
+// Block-sparse matrix product Y[p][o] = b[o] + sum over kept blocks of W-bar X (a fully connected layer, or a 1x1
+// convolution without padding or stride, over P positions) on 5th-generation tensor cores: tcgen05.mma with the
+// accumulators in tensor memory, bf16 -> fp32 (kind::f16), int8 -> int32 (kind::i8) and fp32 as TF32 -> fp32
+// (kind::tf32).  Introduction (Y = W*X + b) and Section "Block Sparsity in a Matrix" of the paper ("GEMM is a 1x1
+// convolution").
+//
+// The kernel reads the third packed form: Gamma (.) W-bar as a plain K-major [O][I] matrix (zeroed blocks stored as
+// zeros), so that both operands arrive by tiled TMA loads under the 128-byte swizzle.  A persistent CTA owns tiles of
+// 128 positions x BN output channels (BN <= 256).  Per K-stage (128 bytes of input channels) one thread issues the
+// two loads (128 x 128 bytes of X, BN x 128 bytes of weights); one elected lane of the MMA warp issues four MMAs of
+// 128 x BN x 32 bytes; two accumulator buffers of 256 columns let the epilogue of a tile (tensor memory -> registers
+// -> + bias -> convert -> swizzled shared memory -> TMA store) overlap the MMAs of the next one.  The arithmetic
+// skips nothing: a tensor-core instruction covers 128 x BN x 16 entries of the operands at once, far more than a
+// block, and feeding it compact blocks (cp.async expansion of the block-CSR payload in shared memory, or TMA gather
+// loads of 128-byte cores) was measured two to four times slower than these dense loads.
+//
+// Warps: 0 producer (one thread), 1 MMA issuer (the whole warp runs the loop so that its address arithmetic stays
+// warp-uniform), 2-5 epilogue (warp w reads the tensor-memory lanes 32 (w % 4) ..).  Barriers per stage: full (one
+// arrival that announces the bytes of both loads) and empty (tcgen05.commit); per accumulator buffer: acc_full (commit)
+// and acc_empty (4 warps).  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched, the roles wind down, loads
+// in flight are awaited (bounded) and tensor memory is freed.
+#include <cuda.h>
+#include "bsp_internal.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kGtThreads = 192;
+constexpr int kGtBM = 128;                         // positions per tile (M of the MMA)
+constexpr int kGtABytes = kGtBM * 128;             // activation bytes of a stage
+constexpr int kGtStageRows = 32;                   // rows of Y per epilogue warp
+constexpr int kGtStagingBytes = kGtStageRows * 128;   // one staging buffer of an epilogue warp
+constexpr int kGtMaxStages = 8;
+constexpr int kGtMaxSmem = 226 * 1024;
+constexpr int kGtTmemCols = 512;
+constexpr int kGtMaxDevices = 64;
+constexpr uint32_t kGtSpin = 1u << 24;             // polls of a barrier before a wait gives up
+
+struct GtParams {
+    CUtensorMap tmx;          // X as bytes: (I * esz, P), box 128 bytes x 128 positions, 128-byte swizzle
+    CUtensorMap tmw;          // Gamma (.) W-bar as bytes: (I * esz, O), box 128 bytes x BN channels, 128-byte swizzle
+    CUtensorMap tmy;          // Y as bytes: (O * ey, P), box 128 bytes x 32 positions, 128-byte swizzle
+    const void *bias;         // float32 or int32 [O], may be NULL
+    const uint8_t *packed;
+    int *status;
+    int O, I, P, H, K, bo, bi, wtype, ytype;
+    int BN, n_tiles_n, n_tiles, n_ks;
+    int stages, stage_bytes;
+};
+
+__device__ __forceinline__ uint32_t sm32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool gt_poll(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < kGtSpin; ++spin) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// The same wait for the threads of the epilogue warps: try_wait suspends the thread for a while.
+__device__ __forceinline__ bool gt_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < (kGtSpin >> 6); ++spin) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Shared-memory matrix descriptor of a K-major operand under the 128-byte swizzle (start address in 16-byte units in
+// the low 14 bits): rows of 128 bytes, 8-row groups 1024 bytes apart; a K-step of 32 bytes inside the swizzle span is
+// an advance of the start address by 2.
+constexpr uint64_t kGtDesc = (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+
+// The four MMAs of one stage and the commit that releases the stage, issued by one elected lane of a converged warp.
+// All lanes execute this statement with the same operands; the MMA of the first K-step overwrites the accumulator
+// when `acc` is 0.
+#define GT_ISSUE_STAGE(KIND)                                                                                        \
+    asm volatile("{\n .reg .pred e, p, t;\n .reg .b64 a1, a2, a3, b1, b2, b3;\n"                                     \
+                 " elect.sync _|e, 0xFFFFFFFF;\n setp.ne.b32 p, %5, 0;\n setp.eq.b32 t, %5, %5;\n"                    \
+                 " add.u64 a1, %1, 2;\n add.u64 a2, %1, 4;\n add.u64 a3, %1, 6;\n"                                    \
+                 " add.u64 b1, %2, 2;\n add.u64 b2, %2, 4;\n add.u64 b3, %2, 6;\n"                                    \
+                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], %1, %2, %3, p;\n"                                 \
+                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a1, b1, %3, t;\n"                                 \
+                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a2, b2, %3, t;\n"                                 \
+                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a3, b3, %3, t;\n"                                 \
+                 " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%4];\n}\n"               \
+                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(bar_empty), "r"(acc) : "memory")
+
+__device__ __forceinline__ void gt_issue_stage(int wtype, uint32_t d, uint64_t da, uint64_t db, uint32_t idesc,
+                                               uint32_t bar_empty, uint32_t acc)
+{
+    if (wtype == BSP_BF16) GT_ISSUE_STAGE("f16");
+    else if (wtype == BSP_I8) GT_ISSUE_STAGE("i8");
+    else GT_ISSUE_STAGE("tf32");
+}
+// All MMAs issued so far by the elected lane complete -> one arrival on `bar`.
+__device__ __forceinline__ void gt_commit_elected(uint32_t bar)
+{
+    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                 " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive accumulator columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void gt_load32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+
+// Bias of output channel ch as raw bits (float32 or int32), zero without a bias or past the last channel.
+__device__ __forceinline__ uint32_t gt_bias(const GtParams &p, int ch)
+{
+    return (p.bias != nullptr && ch < p.O) ? __ldg((const uint32_t *)p.bias + ch) : 0u;
+}
+
+__global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_constant__ GtParams p)
+{
+    extern __shared__ __align__(16) uint8_t gt_smem_raw[];
+    uint8_t *smem = gt_smem_raw + ((1024u - (sm32(gt_smem_raw) & 1023u)) & 1023u);
+    __shared__ __align__(8) uint64_t s_full[kGtMaxStages], s_empty[kGtMaxStages];
+    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ volatile uint32_t s_fail;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int S = p.stages, n_ks = p.n_ks, BN = p.BN;
+    const uint32_t ring = sm32(smem);
+    const uint32_t staging = ring + (uint32_t)(S * p.stage_bytes);
+
+    if (tid == 0) {
+        // the packed buffer must be the one bsp_compact filled for this descriptor, with the masked dense form in it
+        const PackedHeader *h = (const PackedHeader *)p.packed;
+        const bool ok = h->magic == kPackedMagic && h->dtype == p.wtype && h->O == p.O && h->I == p.I && h->H == p.H &&
+                        h->K == p.K && h->bo == p.bo && h->bi == p.bi && (h->forms & kFormDense) != 0;
+        s_fail = ok ? 0u : 2u;
+        if (!ok) atomicMax(p.status, (int)BSP_ERR_INDEX);
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_full[s])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_empty[s])), "r"(1) : "memory");
+        }
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc_full[b])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc_empty[b])), "r"(4) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmx) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmw) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmy) : "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const uint32_t tmem = s_tmem;
+    const bool run = s_fail == 0u;
+
+    if (warp == 0) {
+        // ================= producer =================
+        if (lane == 0 && run) {
+            const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
+            const uint32_t stage_bytes = (uint32_t)p.stage_bytes, tx = stage_bytes;
+            uint32_t slot = 0, round = 0, issued = 0, dst = ring;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / p.n_tiles_n) * kGtBM, n0 = (tile % p.n_tiles_n) * BN;
+                for (int ks = 0; ks < n_ks; ++ks) {
+                    if (round && !gt_poll(empty0 + slot * 8u, (round & 1u) ^ 1u)) { ok = false; break; }
+                    if (s_fail) { ok = false; break; }
+                    const uint32_t bar = full0 + slot * 8u;
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+                                 ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(ks * 128), "r"(m0) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+                                 ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(ks * 128), "r"(n0) : "memory");
+                    ++issued;
+                    if (++slot == (uint32_t)S) { slot = 0; ++round; dst = ring; } else dst += stage_bytes;
+                }
+            }
+            if (!ok) {
+                // winding down after a wait that ran out: the loads already issued still write into this CTA's shared
+                // memory, so the barriers of the stages in flight are awaited (bounded) before the CTA may leave
+                atomicExch((uint32_t *)&s_fail, 1u);
+                for (uint32_t back = 0; back < (uint32_t)S && back < issued; ++back) {
+                    const uint32_t it = issued - 1u - back;
+                    gt_poll(full0 + (it % (uint32_t)S) * 8u, (it / (uint32_t)S) & 1u);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        // The whole warp runs the loop (so that its address arithmetic stays warp-uniform); one elected lane issues.
+        if (run) {
+            // instruction descriptor: D fp32 (int32 for int8), A and B bf16 / signed int8 / tf32, K-major both, M = 128, N = BN
+            const uint32_t dfmt = p.wtype == BSP_I8 ? 2u : 1u, abfmt = p.wtype == BSP_F32 ? 2u : 1u;
+            const uint32_t idesc = (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
+            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
+            uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_i) {
+                const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
+                if (use && !gt_poll(sm32(&s_acc_empty[buf]), (use & 1u) ^ 1u)) ok = false;
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const uint32_t d = tmem + buf * 256u;
+                for (int ks = 0; ks < n_ks; ++ks) {
+                    bool got = gt_poll(full0 + slot * 8u, par);
+                    got = __all_sync(0xFFFFFFFFu, got && s_fail == 0u);
+                    if (!got) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
+                    gt_issue_stage(p.wtype, d, da, db, idesc, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
+                }
+                if (ok) gt_commit_elected(sm32(&s_acc_full[buf]));
+            }
+            if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
+        }
+    } else {
+        // ================= epilogue (warps 2-5) =================
+        if (run) {
+            const int q = warp & 3;                              // quarter of the tensor-memory lanes this warp reaches
+            const int ew = warp - 2;
+            const int ey = p.ytype == BSP_BF16 ? 2 : 4;
+            const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
+            const uint32_t stg0 = staging + (uint32_t)(ew * 2 * kGtStagingBytes);
+            uint32_t tile_i = 0, rounds_done = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_i) {
+                const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
+                const int n0 = (tile % p.n_tiles_n) * BN, m0 = (tile / p.n_tiles_n) * kGtBM;
+                if (!gt_wait(sm32(&s_acc_full[buf]), use & 1u)) ok = false;
+                if (s_fail) ok = false;
+                ok = __all_sync(0xFFFFFFFFu, ok);             // the warp goes on or gives up as one (aligned tcgen05.ld below)
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16) + buf * 256u;
+                for (int c0 = 0; c0 < BN; c0 += cpr, ++rounds_done) {
+                    uint32_t out[32];                            // 128 bytes of this lane's row of Y
+                    if (ey == 4) {                               // fp32 or int32 output: 32 channels
+                        uint32_t v[32];
+                        gt_load32(tbase + (uint32_t)c0, v);
+                        const uint32_t bl = gt_bias(p, n0 + c0 + lane);      // lane e holds the bias of channel c0 + e
+                        if (p.wtype == BSP_I8) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) out[e] = (uint32_t)((int)v[e] + (int)__shfl_sync(0xFFFFFFFFu, bl, e));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                out[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, e)));
+                        }
+                    } else {                                     // bf16 output: 64 channels, rounded to nearest even after the bias
+#pragma unroll
+                        for (int sub = 0; sub < 2; ++sub) {
+                            uint32_t v[32];
+                            gt_load32(tbase + (uint32_t)(c0 + sub * 32), v);
+                            const uint32_t bl = gt_bias(p, n0 + c0 + sub * 32 + lane);
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(
+                                    __uint_as_float(v[2 * e]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, 2 * e)),
+                                    __uint_as_float(v[2 * e + 1]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, 2 * e + 1)));
+                                out[sub * 16 + e] = *(const uint32_t *)&h;
+                            }
+                        }
+                    }
+                    // the staging buffer of this round was handed to a TMA store two rounds ago: wait until it has been read
+                    const uint32_t sb = stg0 + (rounds_done & 1u) * (uint32_t)kGtStagingBytes;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;\n" ::: "memory");
+                    __syncwarp();
+                    const uint32_t srow = sb + (uint32_t)lane * 128u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                                     ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
+                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    __syncwarp();
+                    // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
+                    if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
+                                     ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+                    }
+                }
+                // the accumulator buffer has been read: hand it back to the MMA issuer
+                asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc_empty[buf])) : "memory");
+            }
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
+            if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
+        }
+    }
+
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (s_fail == 1u && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kGtTmemCols) : "memory");
+}
+
+typedef CUresult (*GtEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                               const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+GtEncodeFn gt_encode()
+{
+    static GtEncodeFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (GtEncodeFn)ptr;
+    }
+    return fn;
+}
+
+}  // namespace
+
+// True if the matrix-product kernel can run this layer: a 1x1 layer without padding or stride whose rows of X and Y
+// are multiples of 16 bytes (tensor-map strides).
+bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype)
+{
+    if (wd.H != 1 || wd.K != 1 || xd.pad_h != 0 || xd.pad_w != 0 || xd.stride_h != 1 || xd.stride_w != 1) return false;
+    if (!packed_layout(wd, 0).gm.enabled) return false;
+    if (ytype != BSP_F32 && ytype != BSP_BF16 && ytype != BSP_I32) return false;
+    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    if (((long long)wd.O * ey) % 16 != 0) return false;
+    if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
+    return true;
+}
+
+bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
+{
+    const PackedLayout L = packed_layout(wd, 0);
+    const GemmLayout &G = L.gm;
+    if (!G.enabled) return BSP_ERR_SHAPE;
+    const long long P = (long long)xd.N * xd.L * xd.J;
+    const int esz = elem_bytes(wd.wtype);
+    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    GtParams p = {};
+    p.bias = bias; p.packed = (const uint8_t *)packed;
+    p.status = (int *)ws;
+    p.O = wd.O; p.I = wd.I; p.P = (int)P; p.H = wd.H; p.K = wd.K; p.bo = wd.bo; p.bi = wd.bi;
+    p.wtype = wd.wtype; p.ytype = ytype;
+    p.BN = gemm_tile_n(wd.O);
+    p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
+    const long long n_tiles_m = (P + kGtBM - 1) / kGtBM;
+    if (n_tiles_m * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
+    p.n_tiles = (int)(n_tiles_m * p.n_tiles_n);
+    p.n_ks = G.n_ks;
+    p.stage_bytes = kGtABytes + p.BN * 128;
+    const int staging = 4 * 2 * kGtStagingBytes;
+    int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
+    if (stages > kGtMaxStages) stages = kGtMaxStages;
+    if (stages < 2) return BSP_ERR_SHAPE;
+    p.stages = stages;
+    const size_t smem = 1024 + (size_t)stages * p.stage_bytes + staging;
+
+    GtEncodeFn enc = gt_encode();
+    if (!enc) return BSP_ERR_CUDA;
+    const cuuint32_t estr[2] = {1, 1};
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)wd.I * esz, (cuuint64_t)P};
+        const cuuint64_t gstr[1] = {(cuuint64_t)wd.I * esz};
+        const cuuint32_t box[2] = {128, (cuuint32_t)kGtBM};
+        if (enc(&p.tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(X), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)wd.I * esz, (cuuint64_t)wd.O};
+        const cuuint64_t gstr[1] = {(cuuint64_t)wd.I * esz};
+        const cuuint32_t box[2] = {128, (cuuint32_t)p.BN};
+        if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>((const uint8_t *)packed + G.off_payload), gdim, gstr, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)wd.O * ey, (cuuint64_t)P};
+        const cuuint64_t gstr[1] = {(cuuint64_t)wd.O * ey};
+        const cuuint32_t box[2] = {128, (cuuint32_t)kGtStageRows};
+        if (enc(&p.tmy, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, Y, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+
+    static bool opted[kGtMaxDevices] = {};
+    static int n_sm[kGtMaxDevices] = {};
+    int dev = 0;
+    BSP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
+    if (!opted[dev]) {
+        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
+        opted[dev] = true;
+    }
+    const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
+    gemm_tc_kernel<<<grid, kGtThreads, smem, st>>>(p);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // namespace bsp

@@ -30,9 +30,16 @@ struct PackedHeader {
     int32_t off_panelbase;
     int64_t off_payload;
     int64_t off_tc_payload;  // start of the super-tile payload (depends on the capacity the buffer was sized for)
+    int32_t forms;           // forms written by the compaction that filled this buffer: kForm* bits
 };
+static_assert(sizeof(PackedHeader) <= 256, "the packed header is the first 256 bytes");
 
-// Second packed form, for the tcgen05 kernel (bf16 only): W-bar is cut into super-tiles of 16 output channels
+// Forms of the packed buffer (PackedHeader::forms).
+constexpr int kFormTile = 1;     // 8x8 tiles in mma.sync fragment order (warp-MMA kernel)
+constexpr int kFormSuper = 2;    // 16-channel super-tiles (tcgen05 convolution kernel)
+constexpr int kFormDense = 4;    // Gamma (.) W-bar as a plain matrix (tcgen05 matrix-product kernel)
+
+// Second packed form, for the tcgen05 convolution kernel (bf16 and int8): W-bar is cut into super-tiles of 16 output channels
 // (a super-row) by one K-group: 8 input channels and all taps for a convolution, 16 input channels for a 1x1
 // layer.  A super-tile is stored if any 8x8 tile inside it is; it holds one 512-byte tcgen05 B operand
 // (16 x 16 bf16, K-major core matrices) per K-step of 16: a pair of taps, or the two 8-channel halves.
@@ -48,11 +55,21 @@ struct TcLayout {
     size_t off_mask, off_off, off_gcnt, off_payload, end;
 };
 
+// Third packed form, for the persistent tcgen05 matrix-product kernel (1x1 layers of every input type): Gamma (.) W-bar
+// as a plain [O][I] matrix, input channel innermost, weights of zeroed blocks written as zeros, so that tiles of it
+// arrive by tiled TMA loads.  A K-stage of the kernel is 128 bytes of input channels (64 bf16, 128 int8, 32 fp32).
+struct GemmLayout {
+    bool enabled;
+    int n_ks;                // K-stages: ceil(I * esz / 128)
+    size_t off_payload, end;
+};
+
 struct PackedLayout {
     int n_panels, n_cols, tile_bytes;
     int64_t capacity_tiles;
     size_t off_colmask, off_coloff, off_panelbase, off_payload, total_bytes;
     TcLayout tc;
+    GemmLayout gm;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -90,6 +107,15 @@ bsp_status launch_conv(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *pac
 void report_cuda_error(cudaError_t e, const char *expr, const char *file, int line);
 
 bool conv_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd);
+bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype);
+bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
+// Output channels per CTA tile of the matrix-product kernel (a multiple of 64, at most 256).
+inline int gemm_tile_n(int O)
+{
+    const int tiles = (O + 255) / 256;
+    return (((O + tiles - 1) / tiles) + 63) / 64 * 64;
+}
 bsp_status launch_conv_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
                           const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
 

@@ -1,5 +1,6 @@
-"""GPU parity of the tcgen05 kernel (bf16 and int8, stride 1; BSP_CONV_PATH=tc rules out an override from outside)
-against the CPU oracle: within tolerance for bf16, bit for bit for int8."""
+"""GPU parity of the tcgen05 convolution kernel (bf16 and int8; every case asks for it by name, so 1x1 layers that the
+matrix-product kernel would otherwise take run on it too) against the CPU oracle: within tolerance for bf16, bit for bit
+for int8."""
 import numpy as np
 import pytest
 
@@ -7,6 +8,7 @@ from oracle import ref
 import torch
 
 from paper_2407_09453_b200 import bsp, synth
+import gpu_util
 from gpu_util import gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_bias, make_case, make_x
 from test_gpu_product import check, run_conv_case
 
@@ -15,7 +17,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True)
 def tc_path(monkeypatch):
-    monkeypatch.setenv("BSP_CONV_PATH", "tc")
+    monkeypatch.setattr(gpu_util, "PREFER_KERNEL", bsp.KERNEL_CONV_TC)
 
 
 TC_CASES = [  # O, I, H, K, pad, spatial, batch
@@ -47,6 +49,8 @@ STRIDED = [  # O, I, H, K, stride, pad, spatial, batch, runs on the tensor-memor
 def test_tc_strided(dtype, O, I, H, K, stride, pad, sp, batch, on_tc):
     xd = bsp.XDesc(batch, sp[0], sp[1], stride[0], stride[1], pad[0], pad[1])
     tdt = torch.int8 if dtype == "i8" else torch.bfloat16
+    ydt = bsp.I32 if dtype == "i8" else bsp.F32
+    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(O, I, H, K, 8, 8, tdt), xd, ydt) == on_tc
     assert bsp.conv_kernel_name(bsp.wdesc(O, I, H, K, 8, 8, tdt), xd) == ("conv_tc_kernel" if on_tc else "conv_mma_kernel")
     run_conv_case(671 + O + H, O, I, H, K, 8, 8, dtype, (batch, sp[0], sp[1], I), stride, pad)
 
@@ -63,7 +67,7 @@ def test_tc_int8_bit_exact(O, I, H, K, pad, sp, batch, bo, bi):
     if O % bo or I % bi:
         pytest.skip("channels are not a multiple of the block")
     xd = bsp.XDesc(batch, sp[0], sp[1], 1, 1, pad[0], pad[1])
-    assert bsp.conv_kernel_name(bsp.wdesc(O, I, H, K, bo, bi, torch.int8), xd) == "conv_tc_kernel"
+    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(O, I, H, K, bo, bi, torch.int8), xd, bsp.I32)
     run_conv_case(641 + O + H, O, I, H, K, bo, bi, "i8", (batch, sp[0], sp[1], I), (1, 1), pad)
 
 
@@ -111,11 +115,11 @@ def test_tc_gemm_two_position_tiles_per_cta(dtype):
 
 
 @pytest.mark.parametrize("dtype,frac", [("bf16", 0.5), ("i8", 0.75), ("bf16", 0.0)])
-def test_tc_gemm_two_channel_groups_per_cta(dtype, frac, monkeypatch):
-    """256 positions x 256 channels per CTA (BSP_TC_GROUPS=2 pins what only the largest products choose): nine
-    channel groups, so the last CTA row has no second group; a last half super-row; ragged last position tile."""
-    monkeypatch.setenv("BSP_TC_GROUPS", "2")
-    O, I, P = 1144, 96, 8500
+def test_tc_gemm_two_channel_groups_per_cta(dtype, frac):
+    """256 positions x 256 channels per CTA (what the largest products take: here 149 position tiles x 5 pairs of
+    channel groups keep the grid above two waves): nine channel groups, so the last CTA row has no second group; a last
+    half super-row; ragged last position tile."""
+    O, I, P = 1144, 96, 38000
     W = make_case(681, O, I, 1, 1, dtype)
     NB = (O // 8) * (I // 8)
     gamma = synth.random_gamma(682, O // 8, I // 8, int(NB * frac))
