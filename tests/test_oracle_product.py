@@ -214,3 +214,49 @@ def test_int8_overflow_is_reported():
     b = np.full(8, 2**31 - 1, dtype=np.int32)
     with pytest.raises(RuntimeError):
         ref.gemm(8, 8, bo, bi, rp, ci, pl.reshape(-1, 8, 8), X, b)
+
+
+def test_gemm_f32_sampled_rows_against_numpy():
+    """The sampled-rows branch of the float product (the one the large GPU cases lean on): listed rows, in the listed
+    order and with repeats, equal the same rows of the full result bit for bit, and numpy's matmul of Gamma (.) W on
+    those rows of X to rounding."""
+    O, I, P, bo, bi = 64, 96, 41, 16, 4
+    W, gamma, (rp, ci, pl) = sparse_setup(301, O, I, 1, 1, bo, bi, "f32")
+    X = synth.normal(303, (P, I)).astype(np.float32)
+    b = synth.normal(304, (O,), 0.1).astype(np.float32)
+    pix = np.array([40, 0, 13, 13, 7, 39])
+    full = ref.gemm(O, I, bo, bi, rp, ci, pl, X, b)
+    sub = ref.gemm(O, I, bo, bi, rp, ci, pl, X, b, pix=pix)
+    assert sub.shape == (len(pix), O) and np.array_equal(sub, full[pix])
+    Wm = ref.apply_mask(W, gamma, bo, bi)[:, 0, 0, :].astype(np.float64)
+    assert np.allclose(sub, X[pix].astype(np.float64) @ Wm.T + b, rtol=1e-12, atol=1e-12)
+    # a subset taken from the wrong rows (an off-by-one in the position list) must not pass
+    assert not np.allclose(sub, X[(pix + 1) % P].astype(np.float64) @ Wm.T + b, atol=1e-3)
+
+
+@pytest.mark.parametrize("stride,pad", [((1, 1), (1, 1)), ((2, 2), (1, 1)), ((1, 2), (0, 1))])
+def test_conv_int8_sampled_positions_against_brute_force(stride, pad):
+    """The sampled-positions branch of the int8 convolution: positions across images, on the border (padding) and
+    inside, against the pure-Python brute force of the same positions and against the full result."""
+    O, I, H, K, bo, bi = 16, 32, 3, 3, 8, 8
+    W, gamma, (rp, ci, pl) = sparse_setup(311, O, I, H, K, bo, bi, "i8")
+    X = synth.uniform_int(313, (2, 6, 7, I), -127, 127).astype(np.int8)
+    b = synth.uniform_int(314, (O,), -(1 << 15), 1 << 15).astype(np.int32)
+    M, Nw = ref.out_hw(6, 7, H, K, stride[0], stride[1], pad[0], pad[1])
+    P = 2 * M * Nw
+    pix = np.array([P - 1, 0, Nw - 1, Nw, M * Nw, M * Nw + Nw + 1, 5, 5])
+    want = brute_conv(ref.apply_mask(W, gamma, bo, bi), X, b, stride, pad)
+    sub = ref.conv2d(W.shape, bo, bi, rp, ci, pl, X, b, stride, pad, pix=pix)
+    assert sub.dtype == np.int32 and np.array_equal(sub, want[pix])
+    assert np.array_equal(sub, ref.conv2d(W.shape, bo, bi, rp, ci, pl, X, b, stride, pad)[pix])
+
+
+def test_conv_f32_sampled_positions_against_scipy():
+    O, I, H, K, bo, bi = 16, 16, 3, 3, 4, 16
+    W, gamma, (rp, ci, pl) = sparse_setup(321, O, I, H, K, bo, bi, "f32")
+    X = synth.normal(323, (2, 5, 6, I)).astype(np.float32)
+    b = synth.normal(324, (O,), 0.1).astype(np.float32)
+    want = scipy_dense_conv(ref.apply_mask(W, gamma, bo, bi), X, b, (1, 1), (1, 1))
+    pix = np.array([59, 0, 5, 6, 30, 31])
+    sub = ref.conv2d(W.shape, bo, bi, rp, ci, pl, X, b, (1, 1), (1, 1), pix=pix)
+    assert np.allclose(sub, want[pix], rtol=1e-12, atol=1e-12)
