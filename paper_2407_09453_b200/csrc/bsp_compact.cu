@@ -46,16 +46,16 @@ PackedLayout packed_layout(const bsp_wdesc &wd, int64_t nnz_blocks)
         T.off_gcnt = align_up(T.off_off + (size_t)T.n_groups * T.n_kc * 4, 256);
         meta_end = align_up(T.off_gcnt + (size_t)(T.n_groups + 1) * 4, 256);
     }
-    // third form (1x1 layers whose rows are multiples of 16 bytes): the masked dense matrix; it comes first among the
-    // payloads, so that its offset does not depend on the capacity
+    // third form (layers whose rows of input channels are multiples of 16 bytes): Gamma (.) W as it is laid out,
+    // [O][H][K][I]; it comes first among the payloads, so that its offset does not depend on the capacity
     GemmLayout &G = L.gm;
     G = GemmLayout{};
     const int esz = elem_bytes(wd.wtype);
-    G.enabled = HK == 1 && ((long long)wd.I * esz) % 16 == 0 && wd.O % 8 == 0;
+    G.enabled = ((long long)wd.I * esz) % 16 == 0 && wd.O % 8 == 0;
     if (G.enabled) {
-        G.n_ks = (int)(((long long)wd.I * esz + 127) / 128);
+        G.n_ks = HK * (int)(((long long)wd.I * esz + 127) / 128);
         G.off_payload = meta_end;
-        G.end = align_up(G.off_payload + (size_t)wd.O * wd.I * esz + 256, 256);
+        G.end = align_up(G.off_payload + (size_t)wd.O * HK * wd.I * esz + 256, 256);
         meta_end = G.end;
     }
     L.off_payload = meta_end;
@@ -828,33 +828,34 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const FillPackA
     }
 }
 
-// Third packed form: Gamma (.) W-bar as a plain matrix, one 16-byte chunk of a weight row per thread and step (four
-// loads in flight per thread), the channels of zeroed blocks cleared.
+// Third packed form: Gamma (.) W in the layout of W, [O][H][K][I], one 16-byte chunk of input channels per thread and
+// step (four loads in flight per thread), the channels of zeroed blocks cleared.  A "row" below is one (o, tap).
 template <int esz>
 __global__ void __launch_bounds__(kThreads)
-masked_dense_kernel(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I, int bo, int bi, int NBi,
-                    uint8_t *__restrict__ out)
+masked_dense_kernel(const void *__restrict__ W, const uint8_t *__restrict__ gamma, int O, int I, int HK, int bo, int bi,
+                    int NBi, uint8_t *__restrict__ out)
 {
     const bool aligned = (((uintptr_t)W) & 15u) == 0;
     const int cpr = I * esz / 16;                     // chunks per row
     constexpr int cpc = 16 / esz;
-    const long long total = (long long)O * cpr, stride = (long long)gridDim.x * kThreads;
+    const long long total = (long long)O * HK * cpr, stride = (long long)gridDim.x * kThreads;
     for (long long e0 = (long long)blockIdx.x * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const long long e = e0 + u * stride;
             if (e >= total) continue;
-            const int o = (int)(e / cpr), c = (int)(e - (long long)o * cpr);
+            const int ot = (int)(e / cpr), c = (int)(e - (long long)ot * cpr);
+            const int o = ot / HK, tap = ot - o * HK;
             if (aligned) {
-                v[u] = w_chunk<esz>(W, gamma, o, 0, c * cpc, O, I, 1, bo, bi, NBi);
+                v[u] = w_chunk<esz>(W, gamma, o, tap, c * cpc, O, I, HK, bo, bi, NBi);
             } else {
                 // W only 4-byte aligned: word by word (the channels of a word lie in one block: b_i is a multiple of 4)
                 uint32_t w[4];
                 for (int q = 0; q < 4; ++q) {
                     const int ch = c * cpc + q * (4 / esz);
                     const bool on = gamma[(size_t)(o >> lg(bo)) * NBi + (ch >> lg(bi))] != 0;
-                    w[q] = on ? *(const uint32_t *)((const uint8_t *)W + ((size_t)o * I + ch) * esz) : 0u;
+                    w[q] = on ? *(const uint32_t *)((const uint8_t *)W + ((size_t)ot * I + ch) * esz) : 0u;
                 }
                 v[u] = make_uint4(w[0], w[1], w[2], w[3]);
             }
@@ -914,14 +915,14 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     h.forms = pk ? (kFormTile | (L.tc.enabled ? kFormSuper : 0) | (gm_on ? kFormDense : 0)) : 0;
     auto pack_dense = [&]() -> bsp_status {
         if (!gm_on) return BSP_OK;
-        const long long chunks = (long long)wd.O * wd.I * elem_bytes(wd.wtype) / 16;
+        const long long chunks = (long long)wd.O * HK * wd.I * elem_bytes(wd.wtype) / 16;
         long long g = (chunks + 4LL * kThreads - 1) / (4LL * kThreads);
         if (g > 2368) g = 2368;
         if (g < 1) g = 1;
         uint8_t *out = pk + L.gm.off_payload;
-        if (wd.wtype == BSP_I8) masked_dense_kernel<1><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, wd.bo, wd.bi, NBi, out);
-        else if (wd.wtype == BSP_BF16) masked_dense_kernel<2><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, wd.bo, wd.bi, NBi, out);
-        else masked_dense_kernel<4><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, wd.bo, wd.bi, NBi, out);
+        if (wd.wtype == BSP_I8) masked_dense_kernel<1><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, out);
+        else if (wd.wtype == BSP_BF16) masked_dense_kernel<2><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, out);
+        else masked_dense_kernel<4><<<(unsigned)g, kThreads, 0, st>>>(W, gamma, wd.O, wd.I, HK, wd.bo, wd.bi, NBi, out);
         BSP_CUDA_OK(cudaGetLastError());
         return BSP_OK;
     };

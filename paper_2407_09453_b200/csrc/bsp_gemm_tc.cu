@@ -37,15 +37,22 @@ constexpr int kGtMaxDevices = 64;
 constexpr uint32_t kGtSpin = 1u << 24;             // polls of a barrier before a wait gives up
 
 struct GtParams {
-    CUtensorMap tmx;          // X as bytes: (I * esz, P), box 128 bytes x 128 positions, 128-byte swizzle
-    CUtensorMap tmw;          // Gamma (.) W-bar as bytes: (I * esz, O), box 128 bytes x BN channels, 128-byte swizzle
-    CUtensorMap tmy;          // Y as bytes: (O * ey, P), box 128 bytes x 32 positions, 128-byte swizzle
+    CUtensorMap tmx;          // X as bytes: (I * esz, J, L, N), box 128 bytes x Wt x Ht x Nt positions (in steps of the strides), 128-byte swizzle
+    CUtensorMap tmw;          // Gamma (.) W as bytes: (I * esz, H K, O), box 128 bytes x 1 tap x BN channels, 128-byte swizzle
+    CUtensorMap tmy;          // Y as bytes: (O * ey, P), box 128 bytes x 32 positions, 128-byte swizzle (store_tma only)
     const void *bias;         // float32 or int32 [O], may be NULL
     const uint8_t *packed;
     int *status;
     int O, I, P, H, K, bo, bi, wtype, ytype;
     int BN, n_tiles_n, n_tiles, n_ks;
     int stages, stage_bytes;
+    // position tiles: Wt x Ht output positions of Nt images (at most 128), tiles_x x tiles_y of them per Nt images
+    int N, M, Nw, Wt, Ht, Nt, tiles_x, tiles_y, rows_tile;
+    int sh, sw, ph, pw, cpt;          // strides, padding, 128-byte channel chunks per tap
+    int a_bytes;                      // bytes of one activation box
+    int store_tma;                    // a tile is 128 consecutive rows of Y: the epilogue stores by TMA
+    uint8_t *Y;
+    int ey;
 };
 
 __device__ __forceinline__ uint32_t sm32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -104,6 +111,13 @@ __device__ __forceinline__ void gt_commit_elected(uint32_t bar)
 {
     asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
                  " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
+}
+
+// First output position (image, row, column) of position tile mt.
+__device__ __forceinline__ void gt_tile_origin(const GtParams &p, int mt, int &n0, int &y0, int &x0)
+{
+    const int tx = mt % p.tiles_x, r = mt / p.tiles_x;
+    x0 = tx * p.Wt; y0 = (r % p.tiles_y) * p.Ht; n0 = (r / p.tiles_y) * p.Nt;
 }
 
 // 32 consecutive accumulator columns of this thread's tensor-memory lane.
@@ -173,22 +187,30 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
         // ================= producer =================
         if (lane == 0 && run) {
             const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
-            const uint32_t stage_bytes = (uint32_t)p.stage_bytes, tx = stage_bytes;
+            const uint32_t stage_bytes = (uint32_t)p.stage_bytes, tx = (uint32_t)(p.a_bytes + BN * 128);
             uint32_t slot = 0, round = 0, issued = 0, dst = ring;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / p.n_tiles_n) * kGtBM, n0 = (tile % p.n_tiles_n) * BN;
-                for (int ks = 0; ks < n_ks; ++ks) {
-                    if (round && !gt_poll(empty0 + slot * 8u, (round & 1u) ^ 1u)) { ok = false; break; }
-                    if (s_fail) { ok = false; break; }
-                    const uint32_t bar = full0 + slot * 8u;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
-                                 ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(ks * 128), "r"(m0) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
-                                 ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(ks * 128), "r"(n0) : "memory");
-                    ++issued;
-                    if (++slot == (uint32_t)S) { slot = 0; ++round; dst = ring; } else dst += stage_bytes;
+                const int ch0 = (tile % p.n_tiles_n) * BN;
+                int n0, y0, x0;
+                gt_tile_origin(p, tile / p.n_tiles_n, n0, y0, x0);
+                // input position of the tile's first output position at tap (0, 0); a tap is a shift of the box, positions
+                // outside the image read as zeros (the padding)
+                const int xi0 = x0 * p.sw - p.pw, yi0 = y0 * p.sh - p.ph;
+                for (int tap = 0, h = 0, k = 0; tap < p.H * p.K && ok; ++tap) {
+                    for (int c = 0; c < p.cpt; ++c) {
+                        if (round && !gt_poll(empty0 + slot * 8u, (round & 1u) ^ 1u)) { ok = false; break; }
+                        if (s_fail) { ok = false; break; }
+                        const uint32_t bar = full0 + slot * 8u;
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
+                        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+                                     ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(c * 128), "r"(xi0 + k), "r"(yi0 + h), "r"(n0) : "memory");
+                        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
+                                     ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(c * 128), "r"(tap), "r"(ch0) : "memory");
+                        ++issued;
+                        if (++slot == (uint32_t)S) { slot = 0; ++round; dst = ring; } else dst += stage_bytes;
+                    }
+                    if (++k == p.K) { k = 0; ++h; }
                 }
             }
             if (!ok) {
@@ -237,14 +259,23 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
         if (run) {
             const int q = warp & 3;                              // quarter of the tensor-memory lanes this warp reaches
             const int ew = warp - 2;
-            const int ey = p.ytype == BSP_BF16 ? 2 : 4;
+            const int ey = p.ey;
             const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
             const uint32_t stg0 = staging + (uint32_t)(ew * 2 * kGtStagingBytes);
             uint32_t tile_i = 0, rounds_done = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_i) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
-                const int n0 = (tile % p.n_tiles_n) * BN, m0 = (tile / p.n_tiles_n) * kGtBM;
+                const int n0 = (tile % p.n_tiles_n) * BN;
+                // this lane's row of the tile: position (w, h, image i) of the tile's box, w fastest
+                int in0, y0, x0;
+                gt_tile_origin(p, tile / p.n_tiles_n, in0, y0, x0);
+                const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
+                const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
+                // byte offset of the row in Y (rows of O * ey bytes); m0: the tile's first row when rows are consecutive
+                const long long pos = ((long long)(in0 + ri) * p.M + (y0 + rh)) * p.Nw + (x0 + rw);
+                const unsigned long long row_off = (unsigned long long)pos * (unsigned long long)(p.O * ey);
+                const int m0 = (int)(((long long)in0 * p.M + y0) * p.Nw + x0);
                 if (!gt_wait(sm32(&s_acc_full[buf]), use & 1u)) ok = false;
                 if (s_fail) ok = false;
                 ok = __all_sync(0xFFFFFFFFu, ok);             // the warp goes on or gives up as one (aligned tcgen05.ld below)
@@ -282,20 +313,40 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                     }
                     // the staging buffer of this round was handed to a TMA store two rounds ago: wait until it has been read
                     const uint32_t sb = stg0 + (rounds_done & 1u) * (uint32_t)kGtStagingBytes;
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;\n" ::: "memory");
+                    if (lane == 0 && p.store_tma) asm volatile("cp.async.bulk.wait_group.read 1;\n" ::: "memory");
                     __syncwarp();
                     const uint32_t srow = sb + (uint32_t)lane * 128u;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
                                      ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
-                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-                    __syncwarp();
-                    // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
-                    if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
-                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
-                                     ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+                    if (p.store_tma) {
+                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                        __syncwarp();
+                        // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
+                        if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
+                                         ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
+                            asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+                        }
+                    } else {
+                        // rows of the tile are scattered over Y (a box of positions): the warp reads the staged rows back
+                        // four at a time, eight lanes per row, and writes whole 128-byte pieces of rows
+                        __syncwarp();
+                        const int chunk = lane & 7;
+                        const bool ch_ok = (n0 + c0) * ey + chunk * 16 < p.O * ey;
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const int row = it * 4 + (lane >> 3);
+                            const unsigned long long off = __shfl_sync(0xFFFFFFFFu, row_off, row);
+                            const int okr = __shfl_sync(0xFFFFFFFFu, (int)row_ok, row);
+                            uint32_t a0, a1, a2, a3;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];\n"
+                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(sb + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4)) : "memory");
+                            if (okr && ch_ok)
+                                *(uint4 *)(p.Y + off + (unsigned long long)((n0 + c0) * ey + chunk * 16)) = make_uint4(a0, a1, a2, a3);
+                        }
+                        __syncwarp();
                     }
                 }
                 // the accumulator buffer has been read: hand it back to the MMA issuer
@@ -334,17 +385,43 @@ GtEncodeFn gt_encode()
 
 }  // namespace
 
-// True if the matrix-product kernel can run this layer: a 1x1 layer without padding or stride whose rows of X and Y
-// are multiples of 16 bytes (tensor-map strides).
+namespace {
+// Position tile of a layer: Wt x Ht output positions of Nt images, at most 128, chosen for the fewest tiles (ties: the
+// smaller box).  Several images share a tile only when a tile holds whole images.  A box of the tensor map spans
+// Wt * s_w x Ht * s_h input positions and may not exceed 256 in any extent.
+struct GtTile { int Wt, Ht, Nt; long long tiles; };
+
+GtTile gt_pick_tile(int N, int M, int Nw, int sh, int sw)
+{
+    GtTile best = {0, 0, 0, -1};
+    for (int w = 1; w <= Nw && w <= kGtBM; ++w) {
+        if (w * sw > 256) break;
+        for (int h = 1; h <= M && h * w <= kGtBM; ++h) {
+            if (h * sh > 256) break;
+            int b = 1;
+            if (w == Nw && h == M) { b = kGtBM / (w * h); if (b > N) b = N; if (b > 256) b = 256; if (b < 1) b = 1; }
+            const long long cnt = (long long)((N + b - 1) / b) * ((M + h - 1) / h) * ((Nw + w - 1) / w);
+            const long long area = (long long)b * h * w, best_area = (long long)best.Wt * best.Ht * best.Nt;
+            if (best.tiles < 0 || cnt < best.tiles || (cnt == best.tiles && area < best_area)) best = {w, h, b, cnt};
+        }
+    }
+    return best;
+}
+}  // namespace
+
+// True if the kernel can run this layer: rows of X, W and Y that are multiples of 16 bytes (tensor-map strides), a
+// position count that fits 32 bits, and a position tile whose box the tensor map can express.
 bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype)
 {
-    if (wd.H != 1 || wd.K != 1 || xd.pad_h != 0 || xd.pad_w != 0 || xd.stride_h != 1 || xd.stride_w != 1) return false;
     if (!packed_layout(wd, 0).gm.enabled) return false;
     if (ytype != BSP_F32 && ytype != BSP_BF16 && ytype != BSP_I32) return false;
     const int ey = ytype == BSP_BF16 ? 2 : 4;
     if (((long long)wd.O * ey) % 16 != 0) return false;
-    if ((long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
-    return true;
+    const int M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1, Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
+    if (M <= 0 || Nw <= 0) return false;
+    if ((long long)xd.N * M * Nw > 0x7FFFFFFF || (long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
+    if ((long long)xd.N * M * Nw * wd.O * ey >= (1LL << 46)) return false;
+    return gt_pick_tile(xd.N, M, Nw, xd.stride_h, xd.stride_w).tiles > 0;
 }
 
 bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
@@ -353,20 +430,32 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
     const PackedLayout L = packed_layout(wd, 0);
     const GemmLayout &G = L.gm;
     if (!G.enabled) return BSP_ERR_SHAPE;
-    const long long P = (long long)xd.N * xd.L * xd.J;
     const int esz = elem_bytes(wd.wtype);
     const int ey = ytype == BSP_BF16 ? 2 : 4;
+    const int HK = wd.H * wd.K;
     GtParams p = {};
     p.bias = bias; p.packed = (const uint8_t *)packed;
     p.status = (int *)ws;
-    p.O = wd.O; p.I = wd.I; p.P = (int)P; p.H = wd.H; p.K = wd.K; p.bo = wd.bo; p.bi = wd.bi;
-    p.wtype = wd.wtype; p.ytype = ytype;
+    p.O = wd.O; p.I = wd.I; p.H = wd.H; p.K = wd.K; p.bo = wd.bo; p.bi = wd.bi;
+    p.wtype = wd.wtype; p.ytype = ytype; p.ey = ey; p.Y = (uint8_t *)Y;
+    p.N = xd.N; p.sh = xd.stride_h; p.sw = xd.stride_w; p.ph = xd.pad_h; p.pw = xd.pad_w;
+    p.M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1;
+    p.Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
+    const long long P = (long long)xd.N * p.M * p.Nw;
+    p.P = (int)P;
+    const GtTile T = gt_pick_tile(xd.N, p.M, p.Nw, p.sh, p.sw);
+    if (T.tiles <= 0) return BSP_ERR_SHAPE;
+    p.Wt = T.Wt; p.Ht = T.Ht; p.Nt = T.Nt; p.rows_tile = T.Wt * T.Ht * T.Nt;
+    p.tiles_x = (p.Nw + T.Wt - 1) / T.Wt; p.tiles_y = (p.M + T.Ht - 1) / T.Ht;
+    p.a_bytes = p.rows_tile * 128;
+    // a tile of 128 rows that are consecutive in Y (whole images, or the positions of a matrix product) is stored by TMA
+    p.store_tma = (T.Wt == p.Nw && T.Ht == p.M && p.rows_tile == kGtBM) ? 1 : 0;
     p.BN = gemm_tile_n(wd.O);
     p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
-    const long long n_tiles_m = (P + kGtBM - 1) / kGtBM;
-    if (n_tiles_m * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
-    p.n_tiles = (int)(n_tiles_m * p.n_tiles_n);
-    p.n_ks = G.n_ks;
+    if (T.tiles * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
+    p.n_tiles = (int)(T.tiles * p.n_tiles_n);
+    p.cpt = (int)(((long long)wd.I * esz + 127) / 128);
+    p.n_ks = HK * p.cpt;
     p.stage_bytes = kGtABytes + p.BN * 128;
     const int staging = 4 * 2 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
@@ -377,20 +466,24 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
 
     GtEncodeFn enc = gt_encode();
     if (!enc) return BSP_ERR_CUDA;
-    const cuuint32_t estr[2] = {1, 1};
     {
-        const cuuint64_t gdim[2] = {(cuuint64_t)wd.I * esz, (cuuint64_t)P};
-        const cuuint64_t gstr[1] = {(cuuint64_t)wd.I * esz};
-        const cuuint32_t box[2] = {128, (cuuint32_t)kGtBM};
-        if (enc(&p.tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(X), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        const cuuint64_t row = (cuuint64_t)wd.I * esz;
+        const cuuint64_t gdim[4] = {row, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N};
+        const cuuint64_t gstr[3] = {row, row * xd.J, row * xd.J * xd.L};
+        // a box spans Wt * s_w x Ht * s_h input positions in steps of the strides: Wt x Ht positions arrive
+        const cuuint32_t box[4] = {128, (cuuint32_t)(T.Wt * p.sw), (cuuint32_t)(T.Ht * p.sh), (cuuint32_t)T.Nt};
+        const cuuint32_t estr[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
+        if (enc(&p.tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(X), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
     }
     {
-        const cuuint64_t gdim[2] = {(cuuint64_t)wd.I * esz, (cuuint64_t)wd.O};
-        const cuuint64_t gstr[1] = {(cuuint64_t)wd.I * esz};
-        const cuuint32_t box[2] = {128, (cuuint32_t)p.BN};
-        if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>((const uint8_t *)packed + G.off_payload), gdim, gstr, box, estr,
+        const cuuint64_t row = (cuuint64_t)wd.I * esz;
+        const cuuint64_t gdim[3] = {row, (cuuint64_t)HK, (cuuint64_t)wd.O};
+        const cuuint64_t gstr[2] = {row, row * HK};
+        const cuuint32_t box[3] = {128, 1, (cuuint32_t)p.BN};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed + G.off_payload), gdim, gstr, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
@@ -399,6 +492,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         const cuuint64_t gdim[2] = {(cuuint64_t)wd.O * ey, (cuuint64_t)P};
         const cuuint64_t gstr[1] = {(cuuint64_t)wd.O * ey};
         const cuuint32_t box[2] = {128, (cuuint32_t)kGtStageRows};
+        const cuuint32_t estr[2] = {1, 1};
         if (enc(&p.tmy, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, Y, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;

@@ -55,12 +55,12 @@ struct TcLayout {
     size_t off_mask, off_off, off_gcnt, off_payload, end;
 };
 
-// Third packed form, for the persistent tcgen05 matrix-product kernel (1x1 layers of every input type): Gamma (.) W-bar
-// as a plain [O][I] matrix, input channel innermost, weights of zeroed blocks written as zeros, so that tiles of it
-// arrive by tiled TMA loads.  A K-stage of the kernel is 128 bytes of input channels (64 bf16, 128 int8, 32 fp32).
+// Third packed form, for the persistent tcgen05 kernel (layers of every input type): Gamma (.) W in the layout of W,
+// [O][H][K][I], weights of zeroed blocks written as zeros, so that tiles of it arrive by tiled TMA loads.  A K-stage
+// of the kernel is 128 bytes of the input channels of one tap (64 bf16, 128 int8, 32 fp32).
 struct GemmLayout {
     bool enabled;
-    int n_ks;                // K-stages: ceil(I * esz / 128)
+    int n_ks;                // K-stages: H K ceil(I * esz / 128)
     size_t off_payload, end;
 };
 

@@ -67,28 +67,25 @@ def test_host_validation_without_gpu(lib):
 
 
 def test_product_kernel_choice():
-    """1x1 layers without padding or stride take the matrix-product kernel, whatever their type; other bf16 and int8
-    layers the tensor-memory convolution kernel, strided ones included; the rest the warp-MMA kernel (a host-side
-    decision: no GPU needed)."""
+    """Every layer whose rows of input channels are multiples of 16 bytes takes the persistent tensor-memory kernel,
+    whatever its type, taps and strides; the other kernels are reached by name (a host-side decision: no GPU needed)."""
     import torch
     s1 = bsp.XDesc(2, 14, 14, 1, 1, 1, 1)
     s2 = bsp.XDesc(2, 14, 14, 2, 2, 1, 1)
-    for dt, want in ((torch.bfloat16, "conv_tc_kernel"), (torch.int8, "conv_tc_kernel"), (torch.float32, "conv_mma_kernel")):
-        wd = bsp.wdesc(64, 64, 3, 3, 8, 8, dt)
-        assert bsp.conv_kernel_name(wd, s1) == want
-        assert bsp.conv_kernel_name(wd, s2) == want
-    # a stride of 3 over a 5x5 kernel would need nine phase images: more than the kernel stages
-    assert bsp.conv_kernel_name(bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16), bsp.XDesc(2, 20, 20, 3, 3, 2, 2)) == "conv_mma_kernel"
-    flat = bsp.XDesc(2, 7, 7, 1, 1, 0, 0)
     for dt in (torch.bfloat16, torch.int8, torch.float32):
-        assert bsp.conv_kernel_name(bsp.wdesc(64, 48, 1, 1, 8, 8, dt), flat) == "gemm_tc_kernel"
-    # a strided or padded 1x1 layer is not a plain matrix product
-    assert bsp.conv_kernel_name(bsp.wdesc(64, 64, 1, 1, 8, 8, torch.bfloat16), bsp.XDesc(2, 14, 14, 2, 2, 0, 0)) == "conv_tc_kernel"
+        wd = bsp.wdesc(64, 64, 3, 3, 8, 8, dt)
+        assert bsp.conv_kernel_name(wd, s1) == "gemm_tc_kernel"
+        assert bsp.conv_kernel_name(wd, s2) == "gemm_tc_kernel"
+        assert bsp.conv_kernel_name(bsp.wdesc(64, 48, 1, 1, 8, 8, dt), bsp.XDesc(2, 7, 7, 1, 1, 0, 0)) == "gemm_tc_kernel"
     wd = bsp.wdesc(64, 64, 3, 3, 8, 8, torch.bfloat16)
     assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_MMA, wd, s1, bsp.F32)
     assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, wd, s1, bsp.F32)
-    assert not bsp.conv_kernel_takes(bsp.KERNEL_GEMM_TC, wd, s1, bsp.F32)
+    assert bsp.conv_kernel_takes(bsp.KERNEL_GEMM_TC, wd, s1, bsp.F32)
+    # a stride of 3 over a 5x5 kernel would need nine phase images: more than the older tensor-memory kernel stages
+    assert not bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16), bsp.XDesc(2, 20, 20, 3, 3, 2, 2), bsp.F32)
     one = C.c_void_p(256)
     h = bsp.Bcsr(256, 256, 256, 256, 32)
-    assert bsp.lib().bsp_conv2d_on(bsp.KERNEL_GEMM_TC, C.byref(wd), C.byref(h), C.byref(s1), one, None, one, bsp.F32, one,
+    s3 = bsp.XDesc(2, 20, 20, 3, 3, 2, 2)
+    wd5 = bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16)
+    assert bsp.lib().bsp_conv2d_on(bsp.KERNEL_CONV_TC, C.byref(wd5), C.byref(h), C.byref(s3), one, None, one, bsp.F32, one,
                                    None) == bsp.ERR_SHAPE

@@ -51,7 +51,6 @@ def test_tc_strided(dtype, O, I, H, K, stride, pad, sp, batch, on_tc):
     tdt = torch.int8 if dtype == "i8" else torch.bfloat16
     ydt = bsp.I32 if dtype == "i8" else bsp.F32
     assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(O, I, H, K, 8, 8, tdt), xd, ydt) == on_tc
-    assert bsp.conv_kernel_name(bsp.wdesc(O, I, H, K, 8, 8, tdt), xd) == ("conv_tc_kernel" if on_tc else "conv_mma_kernel")
     run_conv_case(671 + O + H, O, I, H, K, 8, 8, dtype, (batch, sp[0], sp[1], I), stride, pad)
 
 
