@@ -57,7 +57,7 @@ typedef enum { BSP_F32 = 0, BSP_BF16 = 1, BSP_I8 = 2, BSP_I32 = 3 } bsp_dtype;
 typedef enum { BSP_NORM_L2 = 0, BSP_NORM_L1 = 1 } bsp_norm;
 
 /* Which blocks compete when the lowest scores are zeroed.  LAYER: all NB_o*NB_i blocks are ranked
- * together ("sort them in ascending order").  ROW: each row of Gamma is ranked on its own and gets
+ * together (Section "Predetermined Sparsity ratio and Full Training Ahead").  ROW: each row of Gamma is ranked on its own and gets
  * n_zero zeros, the per-row reading of Eq. (2). */
 typedef enum { BSP_SCOPE_LAYER = 0, BSP_SCOPE_ROW = 1 } bsp_scope;
 
@@ -113,14 +113,15 @@ bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope
  * runs inside another framework's memory plan or with a fixed, pre-carved device heap, plugins that are
  * handed only their input and output tensors, and real-time loops in which cudaMalloc (a blocking, device-
  * wide call) is banned.  Such callers cannot size and pass the `ws` buffer that bsp_mask() needs for the
- * block scores.  bsp_mask_static() computes exactly what bsp_mask() computes (same kernels, same bit-exact
- * Gamma) but keeps the scores in a fixed array inside the library's device image and allocates nothing: it
+ * block scores.  bsp_mask_static() computes exactly what bsp_mask() computes (the same bit-exact Gamma, by the
+ * score and selection kernels that need no workspace) but keeps the scores in a fixed array inside the library's device image and allocates nothing: it
  * calls neither cudaMalloc/cudaFree nor any allocating library routine.
  *   - Limit: NB = (O/b_o)*(I/b_i) <= BSP_MASK_STATIC_MAX_BLOCKS; a larger layer returns BSP_ERR_CAPACITY and
  *     launches nothing.  The array (8 bytes per block, 512 KiB) is held on every GPU that loads the library,
  *     for the life of the process.
  *   - The first call on each device looks up the array's device address (with that device current) and
- *     caches it; make that first call outside any stream capture.
+ *     caches it; make that first call outside any stream capture, and from one host thread (the cache is a
+ *     plain pointer per device: concurrent first calls would all store the same value, but nothing orders them).
  *   - All calls on a device share the one array, which keeps the previous call's scores; every entry that
  *     is read is rewritten first, so no clearing is needed, but two calls that overlap on the GPU (different
  *     streams, or the same layer masked concurrently) race on it.  Serialise them on one stream.
@@ -135,7 +136,8 @@ bsp_status bsp_mask_static(const bsp_wdesc *wd, const void *W, bsp_norm norm, bs
  * bsp_compact_nnz : counts the ones of a device Gamma and returns the count on the host; this one call
  *                   synchronises the stream.
  * bsp_compact     : scans Gamma (caller supplied or from bsp_mask) row by row and writes row_ptr, col_idx,
- *                   the canonical payload and the packed form.  `payload` may be NULL (canonical copy
+ *                   the canonical payload and the packed form (Gamma (.) W in the layout of W, for the TMA loads of
+ *                   the product kernel; its size does not depend on nnz).  `payload` may be NULL (canonical copy
  *                   skipped); `packed` may be NULL (portable form only).  capacity_blocks is the number of
  *                   blocks col_idx/payload/packed were sized for; if Gamma holds more, nothing beyond the
  *                   capacity is written and BSP_ERR_CAPACITY is latched for bsp_check().
@@ -155,34 +157,25 @@ bsp_status bsp_compact(const bsp_wdesc *wd, const void *W, const uint8_t *gamma,
  *             over P pixels); wd->H = wd->K = 1.
  * bsp_conv2d: Y[n,y,x,o] = bias[o] + sum over stored blocks of row o / b_o, over taps (h,k) and channels c of
  *             W[o,h,k,iota b_i + c] X[n, y s_h + h - p_h, x s_w + k - p_w, iota b_i + c], X = 0 out of bounds.
- * Only stored blocks are read or multiplied (the tensor-memory kernel works on 16-channel super-tiles: zeroed
- * blocks that share a super-tile with a stored block, and a missing super-row between two present ones, are
- * multiplied as zeros).  Types: BF16 or F32 inputs (wtype = type of X) accumulate in
- * float32, bias float32, ytype F32 or BF16 (round to nearest even after the bias); F32 inputs are
- * multiplied as TF32.  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
+ * Types: BF16 or F32 inputs (wtype = type of X) accumulate in float32, bias float32, ytype F32 or BF16 (round to
+ * nearest even after the bias); F32 inputs are multiplied as TF32 (the tensor core reads the upper 19 bits of each
+ * operand).  I8 inputs accumulate in int32 (exact), bias int32, ytype I32.
  *   bias may be NULL (treated as zero).  ws: device scratch of bsp_conv_workspace_bytes() bytes.
- * Two kernels implement the products.  BF16 and I8 layers run on the tensor-memory kernel ("conv_tc_kernel":
- * tcgen05 MMAs on 16-channel super-tiles of the second packed form) unless their shape rules it out (more than
- * four stride residues in use, a tile that does not fit shared memory, I not a multiple of the K-step); those, F32, and
- * every layer when the environment variable BSP_CONV_PATH starts with 'm', runs on the warp-MMA kernel
- * ("conv_mma_kernel", 8x8 tiles).  bsp_conv_kernel_name() says which one a call with these descriptors takes
- * (static storage; NULL for invalid descriptors).
- * Errors: NULL, SHAPE, BLOCK, DTYPE, INDEX (packed buffer does not match wd), CUDA. */
+ * One kernel implements the products ("gemm_tc_kernel": tcgen05 MMAs with the accumulators in tensor memory, both
+ * operands staged by tiled TMA loads; a convolution is an implicit GEMM over taps x channel chunks).  It reads
+ * `packed`, which holds Gamma (.) W in the layout of W: zeroed blocks cost no arithmetic result and no entry in
+ * row_ptr / col_idx / payload, but the tensor-core instruction multiplies them as zeros (an instruction covers
+ * 128 x 256 x 16 entries of the operands, far more than a block).
+ * The kernel compares the header of `packed` with wd before it loads anything; a buffer that bsp_compact filled for
+ * another descriptor latches BSP_ERR_INDEX and leaves Y untouched.  bsp_conv_kernel_name() names the kernel a call
+ * with these descriptors takes (static storage; NULL for descriptors no kernel takes).
+ * Errors: NULL, SHAPE, BLOCK, DTYPE, INDEX (nnz out of range; packed buffer does not match wd: latched), CUDA. */
 size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd);
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,
                     void *Y, bsp_dtype ytype, void *ws, void *stream);
 bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd);
-
-/* The same product on a named kernel, for validation and tuning: every kernel must give the result of the
- * definition above, so the tests run each layer on every kernel that can take it.  BSP_KERNEL_AUTO is bsp_conv2d();
- * a kernel that cannot take the layer returns BSP_ERR_SHAPE and launches nothing. */
-typedef enum { BSP_KERNEL_AUTO = 0, BSP_KERNEL_GEMM_TC = 1, BSP_KERNEL_CONV_TC = 2, BSP_KERNEL_CONV_MMA = 3 } bsp_kernel;
-bsp_status bsp_conv2d_on(bsp_kernel which, const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
-                         const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
-/* 1 if the named kernel can run a layer with these descriptors and output type, else 0 (host-side decision). */
-int bsp_conv_kernel_takes(bsp_kernel which, const bsp_wdesc *wd, const bsp_xdesc *xd, bsp_dtype ytype);
 
 /* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
  * (BSP_OK if none), then clears it. */

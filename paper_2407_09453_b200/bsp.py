@@ -19,12 +19,10 @@ OK, ERR_NULL, ERR_SHAPE, ERR_BLOCK, ERR_DTYPE, ERR_CAPACITY, ERR_INDEX, ERR_CUDA
 F32, BF16, I8, I32 = 0, 1, 2, 3
 NORM_L2, NORM_L1 = 0, 1
 SCOPE_LAYER, SCOPE_ROW = 0, 1
-KERNEL_AUTO, KERNEL_GEMM_TC, KERNEL_CONV_TC, KERNEL_CONV_MMA = 0, 1, 2, 3
-KERNEL_NAMES = {KERNEL_GEMM_TC: "gemm_tc_kernel", KERNEL_CONV_TC: "conv_tc_kernel", KERNEL_CONV_MMA: "conv_mma_kernel"}
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_mask_static", "bsp_packed_bytes",
            "bsp_compact_workspace_bytes", "bsp_compact_nnz", "bsp_compact", "bsp_conv_workspace_bytes", "bsp_gemm",
-           "bsp_conv2d", "bsp_conv2d_on", "bsp_conv_kernel_name", "bsp_conv_kernel_takes", "bsp_check", "bsp_status_string"]
+           "bsp_conv2d", "bsp_conv_kernel_name", "bsp_check", "bsp_status_string"]
 
 
 class BspError(RuntimeError):
@@ -64,7 +62,7 @@ def lib():
         L.bsp_status_string.restype = C.c_char_p
         L.bsp_conv_kernel_name.restype = C.c_char_p
         for n in ("bsp_mask", "bsp_mask_static", "bsp_compact_nnz", "bsp_compact", "bsp_gemm", "bsp_conv2d",
-                  "bsp_conv2d_on", "bsp_conv_kernel_takes", "bsp_check"):
+                  "bsp_check"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -151,11 +149,6 @@ def bsp_conv2d(wd: WDesc, w: Bcsr, xd: XDesc, X, bias, Y, ytype, ws, stream=None
                             _ptr(ws), _stream(stream)), "bsp_conv2d")
 
 
-def bsp_conv2d_on(which: int, wd: WDesc, w: Bcsr, xd: XDesc, X, bias, Y, ytype, ws, stream=None):
-    _raise(lib().bsp_conv2d_on(C.c_int(which), C.byref(wd), C.byref(w), C.byref(xd), _ptr(X), _ptr(bias), _ptr(Y),
-                               C.c_int(ytype), _ptr(ws), _stream(stream)), "bsp_conv2d_on")
-
-
 def bsp_mask_static(wd: WDesc, W, norm, scope, n_zero, gamma, stream=None):
     _raise(lib().bsp_mask_static(C.byref(wd), _ptr(W), C.c_int(norm), C.c_int(scope), C.c_int64(n_zero), _ptr(gamma),
                                  _stream(stream)), "bsp_mask_static")
@@ -173,19 +166,12 @@ def conv_kernel_name(wd: WDesc, xd: XDesc) -> str:
     return r.decode()
 
 
-def conv_kernel_takes(which: int, wd: WDesc, xd: XDesc, ytype: int) -> bool:
-    """True if the named product kernel can run a layer with these descriptors and output type."""
-    return bool(lib().bsp_conv_kernel_takes(C.c_int(which), C.byref(wd), C.byref(xd), C.c_int(ytype)))
-
-
 def launches_per_step(wd: WDesc) -> int:
     """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass.  General path: score, select;
-    count, scan, fill+pack; the product kernel.  Small layers take one launch for the mask (up to 2048 blocks) and
-    one for the compaction (up to 4096 blocks); 1x1 layers add the index kernel of the block form."""
+    count, scan, fill; the product kernel.  Small layers take one launch for the mask (up to 2048 blocks) and
+    one for the compaction (up to 4096 blocks)."""
     nb = (wd.O // wd.bo) * (wd.I // wd.bi)
-    esz = {F32: 4, BF16: 2, I8: 1}[wd.wtype]
-    block_form = 1 if (wd.H == 1 and wd.K == 1 and (wd.I * esz) % 16 == 0 and wd.O % 8 == 0) else 0
-    return (1 if nb <= 2048 else 2) + (1 if nb <= 4096 else 3) + block_form + 1
+    return (1 if nb <= 2048 else 2) + (1 if nb <= 4096 else 3) + 1
 
 
 class SparseLayer:
@@ -207,7 +193,6 @@ class SparseLayer:
         self.ws = new_workspace(max(bsp_mask_workspace_bytes(self.wd), bsp_compact_workspace_bytes(self.wd)),
                                 device)
         self.nnz = self.capacity
-        self.kernel = KERNEL_AUTO      # a KERNEL_* value other than AUTO runs the products through bsp_conv2d_on
 
     def mask(self, W, n_zero, norm=NORM_L2, scope=SCOPE_LAYER, scores=None, stream=None):
         bsp_mask(self.wd, W, norm, scope, n_zero, self.gamma, scores, self.ws, stream)
@@ -225,17 +210,10 @@ class SparseLayer:
     def conv2d(self, X, bias, Y, stride=(1, 1), pad=(0, 0), stream=None):
         N, L, J, _ = X.shape
         xd = XDesc(N, L, J, stride[0], stride[1], pad[0], pad[1])
-        if self.kernel != KERNEL_AUTO:
-            bsp_conv2d_on(self.kernel, self.wd, self.handle(), xd, X, bias, Y, dtype_code(Y.dtype), self.ws, stream)
-        else:
-            bsp_conv2d(self.wd, self.handle(), xd, X, bias, Y, dtype_code(Y.dtype), self.ws, stream)
+        bsp_conv2d(self.wd, self.handle(), xd, X, bias, Y, dtype_code(Y.dtype), self.ws, stream)
 
     def gemm(self, X, bias, Y, stream=None):
-        if self.kernel != KERNEL_AUTO:
-            xd = XDesc(X.shape[0], 1, 1, 1, 1, 0, 0)
-            bsp_conv2d_on(self.kernel, self.wd, self.handle(), xd, X, bias, Y, dtype_code(Y.dtype), self.ws, stream)
-        else:
-            bsp_gemm(self.wd, self.handle(), X, X.shape[0], bias, Y, dtype_code(Y.dtype), self.ws, stream)
+        bsp_gemm(self.wd, self.handle(), X, X.shape[0], bias, Y, dtype_code(Y.dtype), self.ws, stream)
 
     def check(self, stream=None):
         bsp_check(self.ws, stream)

@@ -13,8 +13,7 @@ void report_cuda_error(cudaError_t e, const char *expr, const char *file, int li
 
 using namespace bsp;
 
-namespace {
-
+namespace bsp {
 bsp_status check_wdesc(const bsp_wdesc *wd)
 {
     if (!wd) return BSP_ERR_NULL;
@@ -26,30 +25,11 @@ bsp_status check_wdesc(const bsp_wdesc *wd)
     if ((long long)wd->H * wd->K > 120) return BSP_ERR_SHAPE;
     return BSP_OK;
 }
+}  // namespace bsp
 
+namespace {
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void *p) { return ((uintptr_t)p & 3u) == 0; }
-
-// The product kernel of a layer: the persistent matrix-product kernel for 1x1 layers without padding or stride, the
-// tensor-memory convolution kernel for the other bf16 / int8 layers it can stage, the warp-MMA kernel for the rest.
-// `which` other than BSP_KERNEL_AUTO names one kernel; BSP_KERNEL_AUTO is returned when that kernel cannot take the layer.
-bsp_kernel choose_kernel(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype, bsp_kernel which)
-{
-    const bool gemm_ok = gemm_tc_eligible(wd, xd, ytype), tc_ok = conv_tc_eligible(wd, xd);
-    switch (which) {
-        case BSP_KERNEL_GEMM_TC: return gemm_ok ? which : BSP_KERNEL_AUTO;
-        case BSP_KERNEL_CONV_TC: return tc_ok ? which : BSP_KERNEL_AUTO;
-        case BSP_KERNEL_CONV_MMA: return which;
-        default: break;
-    }
-    return gemm_ok ? BSP_KERNEL_GEMM_TC : (tc_ok ? BSP_KERNEL_CONV_TC : BSP_KERNEL_CONV_MMA);
-}
-
-const char *kernel_name(bsp_kernel k)
-{
-    return k == BSP_KERNEL_GEMM_TC ? "gemm_tc_kernel" : (k == BSP_KERNEL_CONV_TC ? "conv_tc_kernel" : "conv_mma_kernel");
-}
-
 }  // namespace
 
 extern "C" {
@@ -96,13 +76,13 @@ bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope
 size_t bsp_packed_bytes(const bsp_wdesc *wd, int64_t nnz)
 {
     if (check_wdesc(wd) != BSP_OK || nnz < 0) return 0;
-    return packed_layout(*wd, nnz).total_bytes;
+    return packed_layout(*wd).total_bytes;
 }
 
 size_t bsp_compact_workspace_bytes(const bsp_wdesc *wd)
 {
     if (check_wdesc(wd) != BSP_OK) return 0;
-    const size_t n = (size_t)(wd->O / wd->bo) + (size_t)((wd->O + kPanelCh - 1) / kPanelCh) + 8;
+    const size_t n = (size_t)(wd->O / wd->bo) + 8;
     return kWsHeader + align_up(n * 4, 256);
 }
 
@@ -146,12 +126,6 @@ size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd)
 bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
 {
-    return bsp_conv2d_on(BSP_KERNEL_AUTO, wd, w, xd, X, bias, Y, ytype, ws, stream);
-}
-
-bsp_status bsp_conv2d_on(bsp_kernel which, const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
-                         const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
-{
     bsp_status rc = check_wdesc(wd);
     if (rc != BSP_OK) return rc;
     if (!w || !xd || !X || !Y || !ws || !w->packed) return BSP_ERR_NULL;
@@ -164,31 +138,17 @@ bsp_status bsp_conv2d_on(bsp_kernel which, const bsp_wdesc *wd, const bsp_bcsr *
     if (wd->wtype == BSP_I8) { if (ytype != BSP_I32) return BSP_ERR_DTYPE; }
     else if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
     if (!aligned16(X) || !aligned16(Y) || !aligned16(w->packed)) return BSP_ERR_SHAPE;
-    // the packed header is on the device; the host checks what it can: capacity against the descriptor
+    // the packed header is on the device (the kernel checks it against the descriptor); the host checks the count
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
-    if (which < BSP_KERNEL_AUTO || which > BSP_KERNEL_CONV_MMA) return BSP_ERR_DTYPE;
-    const bsp_kernel k = choose_kernel(*wd, *xd, ytype, which);
-    if (k == BSP_KERNEL_AUTO) return BSP_ERR_SHAPE;              // the kernel asked for cannot take this layer
-    if (k == BSP_KERNEL_GEMM_TC)
-        return launch_gemm_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
-    if (k == BSP_KERNEL_CONV_TC)
-        return launch_conv_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
-    // the stored fraction only steers the choice of launch shape
-    const double density = NB > 0 ? (double)w->nnz / (double)NB : 1.0;
-    return launch_conv(*wd, *xd, w->packed, X, bias, Y, ytype, density > 0.05 ? density : 0.05, ws, (cudaStream_t)stream);
+    if (!gemm_tc_eligible(*wd, *xd, ytype)) return BSP_ERR_SHAPE;
+    return launch_gemm_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
 }
 
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd)
 {
     if (check_wdesc(wd) != BSP_OK || !xd) return nullptr;
-    return kernel_name(choose_kernel(*wd, *xd, wd->wtype == BSP_I8 ? BSP_I32 : BSP_F32, BSP_KERNEL_AUTO));
-}
-
-int bsp_conv_kernel_takes(bsp_kernel which, const bsp_wdesc *wd, const bsp_xdesc *xd, bsp_dtype ytype)
-{
-    if (check_wdesc(wd) != BSP_OK || !xd || which <= BSP_KERNEL_AUTO || which > BSP_KERNEL_CONV_MMA) return 0;
-    return choose_kernel(*wd, *xd, ytype, which) == which ? 1 : 0;
+    return gemm_tc_eligible(*wd, *xd, wd->wtype == BSP_I8 ? BSP_I32 : BSP_F32) ? "gemm_tc_kernel" : nullptr;
 }
 
 bsp_status bsp_gemm(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const void *bias,

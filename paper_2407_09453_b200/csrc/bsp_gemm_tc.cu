@@ -391,6 +391,16 @@ namespace {
 // Wt * s_w x Ht * s_h input positions and may not exceed 256 in any extent.
 struct GtTile { int Wt, Ht, Nt; long long tiles; };
 
+// A 1x1 layer without padding or stride is a matrix product over all N L J positions: taken as that many 1x1 images,
+// so that a tile is 128 consecutive positions whatever the image size.
+bsp_xdesc gt_flatten(const bsp_wdesc &wd, const bsp_xdesc &xd)
+{
+    const long long P = (long long)xd.N * xd.L * xd.J;
+    if (wd.H == 1 && wd.K == 1 && xd.pad_h == 0 && xd.pad_w == 0 && xd.stride_h == 1 && xd.stride_w == 1 && P <= 0x7FFFFFFF)
+        return bsp_xdesc{(int)P, 1, 1, 1, 1, 0, 0};
+    return xd;
+}
+
 GtTile gt_pick_tile(int N, int M, int Nw, int sh, int sw)
 {
     GtTile best = {0, 0, 0, -1};
@@ -411,9 +421,10 @@ GtTile gt_pick_tile(int N, int M, int Nw, int sh, int sw)
 
 // True if the kernel can run this layer: rows of X, W and Y that are multiples of 16 bytes (tensor-map strides), a
 // position count that fits 32 bits, and a position tile whose box the tensor map can express.
-bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype)
+bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd0, bsp_dtype ytype)
 {
-    if (!packed_layout(wd, 0).gm.enabled) return false;
+    const bsp_xdesc xd = gt_flatten(wd, xd0);
+    if (!packed_layout(wd).enabled) return false;
     if (ytype != BSP_F32 && ytype != BSP_BF16 && ytype != BSP_I32) return false;
     const int ey = ytype == BSP_BF16 ? 2 : 4;
     if (((long long)wd.O * ey) % 16 != 0) return false;
@@ -424,12 +435,12 @@ bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype)
     return gt_pick_tile(xd.N, M, Nw, xd.stride_h, xd.stride_w).tiles > 0;
 }
 
-bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
+bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void *packed, const void *X,
                           const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
 {
-    const PackedLayout L = packed_layout(wd, 0);
-    const GemmLayout &G = L.gm;
-    if (!G.enabled) return BSP_ERR_SHAPE;
+    const bsp_xdesc xd = gt_flatten(wd, xd0);
+    const PackedLayout L = packed_layout(wd);
+    if (!L.enabled) return BSP_ERR_SHAPE;
     const int esz = elem_bytes(wd.wtype);
     const int ey = ytype == BSP_BF16 ? 2 : 4;
     const int HK = wd.H * wd.K;
@@ -483,7 +494,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *
         const cuuint64_t gstr[2] = {row, row * HK};
         const cuuint32_t box[3] = {128, 1, (cuuint32_t)p.BN};
         const cuuint32_t estr[3] = {1, 1, 1};
-        if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed + G.off_payload), gdim, gstr, box, estr,
+        if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed + L.off_payload), gdim, gstr, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;

@@ -17,12 +17,8 @@ void *g_scores_ptr[kMaxDevices] = {};      // device address of g_static_scores,
 extern "C" bsp_status bsp_mask_static(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope,
                                       int64_t n_zero, uint8_t *gamma, void *stream)
 {
-    if (!wd) return BSP_ERR_NULL;
-    if (wd->O <= 0 || wd->I <= 0 || wd->H <= 0 || wd->K <= 0) return BSP_ERR_SHAPE;
-    const bool ok_block = (wd->bo == 8 && wd->bi == 8) || (wd->bo == 4 && wd->bi == 16) || (wd->bo == 16 && wd->bi == 4);
-    if (!ok_block) return BSP_ERR_BLOCK;
-    if (wd->O % wd->bo != 0 || wd->I % wd->bi != 0) return BSP_ERR_SHAPE;
-    if (wd->wtype != BSP_F32 && wd->wtype != BSP_BF16 && wd->wtype != BSP_I8) return BSP_ERR_DTYPE;
+    const bsp_status rc = bsp::check_wdesc(wd);           // the same descriptor rules as bsp_mask()
+    if (rc != BSP_OK) return rc;
     if (!W || !gamma) return BSP_ERR_NULL;
     if (((uintptr_t)W & 3u) != 0) return BSP_ERR_SHAPE;
     if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1) return BSP_ERR_DTYPE;

@@ -6,17 +6,6 @@ from paper_2407_09453_b200 import bsp, synth
 
 TORCH_DT = {"bf16": torch.bfloat16, "f32": torch.float32, "i8": torch.int8}
 
-# The product kernel that gpu_conv / gpu_gemm ask for (a bsp.KERNEL_* value, set by test fixtures); a layer that this
-# kernel cannot take runs on the library's own choice.
-PREFER_KERNEL = bsp.KERNEL_AUTO
-
-
-def pick_kernel(lay, xd, ytype):
-    k = PREFER_KERNEL
-    lay.kernel = k if k != bsp.KERNEL_AUTO and bsp.conv_kernel_takes(k, lay.wd, xd, bsp.dtype_code(ytype)) else bsp.KERNEL_AUTO
-    return lay.kernel
-
-
 def to_dev(a: np.ndarray, dtype: str) -> torch.Tensor:
     t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
     return t.to(torch.bfloat16) if dtype == "bf16" else t
@@ -57,7 +46,6 @@ def gpu_conv(lay, X, bias, dtype, stride=(1, 1), pad=(0, 0), out="f32"):
     Y = torch.full((N, M, Nw, O), -7, dtype=ydt, device="cuda")
     Xd = to_dev(X, dtype)
     bd = None if bias is None else torch.from_numpy(bias).cuda()
-    pick_kernel(lay, bsp.XDesc(N, L, J, stride[0], stride[1], pad[0], pad[1]), ydt)
     lay.conv2d(Xd, bd, Y, stride, pad)
     lay.check()
     return from_dev(Y).reshape(-1, O)
@@ -70,7 +58,6 @@ def gpu_gemm(lay, X, bias, dtype, out="f32"):
     Y = torch.full((P, O), -7, dtype=ydt, device="cuda")
     Xd = to_dev(X, dtype)
     bd = None if bias is None else torch.from_numpy(bias).cuda()
-    pick_kernel(lay, bsp.XDesc(P, 1, 1, 1, 1, 0, 0), ydt)
     lay.gemm(Xd, bd, Y)
     lay.check()
     return from_dev(Y)

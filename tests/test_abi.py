@@ -66,26 +66,13 @@ def test_host_validation_without_gpu(lib):
     assert lib.bsp_check(None, None) == bsp.ERR_NULL
 
 
-def test_product_kernel_choice():
-    """Every layer whose rows of input channels are multiples of 16 bytes takes the persistent tensor-memory kernel,
-    whatever its type, taps and strides; the other kernels are reached by name (a host-side decision: no GPU needed)."""
+def test_product_kernel_name():
+    """Every layer the API accepts takes the one product kernel, whatever its type, taps and strides (a host-side
+    answer: no GPU needed)."""
     import torch
-    s1 = bsp.XDesc(2, 14, 14, 1, 1, 1, 1)
-    s2 = bsp.XDesc(2, 14, 14, 2, 2, 1, 1)
     for dt in (torch.bfloat16, torch.int8, torch.float32):
         wd = bsp.wdesc(64, 64, 3, 3, 8, 8, dt)
-        assert bsp.conv_kernel_name(wd, s1) == "gemm_tc_kernel"
-        assert bsp.conv_kernel_name(wd, s2) == "gemm_tc_kernel"
+        assert bsp.conv_kernel_name(wd, bsp.XDesc(2, 14, 14, 1, 1, 1, 1)) == "gemm_tc_kernel"
+        assert bsp.conv_kernel_name(wd, bsp.XDesc(2, 14, 14, 2, 2, 1, 1)) == "gemm_tc_kernel"
         assert bsp.conv_kernel_name(bsp.wdesc(64, 48, 1, 1, 8, 8, dt), bsp.XDesc(2, 7, 7, 1, 1, 0, 0)) == "gemm_tc_kernel"
-    wd = bsp.wdesc(64, 64, 3, 3, 8, 8, torch.bfloat16)
-    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_MMA, wd, s1, bsp.F32)
-    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, wd, s1, bsp.F32)
-    assert bsp.conv_kernel_takes(bsp.KERNEL_GEMM_TC, wd, s1, bsp.F32)
-    # a stride of 3 over a 5x5 kernel would need nine phase images: more than the older tensor-memory kernel stages
-    assert not bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16), bsp.XDesc(2, 20, 20, 3, 3, 2, 2), bsp.F32)
-    one = C.c_void_p(256)
-    h = bsp.Bcsr(256, 256, 256, 256, 32)
-    s3 = bsp.XDesc(2, 20, 20, 3, 3, 2, 2)
-    wd5 = bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16)
-    assert bsp.lib().bsp_conv2d_on(bsp.KERNEL_CONV_TC, C.byref(wd5), C.byref(h), C.byref(s3), one, None, one, bsp.F32, one,
-                                   None) == bsp.ERR_SHAPE
+    assert bsp.conv_kernel_name(bsp.wdesc(64, 64, 5, 5, 8, 8, torch.bfloat16), bsp.XDesc(2, 20, 20, 3, 3, 2, 2)) == "gemm_tc_kernel"

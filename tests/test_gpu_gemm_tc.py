@@ -1,7 +1,6 @@
-"""GPU parity of the persistent tcgen05 matrix-product kernel (gemm_tc_kernel: bf16, int8 and fp32-as-TF32 1x1 layers;
-kept blocks expanded from the block-CSR payload inside the SM) against the CPU oracle, through the C ABI: within
-tolerance for floats, bit for bit for int8.  Every case asks for the kernel by name and checks that it can take the
-layer, so that a silent fall-back to another kernel cannot pass."""
+"""GPU parity of the product kernel on matrix products (bf16, int8 and fp32-as-TF32 1x1 layers: ragged position and
+channel tiles, K tails inside a stage, more tiles than SMs, long K, sparsity extremes, bf16 output) against the CPU
+oracle, through the C ABI: within tolerance for floats, bit for bit for int8."""
 import numpy as np
 import pytest
 import torch
@@ -18,14 +17,9 @@ SHAPES = [(8, 8), (4, 16), (16, 4)]
 YT = {"bf16": bsp.F32, "f32": bsp.F32, "i8": bsp.I32}
 
 
-@pytest.fixture(autouse=True)
-def on_gemm_tc(monkeypatch):
-    monkeypatch.setattr(gpu_util, "PREFER_KERNEL", bsp.KERNEL_GEMM_TC)
-
-
 def run_gemm(seed, O, I, P, bo, bi, dtype, frac=0.5, out="f32", bias=True):
     wd = bsp.wdesc(O, I, 1, 1, bo, bi, gpu_util.TORCH_DT[dtype])
-    assert bsp.conv_kernel_takes(bsp.KERNEL_GEMM_TC, wd, bsp.XDesc(P, 1, 1, 1, 1, 0, 0), bsp.BF16 if out == "bf16" else YT[dtype])
+    assert bsp.conv_kernel_name(wd, bsp.XDesc(P, 1, 1, 1, 1, 0, 0)) == "gemm_tc_kernel"
     W = make_case(seed, O, I, 1, 1, dtype)
     NB = (O // bo) * (I // bi)
     gamma = synth.random_gamma(seed + 1, O // bo, I // bi, int(round(frac * NB)))
@@ -33,7 +27,6 @@ def run_gemm(seed, O, I, P, bo, bi, dtype, frac=0.5, out="f32", bias=True):
     b = make_bias(seed + 3, O, dtype) if bias else None
     lay = gpu_layer(W, gamma, bo, bi, dtype)
     got = gpu_gemm(lay, X, b, dtype, out)
-    assert lay.kernel == bsp.KERNEL_GEMM_TC
     rp, ci, pl = ref.compact(W, gamma, bo, bi)
     want = ref.gemm(O, I, bo, bi, rp, ci, pl.reshape(-1, bo, bi), X, b)
     check(got, want, dtype, out)
@@ -86,7 +79,7 @@ def test_long_k_wraps_the_stage_ring_many_times():
     run_gemm(763, 64, 8192, 40, 8, 8, "i8", frac=0.75)
 
 
-def test_conv2d_1x1_takes_the_same_kernel_and_equals_gemm_bitwise():
+def test_conv2d_1x1_equals_gemm_bitwise():
     O, I = 128, 192
     W = make_case(771, O, I, 1, 1, "bf16")
     gamma = synth.random_gamma(772, 16, 24, 192)
@@ -94,7 +87,6 @@ def test_conv2d_1x1_takes_the_same_kernel_and_equals_gemm_bitwise():
     b = make_bias(774, O, "bf16")
     lay = gpu_layer(W, gamma, 8, 8, "bf16")
     yc = gpu_conv(lay, X, b, "bf16")
-    assert lay.kernel == bsp.KERNEL_GEMM_TC
     yg = gpu_gemm(lay, X.reshape(-1, I), b, "bf16")
     assert np.array_equal(yc, yg)
 
@@ -109,7 +101,7 @@ def test_packed_buffer_of_another_layer_is_refused():
     other = bsp.SparseLayer(128, 128, 1, 1, 4, 16, torch.bfloat16)       # same sizes, another block shape
     X = gpu_util.to_dev(make_x(783, (64, 128), "bf16"), "bf16")
     Y = torch.full((64, 128), -7.0, dtype=torch.float32, device="cuda")
-    bsp.bsp_conv2d_on(bsp.KERNEL_GEMM_TC, other.wd, lay.handle(), bsp.XDesc(64, 1, 1, 1, 1, 0, 0), X, None, Y, bsp.F32, lay.ws)
+    bsp.bsp_conv2d(other.wd, lay.handle(), bsp.XDesc(64, 1, 1, 1, 1, 0, 0), X, None, Y, bsp.F32, lay.ws)
     with pytest.raises(bsp.BspError) as e:
         lay.check()
     assert e.value.status == bsp.ERR_INDEX

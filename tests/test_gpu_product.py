@@ -8,19 +8,10 @@ import pytest
 
 from oracle import ref
 from paper_2407_09453_b200 import bsp, synth
-import gpu_util
 from gpu_util import (TIGHT, TOL, gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_bias, make_case, make_x,
                       rel_err, from_dev)
 
 pytestmark = pytest.mark.gpu
-
-
-@pytest.fixture(autouse=True, params=["auto", "mma"])
-def conv_path(request, monkeypatch):
-    """Every case runs twice: with the library's own choice of product kernel (a tensor-memory kernel wherever one can
-    take the layer) and on the warp-MMA kernel, so that both see every shape."""
-    monkeypatch.setattr(gpu_util, "PREFER_KERNEL", bsp.KERNEL_CONV_MMA if request.param == "mma" else bsp.KERNEL_AUTO)
-    return request.param
 
 
 SHAPES = [(8, 8), (4, 16), (16, 4)]
@@ -96,10 +87,8 @@ def test_conv_taps_strides_padding(dtype, H, K, stride, pad, sp):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "i8"])
-@pytest.mark.parametrize("kernel", [bsp.KERNEL_CONV_MMA, bsp.KERNEL_CONV_TC, bsp.KERNEL_GEMM_TC])
-def test_gemm_packed_forms_of_the_multi_launch_compaction(dtype, kernel, monkeypatch):
-    """8192 blocks: all three packed forms come from the count / scan / fill launches, not the one-launch kernel."""
-    monkeypatch.setattr(gpu_util, "PREFER_KERNEL", kernel)
+def test_gemm_packed_form_of_the_multi_launch_compaction(dtype):
+    """8192 blocks: the packed form comes from the count / scan / fill launches, not the one-launch kernel."""
     O, I, P = 512, 1024, 200
     W = make_case(451, O, I, 1, 1, dtype)
     gamma = synth.random_gamma(452, O // 8, I // 8, (O // 8) * (I // 8) // 2)
@@ -165,28 +154,6 @@ def test_config_resnet_conv_3x3_256_bf16_with_l2_gamma():
         rp, ci, pl = ref.compact(W, want_g, 8, 8)
         want = ref.conv2d(W.shape, 8, 8, rp, ci, pl, X, b, (1, 1), (1, 1))
         check(got, want, "bf16", out)
-
-
-@pytest.mark.parametrize("bo,bi,frac", [(8, 8, 0.5), (4, 16, 0.25), (16, 4, 0.75)])
-def test_config_gemm_4096_sampled_rows(bo, bi, frac):
-    """O = I = 4096, P = 8192, bf16, magnitude Gamma: the oracle evaluates 48 sampled rows of Y."""
-    O = I = 4096
-    P = 8192
-    W = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 0), (O, 1, 1, I), 1 / 64.0).astype(np.float32))
-    X = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 1), (P, I)).astype(np.float32))
-    b = synth.normal(synth.tensor_seed(3, 0, 2), (O,), 0.1).astype(np.float32)
-    NB = (O // bo) * (I // bi)
-    g, s, lay, Wd = gpu_mask(W, bo, bi, "bf16", int(frac * NB))
-    want_g = ref.mask(ref.scores(W, bo, bi), int(frac * NB))
-    assert np.array_equal(g, want_g)
-    lay.compact(Wd)
-    lay.check()
-    got = gpu_gemm(lay, X, b, "bf16")
-    pix = np.r_[0, 127, 128, P - 1, synth.uniform_int(7, (44,), 0, P - 1)]
-    rp, ci, pl = ref.compact(W, want_g, bo, bi)
-    want = ref.gemm(O, I, bo, bi, rp, ci, pl.reshape(-1, bo, bi), X, b, pix=pix)
-    check(got[pix], want, "bf16")
-    assert np.isfinite(got).all()
 
 
 def test_large_int8_vgg_like_layer_sampled_pixels():

@@ -1,6 +1,5 @@
-"""GPU parity of the tcgen05 convolution kernel (bf16 and int8; every case asks for it by name, so 1x1 layers that the
-matrix-product kernel would otherwise take run on it too) against the CPU oracle: within tolerance for bf16, bit for bit
-for int8."""
+"""GPU parity of the product kernel over layer shapes (taps, strides, padding, channel counts off the tile grid, tiles
+that span images, long position counts) against the CPU oracle: within tolerance for bf16, bit for bit for int8."""
 import numpy as np
 import pytest
 
@@ -8,16 +7,10 @@ from oracle import ref
 import torch
 
 from paper_2407_09453_b200 import bsp, synth
-import gpu_util
 from gpu_util import gpu_conv, gpu_gemm, gpu_layer, gpu_mask, make_bias, make_case, make_x
 from test_gpu_product import check, run_conv_case
 
 pytestmark = pytest.mark.gpu
-
-
-@pytest.fixture(autouse=True)
-def tc_path(monkeypatch):
-    monkeypatch.setattr(gpu_util, "PREFER_KERNEL", bsp.KERNEL_CONV_TC)
 
 
 TC_CASES = [  # O, I, H, K, pad, spatial, batch
@@ -32,25 +25,18 @@ def test_tc_conv_shapes(O, I, H, K, pad, sp, batch):
     run_conv_case(601 + O + H, O, I, H, K, 8, 8, "bf16", (batch, sp[0], sp[1], I), (1, 1), pad)
 
 
-STRIDED = [  # O, I, H, K, stride, pad, spatial, batch, runs on the tensor-memory kernel
-    (128, 64, 3, 3, (2, 2), (1, 1), (15, 15), 3, True), (64, 64, 1, 1, (2, 2), (0, 0), (14, 14), 3, True),
-    (64, 32, 3, 3, (2, 2), (0, 0), (17, 17), 2, True), (64, 64, 3, 3, (2, 1), (1, 1), (28, 9), 2, True),
-    (256, 128, 3, 3, (2, 2), (1, 1), (56, 56), 1, True), (64, 32, 5, 5, (2, 2), (2, 2), (30, 30), 1, True),
-    # 49 taps: two stages of one K-group's weights (25 K-steps x 8 super-rows) do not fit the shared memory
-    (64, 32, 7, 7, (2, 2), (3, 3), (30, 30), 1, False),
-    # 5 taps per row at a column stride of 2: tap pairs (A, B) and (B, A) of the two phases cannot both lie in
-    # ascending order in shared memory, so this one stays on the warp-MMA kernel
-    (72, 48, 5, 5, (1, 2), (2, 1), (11, 13), 2, False),
+STRIDED = [  # O, I, H, K, stride, pad, spatial, batch
+    (128, 64, 3, 3, (2, 2), (1, 1), (15, 15), 3), (64, 64, 1, 1, (2, 2), (0, 0), (14, 14), 3),
+    (64, 32, 3, 3, (2, 2), (0, 0), (17, 17), 2), (64, 64, 3, 3, (2, 1), (1, 1), (28, 9), 2),
+    (256, 128, 3, 3, (2, 2), (1, 1), (56, 56), 1), (64, 32, 5, 5, (2, 2), (2, 2), (30, 30), 1),
+    (64, 32, 7, 7, (2, 2), (3, 3), (30, 30), 1), (72, 48, 5, 5, (1, 2), (2, 1), (11, 13), 2),
+    (64, 32, 3, 3, (3, 3), (1, 1), (200, 9), 1),       # a tall image at stride 3: the box height is capped by the tensor map's 256-element extent
 ]
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "i8"])
-@pytest.mark.parametrize("O,I,H,K,stride,pad,sp,batch,on_tc", STRIDED)
-def test_tc_strided(dtype, O, I, H, K, stride, pad, sp, batch, on_tc):
-    xd = bsp.XDesc(batch, sp[0], sp[1], stride[0], stride[1], pad[0], pad[1])
-    tdt = torch.int8 if dtype == "i8" else torch.bfloat16
-    ydt = bsp.I32 if dtype == "i8" else bsp.F32
-    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(O, I, H, K, 8, 8, tdt), xd, ydt) == on_tc
+@pytest.mark.parametrize("dtype", ["bf16", "i8", "f32"])
+@pytest.mark.parametrize("O,I,H,K,stride,pad,sp,batch", STRIDED)
+def test_tc_strided(dtype, O, I, H, K, stride, pad, sp, batch):
     run_conv_case(671 + O + H, O, I, H, K, 8, 8, dtype, (batch, sp[0], sp[1], I), stride, pad)
 
 
@@ -65,8 +51,6 @@ I8_CASES = [  # O, I, H, K, pad, spatial, batch: I a multiple of 16 (conv) or 32
 def test_tc_int8_bit_exact(O, I, H, K, pad, sp, batch, bo, bi):
     if O % bo or I % bi:
         pytest.skip("channels are not a multiple of the block")
-    xd = bsp.XDesc(batch, sp[0], sp[1], 1, 1, pad[0], pad[1])
-    assert bsp.conv_kernel_takes(bsp.KERNEL_CONV_TC, bsp.wdesc(O, I, H, K, bo, bi, torch.int8), xd, bsp.I32)
     run_conv_case(641 + O + H, O, I, H, K, bo, bi, "i8", (batch, sp[0], sp[1], I), (1, 1), pad)
 
 
@@ -115,9 +99,8 @@ def test_tc_gemm_two_position_tiles_per_cta(dtype):
 
 @pytest.mark.parametrize("dtype,frac", [("bf16", 0.5), ("i8", 0.75), ("bf16", 0.0)])
 def test_tc_gemm_two_channel_groups_per_cta(dtype, frac):
-    """256 positions x 256 channels per CTA (what the largest products take: here 149 position tiles x 5 pairs of
-    channel groups keep the grid above two waves): nine channel groups, so the last CTA row has no second group; a last
-    half super-row; ragged last position tile."""
+    """Five channel tiles of 256 with 120 channels in the last, 297 position tiles with a ragged tail: every persistent CTA
+    takes ten tiles."""
     O, I, P = 1144, 96, 38000
     W = make_case(681, O, I, 1, 1, dtype)
     NB = (O // 8) * (I // 8)
@@ -128,33 +111,3 @@ def test_tc_gemm_two_channel_groups_per_cta(dtype, frac):
     got = gpu_gemm(lay, X, b, dtype)
     rp, ci, pl = ref.compact(W, gamma, 8, 8)
     check(got, ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b), dtype)
-
-
-def test_tc_config_resnet_conv_with_l2_gamma():
-    layer = synth.Layer("cfg2", 256, 256, 3, 3, 32, 14, 14, 1, 1, 1, 1)
-    W, X, b = synth.make_layer_tensors(layer, "bf16", config=2)
-    g, s, lay, Wd = gpu_mask(W, 8, 8, "bf16", 512)
-    lay.compact(Wd)
-    lay.check()
-    got = gpu_conv(lay, X, b, "bf16", (1, 1), (1, 1))
-    want_g = ref.mask(ref.scores(W, 8, 8), 512)
-    rp, ci, pl = ref.compact(W, want_g, 8, 8)
-    want = ref.conv2d(W.shape, 8, 8, rp, ci, pl, X, b, (1, 1), (1, 1))
-    check(got, want, "bf16")
-
-
-def test_tc_config_gemm_4096_sampled_rows():
-    O = I = 4096
-    P = 8192
-    W = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 0), (O, 1, 1, I), 1 / 64.0).astype(np.float32))
-    X = synth.round_to_bf16(synth.normal(synth.tensor_seed(3, 0, 1), (P, I)).astype(np.float32))
-    b = synth.normal(synth.tensor_seed(3, 0, 2), (O,), 0.1).astype(np.float32)
-    NB = (O // 8) * (I // 8)
-    g, s, lay, Wd = gpu_mask(W, 8, 8, "bf16", NB // 2)
-    lay.compact(Wd)
-    lay.check()
-    got = gpu_gemm(lay, X, b, "bf16")
-    pix = np.r_[0, 127, 128, P - 1, synth.uniform_int(7, (28,), 0, P - 1)]
-    rp, ci, pl = ref.compact(W, g, 8, 8)
-    want = ref.gemm(O, I, 8, 8, rp, ci, pl.reshape(-1, 8, 8), X, b, pix=pix)
-    check(got[pix], want, "bf16")
