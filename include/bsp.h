@@ -54,7 +54,7 @@ typedef enum {
 typedef enum { BSP_F32 = 0, BSP_BF16 = 1, BSP_I8 = 2, BSP_I32 = 3 } bsp_dtype;
 
 /* Block importance (Section "Predetermined Sparsity ratio and Full Training Ahead"). */
-typedef enum { BSP_NORM_L2 = 0, BSP_NORM_L1 = 1 } bsp_norm;
+typedef enum { BSP_NORM_L2 = 0, BSP_NORM_L1 = 1, BSP_NORM_VAR = 2 } bsp_norm;
 
 /* Which blocks compete when the lowest scores are zeroed.  LAYER: all NB_o*NB_i blocks are ranked
  * together (Section "Predetermined Sparsity ratio and Full Training Ahead").  ROW: each row of Gamma is ranked on its own and gets
@@ -92,7 +92,8 @@ typedef struct {
 } bsp_bcsr;
 
 /* ---- Gamma builder (Eq. (1), Eq. (2); Section "Predetermined Sparsity ratio ...") ------------------
- * score[l][iota] = sum of w^2 (L2, ranked by its square) or sum of |w| (L1) over the b_o x H x K x b_i
+ * score[l][iota] = sum of w^2 (L2, ranked by its square), sum of |w| (L1) or, for float weights, the variance
+ * of the block's entries about the block's own mean (VAR, n = b_o H K b_i) over the b_o x H x K x b_i
  * block; the n_zero blocks with the lowest (score, block index) pairs get Gamma = 0, all others 1.
  * Float weights: scores are float64, each product exact, summed over (h, k, c) for each output row r of
  * the block and then over r, always in that order, so that the mask is reproducible bit for bit.
@@ -102,7 +103,7 @@ typedef struct {
  *   gamma      [NB_o*NB_i] uint8 device, out
  *   scores_opt [NB_o*NB_i] float64 (float W) or int64 (int8 W) device, out; may be NULL
  *   ws         device scratch of bsp_mask_workspace_bytes() bytes
- * Errors: NULL, SHAPE, BLOCK, DTYPE (wtype I32), CAPACITY (n_zero out of range), CUDA. */
+ * Errors: NULL, SHAPE, BLOCK, DTYPE (wtype I32; VAR with int8 weights), CAPACITY (n_zero out of range), CUDA. */
 size_t bsp_mask_workspace_bytes(const bsp_wdesc *wd);
 bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope scope, int64_t n_zero,
                     uint8_t *gamma, void *scores_opt, void *ws, void *stream);

@@ -17,7 +17,8 @@
  *
  * Parity pins (tests/test_oracle_*.py): every function below is pinned against something other
  * than itself -- the paper's printed index example, Eq. (2) counts, numpy sort, a numpy/scipy
- * dense correlation of Gamma (.) W, closed forms and brute force on tiny shapes.
+ * dense correlation of Gamma (.) W, closed forms and brute force on tiny shapes; the requantising
+ * epilogue against hand-worked values and an exact rational restatement.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -428,5 +429,32 @@ int ref_dense_conv2d_i8(const ref_wdesc *w, const ref_xdesc *x, const int8_t *W,
             Y[p * w->O + o] = acc;
         }
     }
+    return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Requantising epilogue of the 8-bit path (Section "Compiler and its Code generation": an INT8
+ * tensor carries a power-of-two scale, "a position where the fraction starts"; weights 8 bits,
+ * bias 32 bits, scaling factors may differ per output channel; Eq. (quant) rounds to nearest).
+ * The int32 value v = accumulator + bias of output channel o stands at 2^-(f_x + f_w[o]); the int8
+ * output stands at 2^-f_y, so it is v / 2^s with s = shift[o] = f_x + f_w[o] - f_y >= 0, rounded
+ * to the nearest integer, halves away from zero, then saturated to [-128, 127].
+ * ------------------------------------------------------------------------------------------- */
+int ref_requant_i8(int64_t rows, int O, const int32_t *y32, const int32_t *shift, int8_t *y8)
+{
+    if (rows < 0 || O <= 0) return ORACLE_ERR_SHAPE;
+    for (int o = 0; o < O; ++o)
+        if (shift[o] < 0 || shift[o] > 31) return ORACLE_ERR_SHAPE;
+    for (int64_t p = 0; p < rows; ++p)
+        for (int o = 0; o < O; ++o) {
+            const int64_t v = (int64_t)y32[p * O + o];
+            const int s = shift[o];
+            int64_t mag = v < 0 ? -v : v;
+            if (s > 0) mag = (mag + ((int64_t)1 << (s - 1))) >> s;      /* nearest, halves away from zero */
+            int64_t q = v < 0 ? -mag : mag;
+            if (q > 127) q = 127;
+            if (q < -128) q = -128;
+            y8[p * O + o] = (int8_t)q;
+        }
     return ORACLE_OK;
 }

@@ -184,6 +184,17 @@ def gemm(O, I, bo, bi, row_ptr, col_idx, payload, X, bias=None, pix=None) -> np.
     return Y
 
 
+def requant_i8(y32: np.ndarray, shift: np.ndarray) -> np.ndarray:
+    """int32 [rows][O] (accumulator + bias) -> int8: value / 2^shift[o], nearest with halves away from zero, saturated."""
+    y32 = np.ascontiguousarray(y32, dtype=np.int32)
+    shift = np.ascontiguousarray(shift, dtype=np.int32)
+    rows, O = y32.shape
+    assert shift.shape == (O,)
+    y8 = np.empty((rows, O), dtype=np.int8)
+    _check(lib().ref_requant_i8(C.c_int64(rows), C.c_int(O), _p(y32), _p(shift), _p(y8)), "requant_i8")
+    return y8
+
+
 def dense_conv2d(W, X, bias=None, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     """Textbook dense convolution (cross-correlation) with bias; float64 or int64 [pixels][O]."""
     O, H, K, I = W.shape

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libbsp.so")
 
 OK, ERR_NULL, ERR_SHAPE, ERR_BLOCK, ERR_DTYPE, ERR_CAPACITY, ERR_INDEX, ERR_CUDA, ERR_TIMEOUT = range(9)
 F32, BF16, I8, I32 = 0, 1, 2, 3
-NORM_L2, NORM_L1 = 0, 1
+NORM_L2, NORM_L1, NORM_VAR = 0, 1, 2
 SCOPE_LAYER, SCOPE_ROW = 0, 1
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_mask_static", "bsp_packed_bytes",

@@ -64,7 +64,8 @@ bsp_status bsp_mask(const bsp_wdesc *wd, const void *W, bsp_norm norm, bsp_scope
     if (rc != BSP_OK) return rc;
     if (!W || !gamma || !ws) return BSP_ERR_NULL;
     if (!aligned4(W)) return BSP_ERR_SHAPE;
-    if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1) return BSP_ERR_DTYPE;
+    if (norm != BSP_NORM_L2 && norm != BSP_NORM_L1 && norm != BSP_NORM_VAR) return BSP_ERR_DTYPE;
+    if (norm == BSP_NORM_VAR && wd->wtype == BSP_I8) return BSP_ERR_DTYPE;      // the variance is defined for float weights
     if (scope != BSP_SCOPE_LAYER && scope != BSP_SCOPE_ROW) return BSP_ERR_DTYPE;
     const int64_t NBi = wd->I / wd->bi, NB = (int64_t)(wd->O / wd->bo) * NBi;
     const int64_t limit = (scope == BSP_SCOPE_LAYER) ? NB : NBi;

@@ -14,17 +14,28 @@ template <> struct Acc<BSP_F32> { using type = double; };
 template <> struct Acc<BSP_BF16> { using type = double; };
 template <> struct Acc<BSP_I8> { using type = long long; };
 
+// Measures of one weight: BSP_NORM_L2 (w^2), BSP_NORM_L1 (|w|), and for the variance two passes over the block:
+// kNormSum (w, for the block mean) and BSP_NORM_VAR ((w - mean)^2, with the subtraction, the product and the addition
+// each rounded on its own, never fused: the float64 result must not depend on what the compiler contracts).
+constexpr int kNormSum = 3;
+
+template <int NORM>
+__device__ __forceinline__ void add_value(double v, double &acc, double mean)
+{
+    if constexpr (NORM == BSP_NORM_L2) acc += v * v;
+    else if constexpr (NORM == BSP_NORM_L1) acc += fabs(v);
+    else if constexpr (NORM == kNormSum) acc += v;
+    else { const double d = __dsub_rn(v, mean); acc = __dadd_rn(acc, __dmul_rn(d, d)); }
+}
+
 template <int DT, int NORM>
-__device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc)
+__device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc, double mean)
 {
     if constexpr (DT == BSP_F32) {
-        const double v = (double)__uint_as_float(w);
-        acc += (NORM == BSP_NORM_L2) ? v * v : fabs(v);
+        add_value<NORM>((double)__uint_as_float(w), acc, mean);
     } else if constexpr (DT == BSP_BF16) {
-        const double v0 = (double)__uint_as_float(w << 16);
-        const double v1 = (double)__uint_as_float(w & 0xFFFF0000u);
-        acc += (NORM == BSP_NORM_L2) ? v0 * v0 : fabs(v0);
-        acc += (NORM == BSP_NORM_L2) ? v1 * v1 : fabs(v1);
+        add_value<NORM>((double)__uint_as_float(w << 16), acc, mean);
+        add_value<NORM>((double)__uint_as_float(w & 0xFFFF0000u), acc, mean);
     } else {
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
@@ -44,7 +55,8 @@ __device__ __forceinline__ void add_word(uint32_t w, typename Acc<DT>::type &acc
 // Loads of up to nine taps (a whole 3x3 kernel) are issued together, as 16-byte loads when `vec` says that the
 // rows are 16-byte aligned; the adds keep the (h, k, c) order.
 template <int DT, int NORM, int WORDS, int kBatch>
-__device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__restrict__ src, size_t row_words, int HK, bool vec)
+__device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__restrict__ src, size_t row_words, int HK, bool vec,
+                                                            double mean)
 {
     using acc_t = typename Acc<DT>::type;
     acc_t pr = 0;
@@ -78,7 +90,7 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__re
         for (int u = 0; u < kBatch; ++u)
 #pragma unroll
             for (int j = 0; j < WORDS; ++j)
-                if (t + u < HK) add_word<DT, NORM>(w[u][j], pr);
+                if (t + u < HK) add_word<DT, NORM>(w[u][j], pr, mean);
         src += (size_t)kBatch * row_words;
     }
     return pr;
@@ -88,7 +100,7 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum_w(const uint32_t *__re
 // one-tap layers, which then need few registers and keep many CTAs resident.
 template <int DT, int NORM, int kBatch>
 __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi,
-                                                          int NBi, long long B, int r)
+                                                          int NBi, long long B, int r, double mean = 0.0)
 {
     constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
     const int l = (int)(B / NBi), iota = (int)(B % NBi);
@@ -97,11 +109,11 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__rest
     const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
     const bool vec = (((uintptr_t)W) & 15u) == 0 && row_words % 4 == 0;
     switch (words) {
-        case 1: return row_sum_w<DT, NORM, 1, kBatch>(src, row_words, HK, vec);
-        case 2: return row_sum_w<DT, NORM, 2, kBatch>(src, row_words, HK, vec);
-        case 4: return row_sum_w<DT, NORM, 4, kBatch>(src, row_words, HK, vec);
-        case 8: return row_sum_w<DT, NORM, 8, kBatch>(src, row_words, HK, vec);
-        default: return row_sum_w<DT, NORM, 16, kBatch>(src, row_words, HK, vec);
+        case 1: return row_sum_w<DT, NORM, 1, kBatch>(src, row_words, HK, vec, mean);
+        case 2: return row_sum_w<DT, NORM, 2, kBatch>(src, row_words, HK, vec, mean);
+        case 4: return row_sum_w<DT, NORM, 4, kBatch>(src, row_words, HK, vec, mean);
+        case 8: return row_sum_w<DT, NORM, 8, kBatch>(src, row_words, HK, vec, mean);
+        default: return row_sum_w<DT, NORM, 16, kBatch>(src, row_words, HK, vec, mean);
     }
 }
 
@@ -117,6 +129,25 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
     const int r = threadIdx.x / blocks_per_cta;
     const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
     const long long NB = (long long)NBo * NBi;
+    if constexpr (NORM == BSP_NORM_VAR) {
+        // variance about the block's own mean, n = b_o H K b_i entries: the mean from the row sums added in order of r
+        // (every thread of the block adds them the same way), then the squared deviations in the same order, over n
+        const double n_elems = (double)bo * HK * bi;
+        part[threadIdx.x] = (B < NB) ? row_sum<DT, kNormSum, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+        __syncthreads();
+        double s = 0.0;
+        for (int q = 0; q < bo; ++q) s += (double)part[q * blocks_per_cta + bl];
+        const double mean = s / n_elems;
+        __syncthreads();
+        part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r, mean) : (acc_t)0;
+        __syncthreads();
+        if (B < NB && r == 0) {
+            double total = 0.0;
+            for (int q = 0; q < bo; ++q) total += (double)part[q * blocks_per_cta + bl];
+            score[B] = (acc_t)(total / n_elems);
+        }
+        return;
+    }
     part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
     __syncthreads();
     if (B < NB && r == 0) {
@@ -490,6 +521,14 @@ bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *s
     const int HK = wd.H * wd.K;
     const uint32_t *Wp = (const uint32_t *)W;
     acc_t *sc = (acc_t *)scores;
+    if constexpr (DT != BSP_I8) {
+        if (norm == BSP_NORM_VAR) {
+            if (HK == 1) score_kernel<DT, BSP_NORM_VAR, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+            else score_kernel<DT, BSP_NORM_VAR, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+            BSP_CUDA_OK(cudaGetLastError());
+            return BSP_OK;
+        }
+    }
     if (norm == BSP_NORM_L2) {
         if (HK == 1) score_kernel<DT, BSP_NORM_L2, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
         else score_kernel<DT, BSP_NORM_L2, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
@@ -509,7 +548,7 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
     bsp_status rc;
     {
         const long long NB = (long long)(wd.O / wd.bo) * (wd.I / wd.bi);
-        if (ws != nullptr && NB <= kRankMax) {
+        if (ws != nullptr && NB <= kRankMax && norm != BSP_NORM_VAR) {     // (the variance takes the two-pass score kernel)
             const int seg_len = (int)((scope == BSP_SCOPE_LAYER) ? NB : wd.I / wd.bi);
             int *status = (int *)ws;
             unsigned *sync = (unsigned *)ws + kWsSyncWord;

@@ -174,3 +174,33 @@ def test_mask_then_compact_round_trip_to_masked_dense():
         for n in range(rp[l], rp[l + 1]):
             back[l * bo:(l + 1) * bo, :, :, ci[n] * bi:(ci[n] + 1) * bi] = pl[n]
     assert rp[-1] == 512 and np.array_equal(back, ref.apply_mask(W, g, bo, bi))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("bo,bi", SHAPES)
+@pytest.mark.parametrize("H,K,O,I", [(3, 3, 96, 160), (1, 1, 256, 512), (1, 7, 32, 64)])
+def test_variance_scores_and_gamma_bit_exact(dtype, bo, bi, H, K, O, I):
+    """Variance importance (float weights): blocks get their own offsets so that the mean matters and the ranking
+    differs from the L2 one; scores are compared as bit patterns (the kernel keeps the oracle's order of the sums and
+    rounds the subtraction, the square and the addition one by one), Gamma bit for bit."""
+    W = make_case(131, O, I, H, K, dtype)
+    NBo, NBi = O // bo, I // bi
+    shift = synth.normal(132, (NBo, NBi), 0.05).astype(np.float32)
+    W = W + np.repeat(np.repeat(shift, bo, axis=0), bi, axis=1)[:, None, None, :]
+    W = synth.round_to_bf16(W.astype(np.float32)) if dtype == "bf16" else W.astype(np.float32)
+    want_s = ref.scores(W, bo, bi, ref.NORM_VAR)
+    NB = NBo * NBi
+    g, s, _, _ = gpu_mask(W, bo, bi, dtype, NB // 2, bsp.NORM_VAR)
+    assert np.array_equal(s.view(np.uint64), want_s.view(np.uint64))
+    want_g = ref.mask(want_s, NB // 2)
+    assert np.array_equal(g, want_g)
+    assert not np.array_equal(want_g, ref.mask(ref.scores(W, bo, bi, ref.NORM_L2), NB // 2))
+    g_row, _, _, _ = gpu_mask(W, bo, bi, dtype, 3, bsp.NORM_VAR, bsp.SCOPE_ROW)
+    assert np.array_equal(g_row, ref.mask(want_s, 3, ref.SCOPE_ROW))
+
+
+def test_variance_of_int8_weights_is_refused():
+    W = make_case(133, 64, 64, 1, 1, "i8")
+    with pytest.raises(bsp.BspError) as e:
+        gpu_mask(W, 8, 8, "i8", 4, bsp.NORM_VAR)
+    assert e.value.status == bsp.ERR_DTYPE
