@@ -178,6 +178,21 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
                       const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream);
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd);
 
+/* ---- 8-bit products with a requantised int8 output (Section "Compiler and its Code generation": an INT8 tensor
+ * carries a power-of-two scale, weights are 8 bits, the bias 32 bits, scales may differ per output channel; the
+ * round-to-nearest of Eq. (quant)) -----------------------------------------------------------------------------
+ * The same products as bsp_gemm / bsp_conv2d on I8 weights and activations, with the epilogue
+ *   Y[.., o] = saturate_int8( round( (accumulator + bias[o]) / 2^shift[o] ) ),
+ * rounded to the nearest integer with halves away from zero, saturated to [-128, 127].  With X at scale 2^-f_x, the
+ * weights of channel o at 2^-f_w[o] (bias at their product) and Y at 2^-f_y the shift is f_x + f_w[o] - f_y.
+ *   bias   int32 [O] device, may be NULL      shift  int32 [O] device, every entry in 0..31 (only the low 5 bits are read)
+ *   Y      int8, NHWC / [P][O]; O must be a multiple of 16 (rows of Y are 16-byte multiples)
+ * Errors: as bsp_conv2d; NULL shift; DTYPE if the weights are not I8. */
+bsp_status bsp_gemm_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const int32_t *bias,
+                       const int32_t *shift, int8_t *Y, void *ws, void *stream);
+bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                         const int32_t *bias, const int32_t *shift, int8_t *Y, void *ws, void *stream);
+
 /* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
  * (BSP_OK if none), then clears it. */
 bsp_status bsp_check(void *ws, void *stream);

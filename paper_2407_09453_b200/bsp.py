@@ -22,7 +22,7 @@ SCOPE_LAYER, SCOPE_ROW = 0, 1
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_mask_static", "bsp_packed_bytes",
            "bsp_compact_workspace_bytes", "bsp_compact_nnz", "bsp_compact", "bsp_conv_workspace_bytes", "bsp_gemm",
-           "bsp_conv2d", "bsp_conv_kernel_name", "bsp_check", "bsp_status_string"]
+           "bsp_conv2d", "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv_kernel_name", "bsp_check", "bsp_status_string"]
 
 
 class BspError(RuntimeError):
@@ -62,7 +62,7 @@ def lib():
         L.bsp_status_string.restype = C.c_char_p
         L.bsp_conv_kernel_name.restype = C.c_char_p
         for n in ("bsp_mask", "bsp_mask_static", "bsp_compact_nnz", "bsp_compact", "bsp_gemm", "bsp_conv2d",
-                  "bsp_check"):
+                  "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_check"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -149,6 +149,16 @@ def bsp_conv2d(wd: WDesc, w: Bcsr, xd: XDesc, X, bias, Y, ytype, ws, stream=None
                             _ptr(ws), _stream(stream)), "bsp_conv2d")
 
 
+def bsp_conv2d_q8(wd: WDesc, w: Bcsr, xd: XDesc, X, bias, shift, Y, ws, stream=None):
+    _raise(lib().bsp_conv2d_q8(C.byref(wd), C.byref(w), C.byref(xd), _ptr(X), _ptr(bias), _ptr(shift), _ptr(Y), _ptr(ws),
+                               _stream(stream)), "bsp_conv2d_q8")
+
+
+def bsp_gemm_q8(wd: WDesc, w: Bcsr, X, P, bias, shift, Y, ws, stream=None):
+    _raise(lib().bsp_gemm_q8(C.byref(wd), C.byref(w), _ptr(X), C.c_int64(P), _ptr(bias), _ptr(shift), _ptr(Y), _ptr(ws),
+                             _stream(stream)), "bsp_gemm_q8")
+
+
 def bsp_mask_static(wd: WDesc, W, norm, scope, n_zero, gamma, stream=None):
     _raise(lib().bsp_mask_static(C.byref(wd), _ptr(W), C.c_int(norm), C.c_int(scope), C.c_int64(n_zero), _ptr(gamma),
                                  _stream(stream)), "bsp_mask_static")
@@ -214,6 +224,14 @@ class SparseLayer:
 
     def gemm(self, X, bias, Y, stream=None):
         bsp_gemm(self.wd, self.handle(), X, X.shape[0], bias, Y, dtype_code(Y.dtype), self.ws, stream)
+
+    def conv2d_q8(self, X, bias, shift, Y, stride=(1, 1), pad=(0, 0), stream=None):
+        N, L, J, _ = X.shape
+        xd = XDesc(N, L, J, stride[0], stride[1], pad[0], pad[1])
+        bsp_conv2d_q8(self.wd, self.handle(), xd, X, bias, shift, Y, self.ws, stream)
+
+    def gemm_q8(self, X, bias, shift, Y, stream=None):
+        bsp_gemm_q8(self.wd, self.handle(), X, X.shape[0], bias, shift, Y, self.ws, stream)
 
     def check(self, stream=None):
         bsp_check(self.ws, stream)

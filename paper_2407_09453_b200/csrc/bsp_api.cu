@@ -124,8 +124,10 @@ size_t bsp_conv_workspace_bytes(const bsp_wdesc *wd, const bsp_xdesc *xd)
     return kWsHeader;
 }
 
-bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
-                      const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
+namespace {
+// Validation and launch shared by bsp_conv2d and bsp_conv2d_q8 (shift != NULL: int8 output).
+bsp_status conv2d_any(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X, const void *bias,
+                      const int32_t *shift, void *Y, bsp_dtype ytype, void *ws, void *stream)
 {
     bsp_status rc = check_wdesc(wd);
     if (rc != BSP_OK) return rc;
@@ -136,14 +138,42 @@ bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *x
     if (xd->L + 2 * xd->pad_h < wd->H || xd->J + 2 * xd->pad_w < wd->K) return BSP_ERR_SHAPE;
     if (wd->O % 8 != 0 || wd->I % 8 != 0) return BSP_ERR_SHAPE;
     if (wd->wtype == BSP_I8 && wd->I % 16 != 0) return BSP_ERR_SHAPE;   // rows of X must be 16-byte multiples
-    if (wd->wtype == BSP_I8) { if (ytype != BSP_I32) return BSP_ERR_DTYPE; }
+    if (wd->wtype == BSP_I8) { if (ytype != BSP_I32 && ytype != BSP_I8) return BSP_ERR_DTYPE; }
     else if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
+    if (ytype == BSP_I8 && wd->O % 16 != 0) return BSP_ERR_SHAPE;       // rows of an int8 Y must be 16-byte multiples
     if (!aligned16(X) || !aligned16(Y) || !aligned16(w->packed)) return BSP_ERR_SHAPE;
+    if (shift && !aligned4(shift)) return BSP_ERR_SHAPE;
     // the packed header is on the device (the kernel checks it against the descriptor); the host checks the count
     const int64_t NB = (int64_t)(wd->O / wd->bo) * (wd->I / wd->bi);
     if (w->nnz < 0 || w->nnz > NB) return BSP_ERR_INDEX;
     if (!gemm_tc_eligible(*wd, *xd, ytype)) return BSP_ERR_SHAPE;
-    return launch_gemm_tc(*wd, *xd, w->packed, X, bias, Y, ytype, ws, (cudaStream_t)stream);
+    return launch_gemm_tc(*wd, *xd, w->packed, X, bias, shift, Y, ytype, ws, (cudaStream_t)stream);
+}
+}  // namespace
+
+bsp_status bsp_conv2d(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                      const void *bias, void *Y, bsp_dtype ytype, void *ws, void *stream)
+{
+    if (ytype == BSP_I8) return BSP_ERR_DTYPE;           // an int8 output needs its shifts: bsp_conv2d_q8
+    return conv2d_any(wd, w, xd, X, bias, nullptr, Y, ytype, ws, stream);
+}
+
+bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
+                         const int32_t *bias, const int32_t *shift, int8_t *Y, void *ws, void *stream)
+{
+    if (!shift) return BSP_ERR_NULL;
+    if (wd && wd->wtype != BSP_I8) return BSP_ERR_DTYPE;
+    return conv2d_any(wd, w, xd, X, bias, shift, Y, BSP_I8, ws, stream);
+}
+
+bsp_status bsp_gemm_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const int32_t *bias,
+                       const int32_t *shift, int8_t *Y, void *ws, void *stream)
+{
+    if (!wd) return BSP_ERR_NULL;
+    if (wd->H != 1 || wd->K != 1) return BSP_ERR_SHAPE;
+    if (P <= 0 || P > 0x7FFFFFFF) return BSP_ERR_SHAPE;
+    bsp_xdesc xd = {(int)P, 1, 1, 1, 1, 0, 0};
+    return bsp_conv2d_q8(wd, w, &xd, X, bias, shift, Y, ws, stream);
 }
 
 const char *bsp_conv_kernel_name(const bsp_wdesc *wd, const bsp_xdesc *xd)

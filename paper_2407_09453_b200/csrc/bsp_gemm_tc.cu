@@ -41,6 +41,7 @@ struct GtParams {
     CUtensorMap tmw;          // Gamma (.) W as bytes: (I * esz, H K, O), box 128 bytes x 1 tap x BN channels, 128-byte swizzle
     CUtensorMap tmy;          // Y as bytes: (O * ey, P), box 128 bytes x 32 positions, 128-byte swizzle (store_tma only)
     const void *bias;         // float32 or int32 [O], may be NULL
+    const int32_t *shift;     // int8 output only: right shift per output channel, 0..31
     const uint8_t *packed;
     int *status;
     int O, I, P, H, K, bo, bi, wtype, ytype;
@@ -111,6 +112,16 @@ __device__ __forceinline__ void gt_commit_elected(uint32_t bar)
 {
     asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
                  " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
+}
+
+// Requantisation of the 8-bit path (Section "Compiler and its Code generation", Eq. (quant)): v / 2^s rounded to the
+// nearest integer, halves away from zero, saturated to int8.
+__device__ __forceinline__ uint32_t gt_requant(int v, uint32_t s)
+{
+    const uint32_t mag = v < 0 ? 0u - (uint32_t)v : (uint32_t)v;        // at most 2^31
+    const uint32_t r = s ? (mag + (1u << (s - 1u))) >> s : mag;          // no overflow: mag + 2^30 < 2^32
+    const int q = v < 0 ? -(int)min(r, 128u) : (int)min(r, 127u);
+    return (uint32_t)q & 0xFFu;
 }
 
 // First output position (image, row, column) of position tile mt.
@@ -296,6 +307,24 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                             for (int e = 0; e < 32; ++e)
                                 out[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, e)));
                         }
+                    } else if (ey == 1) {                        // int8 output: 128 channels, requantised after the bias
+#pragma unroll
+                        for (int sub = 0; sub < 4; ++sub) {
+                            uint32_t v[32];
+                            gt_load32(tbase + (uint32_t)(c0 + sub * 32), v);
+                            const int ch = n0 + c0 + sub * 32 + lane;
+                            const uint32_t bl = gt_bias(p, ch);
+                            const uint32_t sl = ch < p.O ? (uint32_t)__ldg(p.shift + ch) & 31u : 0u;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                uint32_t w = 0u;
+#pragma unroll
+                                for (int b = 0; b < 4; ++b)
+                                    w |= gt_requant((int)v[4 * e + b] + (int)__shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
+                                                    __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b)) << (8 * b);
+                                out[sub * 8 + e] = w;
+                            }
+                        }
                     } else {                                     // bf16 output: 64 channels, rounded to nearest even after the bias
 #pragma unroll
                         for (int sub = 0; sub < 2; ++sub) {
@@ -324,9 +353,11 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                         __syncwarp();
                         // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
-                        if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
-                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
-                                         ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
+                        // (every round commits a group, an empty one when nothing is stored: the wait above counts rounds)
+                        if (lane == 0) {
+                            if (n0 + c0 < p.O && m0 + q * 32 < p.P)
+                                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
+                                             ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
                             asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
                         }
                     } else {
@@ -425,8 +456,8 @@ bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd0, bsp_dtype ytype
 {
     const bsp_xdesc xd = gt_flatten(wd, xd0);
     if (!packed_layout(wd).enabled) return false;
-    if (ytype != BSP_F32 && ytype != BSP_BF16 && ytype != BSP_I32) return false;
-    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    if (ytype != BSP_F32 && ytype != BSP_BF16 && ytype != BSP_I32 && ytype != BSP_I8) return false;
+    const int ey = ytype == BSP_BF16 ? 2 : (ytype == BSP_I8 ? 1 : 4);
     if (((long long)wd.O * ey) % 16 != 0) return false;
     const int M = (xd.L + 2 * xd.pad_h - wd.H) / xd.stride_h + 1, Nw = (xd.J + 2 * xd.pad_w - wd.K) / xd.stride_w + 1;
     if (M <= 0 || Nw <= 0) return false;
@@ -436,16 +467,17 @@ bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd0, bsp_dtype ytype
 }
 
 bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void *packed, const void *X,
-                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
+                          const void *bias, const int32_t *shift, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
 {
     const bsp_xdesc xd = gt_flatten(wd, xd0);
     const PackedLayout L = packed_layout(wd);
     if (!L.enabled) return BSP_ERR_SHAPE;
     const int esz = elem_bytes(wd.wtype);
-    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    const int ey = ytype == BSP_BF16 ? 2 : (ytype == BSP_I8 ? 1 : 4);
     const int HK = wd.H * wd.K;
+    if (ytype == BSP_I8 && shift == nullptr) return BSP_ERR_NULL;
     GtParams p = {};
-    p.bias = bias; p.packed = (const uint8_t *)packed;
+    p.bias = bias; p.shift = shift; p.packed = (const uint8_t *)packed;
     p.status = (int *)ws;
     p.O = wd.O; p.I = wd.I; p.H = wd.H; p.K = wd.K; p.bo = wd.bo; p.bi = wd.bi;
     p.wtype = wd.wtype; p.ytype = ytype; p.ey = ey; p.Y = (uint8_t *)Y;
@@ -461,7 +493,8 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.a_bytes = p.rows_tile * 128;
     // a tile of 128 rows that are consecutive in Y (whole images, or the positions of a matrix product) is stored by TMA
     p.store_tma = (T.Wt == p.Nw && T.Ht == p.M && p.rows_tile == kGtBM) ? 1 : 0;
-    p.BN = gemm_tile_n(wd.O);
+    // (a staging round of the int8 output covers 128 channels, so those tiles are multiples of 128 channels)
+    p.BN = ytype == BSP_I8 ? (gemm_tile_n(wd.O) + 127) / 128 * 128 : gemm_tile_n(wd.O);
     p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
     if (T.tiles * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
     p.n_tiles = (int)(T.tiles * p.n_tiles_n);

@@ -58,7 +58,7 @@ void report_cuda_error(cudaError_t e, const char *expr, const char *file, int li
 
 bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype);
 bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
-                          const void *bias, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
+                          const void *bias, const int32_t *shift, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
 // Output channels per CTA tile of the product kernel (a multiple of 64, at most 256).
 inline int gemm_tile_n(int O)
 {

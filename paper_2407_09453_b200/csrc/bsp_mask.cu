@@ -236,7 +236,7 @@ select_kernel(const unsigned long long *__restrict__ key, long long seg_len, lon
 // counts arrivals and is reset by the last arriver, `sync[1]` is a generation that the last arriver bumps.
 // Thread 0 of each CTA takes part (release on arrival, acquire on the generation; the CTA barriers around it
 // extend both to the other threads); the wait is bounded.  Returns false if it expired.
-constexpr unsigned kGridSpinLimit = 1u << 24;
+constexpr unsigned kGridSpinLimit = 1u << 22;
 __device__ __forceinline__ bool grid_barrier(unsigned *sync)
 {
     __shared__ int s_bar_ok;

@@ -204,3 +204,24 @@ def test_variance_of_int8_weights_is_refused():
     with pytest.raises(bsp.BspError) as e:
         gpu_mask(W, 8, 8, "i8", 4, bsp.NORM_VAR)
     assert e.value.status == bsp.ERR_DTYPE
+
+
+def test_bounded_wait_runs_out_and_the_workspace_recovers():
+    """A wait that nothing can satisfy ends by itself: the arrival word of the grid barrier in the workspace header is
+    preset (by the host: the contract says it starts at zero) so that no CTA of the one-launch Gamma builder ever counts
+    as the last arriver.  Every CTA's bounded wait expires, the kernel returns, bsp_check reports BSP_ERR_TIMEOUT once and
+    clears the barrier words, and the next call on the same workspace is bit-exact."""
+    W = make_case(141, 128, 128, 3, 3, "bf16")
+    lay = bsp.SparseLayer(128, 128, 3, 3, 8, 8, torch.bfloat16)
+    Wd = to_dev(W, "bf16")
+    lay.ws.view(torch.int32)[2] = 0x40000000          # arrivals so far: far more than any grid
+    lay.mask(Wd, 128)
+    with pytest.raises(bsp.BspError) as e:
+        lay.check()
+    assert e.value.status == bsp.ERR_TIMEOUT
+    assert lay.ws.view(torch.int32)[:4].abs().sum().item() == 0      # status and barrier words cleared by bsp_check
+    lay.check()
+    lay.mask(Wd, 128)
+    lay.check()
+    want = ref.mask(ref.scores(W, 8, 8), 128)
+    assert np.array_equal(from_dev(lay.gamma).reshape(16, 16), want)

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import ref
 from paper_2407_09453_b200 import bsp, build, synth
 
 
@@ -53,5 +54,8 @@ def test_static_variant_matches_workspace_variant_twice_in_a_row():
         assert rc == bsp.OK
         torch.cuda.synchronize()
         assert torch.equal(got, want)                                # masks are compared bit for bit
+        Wh = W.float().cpu().numpy() if dt != torch.int8 else W.cpu().numpy()
+        oracle = ref.mask(ref.scores(Wh, bo, bi), n_zero, ref.SCOPE_LAYER if scope == bsp.SCOPE_LAYER else ref.SCOPE_ROW)
+        assert np.array_equal(got.cpu().numpy().reshape(oracle.shape), oracle)      # and with the CPU oracle
         zeros = int((got == 0).sum())
         assert zeros == (n_zero if scope == bsp.SCOPE_LAYER else n_zero * (O // bo))
