@@ -493,8 +493,31 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.a_bytes = p.rows_tile * 128;
     // a tile of 128 rows that are consecutive in Y (whole images, or the positions of a matrix product) is stored by TMA
     p.store_tma = (T.Wt == p.Nw && T.Ht == p.M && p.rows_tile == kGtBM) ? 1 : 0;
-    // (a staging round of the int8 output covers 128 channels, so those tiles are multiples of 128 channels)
-    p.BN = ytype == BSP_I8 ? (gemm_tile_n(wd.O) + 127) / 128 * 128 : gemm_tile_n(wd.O);
+    static bool opted[kGtMaxDevices] = {};
+    static int n_sm[kGtMaxDevices] = {};
+    int dev = 0;
+    BSP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
+    if (!opted[dev]) {
+        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
+        opted[dev] = true;
+    }
+    // Channels per tile: the widest tile keeps the tensor pipe busiest (a stage costs about 256 + 2 BN cycles of operand
+    // fetch from shared memory), but a layer with few position tiles fills more SMs with narrower ones: the width with
+    // the lowest waves x stage cost wins.  (A staging round of the int8 output covers 128 channels, so those tiles are
+    // multiples of 128 channels.)
+    {
+        const int step = ytype == BSP_I8 ? 128 : 64;
+        const int widest = (gemm_tile_n(wd.O) + step - 1) / step * step;
+        long long best_cost = -1;
+        for (int bn = widest; bn >= step; bn -= step) {
+            if (bn != widest && bn != 128 && bn != 64) continue;
+            const long long tiles = T.tiles * ((wd.O + bn - 1) / bn);
+            const long long cost = ((tiles + n_sm[dev] - 1) / n_sm[dev]) * (256 + 2 * bn);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.BN = bn; }
+        }
+    }
     p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
     if (T.tiles * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
     p.n_tiles = (int)(T.tiles * p.n_tiles_n);
@@ -542,16 +565,6 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
             return BSP_ERR_CUDA;
     }
 
-    static bool opted[kGtMaxDevices] = {};
-    static int n_sm[kGtMaxDevices] = {};
-    int dev = 0;
-    BSP_CUDA_OK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
-    if (!opted[dev]) {
-        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
-        BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
-        opted[dev] = true;
-    }
     const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
     gemm_tc_kernel<<<grid, kGtThreads, smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
