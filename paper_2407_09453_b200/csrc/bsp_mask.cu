@@ -380,7 +380,7 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
 // Small segments (up to kRankMax keys): the keys sit in shared memory and every thread counts the (key, index)
 // pairs below its own, which is its rank in the ascending order; Gamma = 0 for ranks below n_zero.  Same
 // result as the radix select, in one pass instead of nine.
-constexpr int kRankMax = 2048;
+constexpr int kRankMax = 4096;
 constexpr int kRankThreads = 256;
 constexpr int kRankLanes = 8;            // lanes sharing one key; each counts an eighth of the segment
 __global__ void __launch_bounds__(kRankThreads)
