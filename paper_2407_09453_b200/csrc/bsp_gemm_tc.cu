@@ -1,18 +1,22 @@
-// Block-sparse matrix product Y[p][o] = b[o] + sum over kept blocks of W-bar X (a fully connected layer, or a 1x1
-// convolution without padding or stride, over P positions) on 5th-generation tensor cores: tcgen05.mma with the
-// accumulators in tensor memory, bf16 -> fp32 (kind::f16), int8 -> int32 (kind::i8) and fp32 as TF32 -> fp32
-// (kind::tf32).  Introduction (Y = W*X + b) and Section "Block Sparsity in a Matrix" of the paper ("GEMM is a 1x1
-// convolution").
+// Block-sparse products Y = W*X + b on 5th-generation tensor cores, one kernel for all of them: the matrix product
+// Y[p][o] = b[o] + sum over kept blocks of W-bar X (a fully connected layer, "GEMM is a 1x1 convolution") and the NHWC
+// convolution with any taps, strides and zero padding, as an implicit GEMM.  tcgen05.mma with the accumulators in
+// tensor memory: bf16 -> fp32 (kind::f16), int8 -> int32 (kind::i8), fp32 as TF32 -> fp32 (kind::tf32); fused bias;
+// fp32, bf16, int32 or requantised int8 output.  Introduction (Y = W*X + b), Section "Block Sparsity in a Matrix" and
+// Section "Compiler and its Code generation" (8-bit tensors with power-of-two scales) of the paper.
 //
-// The kernel reads the third packed form: Gamma (.) W-bar as a plain K-major [O][I] matrix (zeroed blocks stored as
-// zeros), so that both operands arrive by tiled TMA loads under the 128-byte swizzle.  A persistent CTA owns tiles of
-// 128 positions x BN output channels (BN <= 256).  Per K-stage (128 bytes of input channels) one thread issues the
-// two loads (128 x 128 bytes of X, BN x 128 bytes of weights); one elected lane of the MMA warp issues four MMAs of
-// 128 x BN x 32 bytes; two accumulator buffers of 256 columns let the epilogue of a tile (tensor memory -> registers
-// -> + bias -> convert -> swizzled shared memory -> TMA store) overlap the MMAs of the next one.  The arithmetic
-// skips nothing: a tensor-core instruction covers 128 x BN x 16 entries of the operands at once, far more than a
-// block, and feeding it compact blocks (cp.async expansion of the block-CSR payload in shared memory, or TMA gather
-// loads of 128-byte cores) was measured two to four times slower than these dense loads.
+// The kernel reads the packed form Gamma (.) W in the layout of W, [O][H][K][I] (zeroed blocks stored as zeros), so
+// that both operands arrive by tiled TMA loads under the 128-byte swizzle.  A persistent CTA owns tiles of up to 128
+// output positions (a box of Wt x Ht positions of Nt images; 128 consecutive positions for a matrix product) x BN
+// output channels (BN <= 256).  The reduction runs over taps x 128-byte chunks of input channels: per K-stage one
+// thread issues two loads, the activation box shifted by the tap (out-of-bounds positions arrive as zeros: the
+// padding; strides are the tensor map's element strides) and BN x 128 bytes of that tap's weights; one elected lane
+// of the MMA warp issues four MMAs of 128 x BN x 32 bytes; two accumulator buffers of 256 columns let the epilogue of
+// a tile (tensor memory -> registers -> + bias -> convert -> swizzled shared memory -> global memory, by TMA store
+// when the tile's rows are consecutive in Y) overlap the MMAs of the next one.  The arithmetic skips nothing: a
+// tensor-core instruction covers 128 x BN x 16 entries of the operands at once, far more than a block, and feeding it
+// compact blocks (cp.async expansion of the block-CSR payload in shared memory, or TMA gather loads of 128-byte
+// cores) was measured two to five times slower than these dense loads.
 //
 // Warps: 0 producer (one thread), 1 MMA issuer (the whole warp runs the loop so that its address arithmetic stays
 // warp-uniform), 2-5 epilogue (warp w reads the tensor-memory lanes 32 (w % 4) ..).  Barriers per stage: full (one
