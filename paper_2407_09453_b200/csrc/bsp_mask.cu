@@ -117,6 +117,8 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__rest
     }
 }
 
+// A CTA takes groups of 256 / b_o blocks, every `gridDim.x`-th one (a bounded grid of long-lived CTAs instead of one
+// short CTA per group: a layer of 4096 x 4096 weights is 8192 groups).
 template <int DT, int NORM, int kBatch>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
@@ -127,33 +129,37 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
     const int blocks_per_cta = kScoreThreads / bo;
     const int bl = threadIdx.x % blocks_per_cta;
     const int r = threadIdx.x / blocks_per_cta;
-    const long long B = (long long)blockIdx.x * blocks_per_cta + bl;
     const long long NB = (long long)NBo * NBi;
-    if constexpr (NORM == BSP_NORM_VAR) {
-        // variance about the block's own mean, n = b_o H K b_i entries: the mean from the row sums added in order of r
-        // (every thread of the block adds them the same way), then the squared deviations in the same order, over n
-        const double n_elems = (double)bo * HK * bi;
-        part[threadIdx.x] = (B < NB) ? row_sum<DT, kNormSum, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
-        __syncthreads();
-        double s = 0.0;
-        for (int q = 0; q < bo; ++q) s += (double)part[q * blocks_per_cta + bl];
-        const double mean = s / n_elems;
-        __syncthreads();
-        part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r, mean) : (acc_t)0;
-        __syncthreads();
-        if (B < NB && r == 0) {
-            double total = 0.0;
-            for (int q = 0; q < bo; ++q) total += (double)part[q * blocks_per_cta + bl];
-            score[B] = (acc_t)(total / n_elems);
+    const long long n_groups = (NB + blocks_per_cta - 1) / blocks_per_cta;
+    for (long long grp = blockIdx.x; grp < n_groups; grp += gridDim.x) {
+        const long long B = grp * blocks_per_cta + bl;
+        if constexpr (NORM == BSP_NORM_VAR) {
+            // variance about the block's own mean, n = b_o H K b_i entries: the mean from the row sums added in order of
+            // r (every thread of the block adds them the same way), then the squared deviations in the same order, over n
+            const double n_elems = (double)bo * HK * bi;
+            part[threadIdx.x] = (B < NB) ? row_sum<DT, kNormSum, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+            __syncthreads();
+            double s = 0.0;
+            for (int q = 0; q < bo; ++q) s += (double)part[q * blocks_per_cta + bl];
+            const double mean = s / n_elems;
+            __syncthreads();
+            part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r, mean) : (acc_t)0;
+            __syncthreads();
+            if (B < NB && r == 0) {
+                double total = 0.0;
+                for (int q = 0; q < bo; ++q) total += (double)part[q * blocks_per_cta + bl];
+                score[B] = (acc_t)(total / n_elems);
+            }
+        } else {
+            part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
+            __syncthreads();
+            if (B < NB && r == 0) {
+                acc_t total = 0;
+                for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
+                score[B] = total;
+            }
         }
-        return;
-    }
-    part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
-    __syncthreads();
-    if (B < NB && r == 0) {
-        acc_t total = 0;
-        for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
-        score[B] = total;
+        __syncthreads();
     }
 }
 
@@ -268,70 +274,134 @@ __device__ __forceinline__ bool grid_barrier(unsigned *sync)
 // derives the digit for itself.  Keys equal to the threshold T are zeroed lowest index first: the CTAs publish
 // how many such keys their slices hold (geq[c]), meet again, and each counts those in the slices before its own.
 constexpr int kCoopThreads = 512;
+constexpr int kLocalMax = 2048;          // candidates that the CTAs finish on their own, in shared memory
+
+// The digit d of a 256-bin histogram with cum(d - 1) < need <= cum(d), found by the first warp: each lane sums eight
+// bins, a warp scan finds the lane, the lane walks its bins.  Writes the remaining count, the extended prefix and the
+// number of keys in the chosen bin; the caller synchronises the CTA afterwards.
+__device__ __forceinline__ void select_digit(const unsigned *hist, int tid, unsigned long long prefix, long long *s_k,
+                                             unsigned long long *s_prefix, unsigned *s_left, int width)
+{
+    if (tid >= 32) return;
+    const long long need = *s_k;
+    long long mine = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) mine += hist[tid * 8 + q];
+    long long inc = mine;
+#pragma unroll
+    for (int dd = 1; dd < 32; dd <<= 1) {
+        const long long n = __shfl_up_sync(0xFFFFFFFFu, inc, dd);
+        if (tid >= dd) inc += n;
+    }
+    const unsigned reach = __ballot_sync(0xFFFFFFFFu, inc >= need);
+    const int owner = reach ? __ffs(reach) - 1 : 31;        // need <= total, so some lane reaches it
+    if (tid == owner) {
+        long long cum = inc - mine;
+        int d = tid * 8;
+        for (; d < tid * 8 + 7; ++d) {
+            if (cum + (long long)hist[d] >= need) break;
+            cum += hist[d];
+        }
+        *s_k = need - cum;
+        *s_prefix = (prefix << width) | (unsigned long long)d;
+        *s_left = hist[d];
+    }
+}
+
+// The select starts at the highest bit in which any two keys differ (one grid-wide OR of key ^ key[0]: the bits above
+// it are the same in every key, e.g. the sign and most of the exponent of float scores, or the leading zero bytes of
+// integer ones) and takes digits of eight bits downwards.  Passes run grid-wide (global histograms, a grid barrier
+// each) only while more than kLocalMax keys still match the prefix; then the CTAs append their matching keys to one
+// list (`cand`, counted in gcount[0]; the OR sits in gcount[2..3]; both zeroed by the host with the histograms), meet
+// once, and every CTA finishes the remaining digits on the list in its own shared memory.
 __global__ void __launch_bounds__(kCoopThreads)
 select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long long n_zero, uint8_t *__restrict__ gamma,
-                   unsigned *ghist, unsigned *geq, unsigned *sync, int *status)
+                   unsigned *ghist, unsigned *gcount, unsigned long long *cand, unsigned *geq, unsigned *sync, int *status)
 {
     __shared__ unsigned hist[256];
+    __shared__ unsigned long long s_cand[kLocalMax];
     __shared__ unsigned long long s_prefix;
     __shared__ long long s_k;
+    __shared__ unsigned s_left;
     __shared__ unsigned warp_cnt[kCoopThreads / 32];
     __shared__ long long s_run;
     const int tid = threadIdx.x;
     const long long slice = (n + gridDim.x - 1) / gridDim.x;
     const long long lo = (long long)blockIdx.x * slice, hi = min(n, lo + slice);
-    if (tid == 0) { s_prefix = 0ull; s_k = n_zero; }
-    for (int pass = 7; pass >= 0; --pass) {
+    const unsigned long long k0 = key[0];
+    {
+        unsigned long long d = 0ull;
+        for (long long i = lo + tid; i < hi; i += kCoopThreads) d |= key[i] ^ k0;
+        for (int o = 16; o > 0; o >>= 1) d |= __shfl_xor_sync(0xFFFFFFFFu, d, o);
+        if ((tid & 31) == 0 && d) atomicOr((unsigned long long *)(gcount + 2), d);
+    }
+    if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
+    const unsigned long long diff = __ldcg((const unsigned long long *)(gcount + 2));
+    // bits above `top` are common to all keys: they are the prefix so far (all keys equal: nothing left to select)
+    int top = diff ? 63 - __clzll((long long)diff) : -1;
+    if (tid == 0) { s_prefix = top >= 63 ? 0ull : (k0 >> (top + 1)); s_k = n_zero; s_left = 0xFFFFFFFFu; }
+    int pi = 0;
+    while (top >= 0) {
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
+        if (s_left <= (unsigned)kLocalMax) break;          // few enough candidates: the rest is local
         const unsigned long long prefix = s_prefix;
-        const int shift = 8 * pass;
-        // lanes with the same digit add once (the leading digits of float keys are nearly all alike)
+        const int width = min(8, top + 1), shift = top + 1 - width;
+        const unsigned dmask = (1u << width) - 1u;
+        // lanes with the same digit add once
         for (long long base = lo; base < hi; base += kCoopThreads) {
             const long long i = base + tid;
             unsigned long long v = 0ull;
             bool in = false;
             if (i < hi) {
                 v = key[i];
-                in = (pass == 7) || ((v >> (shift + 8)) == prefix);
+                in = top >= 63 || ((v >> (top + 1)) == prefix);
             }
-            const unsigned digit = in ? (unsigned)((v >> shift) & 0xFFull) : 256u;
+            const unsigned digit = in ? ((unsigned)(v >> shift) & dmask) : 256u;
             const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
             if (in && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
         }
         __syncthreads();
-        if (tid < 256 && hist[tid]) atomicAdd(&ghist[pass * 256 + tid], hist[tid]);
+        if (tid < 256 && hist[tid]) atomicAdd(&ghist[pi * 256 + tid], hist[tid]);
         if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
-        if (tid < 256) hist[tid] = __ldcg(&ghist[pass * 256 + tid]);
+        if (tid < 256) hist[tid] = __ldcg(&ghist[pi * 256 + tid]);
         __syncthreads();
-        if (tid < 32) {
-            // the digit d with cum(d - 1) < need <= cum(d): each lane sums eight bins, a warp scan finds the lane, the
-            // lane walks its bins
-            const long long need = s_k;
-            long long mine = 0;
-#pragma unroll
-            for (int q = 0; q < 8; ++q) mine += hist[tid * 8 + q];
-            long long inc = mine;
-#pragma unroll
-            for (int dd = 1; dd < 32; dd <<= 1) {
-                const long long n = __shfl_up_sync(0xFFFFFFFFu, inc, dd);
-                if (tid >= dd) inc += n;
-            }
-            const unsigned reach = __ballot_sync(0xFFFFFFFFu, inc >= need);
-            const int owner = reach ? __ffs(reach) - 1 : 31;        // need <= total, so some lane reaches it
-            if (tid == owner) {
-                long long cum = inc - mine;
-                int d = tid * 8;
-                for (; d < tid * 8 + 7; ++d) {
-                    if (cum + (long long)hist[d] >= need) break;
-                    cum += hist[d];
-                }
-                s_k = need - cum;
-                s_prefix = (prefix << 8) | (unsigned long long)d;
+        select_digit(hist, tid, prefix, &s_k, &s_prefix, &s_left, width);
+        __syncthreads();
+        top -= width;
+        ++pi;
+    }
+    if (top >= 0) {
+        // bits top .. 0 are still open: gather the keys that match the prefix, then finish locally
+        const unsigned long long prefix = s_prefix;
+        for (long long i = lo + tid; i < hi; i += kCoopThreads) {
+            const unsigned long long v = key[i];
+            if ((v >> (top + 1)) == prefix) {          // (top < 63 here: at least one digit has been taken)
+                const unsigned at = atomicAdd(gcount, 1u);
+                if (at < (unsigned)kLocalMax) cand[at] = v;
             }
         }
+        if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
+        const unsigned cnt = min(__ldcg(gcount), (unsigned)kLocalMax);
+        for (unsigned i = tid; i < cnt; i += kCoopThreads) s_cand[i] = __ldcg(&cand[i]);
         __syncthreads();
+        while (top >= 0) {
+            if (tid < 256) hist[tid] = 0u;
+            __syncthreads();
+            const unsigned long long pre = s_prefix;
+            const int width = min(8, top + 1), shift = top + 1 - width;
+            const unsigned dmask = (1u << width) - 1u;
+            for (unsigned i = tid; i < cnt; i += kCoopThreads) {
+                const unsigned long long v = s_cand[i];
+                if ((v >> (top + 1)) == pre) atomicAdd(&hist[(unsigned)(v >> shift) & dmask], 1u);
+            }
+            __syncthreads();
+            select_digit(hist, tid, pre, &s_k, &s_prefix, &s_left, width);
+            __syncthreads();
+            top -= width;
+        }
     }
+    __syncthreads();
     const unsigned long long T = s_prefix;
     const long long ties = s_k;        // keys equal to T to zero, lowest indices first
     // keys equal to T in this slice
@@ -517,7 +587,8 @@ bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *s
     const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
     const long long NB = (long long)NBo * NBi;
     const int per_cta = kScoreThreads / wd.bo;
-    const unsigned grid = (unsigned)((NB + per_cta - 1) / per_cta);
+    const long long groups = (NB + per_cta - 1) / per_cta;
+    const unsigned grid = (unsigned)(groups < 148 * 8 ? groups : 148 * 8);       // eight CTAs per SM's worth, each looping
     const int HK = wd.H * wd.K;
     const uint32_t *Wp = (const uint32_t *)W;
     acc_t *sc = (acc_t *)scores;
@@ -588,13 +659,15 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
         if (grid > sm_count[dev]) grid = sm_count[dev];
         if (grid > kSelectMaxCtas) grid = kSelectMaxCtas;
         unsigned *ghist = (unsigned *)((char *)ws + kWsHeader + align_up((size_t)NB * 8, 256));
-        unsigned *geq = ghist + 8 * 256;
-        BSP_CUDA_OK(cudaMemsetAsync(ghist, 0, 8 * 256 * sizeof(unsigned), st));
+        unsigned *gcount = ghist + 8 * 256;                      // candidate counter (4 words kept for alignment)
+        unsigned *geq = gcount + 4;
+        unsigned long long *cand = (unsigned long long *)(geq + kSelectMaxCtas);
+        BSP_CUDA_OK(cudaMemsetAsync(ghist, 0, (8 * 256 + 4) * sizeof(unsigned), st));
         const unsigned long long *keys = (const unsigned long long *)scores;
         long long n = seg, nz = n_zero;
         unsigned *sync = (unsigned *)ws + kWsSyncWord;
         int *status = (int *)ws;
-        void *args[] = {&keys, &n, &nz, &gamma, &ghist, &geq, &sync, &status};
+        void *args[] = {&keys, &n, &nz, &gamma, &ghist, &gcount, &cand, &geq, &sync, &status};
         const cudaError_t e = cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, 0, st);
         if (e == cudaErrorCooperativeLaunchTooLarge) {
             (void)cudaGetLastError();
