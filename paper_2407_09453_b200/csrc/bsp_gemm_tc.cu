@@ -49,7 +49,7 @@ struct GtParams {
     const uint8_t *packed;
     int *status;
     int O, I, P, H, K, bo, bi, wtype, ytype;
-    int BN, n_tiles_n, n_tiles, n_ks;
+    int BN, n_tiles_n, n_tiles, n_tile_pairs, n_ks;
     int stages, stage_bytes;
     // position tiles: Wt x Ht output positions of Nt images (at most 128), tiles_x x tiles_y of them per Nt images
     int N, M, Nw, Wt, Ht, Nt, tiles_x, tiles_y, rows_tile;
@@ -92,30 +92,56 @@ constexpr uint64_t kGtDesc = (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1u
 // The four MMAs of one stage and the commit that releases the stage, issued by one elected lane of a converged warp.
 // All lanes execute this statement with the same operands; the MMA of the first K-step overwrites the accumulator
 // when `acc` is 0.
-#define GT_ISSUE_STAGE(KIND)                                                                                        \
+#define GT_ISSUE_STAGE(KIND, CG, COMMIT_TAIL)                                                                       \
     asm volatile("{\n .reg .pred e, p, t;\n .reg .b64 a1, a2, a3, b1, b2, b3;\n"                                     \
                  " elect.sync _|e, 0xFFFFFFFF;\n setp.ne.b32 p, %5, 0;\n setp.eq.b32 t, %5, %5;\n"                    \
                  " add.u64 a1, %1, 2;\n add.u64 a2, %1, 4;\n add.u64 a3, %1, 6;\n"                                    \
                  " add.u64 b1, %2, 2;\n add.u64 b2, %2, 4;\n add.u64 b3, %2, 6;\n"                                    \
-                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], %1, %2, %3, p;\n"                                 \
-                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a1, b1, %3, t;\n"                                 \
-                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a2, b2, %3, t;\n"                                 \
-                 " @e tcgen05.mma.cta_group::1.kind::" KIND " [%0], a3, b3, %3, t;\n"                                 \
-                 " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%4];\n}\n"               \
-                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(bar_empty), "r"(acc) : "memory")
+                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], %1, %2, %3, p;\n"                                 \
+                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a1, b1, %3, t;\n"                                 \
+                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a2, b2, %3, t;\n"                                 \
+                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a3, b3, %3, t;\n"                                 \
+                 " @e tcgen05.commit.cta_group::" CG ".mbarrier::arrive::one.shared::cluster" COMMIT_TAIL ";\n}\n"        \
+                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(bar_empty), "r"(acc), "h"((unsigned short)3) : "memory")
 
+// kPair: the MMAs span a pair of CTAs (cta_group::2, M = 256: each CTA its own 128 positions and half of the weight
+// tile); the commits then arrive on the barrier at the same shared-memory offset in both CTAs.
+template <bool kPair>
 __device__ __forceinline__ void gt_issue_stage(int wtype, uint32_t d, uint64_t da, uint64_t db, uint32_t idesc,
                                                uint32_t bar_empty, uint32_t acc)
 {
-    if (wtype == BSP_BF16) GT_ISSUE_STAGE("f16");
-    else if (wtype == BSP_I8) GT_ISSUE_STAGE("i8");
-    else GT_ISSUE_STAGE("tf32");
+    if constexpr (kPair) {
+        if (wtype == BSP_BF16) GT_ISSUE_STAGE("f16", "2", ".multicast::cluster.b64 [%4], %6");
+        else if (wtype == BSP_I8) GT_ISSUE_STAGE("i8", "2", ".multicast::cluster.b64 [%4], %6");
+        else GT_ISSUE_STAGE("tf32", "2", ".multicast::cluster.b64 [%4], %6");
+    } else {
+        if (wtype == BSP_BF16) GT_ISSUE_STAGE("f16", "1", ".b64 [%4]");
+        else if (wtype == BSP_I8) GT_ISSUE_STAGE("i8", "1", ".b64 [%4]");
+        else GT_ISSUE_STAGE("tf32", "1", ".b64 [%4]");
+    }
 }
-// All MMAs issued so far by the elected lane complete -> one arrival on `bar`.
+// All MMAs issued so far by the elected lane complete -> one arrival on `bar` (in both CTAs of a pair).
+template <bool kPair>
 __device__ __forceinline__ void gt_commit_elected(uint32_t bar)
 {
-    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
-                 " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
+    if constexpr (kPair)
+        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                     " @e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n}\n"
+                     ::"r"(bar), "h"((unsigned short)3) : "memory");
+    else
+        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                     " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
+}
+
+// Synchronises the CTA (the two CTAs of a pair).
+template <bool kPair>
+__device__ __forceinline__ void gt_sync_all()
+{
+    if constexpr (kPair) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+    } else {
+        __syncthreads();
+    }
 }
 
 // Requantisation of the 8-bit path (Section "Compiler and its Code generation", Eq. (quant)): v / 2^s rounded to the
@@ -154,6 +180,7 @@ __device__ __forceinline__ uint32_t gt_bias(const GtParams &p, int ch)
     return (p.bias != nullptr && ch < p.O) ? __ldg((const uint32_t *)p.bias + ch) : 0u;
 }
 
+template <bool kPair>
 __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_constant__ GtParams p)
 {
     extern __shared__ __align__(16) uint8_t gt_smem_raw[];
@@ -167,6 +194,18 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
     const int S = p.stages, n_ks = p.n_ks, BN = p.BN;
     const uint32_t ring = sm32(smem);
     const uint32_t staging = ring + (uint32_t)(S * p.stage_bytes);
+    // Work items: tiles, or for CTA pairs two position tiles side by side on one channel tile (CTA r of the pair takes
+    // position tile 2 mp + r; a pair past an odd count loads zeros and stores nothing).
+    uint32_t rank = 0;
+    if constexpr (kPair) asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(rank));
+    const int t_first = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, t_step = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int t_count = kPair ? p.n_tile_pairs : p.n_tiles;
+    // barriers of the pair's leader (CTA 0), as shared::cluster addresses
+    uint32_t lead_full0 = sm32(&s_full[0]), lead_acc_empty0 = sm32(&s_acc_empty[0]);
+    if constexpr (kPair) {
+        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;\n" : "=r"(lead_full0) : "r"(sm32(&s_full[0])));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;\n" : "=r"(lead_acc_empty0) : "r"(sm32(&s_acc_empty[0])));
+    }
 
     if (tid == 0) {
         // the packed buffer must be the one bsp_compact filled for this descriptor, with the masked dense form in it
@@ -181,7 +220,7 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
         }
         for (int b = 0; b < 2; ++b) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc_full[b])), "r"(1) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc_empty[b])), "r"(4) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc_empty[b])), "r"(kPair ? 8 : 4) : "memory");
         }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmx) : "memory");
@@ -189,11 +228,16 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmy) : "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        if constexpr (kPair) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;\n" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-    __syncthreads();
+    gt_sync_all<kPair>();                   // (a pair: both CTAs' barriers are initialised before either signals the other)
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem = s_tmem;
     const bool run = s_fail == 0u;
@@ -202,13 +246,16 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
         // ================= producer =================
         if (lane == 0 && run) {
             const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
-            const uint32_t stage_bytes = (uint32_t)p.stage_bytes, tx = (uint32_t)(p.a_bytes + BN * 128);
+            // (a pair: each CTA loads its own activation box and its half of the weight tile, all four loads announce their
+            // bytes on the leader's barrier, which the leader arms with the total)
+            const uint32_t stage_bytes = (uint32_t)p.stage_bytes;
+            const uint32_t tx = (uint32_t)(p.a_bytes + (BN >> (kPair ? 1 : 0)) * 128) * (kPair ? 2u : 1u);
             uint32_t slot = 0, round = 0, issued = 0, dst = ring;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-                const int ch0 = (tile % p.n_tiles_n) * BN;
+            for (int tile = t_first; tile < t_count && ok; tile += t_step) {
+                const int ch0 = (tile % p.n_tiles_n) * BN + (kPair ? (int)rank * (BN >> 1) : 0);
                 int n0, y0, x0;
-                gt_tile_origin(p, tile / p.n_tiles_n, n0, y0, x0);
+                gt_tile_origin(p, kPair ? 2 * (tile / p.n_tiles_n) + (int)rank : tile / p.n_tiles_n, n0, y0, x0);
                 // input position of the tile's first output position at tap (0, 0); a tap is a shift of the box, positions
                 // outside the image read as zeros (the padding)
                 const int xi0 = x0 * p.sw - p.pw, yi0 = y0 * p.sh - p.ph;
@@ -216,12 +263,21 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                     for (int c = 0; c < p.cpt; ++c) {
                         if (round && !gt_poll(empty0 + slot * 8u, (round & 1u) ^ 1u)) { ok = false; break; }
                         if (s_fail) { ok = false; break; }
+                        if constexpr (kPair) {
+                            const uint32_t bar = lead_full0 + slot * 8u;
+                            if (rank == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(full0 + slot * 8u), "r"(tx) : "memory");
+                            asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+                                         ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(c * 128), "r"(xi0 + k), "r"(yi0 + h), "r"(n0) : "memory");
+                            asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
+                                         ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(c * 128), "r"(tap), "r"(ch0) : "memory");
+                        } else {
                         const uint32_t bar = full0 + slot * 8u;
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
                         asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
                                      ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(c * 128), "r"(xi0 + k), "r"(yi0 + h), "r"(n0) : "memory");
                         asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
                                      ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(c * 128), "r"(tap), "r"(ch0) : "memory");
+                        }
                         ++issued;
                         if (++slot == (uint32_t)S) { slot = 0; ++round; dst = ring; } else dst += stage_bytes;
                     }
@@ -232,7 +288,9 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                 // winding down after a wait that ran out: the loads already issued still write into this CTA's shared
                 // memory, so the barriers of the stages in flight are awaited (bounded) before the CTA may leave
                 atomicExch((uint32_t *)&s_fail, 1u);
-                for (uint32_t back = 0; back < (uint32_t)S && back < issued; ++back) {
+                // (the follower of a pair has no barrier of its own to watch: its loads announce themselves to the leader;
+                // both CTAs meet at the cluster barrier before they leave)
+                for (uint32_t back = 0; back < (uint32_t)S && back < issued && rank == 0; ++back) {
                     const uint32_t it = issued - 1u - back;
                     gt_poll(full0 + (it % (uint32_t)S) * 8u, (it / (uint32_t)S) & 1u);
                 }
@@ -241,15 +299,16 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
     } else if (warp == 1) {
         // ================= MMA issuer =================
         // The whole warp runs the loop (so that its address arithmetic stays warp-uniform); one elected lane issues.
-        if (run) {
-            // instruction descriptor: D fp32 (int32 for int8), A and B bf16 / signed int8 / tf32, K-major both, M = 128, N = BN
+        if (run && rank == 0) {               // (of a pair, the leader issues for both CTAs)
+            // instruction descriptor: D fp32 (int32 for int8), A and B bf16 / signed int8 / tf32, K-major both, M = 128
+            // (256 over a pair), N = BN
             const uint32_t dfmt = p.wtype == BSP_I8 ? 2u : 1u, abfmt = p.wtype == BSP_F32 ? 2u : 1u;
-            const uint32_t idesc = (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc = (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(BN >> 3) << 17) | (((kPair ? 256u : 128u) >> 4) << 24);
             const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
             uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_i) {
+            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
                 if (use && !gt_poll(sm32(&s_acc_empty[buf]), (use & 1u) ^ 1u)) ok = false;
                 ok = __all_sync(0xFFFFFFFFu, ok);
@@ -262,10 +321,10 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                     if (!got) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
-                    gt_issue_stage(p.wtype, d, da, db, idesc, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    gt_issue_stage<kPair>(p.wtype, d, da, db, idesc, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
                     if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                 }
-                if (ok) gt_commit_elected(sm32(&s_acc_full[buf]));
+                if (ok) gt_commit_elected<kPair>(sm32(&s_acc_full[buf]));
             }
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
@@ -279,12 +338,12 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             const uint32_t stg0 = staging + (uint32_t)(ew * 2 * kGtStagingBytes);
             uint32_t tile_i = 0, rounds_done = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_i) {
+            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
                 const int n0 = (tile % p.n_tiles_n) * BN;
                 // this lane's row of the tile: position (w, h, image i) of the tile's box, w fastest
                 int in0, y0, x0;
-                gt_tile_origin(p, tile / p.n_tiles_n, in0, y0, x0);
+                gt_tile_origin(p, kPair ? 2 * (tile / p.n_tiles_n) + (int)rank : tile / p.n_tiles_n, in0, y0, x0);
                 const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
                 const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
                 // byte offset of the row in Y (rows of O * ey bytes); m0: the tile's first row when rows are consecutive
@@ -387,7 +446,12 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                 // the accumulator buffer has been read: hand it back to the MMA issuer
                 asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
                 __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc_empty[buf])) : "memory");
+                if (lane == 0) {
+                    if constexpr (kPair)
+                        asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(lead_acc_empty0 + buf * 8u) : "memory");
+                    else
+                        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc_empty[buf])) : "memory");
+                }
             }
             if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
@@ -396,9 +460,12 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
 
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-    __syncthreads();
+    gt_sync_all<kPair>();                   // (a pair: neither CTA leaves while the other may still signal its barriers)
     if (s_fail == 1u && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kGtTmemCols) : "memory");
+    if (warp == 0) {
+        if constexpr (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kGtTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kGtTmemCols) : "memory");
+    }
 }
 
 typedef CUresult (*GtEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -503,7 +570,8 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     BSP_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
     if (!opted[dev]) {
-        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
         BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
         opted[dev] = true;
     }
@@ -525,9 +593,13 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
     if (T.tiles * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
     p.n_tiles = (int)(T.tiles * p.n_tiles_n);
+    // Large products run on CTA pairs: two position tiles side by side on one 256-channel tile, every CTA loading its
+    // own activations and half of the weights (the operand fetch per SM and MMA falls from 12 KB to 8 KB).
+    const bool pair = p.BN == 256 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
+    p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
     p.cpt = (int)(((long long)wd.I * esz + 127) / 128);
     p.n_ks = HK * p.cpt;
-    p.stage_bytes = kGtABytes + p.BN * 128;
+    p.stage_bytes = kGtABytes + (pair ? p.BN / 2 : p.BN) * 128;
     const int staging = 4 * 2 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
     if (stages > kGtMaxStages) stages = kGtMaxStages;
@@ -552,7 +624,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
         const cuuint64_t row = (cuuint64_t)wd.I * esz;
         const cuuint64_t gdim[3] = {row, (cuuint64_t)HK, (cuuint64_t)wd.O};
         const cuuint64_t gstr[2] = {row, row * HK};
-        const cuuint32_t box[3] = {128, 1, (cuuint32_t)p.BN};
+        const cuuint32_t box[3] = {128, 1, (cuuint32_t)(pair ? p.BN / 2 : p.BN)};
         const cuuint32_t estr[3] = {1, 1, 1};
         if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed + L.off_payload), gdim, gstr, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -569,8 +641,22 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
             return BSP_ERR_CUDA;
     }
 
+    if (pair) {
+        cudaLaunchConfig_t cfg = {};
+        const int pairs = p.n_tile_pairs < n_sm[dev] / 2 ? p.n_tile_pairs : n_sm[dev] / 2;
+        cfg.gridDim = dim3((unsigned)(2 * pairs));
+        cfg.blockDim = dim3(kGtThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        BSP_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, p));
+        return BSP_OK;
+    }
     const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
-    gemm_tc_kernel<<<grid, kGtThreads, smem, st>>>(p);
+    gemm_tc_kernel<false><<<grid, kGtThreads, smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }
