@@ -595,10 +595,11 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.n_tiles = (int)(T.tiles * p.n_tiles_n);
     // Large products run on CTA pairs: two position tiles side by side on one 256-channel tile, every CTA loading its
     // own activations and half of the weights (the operand fetch per SM and MMA falls from 12 KB to 8 KB).
-    const bool pair = p.BN == 256 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
-    p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
+    // (Tiles of a few K-stages are bound by their epilogue, and there the pair's cross-CTA hand-shakes only cost.)
     p.cpt = (int)(((long long)wd.I * esz + 127) / 128);
     p.n_ks = HK * p.cpt;
+    const bool pair = p.BN == 256 && p.n_ks >= 8 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
+    p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
     p.stage_bytes = kGtABytes + (pair ? p.BN / 2 : p.BN) * 128;
     const int staging = 4 * 2 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
