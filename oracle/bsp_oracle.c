@@ -458,3 +458,67 @@ int ref_requant_i8(int64_t rows, int O, const int32_t *y32, const int32_t *shift
         }
     return ORACLE_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Block-sparse x block-sparse product (Section "Block-Sparse Matrix-Matrix Multiplication"):
+ *   C = (Gamma . A) (Omega . B)^t,   C_{i,j} = sum_k gamma_{i,k} A_{i,k} (omega_{j,k} B_{j,k})^t
+ * with kb x kb blocks.  A and B are stored as compressed block rows (only blocks with a one in
+ * their mask), so the block-column indices of row i of A and of row j of B are two ascending
+ * lists; a product is formed exactly where both lists hold the same k: the lists are merged.
+ * C is dense, [NBa*kb][NBb*kb], float64.
+ * ------------------------------------------------------------------------------------------- */
+int ref_spgemm_f32(int NBa, int NBb, int kb, const int32_t *a_row_ptr, const int32_t *a_col_idx,
+                   const float *a_payload, const int32_t *b_row_ptr, const int32_t *b_col_idx,
+                   const float *b_payload, double *C)
+{
+    if (NBa <= 0 || NBb <= 0 || kb <= 0) return ORACLE_ERR_SHAPE;
+    const size_t ldc = (size_t)NBb * kb;
+    for (int i = 0; i < NBa; ++i)
+        for (int j = 0; j < NBb; ++j) {
+            for (int r = 0; r < kb; ++r)
+                for (int c = 0; c < kb; ++c) C[((size_t)i * kb + r) * ldc + (size_t)j * kb + c] = 0.0;
+            int32_t pa = a_row_ptr[i], pb = b_row_ptr[j];
+            while (pa < a_row_ptr[i + 1] && pb < b_row_ptr[j + 1]) {
+                if (a_col_idx[pa] < b_col_idx[pb]) ++pa;
+                else if (a_col_idx[pa] > b_col_idx[pb]) ++pb;
+                else {
+                    const float *Ab = a_payload + (size_t)pa * kb * kb, *Bb = b_payload + (size_t)pb * kb * kb;
+                    for (int r = 0; r < kb; ++r)
+                        for (int c = 0; c < kb; ++c) {
+                            double acc = 0.0;
+                            for (int t = 0; t < kb; ++t) acc += (double)Ab[r * kb + t] * (double)Bb[c * kb + t];
+                            C[((size_t)i * kb + r) * ldc + (size_t)j * kb + c] += acc;
+                        }
+                    ++pa; ++pb;
+                }
+            }
+        }
+    return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Relative column index (Section "Block Sparsity in a Matrix": "a relative row/col index"): within
+ * each row of Gamma the first kept block keeps its column, every further one stores its distance
+ * to the previous kept block of the row.  Distances are >= 1; both directions are given.
+ * ------------------------------------------------------------------------------------------- */
+int ref_index_to_relative(int NBo, const int32_t *row_ptr, const int32_t *col_idx, int32_t *rel)
+{
+    if (NBo <= 0) return ORACLE_ERR_SHAPE;
+    for (int l = 0; l < NBo; ++l)
+        for (int32_t n = row_ptr[l]; n < row_ptr[l + 1]; ++n)
+            rel[n] = (n == row_ptr[l]) ? col_idx[n] : col_idx[n] - col_idx[n - 1];
+    return ORACLE_OK;
+}
+
+int ref_index_from_relative(int NBo, const int32_t *row_ptr, const int32_t *rel, int32_t *col_idx)
+{
+    if (NBo <= 0) return ORACLE_ERR_SHAPE;
+    for (int l = 0; l < NBo; ++l) {
+        int32_t at = 0;
+        for (int32_t n = row_ptr[l]; n < row_ptr[l + 1]; ++n) {
+            at = (n == row_ptr[l]) ? rel[n] : at + rel[n];
+            col_idx[n] = at;
+        }
+    }
+    return ORACLE_OK;
+}

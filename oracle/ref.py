@@ -195,6 +195,38 @@ def requant_i8(y32: np.ndarray, shift: np.ndarray) -> np.ndarray:
     return y8
 
 
+def spgemm(kb, a, b) -> np.ndarray:
+    """C = (Gamma . A)(Omega . B)^t from two compact forms (row_ptr, col_idx, payload [nnz][kb][kb]) with kb x kb blocks;
+    dense float64 [NBa*kb][NBb*kb]."""
+    (arp, aci, apl), (brp, bci, bpl) = a, b
+    NBa, NBb = len(arp) - 1, len(brp) - 1
+    apl = np.ascontiguousarray(apl, dtype=np.float32).reshape(-1, kb, kb)
+    bpl = np.ascontiguousarray(bpl, dtype=np.float32).reshape(-1, kb, kb)
+    Cm = np.empty((NBa * kb, NBb * kb), dtype=np.float64)
+    _check(lib().ref_spgemm_f32(C.c_int(NBa), C.c_int(NBb), C.c_int(kb),
+                                _p(np.ascontiguousarray(arp, dtype=np.int32)), _p(np.ascontiguousarray(aci, dtype=np.int32)), _p(apl),
+                                _p(np.ascontiguousarray(brp, dtype=np.int32)), _p(np.ascontiguousarray(bci, dtype=np.int32)), _p(bpl),
+                                _p(Cm)), "spgemm_f32")
+    return Cm
+
+
+def index_to_relative(row_ptr, col_idx) -> np.ndarray:
+    """Relative column index of a compact form: first kept block of a row absolute, the others as distances."""
+    row_ptr = np.ascontiguousarray(row_ptr, dtype=np.int32)
+    col_idx = np.ascontiguousarray(col_idx, dtype=np.int32)
+    rel = np.empty_like(col_idx)
+    _check(lib().ref_index_to_relative(C.c_int(len(row_ptr) - 1), _p(row_ptr), _p(col_idx), _p(rel)), "index_to_relative")
+    return rel
+
+
+def index_from_relative(row_ptr, rel) -> np.ndarray:
+    row_ptr = np.ascontiguousarray(row_ptr, dtype=np.int32)
+    rel = np.ascontiguousarray(rel, dtype=np.int32)
+    col = np.empty_like(rel)
+    _check(lib().ref_index_from_relative(C.c_int(len(row_ptr) - 1), _p(row_ptr), _p(rel), _p(col)), "index_from_relative")
+    return col
+
+
 def dense_conv2d(W, X, bias=None, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     """Textbook dense convolution (cross-correlation) with bias; float64 or int64 [pixels][O]."""
     O, H, K, I = W.shape
