@@ -362,6 +362,36 @@ def pass_layers(gpu, bsp, torch, layers, dtype, sparsities, pk, ydt, with_setup,
     return out
 
 
+def pass_spgemm(gpu, bsp, torch, reps=5):
+    """Block-sparse x block-sparse product C = (Gamma . A)(Omega . B)^t, 2048 x 4096 times (2048 x 4096)^t, bf16 8x8 blocks,
+    magnitude masks at 50 % and 75 %: useful FLOPs are those of the block pairs that both masks keep.  The kernel runs on
+    the fp32 pipes (8 x 8 x 8 products), so its roofline is the fp32 FMA rate: 148 SMs x 128 lanes x 2 x 1.965 GHz."""
+    peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    out = []
+    g = torch.Generator(device="cuda")
+    g.manual_seed(77)
+    O, I = 2048, 4096
+    A = (torch.randn((O, 1, 1, I), device="cuda", generator=g) / 64).to(torch.bfloat16)
+    B = (torch.randn((O, 1, 1, I), device="cuda", generator=g) / 64).to(torch.bfloat16)
+    Cm = torch.empty((O, O), dtype=torch.float32, device="cuda")
+    la = bsp.SparseLayer(O, I, 1, 1, 8, 8, torch.bfloat16)
+    lb = bsp.SparseLayer(O, I, 1, 1, 8, 8, torch.bfloat16)
+    NB = la.NBo * la.NBi
+    for s in (0.5, 0.75):
+        for lay, W in ((la, A), (lb, B)):
+            lay.mask(W, int(s * NB + 0.5))
+            lay.compact(W)
+        st = stats(gpu.timed(lambda: bsp.bsp_spgemm(la.wd, la.handle(), lb.wd, lb.handle(), Cm, la.ws), reps, 1))
+        la.check()
+        ga = la.gamma.view(la.NBo, la.NBi).float()
+        gb = lb.gamma.view(lb.NBo, lb.NBi).float()
+        pairs = float((ga @ gb.t()).sum().item())             # block pairs that both masks keep
+        fl = 2.0 * 512 * pairs
+        out.append({"sparsity": s, **st, "useful_flops": fl, "tflops": fl / (st["ms"] * 1e-3) / 1e12,
+                    "roofline": {"bound": "alu", "peak": peak, "unit": "TFLOP/s", "frac": fl / (st["ms"] * 1e-3) / 1e12 / peak}})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -543,6 +573,7 @@ def main():
             "layers": i8, "note": "int8 -> int32, bsp_mask, bsp_compact and the product each timed on their own",
             "sum_ms": {str(s): {k: float(sum(r[k] * r["count"] for r in i8 if r["sparsity"] == s))
                                 for k in ("mask_ms", "compact_ms", "conv_ms", "step_ms")} for s in (0.5, 0.75)}}
+        sweeps["spgemm_2048x4096_bf16_8x8"] = pass_spgemm(gpu, bsp, torch)
     clocks = sampler.stop()
 
     # max over ranks

@@ -193,6 +193,24 @@ bsp_status bsp_gemm_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, in
 bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                          const int32_t *bias, const int32_t *shift, int8_t *Y, void *ws, void *stream);
 
+/* ---- Block-sparse x block-sparse product (Section "Block-Sparse Matrix-Matrix Multiplication") and the relative column
+ * index (Section "Block Sparsity in a Matrix": "a relative row/col index") ------------------------------------------
+ * bsp_spgemm: C = (Gamma . A)(Omega . B)^t, i.e. C_{i,j} = sum over the block columns k that row i of A and row j of B
+ *             both keep of A_{i,k} B_{j,k}^t.  A is wa->O x wa->I, B is wb->O x wb->I with the same I, both with H = K = 1,
+ *             8x8 blocks and the same type (F32 or BF16); `a` and `b` are their compact forms from bsp_compact (row_ptr,
+ *             col_idx and the canonical payload are read; `packed` is not).  C is dense float32 [wa->O][wb->O], 8-byte
+ *             aligned, written in full (blocks without a common column are zero).  Products are accumulated in float32
+ *             in ascending order of k.  A column index outside the matrix is skipped and latches BSP_ERR_INDEX.
+ *             ws: any workspace of at least 256 bytes (status word only).
+ * bsp_index_to_relative / bsp_index_from_relative: within each row of Gamma the first kept block keeps its column, every
+ *             further one stores its distance (>= 1) to the previous kept block of the row; and back.  int32 in, int32
+ *             out, [nnz] device arrays; row_ptr [NB_o + 1] as written by bsp_compact.
+ * Errors: NULL, SHAPE (I differs, H K != 1, more than 12288 block columns), BLOCK (not 8x8), DTYPE, CUDA. */
+bsp_status bsp_spgemm(const bsp_wdesc *wa, const bsp_bcsr *a, const bsp_wdesc *wb, const bsp_bcsr *b, float *C, void *ws,
+                      void *stream);
+bsp_status bsp_index_to_relative(int NBo, const int32_t *row_ptr, const int32_t *col_idx, int32_t *rel, void *stream);
+bsp_status bsp_index_from_relative(int NBo, const int32_t *row_ptr, const int32_t *rel, int32_t *col_idx, void *stream);
+
 /* Synchronises `stream` and returns the status latched in the workspace by the kernels that used it
  * (BSP_OK if none), then clears it. */
 bsp_status bsp_check(void *ws, void *stream);

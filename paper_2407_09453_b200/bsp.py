@@ -22,7 +22,8 @@ SCOPE_LAYER, SCOPE_ROW = 0, 1
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_mask_static", "bsp_packed_bytes",
            "bsp_compact_workspace_bytes", "bsp_compact_nnz", "bsp_compact", "bsp_conv_workspace_bytes", "bsp_gemm",
-           "bsp_conv2d", "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv_kernel_name", "bsp_check", "bsp_status_string"]
+           "bsp_conv2d", "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv_kernel_name", "bsp_spgemm",
+           "bsp_index_to_relative", "bsp_index_from_relative", "bsp_check", "bsp_status_string"]
 
 
 class BspError(RuntimeError):
@@ -62,7 +63,7 @@ def lib():
         L.bsp_status_string.restype = C.c_char_p
         L.bsp_conv_kernel_name.restype = C.c_char_p
         for n in ("bsp_mask", "bsp_mask_static", "bsp_compact_nnz", "bsp_compact", "bsp_gemm", "bsp_conv2d",
-                  "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_check"):
+                  "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_spgemm", "bsp_index_to_relative", "bsp_index_from_relative", "bsp_check"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -157,6 +158,19 @@ def bsp_conv2d_q8(wd: WDesc, w: Bcsr, xd: XDesc, X, bias, shift, Y, ws, stream=N
 def bsp_gemm_q8(wd: WDesc, w: Bcsr, X, P, bias, shift, Y, ws, stream=None):
     _raise(lib().bsp_gemm_q8(C.byref(wd), C.byref(w), _ptr(X), C.c_int64(P), _ptr(bias), _ptr(shift), _ptr(Y), _ptr(ws),
                              _stream(stream)), "bsp_gemm_q8")
+
+
+def bsp_spgemm(wa: WDesc, a: Bcsr, wb: WDesc, b: Bcsr, Cm, ws, stream=None):
+    _raise(lib().bsp_spgemm(C.byref(wa), C.byref(a), C.byref(wb), C.byref(b), _ptr(Cm), _ptr(ws), _stream(stream)), "bsp_spgemm")
+
+
+def bsp_index_to_relative(NBo, row_ptr, col_idx, rel, stream=None):
+    _raise(lib().bsp_index_to_relative(C.c_int(NBo), _ptr(row_ptr), _ptr(col_idx), _ptr(rel), _stream(stream)), "bsp_index_to_relative")
+
+
+def bsp_index_from_relative(NBo, row_ptr, rel, col_idx, stream=None):
+    _raise(lib().bsp_index_from_relative(C.c_int(NBo), _ptr(row_ptr), _ptr(rel), _ptr(col_idx), _stream(stream)),
+           "bsp_index_from_relative")
 
 
 def bsp_mask_static(wd: WDesc, W, norm, scope, n_zero, gamma, stream=None):

@@ -1,0 +1,154 @@
+// Block-sparse x block-sparse product C = (Gamma . A)(Omega . B)^t on the compressed block rows of both operands, and the
+// relative column index.  Section "Block-Sparse Matrix-Matrix Multiplication" and Section "Block Sparsity in a Matrix"
+// ("a relative row/col index") of the paper.
+//
+// C_{i,j} = sum over the block columns k that row i of A and row j of B both keep of A_{i,k} B_{j,k}^t, 8 x 8 blocks.
+// A CTA owns one row i of A: the positions of its kept blocks are spread into a table over the block columns in shared
+// memory (the table replaces one side of the paper's merge of two sorted lists), and every warp takes rows j of B in
+// turn: 32 entries of B's column list are looked up at once, a ballot gives the common columns in ascending order, and
+// for each of them the warp adds the 8 x 8 x 8 product, lane (r, c) holding C[r][2c], C[r][2c + 1] in fp32.  Work and
+// traffic follow the kept blocks only: nothing is read or multiplied where either mask has a zero.
+#include "bsp_internal.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kSpThreads = 256;
+constexpr int kSpEdge = 8;
+
+__device__ __forceinline__ float sp_load(const float *p) { return __ldg(p); }
+__device__ __forceinline__ float sp_load(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+
+template <typename T>
+__global__ void __launch_bounds__(kSpThreads)
+spgemm_kernel(const int32_t *__restrict__ a_row_ptr, const int32_t *__restrict__ a_col_idx, const T *__restrict__ a_payload,
+              const int32_t *__restrict__ b_row_ptr, const int32_t *__restrict__ b_col_idx, const T *__restrict__ b_payload,
+              int NBb, int NBk, float *__restrict__ C, int *status)
+{
+    extern __shared__ int s_pos[];                 // [NBk]: payload position of row i's block in column k, or -1
+    const int i = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int k = threadIdx.x; k < NBk; k += kSpThreads) s_pos[k] = -1;
+    __syncthreads();
+    for (int n = a_row_ptr[i] + threadIdx.x; n < a_row_ptr[i + 1]; n += kSpThreads) {
+        const int k = a_col_idx[n];
+        if (k >= 0 && k < NBk) s_pos[k] = n;
+        else atomicMax(status, (int)BSP_ERR_INDEX);          // a column outside the matrix: skipped
+    }
+    __syncthreads();
+    const int r = lane >> 2, c = (lane & 3) * 2;             // this lane's two entries of the 8 x 8 block of C
+    const size_t ldc = (size_t)NBb * kSpEdge;
+    for (int j = blockIdx.y * (kSpThreads / 32) + warp; j < NBb; j += gridDim.y * (kSpThreads / 32)) {
+        float acc0 = 0.f, acc1 = 0.f;
+        const int lo = b_row_ptr[j], hi = b_row_ptr[j + 1];
+        for (int base = lo; base < hi; base += 32) {
+            const int nb = base + lane;
+            int pa = -1;
+            if (nb < hi) {
+                const int k = b_col_idx[nb];
+                if (k >= 0 && k < NBk) pa = s_pos[k];
+                else atomicMax(status, (int)BSP_ERR_INDEX);
+            }
+            unsigned both = __ballot_sync(0xFFFFFFFFu, pa >= 0);
+            while (both) {                                    // common columns, ascending
+                const int src = __ffs(both) - 1;
+                both &= both - 1;
+                const int na = __shfl_sync(0xFFFFFFFFu, pa, src);
+                const T *Ab = a_payload + ((size_t)na * kSpEdge + r) * kSpEdge;
+                const T *Bb = b_payload + ((size_t)(base + src) * kSpEdge + c) * kSpEdge;
+#pragma unroll
+                for (int t = 0; t < kSpEdge; ++t) {
+                    const float a = sp_load(Ab + t);
+                    acc0 = fmaf(a, sp_load(Bb + t), acc0);
+                    acc1 = fmaf(a, sp_load(Bb + kSpEdge + t), acc1);
+                }
+            }
+        }
+        *(float2 *)(C + ((size_t)i * kSpEdge + r) * ldc + (size_t)j * kSpEdge + c) = make_float2(acc0, acc1);
+    }
+}
+
+// One thread per row of Gamma: the first kept block keeps its column, the others store the distance to their predecessor.
+__global__ void index_to_relative_kernel(int NBo, const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                                         int32_t *__restrict__ rel)
+{
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= NBo) return;
+    int prev = 0;
+    for (int n = row_ptr[l]; n < row_ptr[l + 1]; ++n) {
+        const int cur = col_idx[n];
+        rel[n] = cur - prev;
+        prev = cur;
+    }
+}
+
+__global__ void index_from_relative_kernel(int NBo, const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ rel,
+                                           int32_t *__restrict__ col_idx)
+{
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= NBo) return;
+    int at = 0;
+    for (int n = row_ptr[l]; n < row_ptr[l + 1]; ++n) {
+        at += rel[n];
+        col_idx[n] = at;
+    }
+}
+
+}  // namespace
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+bsp_status bsp_spgemm(const bsp_wdesc *wa, const bsp_bcsr *a, const bsp_wdesc *wb, const bsp_bcsr *b, float *C, void *ws,
+                      void *stream)
+{
+    bsp_status rc = check_wdesc(wa);
+    if (rc != BSP_OK) return rc;
+    rc = check_wdesc(wb);
+    if (rc != BSP_OK) return rc;
+    if (!a || !b || !C || !ws || !a->row_ptr || !a->col_idx || !a->payload || !b->row_ptr || !b->col_idx || !b->payload)
+        return BSP_ERR_NULL;
+    if (wa->H != 1 || wa->K != 1 || wb->H != 1 || wb->K != 1 || wa->I != wb->I) return BSP_ERR_SHAPE;
+    if (wa->bo != kSpEdge || wa->bi != kSpEdge || wb->bo != kSpEdge || wb->bi != kSpEdge) return BSP_ERR_BLOCK;
+    if (wa->wtype != wb->wtype || (wa->wtype != BSP_F32 && wa->wtype != BSP_BF16)) return BSP_ERR_DTYPE;
+    if (((uintptr_t)C & 7u) != 0) return BSP_ERR_SHAPE;
+    const int NBa = wa->O / kSpEdge, NBb = wb->O / kSpEdge, NBk = wa->I / kSpEdge;
+    const size_t smem = (size_t)NBk * sizeof(int);
+    if (smem > 48 * 1024) return BSP_ERR_SHAPE;
+    // rows of B are dealt over the warps of gridDim.y CTAs per row of A: enough CTAs to fill the GPU a few times over
+    int gy = (NBb + kSpThreads / 32 - 1) / (kSpThreads / 32);
+    const int want = (148 * 8 + NBa - 1) / NBa;
+    if (gy > want) gy = want;
+    if (gy < 1) gy = 1;
+    const dim3 grid((unsigned)NBa, (unsigned)gy);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (wa->wtype == BSP_F32)
+        spgemm_kernel<float><<<grid, kSpThreads, smem, st>>>(a->row_ptr, a->col_idx, (const float *)a->payload, b->row_ptr, b->col_idx,
+                                                             (const float *)b->payload, NBb, NBk, C, (int *)ws);
+    else
+        spgemm_kernel<__nv_bfloat16><<<grid, kSpThreads, smem, st>>>(a->row_ptr, a->col_idx, (const __nv_bfloat16 *)a->payload, b->row_ptr,
+                                                                     b->col_idx, (const __nv_bfloat16 *)b->payload, NBb, NBk, C, (int *)ws);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+bsp_status bsp_index_to_relative(int NBo, const int32_t *row_ptr, const int32_t *col_idx, int32_t *rel, void *stream)
+{
+    if (!row_ptr || !col_idx || !rel) return BSP_ERR_NULL;
+    if (NBo <= 0) return BSP_ERR_SHAPE;
+    index_to_relative_kernel<<<(NBo + 127) / 128, 128, 0, (cudaStream_t)stream>>>(NBo, row_ptr, col_idx, rel);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+bsp_status bsp_index_from_relative(int NBo, const int32_t *row_ptr, const int32_t *rel, int32_t *col_idx, void *stream)
+{
+    if (!row_ptr || !col_idx || !rel) return BSP_ERR_NULL;
+    if (NBo <= 0) return BSP_ERR_SHAPE;
+    index_from_relative_kernel<<<(NBo + 127) / 128, 128, 0, (cudaStream_t)stream>>>(NBo, row_ptr, rel, col_idx);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // extern "C"
