@@ -199,7 +199,7 @@ bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc
  *             both keep of A_{i,k} B_{j,k}^t.  A is wa->O x wa->I, B is wb->O x wb->I with the same I, both with H = K = 1,
  *             8x8 blocks and the same type (F32 or BF16); `a` and `b` are their compact forms from bsp_compact (row_ptr,
  *             col_idx and the canonical payload are read; `packed` is not).  C is dense float32 [wa->O][wb->O], 8-byte
- *             aligned, written in full (blocks without a common column are zero).  Products are accumulated in float32
+ *             aligned (the two payloads 16-byte aligned), written in full (blocks without a common column are zero).  Products are accumulated in float32
  *             in ascending order of k.  A column index outside the matrix is skipped and latches BSP_ERR_INDEX.
  *             ws: any workspace of at least 256 bytes (status word only).
  * bsp_index_to_relative / bsp_index_from_relative: within each row of Gamma the first kept block keeps its column, every

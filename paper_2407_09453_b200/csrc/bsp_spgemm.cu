@@ -16,8 +16,22 @@ namespace {
 constexpr int kSpThreads = 256;
 constexpr int kSpEdge = 8;
 
-__device__ __forceinline__ float sp_load(const float *p) { return __ldg(p); }
-__device__ __forceinline__ float sp_load(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+// One row of an 8 x 8 block (8 consecutive values) as floats: two 16-byte loads for fp32, one for bf16.
+__device__ __forceinline__ void sp_row(const float *p, float (&v)[8])
+{
+    const float4 a = __ldg((const float4 *)p), b = __ldg((const float4 *)p + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void sp_row(const __nv_bfloat16 *p, float (&v)[8])
+{
+    const uint4 q = __ldg((const uint4 *)p);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        v[2 * t] = __uint_as_float(w[t] << 16);
+        v[2 * t + 1] = __uint_as_float(w[t] & 0xFFFF0000u);
+    }
+}
 
 template <typename T>
 __global__ void __launch_bounds__(kSpThreads)
@@ -55,11 +69,12 @@ spgemm_kernel(const int32_t *__restrict__ a_row_ptr, const int32_t *__restrict__
                 const int na = __shfl_sync(0xFFFFFFFFu, pa, src);
                 const T *Ab = a_payload + ((size_t)na * kSpEdge + r) * kSpEdge;
                 const T *Bb = b_payload + ((size_t)(base + src) * kSpEdge + c) * kSpEdge;
+                float av[8], b0[8], b1[8];
+                sp_row(Ab, av); sp_row(Bb, b0); sp_row(Bb + kSpEdge, b1);
 #pragma unroll
                 for (int t = 0; t < kSpEdge; ++t) {
-                    const float a = sp_load(Ab + t);
-                    acc0 = fmaf(a, sp_load(Bb + t), acc0);
-                    acc1 = fmaf(a, sp_load(Bb + kSpEdge + t), acc1);
+                    acc0 = fmaf(av[t], b0[t], acc0);
+                    acc1 = fmaf(av[t], b1[t], acc1);
                 }
             }
         }
@@ -112,7 +127,7 @@ bsp_status bsp_spgemm(const bsp_wdesc *wa, const bsp_bcsr *a, const bsp_wdesc *w
     if (wa->H != 1 || wa->K != 1 || wb->H != 1 || wb->K != 1 || wa->I != wb->I) return BSP_ERR_SHAPE;
     if (wa->bo != kSpEdge || wa->bi != kSpEdge || wb->bo != kSpEdge || wb->bi != kSpEdge) return BSP_ERR_BLOCK;
     if (wa->wtype != wb->wtype || (wa->wtype != BSP_F32 && wa->wtype != BSP_BF16)) return BSP_ERR_DTYPE;
-    if (((uintptr_t)C & 7u) != 0) return BSP_ERR_SHAPE;
+    if (((uintptr_t)C & 7u) != 0 || ((uintptr_t)a->payload & 15u) != 0 || ((uintptr_t)b->payload & 15u) != 0) return BSP_ERR_SHAPE;
     const int NBa = wa->O / kSpEdge, NBb = wb->O / kSpEdge, NBk = wa->I / kSpEdge;
     const size_t smem = (size_t)NBk * sizeof(int);
     if (smem > 48 * 1024) return BSP_ERR_SHAPE;
