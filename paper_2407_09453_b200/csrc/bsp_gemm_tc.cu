@@ -58,6 +58,7 @@ struct GtParams {
     int store_tma;                    // a tile is 128 consecutive rows of Y: the epilogue stores by TMA
     uint8_t *Y;
     int ey;
+    uint32_t m_ntn, m_tx, m_ty;       // floor(2^32 / d) of n_tiles_n, tiles_x, tiles_y (division by multiplication)
 };
 
 __device__ __forceinline__ uint32_t sm32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -154,11 +155,22 @@ __device__ __forceinline__ uint32_t gt_requant(int v, uint32_t s)
     return (uint32_t)q & 0xFFu;
 }
 
+// n / d and n % d for 0 <= n < 2^31 by the multiplier m = floor(2^32 / d) (0xFFFFFFFF for d = 1): the product's high
+// word is the quotient or one less, one correction settles it.
+__device__ __forceinline__ void gt_divmod(int n, int d, uint32_t m, int &q, int &r)
+{
+    q = (int)__umulhi((uint32_t)n, m);
+    r = n - q * d;
+    if (r >= d) { ++q; r -= d; }
+}
+
 // First output position (image, row, column) of position tile mt.
 __device__ __forceinline__ void gt_tile_origin(const GtParams &p, int mt, int &n0, int &y0, int &x0)
 {
-    const int tx = mt % p.tiles_x, r = mt / p.tiles_x;
-    x0 = tx * p.Wt; y0 = (r % p.tiles_y) * p.Ht; n0 = (r / p.tiles_y) * p.Nt;
+    int r, tx, ty, ni;
+    gt_divmod(mt, p.tiles_x, p.m_tx, r, tx);
+    gt_divmod(r, p.tiles_y, p.m_ty, ni, ty);
+    x0 = tx * p.Wt; y0 = ty * p.Ht; n0 = ni * p.Nt;
 }
 
 // 32 consecutive accumulator columns of this thread's tensor-memory lane.
@@ -244,47 +256,58 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
 
     if (warp == 0) {
         // ================= producer =================
-        if (lane == 0 && run) {
+        // The whole warp runs the loop with warp-uniform values; one elected lane arms the barrier and issues the loads.
+        if (run) {
             const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
             // (a pair: each CTA loads its own activation box and its half of the weight tile, all four loads announce their
             // bytes on the leader's barrier, which the leader arms with the total)
             const uint32_t stage_bytes = (uint32_t)p.stage_bytes;
             const uint32_t tx = (uint32_t)(p.a_bytes + (BN >> (kPair ? 1 : 0)) * 128) * (kPair ? 2u : 1u);
-            uint32_t slot = 0, round = 0, issued = 0, dst = ring;
+            const int cpt128 = p.cpt * 128, Kw = p.K, ntn = p.n_tiles_n;
+            // (a fresh barrier counts as released: the wait on parity 1 of the first round returns at once)
+            uint32_t slot = 0, epar = 1, issued = 0, dst = ring;
             bool ok = true;
             for (int tile = t_first; tile < t_count && ok; tile += t_step) {
-                const int ch0 = (tile % p.n_tiles_n) * BN + (kPair ? (int)rank * (BN >> 1) : 0);
+                int mt, tn;
+                gt_divmod(tile, ntn, p.m_ntn, mt, tn);
+                const int ch0 = tn * BN + (kPair ? (int)rank * (BN >> 1) : 0);
                 int n0, y0, x0;
-                gt_tile_origin(p, kPair ? 2 * (tile / p.n_tiles_n) + (int)rank : tile / p.n_tiles_n, n0, y0, x0);
+                gt_tile_origin(p, kPair ? 2 * mt + (int)rank : mt, n0, y0, x0);
                 // input position of the tile's first output position at tap (0, 0); a tap is a shift of the box, positions
                 // outside the image read as zeros (the padding)
-                const int xi0 = x0 * p.sw - p.pw, yi0 = y0 * p.sh - p.ph;
-                for (int tap = 0, h = 0, k = 0; tap < p.H * p.K && ok; ++tap) {
-                    for (int c = 0; c < p.cpt; ++c) {
-                        if (round && !gt_poll(empty0 + slot * 8u, (round & 1u) ^ 1u)) { ok = false; break; }
-                        if (s_fail) { ok = false; break; }
-                        if constexpr (kPair) {
-                            const uint32_t bar = lead_full0 + slot * 8u;
-                            if (rank == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(full0 + slot * 8u), "r"(tx) : "memory");
-                            asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
-                                         ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(c * 128), "r"(xi0 + k), "r"(yi0 + h), "r"(n0) : "memory");
-                            asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
-                                         ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(c * 128), "r"(tap), "r"(ch0) : "memory");
-                        } else {
-                        const uint32_t bar = full0 + slot * 8u;
-                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
-                        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
-                                     ::"r"(dst), "l"(&p.tmx), "r"(bar), "r"(c * 128), "r"(xi0 + k), "r"(yi0 + h), "r"(n0) : "memory");
-                        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
-                                     ::"r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(bar), "r"(c * 128), "r"(tap), "r"(ch0) : "memory");
-                        }
-                        ++issued;
-                        if (++slot == (uint32_t)S) { slot = 0; ++round; dst = ring; } else dst += stage_bytes;
+                const int xi0 = x0 * p.sw - p.pw;
+                int c128 = 0, kx = xi0, hy = y0 * p.sh - p.ph, tap = 0, kk = 0;
+                if (s_fail) { ok = false; break; }
+                for (int ks = 0; ks < n_ks; ++ks) {
+                    bool got = gt_poll(empty0 + slot * 8u, epar);
+                    got = __all_sync(0xFFFFFFFFu, got);
+                    if (!got) { ok = false; break; }
+                    if constexpr (kPair) {
+                        asm volatile("{\n .reg .pred e, l;\n elect.sync _|e, 0xFFFFFFFF;\n setp.eq.u32 l, %12, 0;\n and.pred l, l, e;\n"
+                                     " @l mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
+                                     " @e cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%13];\n"
+                                     " @e cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%4, %10, %11}], [%13];\n}\n"
+                                     ::"r"(full0 + slot * 8u), "r"(tx), "r"(dst), "l"(&p.tmx), "r"(c128), "r"(kx), "r"(hy), "r"(n0),
+                                       "r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(tap), "r"(ch0), "r"(rank), "r"(lead_full0 + slot * 8u) : "memory");
+                    } else {
+                        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                                     " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
+                                     " @e cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%0];\n"
+                                     " @e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%4, %10, %11}], [%0];\n}\n"
+                                     ::"r"(full0 + slot * 8u), "r"(tx), "r"(dst), "l"(&p.tmx), "r"(c128), "r"(kx), "r"(hy), "r"(n0),
+                                       "r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(tap), "r"(ch0) : "memory");
                     }
-                    if (++k == p.K) { k = 0; ++h; }
+                    ++issued;
+                    if (++slot == (uint32_t)S) { slot = 0; epar ^= 1u; dst = ring; } else dst += stage_bytes;
+                    // next K-stage: the next 128-byte chunk of channels, then the next tap (columns first)
+                    c128 += 128;
+                    if (c128 == cpt128) {
+                        c128 = 0; ++tap; ++kx;
+                        if (++kk == Kw) { kk = 0; kx = xi0; ++hy; }
+                    }
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // winding down after a wait that ran out: the loads already issued still write into this CTA's shared
                 // memory, so the barriers of the stages in flight are awaited (bounded) before the CTA may leave
                 atomicExch((uint32_t *)&s_fail, 1u);
@@ -310,14 +333,14 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             bool ok = true;
             for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
-                if (use && !gt_poll(sm32(&s_acc_empty[buf]), (use & 1u) ^ 1u)) ok = false;
+                if (!gt_poll(sm32(&s_acc_empty[buf]), (use & 1u) ^ 1u) || s_fail != 0u) ok = false;   // (a fresh barrier counts as released)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t d = tmem + buf * 256u;
                 for (int ks = 0; ks < n_ks; ++ks) {
                     bool got = gt_poll(full0 + slot * 8u, par);
-                    got = __all_sync(0xFFFFFFFFu, got && s_fail == 0u);
+                    got = __all_sync(0xFFFFFFFFu, got);
                     if (!got) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
@@ -338,13 +361,15 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             const uint32_t stg0 = staging + (uint32_t)(ew * 2 * kGtStagingBytes);
             uint32_t tile_i = 0, rounds_done = 0;
             bool ok = true;
+            // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
+            const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
             for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
-                const int n0 = (tile % p.n_tiles_n) * BN;
-                // this lane's row of the tile: position (w, h, image i) of the tile's box, w fastest
+                int mt, tn;
+                gt_divmod(tile, p.n_tiles_n, p.m_ntn, mt, tn);
+                const int n0 = tn * BN;
                 int in0, y0, x0;
-                gt_tile_origin(p, kPair ? 2 * (tile / p.n_tiles_n) + (int)rank : tile / p.n_tiles_n, in0, y0, x0);
-                const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
+                gt_tile_origin(p, kPair ? 2 * mt + (int)rank : mt, in0, y0, x0);
                 const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
                 // byte offset of the row in Y (rows of O * ey bytes); m0: the tile's first row when rows are consecutive
                 const long long pos = ((long long)(in0 + ri) * p.M + (y0 + rh)) * p.Nw + (x0 + rw);
@@ -503,6 +528,8 @@ bsp_xdesc gt_flatten(const bsp_wdesc &wd, const bsp_xdesc &xd)
     return xd;
 }
 
+uint32_t gt_magic(int d) { return d <= 1 ? 0xFFFFFFFFu : (uint32_t)((1ull << 32) / (uint64_t)d); }
+
 GtTile gt_pick_tile(int N, int M, int Nw, int sh, int sw)
 {
     GtTile best = {0, 0, 0, -1};
@@ -600,6 +627,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.n_ks = HK * p.cpt;
     const bool pair = p.BN == 256 && p.n_ks >= 8 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
     p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
+    p.m_ntn = gt_magic(p.n_tiles_n); p.m_tx = gt_magic(p.tiles_x); p.m_ty = gt_magic(p.tiles_y);
     p.stage_bytes = kGtABytes + (pair ? p.BN / 2 : p.BN) * 128;
     const int staging = 4 * 2 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
