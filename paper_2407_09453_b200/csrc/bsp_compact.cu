@@ -195,13 +195,16 @@ __device__ __forceinline__ void dense_body(int idx, int n_ctas, const void *__re
     const int cpr = I * esz / 16;                     // chunks per row
     constexpr int cpc = 16 / esz;
     const long long total = (long long)O * HK * cpr, stride = (long long)n_ctas * kThreads;
+    const bool small = total < (1ll << 31);
     for (long long e0 = (long long)idx * kThreads + threadIdx.x; e0 < total; e0 += 4 * stride) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const long long e = e0 + u * stride;
             if (e >= total) continue;
-            const int ot = (int)(e / cpr), c = (int)(e - (long long)ot * cpr);
+            // (a 64-bit division costs an order of magnitude more than a 32-bit one: taken only by layers that need it)
+            const int ot = small ? (int)((unsigned)e / (unsigned)cpr) : (int)(e / cpr);
+            const int c = (int)(e - (long long)ot * cpr);
             const int o = ot / HK, tap = ot - o * HK;
             if (aligned) {
                 v[u] = w_chunk<esz>(W, gamma, o, tap, c * cpc, O, I, HK, bo, bi, NBi);
@@ -241,43 +244,53 @@ struct CompactArgs {
     int *status;
 };
 
-// Launch 1 of the multi-launch path: ones of one row of Gamma -> row_cnt.
+// Larger layers, first launch: CTA l counts the kept blocks of row l of Gamma; the CTA that finishes last (a ticket in
+// the workspace header, which it hands back as zero) turns the counts into row_ptr, checks the capacity and writes the
+// header of the packed buffer.  Nobody waits for anybody.
 __global__ void __launch_bounds__(kThreads)
-count_kernel(const uint8_t *__restrict__ gamma, int NBi, int *__restrict__ row_cnt)
-{
-    __shared__ int warp_sums[kThreads / 32];
-    const uint8_t *g = gamma + (size_t)blockIdx.x * NBi;
-    int c = 0;
-    for (int i = threadIdx.x; i < NBi; i += kThreads) c += g[i] ? 1 : 0;
-    int tot;
-    block_exclusive_scan(c, warp_sums, tot);
-    if (threadIdx.x == 0) row_cnt[blockIdx.x] = tot;
-}
-
-// Launch 2 (one CTA): exclusive scan row_cnt -> row_ptr, the packed header, and BSP_ERR_CAPACITY if more blocks are
-// stored than the buffers were sized for.
-__global__ void __launch_bounds__(kThreads)
-scan_kernel(const int *__restrict__ row_cnt, int NBo, int32_t *__restrict__ row_ptr, PackedHeader *__restrict__ hdr,
-            PackedHeader hdr_init, long long capacity_blocks, int *__restrict__ status)
+count_scan_kernel(const uint8_t *__restrict__ gamma, int NBi, int NBo, int *row_cnt, int32_t *__restrict__ row_ptr,
+                  PackedHeader *__restrict__ hdr, PackedHeader hdr_init, long long capacity_blocks, int *__restrict__ status,
+                  unsigned *ticket)
 {
     __shared__ int warp_sums[kThreads / 32];
     __shared__ int s_run;
-    if (threadIdx.x == 0) s_run = 0;
+    __shared__ bool s_last;
+    const uint8_t *g = gamma + (size_t)blockIdx.x * NBi;
+    int c = 0;
+    if ((NBi & 15) == 0 && (((uintptr_t)gamma) & 15u) == 0) {
+        for (int i = threadIdx.x; i < (NBi >> 4); i += kThreads) {
+            const uint4 q = __ldg((const uint4 *)g + i);
+            c += __popc(__vsetne4(q.x, 0u)) + __popc(__vsetne4(q.y, 0u)) + __popc(__vsetne4(q.z, 0u)) + __popc(__vsetne4(q.w, 0u));
+        }
+    } else {
+        for (int i = threadIdx.x; i < NBi; i += kThreads) c += g[i] ? 1 : 0;
+    }
+    int tot;
+    block_exclusive_scan(c, warp_sums, tot);
+    if (threadIdx.x == 0) {
+        row_cnt[blockIdx.x] = tot;
+        __threadfence();
+        s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+        s_run = 0;
+    }
     __syncthreads();
+    if (!s_last) return;
+    __threadfence();
     for (int base = 0; base < NBo; base += kThreads) {
         const int i = base + threadIdx.x;
-        const int v = (i < NBo) ? row_cnt[i] : 0;
-        int tot;
-        const int before = block_exclusive_scan(v, warp_sums, tot);
+        const int v = (i < NBo) ? __ldcg(row_cnt + i) : 0;
+        int all;
+        const int before = block_exclusive_scan(v, warp_sums, all);
         if (i < NBo) row_ptr[i] = s_run + before;
         __syncthreads();
-        if (threadIdx.x == 0) s_run += tot;
+        if (threadIdx.x == 0) s_run += all;
         __syncthreads();
     }
     if (threadIdx.x == 0) {
         row_ptr[NBo] = s_run;
         if ((long long)s_run > capacity_blocks) atomicMax(status, (int)BSP_ERR_CAPACITY);
         if (hdr != nullptr) *hdr = hdr_init;
+        *ticket = 0u;
     }
 }
 
@@ -398,9 +411,8 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
         BSP_CUDA_OK(cudaGetLastError());
         return BSP_OK;
     }
-    count_kernel<<<NBo, kThreads, 0, st>>>(gamma, NBi, row_cnt);
-    BSP_CUDA_OK(cudaGetLastError());
-    scan_kernel<<<1, kThreads, 0, st>>>(row_cnt, NBo, row_ptr, (PackedHeader *)pk, a.hdr_init, (long long)capacity_blocks, status);
+    count_scan_kernel<<<NBo, kThreads, 0, st>>>(gamma, NBi, NBo, row_cnt, row_ptr, (PackedHeader *)pk, a.hdr_init, (long long)capacity_blocks,
+                                                status, (unsigned *)ws + kWsTicketWord);
     BSP_CUDA_OK(cudaGetLastError());
     // enough CTAs per row to give every SM some of the payload copy
     a.fill_parts = payload ? (296 + NBo - 1) / NBo : 1;

@@ -38,10 +38,11 @@ PackedLayout packed_layout(const bsp_wdesc &wd);
 // barrier of the single-launch kernels (words kWsSyncWord, kWsSyncWord + 1); scratch starts after them.
 constexpr size_t kWsHeader = 256;
 constexpr int kWsSyncWord = 2;
-// Scratch of the cooperative select after the scores in the mask workspace: 8 x 256 histogram words, 4 counter words,
-// one word per CTA and a list of up to 2048 candidate keys.
+constexpr int kWsTicketWord = 4;          // count of finished CTAs of the row-count launch (left at zero)
+// Scratch of the cooperative select after the scores in the mask workspace: 8 x 256 histogram words, 8 counter and key-span words,
+// one word per CTA and a list of up to 8192 candidate keys.
 constexpr int kSelectMaxCtas = 1024;
-constexpr size_t kSelectScratch = (8 * 256 + 4 + kSelectMaxCtas) * 4 + 2048 * 8;
+constexpr size_t kSelectScratch = (8 * 256 + 8 + kSelectMaxCtas) * 4 + 8192 * 8;
 
 // Host-side validation of a weight descriptor, shared by every entry point.
 bsp_status check_wdesc(const bsp_wdesc *wd);

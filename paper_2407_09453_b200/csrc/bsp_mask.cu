@@ -103,7 +103,8 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__rest
                                                           int NBi, long long B, int r, double mean = 0.0)
 {
     constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
-    const int l = (int)(B / NBi), iota = (int)(B % NBi);
+    const int l = B < (1ll << 31) ? (int)((unsigned)B / (unsigned)NBi) : (int)(B / NBi);     // (64-bit divisions are slow)
+    const int iota = (int)(B - (long long)l * NBi);
     const int words = bi / per_word;
     const size_t row_words = (size_t)I / per_word;
     const uint32_t *src = W + ((size_t)(l * bo + r) * HK) * row_words + (size_t)iota * words;
@@ -117,20 +118,113 @@ __device__ __forceinline__ typename Acc<DT>::type row_sum(const uint32_t *__rest
     }
 }
 
+// OR of the keys' bits and OR of their complements, added to span[0] and span[1] (zeroed by the host): a bit
+// position set in both differs between some two keys.  The select starts at the highest such bit.  One thread per
+// CTA adds, and only bits that are not there yet (atomics on one address are served one after the other).
+// Every thread of the CTA must call it.
+__device__ __forceinline__ void publish_span(unsigned long long or1, unsigned long long or0, unsigned long long *span)
+{
+    __shared__ unsigned long long s_or[2][kScoreThreads / 32];
+    for (int o = 16; o > 0; o >>= 1) {
+        or1 |= __shfl_xor_sync(0xFFFFFFFFu, or1, o);
+        or0 |= __shfl_xor_sync(0xFFFFFFFFu, or0, o);
+    }
+    if ((threadIdx.x & 31) == 0) { s_or[0][threadIdx.x >> 5] = or1; s_or[1][threadIdx.x >> 5] = or0; }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        unsigned long long v = 0ull;
+        for (int w = 0; w < kScoreThreads / 32; ++w) v |= s_or[threadIdx.x][w];
+        if (v & ~__ldcg(span + threadIdx.x)) atomicOr(span + threadIdx.x, v);
+    }
+}
+
+// One-tap layers (H K = 1) with the L2 or L1 measure: one thread per block (consecutive threads take consecutive blocks of
+// a block row, so a warp's load of one row r is one contiguous stretch of input channels).  The rows of a block are
+// WORDS words each; kRows rows (eight, or four when b_o = 4 or the rows are long) are loaded at a time, every row is summed over its channels in order and the row sums
+// are added in order of r: the same order of additions as row_sum followed by the sum over r.
+template <int DT, int NORM, int WORDS, int kRows>
+__device__ __forceinline__ void score_one_tap(const uint32_t *__restrict__ W, int I, int bo, int NBo, int NBi,
+                                              typename Acc<DT>::type *__restrict__ score, unsigned long long *span)
+{
+    using acc_t = typename Acc<DT>::type;
+    constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
+    constexpr int kVec = WORDS % 4 == 0 ? 4 : (WORDS % 2 == 0 ? 2 : 1);       // words per load
+    const long long NB = (long long)NBo * NBi;
+    const size_t row_words = (size_t)I / per_word;
+    const bool vec = kVec > 1 && (((uintptr_t)W) & (4u * kVec - 1u)) == 0 && row_words % kVec == 0;
+    const bool small = NB < (1ll << 31);
+    unsigned long long or1 = 0ull, or0 = 0ull;
+    for (long long B = (long long)blockIdx.x * kScoreThreads + threadIdx.x; B < NB; B += (long long)gridDim.x * kScoreThreads) {
+        // (a 64-bit division costs an order of magnitude more than a 32-bit one: taken only by layers that need it)
+        const int l = small ? (int)((unsigned)B / (unsigned)NBi) : (int)(B / NBi);
+        const int iota = (int)(B - (long long)l * NBi);
+        const uint32_t *src = W + (size_t)l * bo * row_words + (size_t)iota * WORDS;
+        acc_t total = 0;
+        for (int r0 = 0; r0 < bo; r0 += kRows) {             // (b_o is a multiple of kRows)
+            uint32_t w[kRows][WORDS];
+#pragma unroll
+            for (int u = 0; u < kRows; ++u) {
+                const uint32_t *row = src + (size_t)(r0 + u) * row_words;
+                if (vec && kVec == 4) {
+#pragma unroll
+                    for (int j = 0; j + 3 < WORDS; j += 4) {
+                        const uint4 q = __ldg((const uint4 *)(row + j));
+                        w[u][j] = q.x; w[u][j + 1] = q.y; w[u][j + 2] = q.z; w[u][j + 3] = q.w;
+                    }
+                } else if (vec && kVec == 2) {
+#pragma unroll
+                    for (int j = 0; j + 1 < WORDS; j += 2) {
+                        const uint2 q = __ldg((const uint2 *)(row + j));
+                        w[u][j] = q.x; w[u][j + 1] = q.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < WORDS; ++j) w[u][j] = __ldg(row + j);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kRows; ++u) {
+                acc_t pr = 0;
+#pragma unroll
+                for (int j = 0; j < WORDS; ++j) add_word<DT, NORM>(w[u][j], pr, 0.0);
+                total += pr;
+            }
+        }
+        score[B] = total;
+        unsigned long long key;
+        memcpy(&key, &total, 8);
+        or1 |= key; or0 |= ~key;
+    }
+    if (span != nullptr) publish_span(or1, or0, span);
+}
+
 // A CTA takes groups of 256 / b_o blocks, every `gridDim.x`-th one (a bounded grid of long-lived CTAs instead of one
 // short CTA per group: a layer of 4096 x 4096 weights is 8192 groups).
 template <int DT, int NORM, int kBatch>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int NBo, int NBi,
-             typename Acc<DT>::type *__restrict__ score)
+             typename Acc<DT>::type *__restrict__ score, unsigned long long *span)
 {
     using acc_t = typename Acc<DT>::type;
+    if constexpr (kBatch == 1 && NORM != BSP_NORM_VAR) {
+        constexpr int per_word = (DT == BSP_F32) ? 1 : (DT == BSP_BF16 ? 2 : 4);
+        const bool eight = bo % 8 == 0;
+        switch (bi / per_word) {
+            case 1: if (eight) score_one_tap<DT, NORM, 1, 8>(W, I, bo, NBo, NBi, score, span); else score_one_tap<DT, NORM, 1, 4>(W, I, bo, NBo, NBi, score, span); break;
+            case 2: if (eight) score_one_tap<DT, NORM, 2, 8>(W, I, bo, NBo, NBi, score, span); else score_one_tap<DT, NORM, 2, 4>(W, I, bo, NBo, NBi, score, span); break;
+            case 4: if (eight) score_one_tap<DT, NORM, 4, 8>(W, I, bo, NBo, NBi, score, span); else score_one_tap<DT, NORM, 4, 4>(W, I, bo, NBo, NBi, score, span); break;
+            case 8: score_one_tap<DT, NORM, 8, 4>(W, I, bo, NBo, NBi, score, span); break;
+            default: score_one_tap<DT, NORM, 16, 4>(W, I, bo, NBo, NBi, score, span); break;
+        }
+        return;
+    }
     __shared__ acc_t part[kScoreThreads];
     const int blocks_per_cta = kScoreThreads / bo;
     const int bl = threadIdx.x % blocks_per_cta;
     const int r = threadIdx.x / blocks_per_cta;
     const long long NB = (long long)NBo * NBi;
     const long long n_groups = (NB + blocks_per_cta - 1) / blocks_per_cta;
+    unsigned long long or1 = 0ull, or0 = 0ull;
     for (long long grp = blockIdx.x; grp < n_groups; grp += gridDim.x) {
         const long long B = grp * blocks_per_cta + bl;
         if constexpr (NORM == BSP_NORM_VAR) {
@@ -148,7 +242,11 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
             if (B < NB && r == 0) {
                 double total = 0.0;
                 for (int q = 0; q < bo; ++q) total += (double)part[q * blocks_per_cta + bl];
-                score[B] = (acc_t)(total / n_elems);
+                const acc_t out = (acc_t)(total / n_elems);
+                score[B] = out;
+                unsigned long long key;
+                memcpy(&key, &out, 8);
+                or1 |= key; or0 |= ~key;
             }
         } else {
             part[threadIdx.x] = (B < NB) ? row_sum<DT, NORM, kBatch>(W, I, HK, bo, bi, NBi, B, r) : (acc_t)0;
@@ -157,10 +255,14 @@ score_kernel(const uint32_t *__restrict__ W, int I, int HK, int bo, int bi, int 
                 acc_t total = 0;
                 for (int q = 0; q < bo; ++q) total += part[q * blocks_per_cta + bl];
                 score[B] = total;
+                unsigned long long key;
+                memcpy(&key, &total, 8);
+                or1 |= key; or0 |= ~key;
             }
         }
         __syncthreads();
     }
+    if (span != nullptr) publish_span(or1, or0, span);
 }
 
 // Scores are non-negative, so the bit pattern of a float64 orders like the value, as does an int64.
@@ -274,7 +376,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned *sync)
 // derives the digit for itself.  Keys equal to the threshold T are zeroed lowest index first: the CTAs publish
 // how many such keys their slices hold (geq[c]), meet again, and each counts those in the slices before its own.
 constexpr int kCoopThreads = 512;
-constexpr int kLocalMax = 2048;          // candidates that the CTAs finish on their own, in shared memory
+constexpr int kLocalMax = 8192;          // candidates that the CTAs finish on their own, in (dynamic) shared memory
 
 // The digit d of a 256-bin histogram with cum(d - 1) < need <= cum(d), found by the first warp: each lane sums eight
 // bins, a warp scan finds the lane, the lane walks its bins.  Writes the remaining count, the extended prefix and the
@@ -308,38 +410,46 @@ __device__ __forceinline__ void select_digit(const unsigned *hist, int tid, unsi
     }
 }
 
-// The select starts at the highest bit in which any two keys differ (one grid-wide OR of key ^ key[0]: the bits above
-// it are the same in every key, e.g. the sign and most of the exponent of float scores, or the leading zero bytes of
-// integer ones) and takes digits of eight bits downwards.  Passes run grid-wide (global histograms, a grid barrier
+// The select starts at the highest bit in which any two keys differ (the score kernel leaves the OR of all keys in
+// gcount[2..3] and the OR of their complements in gcount[4..5]: the bits above it are the same in every key, e.g. the
+// sign and most of the exponent of float scores, or the leading zero bytes of integer ones) and takes digits of eight
+// bits downwards.  Passes run grid-wide (global histograms, a grid barrier
 // each) only while more than kLocalMax keys still match the prefix; then the CTAs append their matching keys to one
-// list (`cand`, counted in gcount[0]; the OR sits in gcount[2..3]; both zeroed by the host with the histograms), meet
+// list (`cand`, counted in gcount[0], zeroed by the host with the histograms), meet
 // once, and every CTA finishes the remaining digits on the list in its own shared memory.
+constexpr int kSliceMax = 4096;          // keys of a CTA's slice that are kept in shared memory for all phases
+constexpr size_t kCoopSmem = (size_t)(kLocalMax + kSliceMax) * sizeof(unsigned long long);
+
 __global__ void __launch_bounds__(kCoopThreads)
 select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long long n_zero, uint8_t *__restrict__ gamma,
                    unsigned *ghist, unsigned *gcount, unsigned long long *cand, unsigned *geq, unsigned *sync, int *status)
 {
     __shared__ unsigned hist[256];
-    __shared__ unsigned long long s_cand[kLocalMax];
+    extern __shared__ unsigned long long s_dyn[];
+    unsigned long long *s_cand = s_dyn;                  // [kLocalMax]
+    unsigned long long *s_keys = s_dyn + kLocalMax;      // [kSliceMax]
     __shared__ unsigned long long s_prefix;
     __shared__ long long s_k;
-    __shared__ unsigned s_left;
+    __shared__ unsigned s_left, s_n;
     __shared__ unsigned warp_cnt[kCoopThreads / 32];
     __shared__ long long s_run;
     const int tid = threadIdx.x;
     const long long slice = (n + gridDim.x - 1) / gridDim.x;
-    const long long lo = (long long)blockIdx.x * slice, hi = min(n, lo + slice);
+    const long long lo = min(n, (long long)blockIdx.x * slice), hi = min(n, lo + slice);
+    const int len = (int)(hi - lo);                      // (a slice of more than 2^31 keys would need more CTAs than the launch allows)
     const unsigned long long k0 = key[0];
-    {
-        unsigned long long d = 0ull;
-        for (long long i = lo + tid; i < hi; i += kCoopThreads) d |= key[i] ^ k0;
-        for (int o = 16; o > 0; o >>= 1) d |= __shfl_xor_sync(0xFFFFFFFFu, d, o);
-        if ((tid & 31) == 0 && d) atomicOr((unsigned long long *)(gcount + 2), d);
+    // bit positions in which some two keys differ (the score kernel accumulated both ORs)
+    const unsigned long long diff = __ldcg((const unsigned long long *)(gcount + 2)) & __ldcg((const unsigned long long *)(gcount + 4));
+    // the slice is read once: every phase below walks it in shared memory (or in place when it does not fit)
+    const unsigned long long *ks = key + lo;
+    if (len <= kSliceMax) {
+#pragma unroll 4
+        for (int i = tid; i < len; i += kCoopThreads) s_keys[i] = key[lo + i];
+        ks = s_keys;
     }
-    if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
-    const unsigned long long diff = __ldcg((const unsigned long long *)(gcount + 2));
     // bits above `top` are common to all keys: they are the prefix so far (all keys equal: nothing left to select)
     int top = diff ? 63 - __clzll((long long)diff) : -1;
-    if (tid == 0) { s_prefix = top >= 63 ? 0ull : (k0 >> (top + 1)); s_k = n_zero; s_left = 0xFFFFFFFFu; }
+    if (tid == 0) { s_prefix = top >= 63 ? 0ull : (k0 >> (top + 1)); s_k = n_zero; s_left = n > 0xFFFFFFFFll ? 0xFFFFFFFFu : (unsigned)n; }
     int pi = 0;
     while (top >= 0) {
         if (tid < 256) hist[tid] = 0u;
@@ -349,12 +459,12 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
         const int width = min(8, top + 1), shift = top + 1 - width;
         const unsigned dmask = (1u << width) - 1u;
         // lanes with the same digit add once
-        for (long long base = lo; base < hi; base += kCoopThreads) {
-            const long long i = base + tid;
+        for (int base = 0; base < len; base += kCoopThreads) {
+            const int i = base + tid;
             unsigned long long v = 0ull;
             bool in = false;
-            if (i < hi) {
-                v = key[i];
+            if (i < len) {
+                v = ks[i];
                 in = top >= 63 || ((v >> (top + 1)) == prefix);
             }
             const unsigned digit = in ? ((unsigned)(v >> shift) & dmask) : 256u;
@@ -374,40 +484,64 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
     if (top >= 0) {
         // bits top .. 0 are still open: gather the keys that match the prefix, then finish locally
         const unsigned long long prefix = s_prefix;
-        for (long long i = lo + tid; i < hi; i += kCoopThreads) {
-            const unsigned long long v = key[i];
-            if ((v >> (top + 1)) == prefix) {          // (top < 63 here: at least one digit has been taken)
-                const unsigned at = atomicAdd(gcount, 1u);
-                if (at < (unsigned)kLocalMax) cand[at] = v;
-            }
+        for (int base = 0; base < len; base += kCoopThreads) {
+            const int i = base + tid;
+            const unsigned long long v = i < len ? ks[i] : 0ull;
+            const bool in = i < len && (top >= 63 || (v >> (top + 1)) == prefix);
+            // one addition to the counter per warp
+            const unsigned ball = __ballot_sync(0xFFFFFFFFu, in);
+            unsigned at = 0u;
+            if ((tid & 31) == 0 && ball) at = atomicAdd(gcount, (unsigned)__popc(ball));
+            at = __shfl_sync(0xFFFFFFFFu, at, 0) + (unsigned)__popc(ball & ((1u << (tid & 31)) - 1u));
+            if (in && at < (unsigned)kLocalMax) cand[at] = v;
         }
         if (!grid_barrier(sync)) { if (tid == 0) atomicMax(status, (int)BSP_ERR_TIMEOUT); return; }
-        const unsigned cnt = min(__ldcg(gcount), (unsigned)kLocalMax);
+        unsigned cnt = min(__ldcg(gcount), (unsigned)kLocalMax);
         for (unsigned i = tid; i < cnt; i += kCoopThreads) s_cand[i] = __ldcg(&cand[i]);
         __syncthreads();
+        constexpr int kMine = kLocalMax / kCoopThreads;    // candidates per thread
         while (top >= 0) {
             if (tid < 256) hist[tid] = 0u;
+            if (tid == 0) s_n = 0u;
             __syncthreads();
-            const unsigned long long pre = s_prefix;
             const int width = min(8, top + 1), shift = top + 1 - width;
             const unsigned dmask = (1u << width) - 1u;
-            for (unsigned i = tid; i < cnt; i += kCoopThreads) {
-                const unsigned long long v = s_cand[i];
-                if ((v >> (top + 1)) == pre) atomicAdd(&hist[(unsigned)(v >> shift) & dmask], 1u);
+            // every candidate matches the prefix so far (the list is thinned after each digit)
+            unsigned long long mine[kMine];
+#pragma unroll
+            for (int u = 0; u < kMine; ++u) {
+                const unsigned i = (unsigned)u * kCoopThreads + tid;
+                mine[u] = i < cnt ? s_cand[i] : 0ull;
+                if (i < cnt) atomicAdd(&hist[(unsigned)(mine[u] >> shift) & dmask], 1u);
             }
             __syncthreads();
-            select_digit(hist, tid, pre, &s_k, &s_prefix, &s_left, width);
+            select_digit(hist, tid, s_prefix, &s_k, &s_prefix, &s_left, width);
             __syncthreads();
             top -= width;
+            // keep the candidates of the chosen digit (all were read into registers above)
+            const unsigned long long pre = s_prefix;
+#pragma unroll
+            for (int u = 0; u < kMine; ++u) {
+                const unsigned i = (unsigned)u * kCoopThreads + tid;
+                if (i < cnt && (top < 0 ? mine[u] : (mine[u] >> (top + 1))) == pre) s_cand[atomicAdd(&s_n, 1u)] = mine[u];
+            }
+            __syncthreads();
+            cnt = s_n;
+            __syncthreads();
         }
     }
     __syncthreads();
     const unsigned long long T = s_prefix;
     const long long ties = s_k;        // keys equal to T to zero, lowest indices first
+    if (s_left == 1u) {
+        // a single key equals T (every CTA derived the same count): it is the last one zeroed, no order among equals
+        for (int i = tid; i < len; i += kCoopThreads) gamma[lo + i] = ks[i] <= T ? 0 : 1;
+        return;
+    }
     // keys equal to T in this slice
     {
         unsigned c = 0;
-        for (long long i = lo + tid; i < hi; i += kCoopThreads) c += key[i] == T ? 1u : 0u;
+        for (int i = tid; i < len; i += kCoopThreads) c += ks[i] == T ? 1u : 0u;
         for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, d);
         if ((tid & 31) == 0) warp_cnt[tid >> 5] = c;
         __syncthreads();
@@ -425,18 +559,18 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
-    for (long long base = lo; base < hi; base += kCoopThreads) {
-        const long long i = base + tid;
+    for (int base = 0; base < len; base += kCoopThreads) {
+        const int i = base + tid;
         unsigned long long v = ~0ull;
-        if (i < hi) v = key[i];
-        const bool eq = (i < hi) && (v == T);
+        if (i < len) v = ks[i];
+        const bool eq = (i < len) && (v == T);
         const unsigned ball = __ballot_sync(0xFFFFFFFFu, eq);
         if (lane == 0) warp_cnt[warp] = __popc(ball);
         __syncthreads();
         long long before = s_run;
         for (int w = 0; w < warp; ++w) before += warp_cnt[w];
         before += __popc(ball & ((1u << lane) - 1u));
-        if (i < hi) gamma[i] = (v < T || (eq && before < ties)) ? 0 : 1;
+        if (i < len) gamma[lo + i] = (v < T || (eq && before < ties)) ? 0 : 1;
         __syncthreads();
         if (tid == 0) {
             long long tot = 0;
@@ -581,7 +715,7 @@ bsp_status run_mask_small(const bsp_wdesc &wd, const void *W, int seg_len, long 
 }
 
 template <int DT>
-bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *scores, cudaStream_t st)
+bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *scores, unsigned long long *span, cudaStream_t st)
 {
     using acc_t = typename Acc<DT>::type;
     const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
@@ -594,18 +728,21 @@ bsp_status run_scores(const bsp_wdesc &wd, const void *W, bsp_norm norm, void *s
     acc_t *sc = (acc_t *)scores;
     if constexpr (DT != BSP_I8) {
         if (norm == BSP_NORM_VAR) {
-            if (HK == 1) score_kernel<DT, BSP_NORM_VAR, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
-            else score_kernel<DT, BSP_NORM_VAR, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+            if (HK == 1) score_kernel<DT, BSP_NORM_VAR, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
+            else score_kernel<DT, BSP_NORM_VAR, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
             BSP_CUDA_OK(cudaGetLastError());
             return BSP_OK;
         }
     }
+    // (one-tap layers: one thread per block)
+    const long long ctas1 = (NB + kScoreThreads - 1) / kScoreThreads;
+    const unsigned grid1 = (unsigned)(ctas1 < 148 * 8 ? ctas1 : 148 * 8);
     if (norm == BSP_NORM_L2) {
-        if (HK == 1) score_kernel<DT, BSP_NORM_L2, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
-        else score_kernel<DT, BSP_NORM_L2, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+        if (HK == 1) score_kernel<DT, BSP_NORM_L2, 1><<<grid1, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
+        else score_kernel<DT, BSP_NORM_L2, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
     } else {
-        if (HK == 1) score_kernel<DT, BSP_NORM_L1, 1><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
-        else score_kernel<DT, BSP_NORM_L1, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc);
+        if (HK == 1) score_kernel<DT, BSP_NORM_L1, 1><<<grid1, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
+        else score_kernel<DT, BSP_NORM_L1, 9><<<grid, kScoreThreads, 0, st>>>(Wp, wd.I, HK, wd.bo, wd.bi, NBo, NBi, sc, span);
     }
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
@@ -637,38 +774,45 @@ bsp_status launch_mask(const bsp_wdesc &wd, const void *W, bsp_norm norm, bsp_sc
             if (small != BSP_ERR_CAPACITY) return small;
         }
     }
-    if (wd.wtype == BSP_F32) rc = run_scores<BSP_F32>(wd, W, norm, scores, st);
-    else if (wd.wtype == BSP_BF16) rc = run_scores<BSP_BF16>(wd, W, norm, scores, st);
-    else rc = run_scores<BSP_I8>(wd, W, norm, scores, st);
-    if (rc != BSP_OK) return rc;
     const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi;
     const long long NB = (long long)NBo * NBi;
     const long long seg = (scope == BSP_SCOPE_LAYER) ? NB : NBi;
     const unsigned nseg = (scope == BSP_SCOPE_LAYER) ? 1u : (unsigned)NBo;
+    // one large segment: the select runs on a cooperative grid; its histograms, counter and the span of the keys (filled
+    // by the score kernel) are zeroed first
+    const bool coop = ws != nullptr && nseg == 1 && seg > kRankMax && n_zero > 0 && n_zero < seg;
+    unsigned *ghist = coop ? (unsigned *)((char *)ws + kWsHeader + align_up((size_t)NB * 8, 256)) : nullptr;
+    unsigned *gcount = coop ? ghist + 8 * 256 : nullptr;     // [0] candidate counter, [2..3] OR of the keys, [4..5] OR of their complements
+    if (coop) BSP_CUDA_OK(cudaMemsetAsync(ghist, 0, (8 * 256 + 8) * sizeof(unsigned), st));
+    unsigned long long *span = coop ? (unsigned long long *)(gcount + 2) : nullptr;
+    if (wd.wtype == BSP_F32) rc = run_scores<BSP_F32>(wd, W, norm, scores, span, st);
+    else if (wd.wtype == BSP_BF16) rc = run_scores<BSP_BF16>(wd, W, norm, scores, span, st);
+    else rc = run_scores<BSP_I8>(wd, W, norm, scores, span, st);
+    if (rc != BSP_OK) return rc;
     if (seg <= kRankMax)
         rank_kernel<<<dim3(nseg, (unsigned)((seg * kRankLanes + kRankThreads - 1) / kRankThreads)), kRankThreads, 0, st>>>(
             (const unsigned long long *)scores, (int)seg, n_zero, gamma);
-    else if (ws != nullptr && nseg == 1 && n_zero > 0 && n_zero < seg) {
-        // one large segment: the select runs on a cooperative grid of at most one CTA per SM
+    else if (coop) {
+        // at most one CTA per SM
         static int sm_count[64] = {};
         int dev = 0;
         BSP_CUDA_OK(cudaGetDevice(&dev));
         if (dev < 0 || dev >= 64) return BSP_ERR_CUDA;
-        if (sm_count[dev] == 0) BSP_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        if (sm_count[dev] == 0) {
+            BSP_CUDA_OK(cudaFuncSetAttribute(select_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCoopSmem));
+            BSP_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        }
         long long grid = (seg + 2 * kCoopThreads - 1) / (2 * kCoopThreads);
         if (grid > sm_count[dev]) grid = sm_count[dev];
         if (grid > kSelectMaxCtas) grid = kSelectMaxCtas;
-        unsigned *ghist = (unsigned *)((char *)ws + kWsHeader + align_up((size_t)NB * 8, 256));
-        unsigned *gcount = ghist + 8 * 256;                      // candidate counter (4 words kept for alignment)
-        unsigned *geq = gcount + 4;
+        unsigned *geq = gcount + 8;
         unsigned long long *cand = (unsigned long long *)(geq + kSelectMaxCtas);
-        BSP_CUDA_OK(cudaMemsetAsync(ghist, 0, (8 * 256 + 4) * sizeof(unsigned), st));
         const unsigned long long *keys = (const unsigned long long *)scores;
         long long n = seg, nz = n_zero;
         unsigned *sync = (unsigned *)ws + kWsSyncWord;
         int *status = (int *)ws;
         void *args[] = {&keys, &n, &nz, &gamma, &ghist, &gcount, &cand, &geq, &sync, &status};
-        const cudaError_t e = cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, 0, st);
+        const cudaError_t e = cudaLaunchCooperativeKernel((const void *)select_coop_kernel, dim3((unsigned)grid), dim3(kCoopThreads), args, kCoopSmem, st);
         if (e == cudaErrorCooperativeLaunchTooLarge) {
             (void)cudaGetLastError();
             select_kernel<<<nseg, kSelectThreads, 0, st>>>((const unsigned long long *)scores, seg, n_zero, gamma);
