@@ -458,18 +458,9 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
         const unsigned long long prefix = s_prefix;
         const int width = min(8, top + 1), shift = top + 1 - width;
         const unsigned dmask = (1u << width) - 1u;
-        // lanes with the same digit add once
-        for (int base = 0; base < len; base += kCoopThreads) {
-            const int i = base + tid;
-            unsigned long long v = 0ull;
-            bool in = false;
-            if (i < len) {
-                v = ks[i];
-                in = top >= 63 || ((v >> (top + 1)) == prefix);
-            }
-            const unsigned digit = in ? ((unsigned)(v >> shift) & dmask) : 256u;
-            const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
-            if (in && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+        for (int i = tid; i < len; i += kCoopThreads) {
+            const unsigned long long v = ks[i];
+            if (top >= 63 || ((v >> (top + 1)) == prefix)) atomicAdd(&hist[(unsigned)(v >> shift) & dmask], 1u);
         }
         __syncthreads();
         if (tid < 256 && hist[tid]) atomicAdd(&ghist[pi * 256 + tid], hist[tid]);
@@ -500,7 +491,7 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
         for (unsigned i = tid; i < cnt; i += kCoopThreads) s_cand[i] = __ldcg(&cand[i]);
         __syncthreads();
         constexpr int kMine = kLocalMax / kCoopThreads;    // candidates per thread
-        while (top >= 0) {
+        while (top >= 0 && cnt > (unsigned)kCoopThreads) {
             if (tid < 256) hist[tid] = 0u;
             if (tid == 0) s_n = 0u;
             __syncthreads();
@@ -528,6 +519,23 @@ select_coop_kernel(const unsigned long long *__restrict__ key, long long n, long
             __syncthreads();
             cnt = s_n;
             __syncthreads();
+        }
+        if (top >= 0) {
+            // at most one candidate per thread is left: each counts the candidates below its own and equal to it; the
+            // s_k-th smallest is the threshold (threads holding equal keys write the same values)
+            const long long need = s_k;
+            __syncthreads();
+            if ((unsigned)tid < cnt) {
+                const unsigned long long v = s_cand[tid];
+                unsigned less = 0u, same = 0u;
+                for (unsigned j = 0; j < cnt; ++j) {
+                    const unsigned long long o = s_cand[j];
+                    less += o < v ? 1u : 0u;
+                    same += o == v ? 1u : 0u;
+                }
+                if ((long long)less < need && need <= (long long)(less + same)) { s_prefix = v; s_k = need - less; s_left = same; }
+            }
+            top = -1;
         }
     }
     __syncthreads();
