@@ -18,8 +18,9 @@
 // compact blocks (cp.async expansion of the block-CSR payload in shared memory, or TMA gather loads of 128-byte
 // cores) was measured two to five times slower than these dense loads.
 //
-// Warps: 0 producer (one thread), 1 MMA issuer (the whole warp runs the loop so that its address arithmetic stays
-// warp-uniform), 2-5 epilogue (warp w reads the tensor-memory lanes 32 (w % 4) ..).  Barriers per stage: full (one
+// Warps: 0 producer and 1 MMA issuer (each runs its loop as a whole, converged warp with warp-uniform values; one
+// elected lane issues), 2-9 epilogue in two groups of four (warp w reads the tensor-memory lanes 32 (w % 4) ..; group g
+// drains accumulator buffer g, so the epilogues of two consecutive tiles overlap).  Barriers per stage: full (one
 // arrival that announces the bytes of both loads) and empty (tcgen05.commit); per accumulator buffer: acc_full (commit)
 // and acc_empty (4 warps).  Every wait is bounded; on expiry BSP_ERR_TIMEOUT is latched, the roles wind down, loads
 // in flight are awaited (bounded) and tensor memory is freed.
@@ -29,7 +30,7 @@
 namespace bsp {
 namespace {
 
-constexpr int kGtThreads = 192;
+constexpr int kGtThreads = 320;                    // producer warp, MMA warp, two groups of four epilogue warps
 constexpr int kGtBM = 128;                         // positions per tile (M of the MMA)
 constexpr int kGtABytes = kGtBM * 128;             // activation bytes of a stage
 constexpr int kGtStageRows = 32;                   // rows of Y per epilogue warp
@@ -352,18 +353,20 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
     } else {
-        // ================= epilogue (warps 2-5) =================
+        // ================= epilogue (warps 2-9) =================
+        // Two groups of four warps: group g drains accumulator buffer g, that is every second tile of the CTA, so the
+        // epilogues of two consecutive tiles run side by side.
         if (run) {
             const int q = warp & 3;                              // quarter of the tensor-memory lanes this warp reaches
-            const int ew = warp - 2;
+            const int ew = warp - 2, grp = ew >> 2;
             const int ey = p.ey;
             const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
-            const uint32_t stg0 = staging + (uint32_t)(ew * 2 * kGtStagingBytes);
-            uint32_t tile_i = 0, rounds_done = 0;
+            const uint32_t sb = staging + (uint32_t)(ew * kGtStagingBytes);      // this warp's staging buffer
+            uint32_t tile_i = (uint32_t)grp;
             bool ok = true;
             // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
             const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
-            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
+            for (int tile = t_first + grp * t_step; tile < t_count && ok; tile += 2 * t_step, tile_i += 2) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
                 int mt, tn;
                 gt_divmod(tile, p.n_tiles_n, p.m_ntn, mt, tn);
@@ -381,7 +384,7 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16) + buf * 256u;
-                for (int c0 = 0; c0 < BN; c0 += cpr, ++rounds_done) {
+                for (int c0 = 0; c0 < BN; c0 += cpr) {
                     uint32_t out[32];                            // 128 bytes of this lane's row of Y
                     if (ey == 4) {                               // fp32 or int32 output: 32 channels
                         uint32_t v[32];
@@ -428,9 +431,9 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                             }
                         }
                     }
-                    // the staging buffer of this round was handed to a TMA store two rounds ago: wait until it has been read
-                    const uint32_t sb = stg0 + (rounds_done & 1u) * (uint32_t)kGtStagingBytes;
-                    if (lane == 0 && p.store_tma) asm volatile("cp.async.bulk.wait_group.read 1;\n" ::: "memory");
+                    // the staging buffer was handed to a TMA store in the previous round: wait until it has been read (the
+                    // loads and the arithmetic of this round ran meanwhile)
+                    if (lane == 0 && p.store_tma) asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
                     __syncwarp();
                     const uint32_t srow = sb + (uint32_t)lane * 128u;
 #pragma unroll
@@ -441,11 +444,9 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                         __syncwarp();
                         // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
-                        // (every round commits a group, an empty one when nothing is stored: the wait above counts rounds)
-                        if (lane == 0) {
-                            if (n0 + c0 < p.O && m0 + q * 32 < p.P)
-                                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
-                                             ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
+                        if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
+                                         ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
                             asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
                         }
                     } else {
@@ -618,7 +619,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
         }
     }
     p.n_tiles_n = (wd.O + p.BN - 1) / p.BN;
-    if (T.tiles * p.n_tiles_n > 0x7FFFFFFF) return BSP_ERR_SHAPE;
+    if (T.tiles * p.n_tiles_n > 0x7FFFFFFF - 4096) return BSP_ERR_SHAPE;      // (tile counters step by up to twice the grid)
     p.n_tiles = (int)(T.tiles * p.n_tiles_n);
     // Large products run on CTA pairs: two position tiles side by side on one 256-channel tile, every CTA loading its
     // own activations and half of the weights (the operand fetch per SM and MMA falls from 12 KB to 8 KB).
@@ -629,7 +630,7 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
     p.m_ntn = gt_magic(p.n_tiles_n); p.m_tx = gt_magic(p.tiles_x); p.m_ty = gt_magic(p.tiles_y);
     p.stage_bytes = kGtABytes + (pair ? p.BN / 2 : p.BN) * 128;
-    const int staging = 4 * 2 * kGtStagingBytes;
+    const int staging = 8 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
     if (stages > kGtMaxStages) stages = kGtMaxStages;
     if (stages < 2) return BSP_ERR_SHAPE;
