@@ -23,6 +23,7 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -456,6 +457,41 @@ int ref_requant_i8(int64_t rows, int O, const int32_t *y32, const int32_t *shift
             if (q < -128) q = -128;
             y8[p * O + o] = (int8_t)q;
         }
+    return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Two consecutive layers evaluated tile by tile with the tensor between them kept on chip
+ * (Section "Depth-wise Tiling").  The result is that of running the layers one after the other;
+ * what the fused evaluation fixes is the precision of the tensor in between, which is stored as
+ * bfloat16.  ref_round_bf16 rounds float64 values to the nearest bfloat16 (8 significant bits,
+ * ties to the even mantissa) and returns them as float32; ref_relu_f64 is max(v, 0).
+ * The chain itself is composed by the caller from ref_conv2d_f32, these two and ref_gemm_f32.
+ * Values are assumed finite and inside the normal range of bfloat16.
+ * ------------------------------------------------------------------------------------------- */
+int ref_round_bf16(int64_t n, const double *in, float *out)
+{
+    if (n < 0) return ORACLE_ERR_SHAPE;
+    for (int64_t i = 0; i < n; ++i) {
+        const double v = in[i];
+        if (v == 0.0) { out[i] = 0.0f; continue; }
+        int e;
+        const double m = frexp(fabs(v), &e);              /* |v| = m 2^e, 0.5 <= m < 1 */
+        const double scaled = ldexp(m, 8);                /* 128 <= scaled < 256: 8 significant bits */
+        double q = floor(scaled);
+        const double rest = scaled - q;
+        if (rest > 0.5 || (rest == 0.5 && fmod(q, 2.0) == 1.0)) q += 1.0;
+        const double r = ldexp(q, e - 8);
+        out[i] = (float)(v < 0 ? -r : r);                  /* exact: 8 bits fit a float */
+    }
+    return ORACLE_OK;
+}
+
+int ref_relu_f64(int64_t n, double *v)
+{
+    if (n < 0) return ORACLE_ERR_SHAPE;
+    for (int64_t i = 0; i < n; ++i)
+        if (v[i] < 0.0) v[i] = 0.0;
     return ORACLE_OK;
 }
 

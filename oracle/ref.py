@@ -195,6 +195,26 @@ def requant_i8(y32: np.ndarray, shift: np.ndarray) -> np.ndarray:
     return y8
 
 
+def round_bf16(v: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bfloat16 (ties to even), returned as float32."""
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.float32)
+    _check(lib().ref_round_bf16(C.c_int64(v.size), _p(v), _p(out)), "round_bf16")
+    return out
+
+
+def chain2(w1shape, bo1, bi1, c1, X, b1, relu, O2, bo2, bi2, c2, b2, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
+    """Two consecutive layers with the tensor between them stored as bfloat16 (Section "Depth-wise Tiling"):
+    T = bf16(act(W1 * X + b1)), Y = W2 * T + b2 with a 1x1 second layer.  c1, c2 are (row_ptr, col_idx, payload) of
+    the two layers; rows of the result = output positions."""
+    T = conv2d(w1shape, bo1, bi1, c1[0], c1[1], c1[2], X, b1, stride, pad)
+    if relu:
+        _check(lib().ref_relu_f64(C.c_int64(T.size), _p(T)), "relu")
+    Tb = round_bf16(T)
+    O1 = w1shape[0]
+    return gemm(O2, O1, bo2, bi2, c2[0], c2[1], np.asarray(c2[2]).reshape(-1, bo2, bi2), Tb, b2)
+
+
 def spgemm(kb, a, b) -> np.ndarray:
     """C = (Gamma . A)(Omega . B)^t from two compact forms (row_ptr, col_idx, payload [nnz][kb][kb]) with kb x kb blocks;
     dense float64 [NBa*kb][NBb*kb]."""
