@@ -193,6 +193,22 @@ bsp_status bsp_gemm_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, in
 bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc *xd, const void *X,
                          const int32_t *bias, const int32_t *shift, int8_t *Y, void *ws, void *stream);
 
+/* ---- Two consecutive layers in one kernel (Section "Depth-wise Tiling": the output is cut into tiles, each tile is
+ * carried through the chain of layers, and the tensors between the layers stay on chip) ----------------------------
+ * bsp_conv2d_chain: T = act(W1 * X + bias1) rounded to bfloat16 (nearest even), Y = W2 * T + bias2, where layer one is
+ *             any convolution that bsp_conv2d takes (taps, strides, zero padding as given by xd) with at most 256
+ *             output channels, act is max(., 0) if relu != 0 and the identity otherwise, and layer two is a 1x1
+ *             layer on those channels (wd2->H = wd2->K = 1, wd2->I = wd1->O).  Both layers BF16 (weights and X),
+ *             accumulation and both biases float32 (device, may be NULL), Y [N][M][N_w][O2] F32 or BF16.  T is never
+ *             written to memory: a tile of 128 output positions of layer one is its own input tile of layer two.
+ *             w1 / w2: compact forms of the two layers from bsp_compact (`packed` is read; its header is compared with
+ *             the descriptors as in bsp_conv2d).  ws: any workspace of at least 256 bytes (status word only).
+ * Errors: NULL, SHAPE (second layer not 1x1 on O1 channels, O1 > 256, misaligned buffers), BLOCK, DTYPE (not BF16;
+ *         ytype not F32 / BF16), INDEX (nnz out of range; a packed buffer does not match: latched), CUDA. */
+bsp_status bsp_conv2d_chain(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
+                            const bsp_xdesc *xd, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
+                            bsp_dtype ytype, void *ws, void *stream);
+
 /* ---- Block-sparse x block-sparse product (Section "Block-Sparse Matrix-Matrix Multiplication") and the relative column
  * index (Section "Block Sparsity in a Matrix": "a relative row/col index") ------------------------------------------
  * bsp_spgemm: C = (Gamma . A)(Omega . B)^t, i.e. C_{i,j} = sum over the block columns k that row i of A and row j of B

@@ -1,0 +1,453 @@
+// Two consecutive block-sparse layers in one kernel: T = act(W1 * X + b1) stored as bfloat16, Y = W2 * T + b2 with a 1x1
+// second layer.  Section "Depth-wise Tiling" of the paper: the output is cut into tiles, every tile is carried through
+// the whole chain, and the tensor between the layers never goes to external memory.  A 1x1 second layer needs no
+// overlap between tiles (its projection of one output position is one position of T), so the tiles are those of the
+// first layer.
+//
+// Per tile of up to 128 output positions a persistent CTA runs
+//   1. the first layer as an implicit GEMM over taps x 128-byte channel chunks (activation box + weight tile per
+//      K-stage, both by tiled TMA loads) into accumulator one, all O1 <= 256 channels in tensor memory;
+//   2. its epilogue: tensor memory -> registers -> + b1 -> max(., 0) if asked -> bfloat16 -> shared memory, written in
+//      the K-major 128-byte-swizzled layout that an MMA reads as its A operand (64 channels per 16 KB chunk);
+//   3. the second layer: for every tile of 128 output channels, MMAs of that tensor against weight chunks that arrive
+//      through the same ring of stages, into one of two 128-column accumulators;
+//   4. its epilogue: + b2 -> convert -> global memory, overlapping the MMAs of the next 128 channels.
+// Warps: 0 producer, 1 MMA issuer (both converged, one elected lane issues), 2-5 epilogue.  Every wait is bounded.
+#include "bsp_tc.cuh"
+
+namespace bsp {
+namespace {
+
+constexpr int kCtThreads = 192;
+constexpr int kCtBN2 = 128;                        // channels of layer two per accumulator buffer
+constexpr int kCtChunk = kGtBM * 128;              // bytes of one 64-channel chunk of the tensor between the layers
+
+struct CtParams {
+    CUtensorMap tmx;          // X as bytes: (I1 * 2, J, L, N), box 128 bytes x Wt x Ht x Nt positions
+    CUtensorMap tmw1;         // Gamma1 (.) W1 as bytes: (I1 * 2, H K, O1), box 128 bytes x 1 tap x O1p channels
+    CUtensorMap tmw2;         // Gamma2 (.) W2 as bytes: (O1 * 2, 1, O2), box 128 bytes x 1 x 128 channels
+    const float *bias1, *bias2;
+    const uint8_t *packed1, *packed2;
+    int *status;
+    int O1, I1, H, K, bo1, bi1, O2, bo2, bi2, relu, ytype, ey;
+    int O1p;                  // O1 rounded up to 64: columns of accumulator one
+    int n_ks1, cpt1, n_c2, n_t2;      // K-stages of layer one, its channel chunks per tap; chunks of T; channel tiles of layer two
+    int stages, stage_bytes, n_tiles;
+    int N, M, Nw, Wt, Ht, Nt, tiles_x, tiles_y, rows_tile, P;
+    int sh, sw, ph, pw, a_bytes;
+    uint32_t m_tx, m_ty;
+    uint8_t *Y;
+};
+
+__device__ __forceinline__ void ct_tile_origin(const CtParams &p, int mt, int &n0, int &y0, int &x0)
+{
+    int r, tx, ty, ni;
+    gt_divmod(mt, p.tiles_x, p.m_tx, r, tx);
+    gt_divmod(r, p.tiles_y, p.m_ty, ni, ty);
+    x0 = tx * p.Wt; y0 = ty * p.Ht; n0 = ni * p.Nt;
+}
+
+__device__ __forceinline__ bool ct_header_ok(const uint8_t *packed, int O, int I, int H, int K, int bo, int bi)
+{
+    const PackedHeader *h = (const PackedHeader *)packed;
+    return h->magic == kPackedMagic && h->dtype == BSP_BF16 && h->O == O && h->I == I && h->H == H && h->K == K && h->bo == bo &&
+           h->bi == bi && (h->forms & kFormDense) != 0;
+}
+
+__global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_constant__ CtParams p)
+{
+    extern __shared__ __align__(16) uint8_t ct_smem_raw[];
+    uint8_t *smem = ct_smem_raw + ((1024u - (sm32(ct_smem_raw) & 1023u)) & 1023u);
+    __shared__ __align__(8) uint64_t s_full[kGtMaxStages], s_empty[kGtMaxStages];
+    __shared__ __align__(8) uint64_t s_acc1_full, s_acc1_empty, s_t_full, s_t_empty, s_acc2_full[2], s_acc2_empty[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ volatile uint32_t s_fail;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int S = p.stages;
+    const uint32_t ring = sm32(smem);
+    const uint32_t tbuf = ring + (uint32_t)(S * p.stage_bytes);          // the tensor between the layers: n_c2 chunks
+    const uint32_t staging = tbuf + (uint32_t)(p.n_c2 * kCtChunk);
+    const int t_first = (int)blockIdx.x, t_step = (int)gridDim.x, t_count = p.n_tiles;
+
+    if (tid == 0) {
+        const bool ok = ct_header_ok(p.packed1, p.O1, p.I1, p.H, p.K, p.bo1, p.bi1) && ct_header_ok(p.packed2, p.O2, p.O1, 1, 1, p.bo2, p.bi2);
+        s_fail = ok ? 0u : 2u;
+        if (!ok) atomicMax(p.status, (int)BSP_ERR_INDEX);
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_full[s])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_empty[s])), "r"(1) : "memory");
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_full)), "r"(1) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_empty)), "r"(4) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_full)), "r"(4) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_empty)), "r"(1) : "memory");
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc2_full[b])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc2_empty[b])), "r"(4) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmx) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmw1) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmw2) : "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const uint32_t tmem = s_tmem;
+    const bool run = s_fail == 0u;
+    const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
+
+    if (warp == 0) {
+        // ================= producer =================
+        if (run) {
+            const uint32_t stage_bytes = (uint32_t)p.stage_bytes;
+            const uint32_t tx1 = (uint32_t)(p.a_bytes + p.O1p * 128), tx2 = (uint32_t)(kCtBN2 * 128);
+            const int cpt128 = p.cpt1 * 128, Kw = p.K;
+            uint32_t slot = 0, epar = 1, issued = 0, dst = ring;      // (a fresh barrier counts as released)
+            bool ok = true;
+            for (int tile = t_first; tile < t_count && ok; tile += t_step) {
+                int n0, y0, x0;
+                ct_tile_origin(p, tile, n0, y0, x0);
+                const int xi0 = x0 * p.sw - p.pw;
+                int c128 = 0, kx = xi0, hy = y0 * p.sh - p.ph, tap = 0, kk = 0;
+                if (s_fail) { ok = false; break; }
+                // layer one: the activation box shifted by the tap and that tap's weights, per 128-byte chunk of channels
+                for (int ks = 0; ks < p.n_ks1; ++ks) {
+                    bool got = gt_poll(empty0 + slot * 8u, epar);
+                    got = __all_sync(0xFFFFFFFFu, got);
+                    if (!got) { ok = false; break; }
+                    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                                 " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
+                                 " @e cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%0];\n"
+                                 " @e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%4, %10, %11}], [%0];\n}\n"
+                                 ::"r"(full0 + slot * 8u), "r"(tx1), "r"(dst), "l"(&p.tmx), "r"(c128), "r"(kx), "r"(hy), "r"(n0),
+                                   "r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw1), "r"(tap), "r"(0) : "memory");
+                    ++issued;
+                    if (++slot == (uint32_t)S) { slot = 0; epar ^= 1u; dst = ring; } else dst += stage_bytes;
+                    c128 += 128;
+                    if (c128 == cpt128) {
+                        c128 = 0; ++tap; ++kx;
+                        if (++kk == Kw) { kk = 0; kx = xi0; ++hy; }
+                    }
+                }
+                // layer two: for every tile of 128 output channels, the weight chunk of each 64 channels of T
+                for (int t2 = 0; t2 < p.n_t2 && ok; ++t2)
+                    for (int c2 = 0; c2 < p.n_c2; ++c2) {
+                        bool got = gt_poll(empty0 + slot * 8u, epar);
+                        got = __all_sync(0xFFFFFFFFu, got);
+                        if (!got) { ok = false; break; }
+                        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
+                                     " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
+                                     " @e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6}], [%0];\n}\n"
+                                     ::"r"(full0 + slot * 8u), "r"(tx2), "r"(dst), "l"(&p.tmw2), "r"(c2 * 128), "r"(0), "r"(t2 * kCtBN2) : "memory");
+                        ++issued;
+                        if (++slot == (uint32_t)S) { slot = 0; epar ^= 1u; dst = ring; } else dst += stage_bytes;
+                    }
+            }
+            if (!ok && lane == 0) {
+                // winding down after a wait that ran out: the loads already issued still write into this CTA's shared
+                // memory, so the barriers of the stages in flight are awaited (bounded) before the CTA may leave
+                atomicExch((uint32_t *)&s_fail, 1u);
+                for (uint32_t back = 0; back < (uint32_t)S && back < issued; ++back) {
+                    const uint32_t it = issued - 1u - back;
+                    gt_poll(full0 + (it % (uint32_t)S) * 8u, (it / (uint32_t)S) & 1u);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (run) {
+            // instruction descriptors: D fp32, A and B bf16, K-major both, M = 128; N = O1p for layer one, 128 for layer two
+            const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.O1p >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCtBN2 >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
+            uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0, u2 = 0;
+            bool ok = true;
+            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
+                // accumulator one is free once the previous tile's first epilogue has read it
+                if (!gt_poll(sm32(&s_acc1_empty), (tile_i & 1u) ^ 1u) || s_fail != 0u) ok = false;
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                for (int ks = 0; ks < p.n_ks1; ++ks) {
+                    bool got = gt_poll(full0 + slot * 8u, par);
+                    got = __all_sync(0xFFFFFFFFu, got);
+                    if (!got) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
+                    gt_issue_stage<false>(BSP_BF16, tmem, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
+                }
+                if (!ok) break;
+                gt_commit_elected<false>(sm32(&s_acc1_full));
+                // the tensor between the layers is in shared memory once the first epilogue has written it
+                if (!gt_poll(sm32(&s_t_full), tile_i & 1u)) ok = false;
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                for (int t2 = 0; t2 < p.n_t2 && ok; ++t2, ++u2) {
+                    const uint32_t buf = u2 & 1u, use = u2 >> 1;
+                    if (!gt_poll(sm32(&s_acc2_empty[buf]), (use & 1u) ^ 1u)) ok = false;
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    const uint32_t d = tmem + 256u + buf * (uint32_t)kCtBN2;
+                    for (int c2 = 0; c2 < p.n_c2; ++c2) {
+                        bool got = gt_poll(full0 + slot * 8u, par);
+                        got = __all_sync(0xFFFFFFFFu, got);
+                        if (!got) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                        const uint64_t da = kGtDesc | (uint64_t)(((tbuf + (uint32_t)(c2 * kCtChunk)) >> 4) & 0x3FFFu);
+                        const uint64_t db = kGtDesc | (uint64_t)(a16 & 0x3FFFu);
+                        gt_issue_stage<false>(BSP_BF16, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
+                        if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
+                    }
+                    if (ok) gt_commit_elected<false>(sm32(&s_acc2_full[buf]));
+                }
+                // all MMAs that read the tensor have been issued: their completion frees it for the next tile
+                if (ok) gt_commit_elected<false>(sm32(&s_t_empty));
+            }
+            if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
+        }
+    } else {
+        // ================= epilogues (warps 2-5) =================
+        if (run) {
+            const int q = warp & 3;                              // quarter of the tensor-memory lanes this warp reaches
+            const int ey = p.ey;
+            const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
+            const uint32_t sb = staging + (uint32_t)((warp - 2) * kGtStagingBytes);
+            uint32_t tile_i = 0, u2 = 0;
+            bool ok = true;
+            // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
+            const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
+            const uint32_t trow = tbuf + (uint32_t)r * 128u;     // this lane's row of a chunk of T
+            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
+                int in0, y0, x0;
+                ct_tile_origin(p, tile, in0, y0, x0);
+                const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
+                const long long pos = ((long long)(in0 + ri) * p.M + (y0 + rh)) * p.Nw + (x0 + rw);
+                const unsigned long long row_off = (unsigned long long)pos * (unsigned long long)(p.O2 * ey);
+                // ---- first epilogue: accumulator one -> + b1 -> activation -> bfloat16 -> T in shared memory ----
+                // (T may be overwritten once the MMAs of the previous tile's second layer have read it)
+                if (!gt_wait(sm32(&s_acc1_full), tile_i & 1u) || !gt_wait(sm32(&s_t_empty), (tile_i & 1u) ^ 1u)) ok = false;
+                if (s_fail) ok = false;
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const uint32_t t1 = tmem + ((uint32_t)(q * 32) << 16);
+                for (int c2 = 0; c2 < p.n_c2; ++c2) {
+                    uint32_t out[32];                            // 64 channels of this lane's row of T
+#pragma unroll
+                    for (int sub = 0; sub < 2; ++sub) {
+                        uint32_t v[32];
+                        gt_load32(t1 + (uint32_t)(c2 * 64 + sub * 32), v);
+                        const int ch = c2 * 64 + sub * 32 + lane;
+                        const float bl = (p.bias1 != nullptr && ch < p.O1) ? __ldg(p.bias1 + ch) : 0.f;     // lane e: bias of channel .. + e
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            float a = __uint_as_float(v[2 * e]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e);
+                            float b = __uint_as_float(v[2 * e + 1]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e + 1);
+                            if (p.relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                            out[sub * 16 + e] = *(const uint32_t *)&h;
+                        }
+                    }
+                    // K-major rows of 128 bytes under the 128-byte swizzle: the 16-byte piece j of row r sits at piece j ^ (r % 8)
+                    const uint32_t dst = trow + (uint32_t)(c2 * kCtChunk);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                                     ::"r"(dst + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
+                }
+                // the MMAs read T through the asynchronous proxy
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc1_empty)) : "memory");
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_t_full)) : "memory");
+                }
+                // ---- second epilogue, per tile of 128 output channels: + b2 -> convert -> Y ----
+                for (int t2 = 0; t2 < p.n_t2 && ok; ++t2, ++u2) {
+                    const uint32_t buf = u2 & 1u, use = u2 >> 1;
+                    const int n0 = t2 * kCtBN2;
+                    if (!gt_wait(sm32(&s_acc2_full[buf]), use & 1u)) ok = false;
+                    if (s_fail) ok = false;
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    const uint32_t t2base = t1 + 256u + buf * (uint32_t)kCtBN2;
+                    for (int c0 = 0; c0 < kCtBN2; c0 += cpr) {
+                        uint32_t out[32];                        // 128 bytes of this lane's row of Y
+                        if (ey == 4) {
+                            uint32_t v[32];
+                            gt_load32(t2base + (uint32_t)c0, v);
+                            const int ch = n0 + c0 + lane;
+                            const float bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg(p.bias2 + ch) : 0.f;
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) out[e] = __float_as_uint(__uint_as_float(v[e]) + __shfl_sync(0xFFFFFFFFu, bl, e));
+                        } else {
+#pragma unroll
+                            for (int sub = 0; sub < 2; ++sub) {
+                                uint32_t v[32];
+                                gt_load32(t2base + (uint32_t)(c0 + sub * 32), v);
+                                const int ch = n0 + c0 + sub * 32 + lane;
+                                const float bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg(p.bias2 + ch) : 0.f;
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * e]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e),
+                                                                                   __uint_as_float(v[2 * e + 1]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e + 1));
+                                    out[sub * 16 + e] = *(const uint32_t *)&h;
+                                }
+                            }
+                        }
+                        // staged in shared memory, read back four rows at a time, eight lanes per row: whole 128-byte pieces of rows of Y
+                        __syncwarp();
+                        const uint32_t srow = sb + (uint32_t)lane * 128u;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                                         ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
+                        __syncwarp();
+                        const int chunk = lane & 7;
+                        const bool ch_ok = (n0 + c0) * ey + chunk * 16 < p.O2 * ey;
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const int row = it * 4 + (lane >> 3);
+                            const unsigned long long off = __shfl_sync(0xFFFFFFFFu, row_off, row);
+                            const int okr = __shfl_sync(0xFFFFFFFFu, (int)row_ok, row);
+                            uint32_t a0, a1, a2, a3;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];\n"
+                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(sb + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4)) : "memory");
+                            if (okr && ch_ok)
+                                *(uint4 *)(p.Y + off + (unsigned long long)((n0 + c0) * ey + chunk * 16)) = make_uint4(a0, a1, a2, a3);
+                        }
+                    }
+                    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc2_empty[buf])) : "memory");
+                }
+            }
+            if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
+        }
+    }
+
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (s_fail == 1u && tid == 0) atomicMax(p.status, (int)BSP_ERR_TIMEOUT);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kGtTmemCols) : "memory");
+}
+
+}  // namespace
+
+// True if the fused kernel can run this pair: bfloat16 layers, a 1x1 second layer on the first one's output channels,
+// at most 256 of them (accumulator one holds them all), rows of X, of both weights and of Y that are multiples of 16 bytes.
+bool chain_tc_eligible(const bsp_wdesc &wd1, const bsp_wdesc &wd2, const bsp_xdesc &xd0, bsp_dtype ytype)
+{
+    if (wd1.wtype != BSP_BF16 || wd2.wtype != BSP_BF16) return false;
+    if (wd2.H != 1 || wd2.K != 1 || wd2.I != wd1.O) return false;
+    if (wd1.O > 256 || wd1.O % 8 != 0 || wd1.I % 8 != 0 || wd2.O % 8 != 0) return false;
+    if (ytype != BSP_F32 && ytype != BSP_BF16) return false;
+    if (!packed_layout(wd1).enabled || !packed_layout(wd2).enabled) return false;
+    const bsp_xdesc xd = gt_flatten(wd1, xd0);
+    const int M = (xd.L + 2 * xd.pad_h - wd1.H) / xd.stride_h + 1, Nw = (xd.J + 2 * xd.pad_w - wd1.K) / xd.stride_w + 1;
+    if (M <= 0 || Nw <= 0) return false;
+    if ((long long)xd.N * M * Nw > 0x7FFFFFFF - 4096 || (long long)xd.N * xd.L * xd.J > 0x7FFFFFFF) return false;
+    return gt_pick_tile(xd.N, M, Nw, xd.stride_h, xd.stride_w).tiles > 0;
+}
+
+bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_wdesc &wd2, const void *packed2,
+                           const bsp_xdesc &xd0, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
+                           bsp_dtype ytype, void *ws, cudaStream_t st)
+{
+    const bsp_xdesc xd = gt_flatten(wd1, xd0);
+    const PackedLayout L1 = packed_layout(wd1), L2 = packed_layout(wd2);
+    if (!L1.enabled || !L2.enabled) return BSP_ERR_SHAPE;
+    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    CtParams p = {};
+    p.bias1 = bias1; p.bias2 = bias2; p.packed1 = (const uint8_t *)packed1; p.packed2 = (const uint8_t *)packed2;
+    p.status = (int *)ws;
+    p.O1 = wd1.O; p.I1 = wd1.I; p.H = wd1.H; p.K = wd1.K; p.bo1 = wd1.bo; p.bi1 = wd1.bi;
+    p.O2 = wd2.O; p.bo2 = wd2.bo; p.bi2 = wd2.bi; p.relu = relu ? 1 : 0; p.ytype = ytype; p.ey = ey; p.Y = (uint8_t *)Y;
+    p.O1p = (wd1.O + 63) / 64 * 64;
+    p.N = xd.N; p.sh = xd.stride_h; p.sw = xd.stride_w; p.ph = xd.pad_h; p.pw = xd.pad_w;
+    p.M = (xd.L + 2 * xd.pad_h - wd1.H) / xd.stride_h + 1;
+    p.Nw = (xd.J + 2 * xd.pad_w - wd1.K) / xd.stride_w + 1;
+    const long long P = (long long)xd.N * p.M * p.Nw;
+    p.P = (int)P;
+    const GtTile T = gt_pick_tile(xd.N, p.M, p.Nw, p.sh, p.sw);
+    if (T.tiles <= 0 || T.tiles > 0x7FFFFFFF - 4096) return BSP_ERR_SHAPE;
+    p.Wt = T.Wt; p.Ht = T.Ht; p.Nt = T.Nt; p.rows_tile = T.Wt * T.Ht * T.Nt;
+    p.tiles_x = (p.Nw + T.Wt - 1) / T.Wt; p.tiles_y = (p.M + T.Ht - 1) / T.Ht;
+    p.m_tx = gt_magic(p.tiles_x); p.m_ty = gt_magic(p.tiles_y);
+    p.a_bytes = p.rows_tile * 128;
+    p.n_tiles = (int)T.tiles;
+    p.cpt1 = (wd1.I * 2 + 127) / 128;
+    p.n_ks1 = wd1.H * wd1.K * p.cpt1;
+    p.n_c2 = p.O1p / 64;
+    p.n_t2 = (wd2.O + kCtBN2 - 1) / kCtBN2;
+    p.stage_bytes = kGtABytes + p.O1p * 128;
+    const int fixed = 1024 + p.n_c2 * kCtChunk + 4 * kGtStagingBytes;
+    int stages = (kGtMaxSmem - fixed) / p.stage_bytes;
+    if (stages > kGtMaxStages) stages = kGtMaxStages;
+    if (stages < 2) return BSP_ERR_SHAPE;
+    p.stages = stages;
+    const size_t smem = (size_t)fixed + (size_t)stages * p.stage_bytes;
+
+    static bool opted[kGtMaxDevices] = {};
+    static int n_sm[kGtMaxDevices] = {};
+    int dev = 0;
+    BSP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
+    if (!opted[dev]) {
+        BSP_CUDA_OK(cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
+        opted[dev] = true;
+    }
+    GtEncodeFn enc = gt_encode();
+    if (!enc) return BSP_ERR_CUDA;
+    {
+        const cuuint64_t row = (cuuint64_t)wd1.I * 2;
+        const cuuint64_t gdim[4] = {row, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N};
+        const cuuint64_t gstr[3] = {row, row * xd.J, row * xd.J * xd.L};
+        const cuuint32_t box[4] = {128, (cuuint32_t)(T.Wt * p.sw), (cuuint32_t)(T.Ht * p.sh), (cuuint32_t)T.Nt};
+        const cuuint32_t estr[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
+        if (enc(&p.tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(X), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t row = (cuuint64_t)wd1.I * 2;
+        const cuuint64_t gdim[3] = {row, (cuuint64_t)(wd1.H * wd1.K), (cuuint64_t)wd1.O};
+        const cuuint64_t gstr[2] = {row, row * wd1.H * wd1.K};
+        const cuuint32_t box[3] = {128, 1, (cuuint32_t)p.O1p};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (enc(&p.tmw1, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed1 + L1.off_payload), gdim, gstr, box,
+                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t row = (cuuint64_t)wd2.I * 2;
+        const cuuint64_t gdim[3] = {row, 1, (cuuint64_t)wd2.O};
+        const cuuint64_t gstr[2] = {row, row};
+        const cuuint32_t box[3] = {128, 1, (cuuint32_t)kCtBN2};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (enc(&p.tmw2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed2 + L2.off_payload), gdim, gstr, box,
+                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
+    chain_tc_kernel<<<grid, kCtThreads, smem, st>>>(p);
+    BSP_CUDA_OK(cudaGetLastError());
+    return BSP_OK;
+}
+
+}  // namespace bsp
