@@ -392,6 +392,53 @@ def pass_spgemm(gpu, bsp, torch, reps=5):
     return out
 
 
+def pass_chain(gpu, bsp, torch, pk, reps=10):
+    """Fused pairs of layers (bsp_conv2d_chain) against the two separate calls through a bfloat16 tensor in memory: the
+    3x3 -> 1x1 tails of the ResNet50 bottlenecks, batch 64, bf16, 8x8 at 50 %, bf16 output.  The HBM roofline of the
+    fused call counts X in and Y out only: the tensor between the layers never leaves the chip."""
+    out = []
+    g = torch.Generator(device="cuda")
+    g.manual_seed(91)
+    for name, L, I, O1, O2 in (("c2.3x3.64-64+1x1.64-256", 56, 64, 64, 256), ("c3.3x3.128-128+1x1.128-512", 28, 128, 128, 512),
+                               ("c4.3x3.256-256+1x1.256-1024", 14, 256, 256, 1024)):
+        N = 64
+        W1 = (torch.randn((O1, 3, 3, I), device="cuda", generator=g) * (2.0 / (9 * I)) ** 0.5).to(torch.bfloat16)
+        W2 = (torch.randn((O2, 1, 1, O1), device="cuda", generator=g) * (2.0 / O1) ** 0.5).to(torch.bfloat16)
+        X = torch.randn((N, L, L, I), device="cuda", generator=g).to(torch.bfloat16)
+        b1 = torch.randn((O1,), device="cuda", generator=g) * 0.1
+        b2 = torch.randn((O2,), device="cuda", generator=g) * 0.1
+        l1 = bsp.SparseLayer(O1, I, 3, 3, 8, 8, torch.bfloat16, canonical=False)
+        l2 = bsp.SparseLayer(O2, O1, 1, 1, 8, 8, torch.bfloat16, canonical=False)
+        for lay, W in ((l1, W1), (l2, W2)):
+            lay.mask(W, lay.NBo * lay.NBi // 2)
+            lay.compact(W)
+        T = torch.empty((N, L, L, O1), dtype=torch.bfloat16, device="cuda")
+        Ya = torch.empty((N, L, L, O2), dtype=torch.bfloat16, device="cuda")
+        Yb = torch.empty_like(Ya)
+        xd = bsp.XDesc(N, L, L, 1, 1, 1, 1)
+
+        def separate():
+            l1.conv2d(X, b1, T, (1, 1), (1, 1))
+            l2.conv2d(T, b2, Ya)
+
+        def fused():
+            bsp.bsp_conv2d_chain(l1.wd, l1.handle(), l2.wd, l2.handle(), xd, X, b1, 0, b2, Yb, bsp.BF16, l1.ws)
+
+        ts = stats(gpu.timed(separate, reps, 2))
+        tf = stats(gpu.timed(fused, reps, 1))
+        l1.check()
+        l2.check()
+        P = N * L * L
+        useful = 2.0 * P * (l1.NBo * l1.NBi // 2) * 64 * 9 + 2.0 * P * (l2.NBo * l2.NBi // 2) * 64
+        hbm = X.numel() * 2 + Yb.numel() * 2 + (W1.numel() + W2.numel())
+        t_roof = max(useful / (pk["bf16_tflops"] * 1e12), hbm / (pk["hbm_gbs"] * 1e9)) * 1e3
+        out.append({"pair": name, "separate_ms": ts["ms"], "fused_ms": tf["ms"], "speedup": ts["ms"] / tf["ms"],
+                    "bit_identical": bool(torch.equal(Ya, Yb)), "effective_tflops": useful / (tf["ms"] * 1e-3) / 1e12,
+                    "algorithmic_bytes": hbm, "bytes_saved_vs_separate": 2 * T.numel() * 2, "roofline_ms": t_roof,
+                    "frac": t_roof / tf["ms"]})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -574,6 +621,7 @@ def main():
             "sum_ms": {str(s): {k: float(sum(r[k] * r["count"] for r in i8 if r["sparsity"] == s))
                                 for k in ("mask_ms", "compact_ms", "conv_ms", "step_ms")} for s in (0.5, 0.75)}}
         sweeps["spgemm_2048x4096_bf16_8x8"] = pass_spgemm(gpu, bsp, torch)
+        sweeps["chain_resnet50_tails_b64_bf16_8x8_50"] = pass_chain(gpu, bsp, torch, pk)
     clocks = sampler.stop()
 
     # max over ranks

@@ -12,13 +12,15 @@
 //   3. the second layer: for every tile of 128 output channels, MMAs of that tensor against weight chunks that arrive
 //      through the same ring of stages, into one of two 128-column accumulators;
 //   4. its epilogue: + b2 -> convert -> global memory, overlapping the MMAs of the next 128 channels.
-// Warps: 0 producer, 1 MMA issuer (both converged, one elected lane issues), 2-5 epilogue.  Every wait is bounded.
+// Warps: 0 producer, 1 MMA issuer (both converged, one elected lane issues), 2-9 epilogue in two groups of four: the
+// groups share the first epilogue (alternate 64-channel chunks) and each drains one of the two second accumulators.
+// Every wait is bounded.
 #include "bsp_tc.cuh"
 
 namespace bsp {
 namespace {
 
-constexpr int kCtThreads = 192;
+constexpr int kCtThreads = 320;                    // producer warp, MMA warp, two groups of four epilogue warps
 constexpr int kCtBN2 = 128;                        // channels of layer two per accumulator buffer
 constexpr int kCtChunk = kGtBM * 128;              // bytes of one 64-channel chunk of the tensor between the layers
 
@@ -79,8 +81,8 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_empty[s])), "r"(1) : "memory");
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_full)), "r"(1) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_empty)), "r"(4) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_full)), "r"(4) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_empty)), "r"(8) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_full)), "r"(8) : "memory");
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_empty)), "r"(1) : "memory");
         for (int b = 0; b < 2; ++b) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc2_full[b])), "r"(1) : "memory");
@@ -215,9 +217,10 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
     } else {
-        // ================= epilogues (warps 2-5) =================
+        // ================= epilogues (warps 2-9) =================
         if (run) {
             const int q = warp & 3;                              // quarter of the tensor-memory lanes this warp reaches
+            const int grp = (warp - 2) >> 2;
             const int ey = p.ey;
             const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
             const uint32_t sb = staging + (uint32_t)((warp - 2) * kGtStagingBytes);
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t t1 = tmem + ((uint32_t)(q * 32) << 16);
-                for (int c2 = 0; c2 < p.n_c2; ++c2) {
+                for (int c2 = grp; c2 < p.n_c2; c2 += 2) {
                     uint32_t out[32];                            // 64 channels of this lane's row of T
 #pragma unroll
                     for (int sub = 0; sub < 2; ++sub) {
@@ -275,6 +278,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 // ---- second epilogue, per tile of 128 output channels: + b2 -> convert -> Y ----
                 for (int t2 = 0; t2 < p.n_t2 && ok; ++t2, ++u2) {
                     const uint32_t buf = u2 & 1u, use = u2 >> 1;
+                    if ((int)buf != grp) continue;               // (the other group drains this accumulator)
                     const int n0 = t2 * kCtBN2;
                     if (!gt_wait(sm32(&s_acc2_full[buf]), use & 1u)) ok = false;
                     if (s_fail) ok = false;
@@ -393,7 +397,7 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
     p.n_c2 = p.O1p / 64;
     p.n_t2 = (wd2.O + kCtBN2 - 1) / kCtBN2;
     p.stage_bytes = kGtABytes + p.O1p * 128;
-    const int fixed = 1024 + p.n_c2 * kCtChunk + 4 * kGtStagingBytes;
+    const int fixed = 1024 + p.n_c2 * kCtChunk + 8 * kGtStagingBytes;
     int stages = (kGtMaxSmem - fixed) / p.stage_bytes;
     if (stages > kGtMaxStages) stages = kGtMaxStages;
     if (stages < 2) return BSP_ERR_SHAPE;
