@@ -448,6 +448,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweeps", action="store_true", help="headline only: skip the block-shape sweep and the layer-table passes")
+    ap.add_argument("--only-chain", action="store_true", help="of the extra passes run the fused pairs of layers only (for profiling)")
     ap.add_argument("--no-graph", action="store_true", help="launch the three calls of a step one by one instead of replaying a CUDA graph of them")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -600,7 +601,11 @@ def main():
 
     # ---- the sweeps (rank 0 of a single-GPU run): block shapes x sparsities on the headline layer, then the layer tables
     sweeps = {}
-    if rank == 0 and world == 1 and not args.no_sweeps:
+    if rank == 0 and world == 1 and args.only_chain:
+        del Xd, Y, Wh, Xh, Yh
+        torch.cuda.empty_cache()
+        sweeps["chain_resnet50_tails_b64_bf16_8x8_50"] = pass_chain(gpu, bsp, torch, pk, reps=2)
+    elif rank == 0 and world == 1 and not args.no_sweeps:
         gemm_layer, gdt, _, _, _, gsig = workload("gemm_4096_p8192")
         if layer.name == gemm_layer.name:
             sweeps["sweep_gemm_4096_p8192"] = sweep_product(gpu, bsp, torch, layer, dtype, Wd, Xd, bd, Y, pk)
