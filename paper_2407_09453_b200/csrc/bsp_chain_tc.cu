@@ -35,6 +35,7 @@ struct CtParams {
     int O1p;                  // O1 rounded up to 64: columns of accumulator one
     int n_ks1, cpt1, n_c2, n_t2;      // K-stages of layer one, its channel chunks per tap; chunks of T; channel tiles of layer two
     int stages, stage_bytes, n_tiles;
+    int db;                   // O1p <= 128: accumulator one and the tensor between the layers are double-buffered
     int N, M, Nw, Wt, Ht, Nt, tiles_x, tiles_y, rows_tile, P;
     int sh, sw, ph, pw, a_bytes;
     uint32_t m_tx, m_ty;
@@ -61,7 +62,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
     extern __shared__ __align__(16) uint8_t ct_smem_raw[];
     uint8_t *smem = ct_smem_raw + ((1024u - (sm32(ct_smem_raw) & 1023u)) & 1023u);
     __shared__ __align__(8) uint64_t s_full[kGtMaxStages], s_empty[kGtMaxStages];
-    __shared__ __align__(8) uint64_t s_acc1_full, s_acc1_empty, s_t_full, s_t_empty, s_acc2_full[2], s_acc2_empty[2];
+    __shared__ __align__(8) uint64_t s_acc1_full[2], s_acc1_empty[2], s_t_full[2], s_t_empty[2], s_acc2_full[2], s_acc2_empty[2];
     __shared__ uint32_t s_tmem;
     __shared__ volatile uint32_t s_fail;
 
@@ -69,7 +70,8 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
     const int S = p.stages;
     const uint32_t ring = sm32(smem);
     const uint32_t tbuf = ring + (uint32_t)(S * p.stage_bytes);          // the tensor between the layers: n_c2 chunks
-    const uint32_t staging = tbuf + (uint32_t)(p.n_c2 * kCtChunk);
+    const uint32_t tbytes = (uint32_t)(p.n_c2 * kCtChunk);
+    const uint32_t staging = tbuf + (p.db ? 2u : 1u) * tbytes;
     const int t_first = (int)blockIdx.x, t_step = (int)gridDim.x, t_count = p.n_tiles;
 
     if (tid == 0) {
@@ -80,10 +82,12 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_full[s])), "r"(1) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_empty[s])), "r"(1) : "memory");
         }
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_full)), "r"(1) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_empty)), "r"(8) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_full)), "r"(8) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_empty)), "r"(1) : "memory");
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_full[b])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc1_empty[b])), "r"(8) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_full[b])), "r"(8) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_t_empty[b])), "r"(1) : "memory");
+        }
         for (int b = 0; b < 2; ++b) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc2_full[b])), "r"(1) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(sm32(&s_acc2_empty[b])), "r"(4) : "memory");
@@ -112,17 +116,16 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             const int cpt128 = p.cpt1 * 128, Kw = p.K;
             uint32_t slot = 0, epar = 1, issued = 0, dst = ring;      // (a fresh barrier counts as released)
             bool ok = true;
-            for (int tile = t_first; tile < t_count && ok; tile += t_step) {
+            // layer one of a tile: the activation box shifted by the tap and that tap's weights, per 128-byte chunk of channels
+            auto load_layer_one = [&](int tile) {
                 int n0, y0, x0;
                 ct_tile_origin(p, tile, n0, y0, x0);
                 const int xi0 = x0 * p.sw - p.pw;
                 int c128 = 0, kx = xi0, hy = y0 * p.sh - p.ph, tap = 0, kk = 0;
-                if (s_fail) { ok = false; break; }
-                // layer one: the activation box shifted by the tap and that tap's weights, per 128-byte chunk of channels
                 for (int ks = 0; ks < p.n_ks1; ++ks) {
                     bool got = gt_poll(empty0 + slot * 8u, epar);
                     got = __all_sync(0xFFFFFFFFu, got);
-                    if (!got) { ok = false; break; }
+                    if (!got) { ok = false; return; }
                     asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
                                  " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
                                  " @e cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%0];\n"
@@ -137,12 +140,14 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         if (++kk == Kw) { kk = 0; kx = xi0; ++hy; }
                     }
                 }
-                // layer two: for every tile of 128 output channels, the weight chunk of each 64 channels of T
-                for (int t2 = 0; t2 < p.n_t2 && ok; ++t2)
+            };
+            // layer two: for every tile of 128 output channels, the weight chunk of each 64 channels of T
+            auto load_layer_two = [&]() {
+                for (int t2 = 0; t2 < p.n_t2; ++t2)
                     for (int c2 = 0; c2 < p.n_c2; ++c2) {
                         bool got = gt_poll(empty0 + slot * 8u, epar);
                         got = __all_sync(0xFFFFFFFFu, got);
-                        if (!got) { ok = false; break; }
+                        if (!got) { ok = false; return; }
                         asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
                                      " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
                                      " @e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6}], [%0];\n}\n"
@@ -150,6 +155,15 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         ++issued;
                         if (++slot == (uint32_t)S) { slot = 0; epar ^= 1u; dst = ring; } else dst += stage_bytes;
                     }
+            };
+            // the stages follow the order in which the MMA warp consumes them: with double buffers, layer one of the next
+            // tile goes before layer two of this one
+            if (p.db && t_first < t_count) load_layer_one(t_first);
+            for (int tile = t_first; tile < t_count && ok; tile += t_step) {
+                if (s_fail) { ok = false; break; }
+                if (p.db) { if (tile + t_step < t_count) load_layer_one(tile + t_step); }
+                else load_layer_one(tile);
+                if (ok) load_layer_two();
             }
             if (!ok && lane == 0) {
                 // winding down after a wait that ran out: the loads already issued still write into this CTA's shared
@@ -170,49 +184,60 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
             uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0, u2 = 0;
             bool ok = true;
-            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
-                // accumulator one is free once the previous tile's first epilogue has read it
-                if (!gt_poll(sm32(&s_acc1_empty), (tile_i & 1u) ^ 1u) || s_fail != 0u) ok = false;
+            // layer one of the CTA's i-th tile into accumulator one (buffer b, used for the u-th time)
+            auto layer_one = [&](uint32_t i) {
+                const uint32_t b = p.db ? (i & 1u) : 0u, u = p.db ? (i >> 1) : i;
+                // the buffer is free once the first epilogue of its previous tile has read it
+                if (!gt_poll(sm32(&s_acc1_empty[b]), (u & 1u) ^ 1u) || s_fail != 0u) ok = false;
                 ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
+                if (!ok) return;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const uint32_t d = tmem + b * 128u;
                 for (int ks = 0; ks < p.n_ks1; ++ks) {
                     bool got = gt_poll(full0 + slot * 8u, par);
                     got = __all_sync(0xFFFFFFFFu, got);
-                    if (!got) { ok = false; break; }
+                    if (!got) { ok = false; return; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
-                    gt_issue_stage<false>(BSP_BF16, tmem, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    gt_issue_stage<false>(BSP_BF16, d, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
                     if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                 }
-                if (!ok) break;
-                gt_commit_elected<false>(sm32(&s_acc1_full));
-                // the tensor between the layers is in shared memory once the first epilogue has written it
-                if (!gt_poll(sm32(&s_t_full), tile_i & 1u)) ok = false;
+                gt_commit_elected<false>(sm32(&s_acc1_full[b]));
+            };
+            // layer two of the i-th tile: the tensor between the layers is in shared memory once the first epilogue has written it
+            auto layer_two = [&](uint32_t i) {
+                const uint32_t b = p.db ? (i & 1u) : 0u, u = p.db ? (i >> 1) : i;
+                if (!gt_poll(sm32(&s_t_full[b]), u & 1u)) ok = false;
                 ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
+                if (!ok) return;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 for (int t2 = 0; t2 < p.n_t2 && ok; ++t2, ++u2) {
                     const uint32_t buf = u2 & 1u, use = u2 >> 1;
                     if (!gt_poll(sm32(&s_acc2_empty[buf]), (use & 1u) ^ 1u)) ok = false;
                     ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
+                    if (!ok) return;
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint32_t d = tmem + 256u + buf * (uint32_t)kCtBN2;
                     for (int c2 = 0; c2 < p.n_c2; ++c2) {
                         bool got = gt_poll(full0 + slot * 8u, par);
                         got = __all_sync(0xFFFFFFFFu, got);
-                        if (!got) { ok = false; break; }
+                        if (!got) { ok = false; return; }
                         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                        const uint64_t da = kGtDesc | (uint64_t)(((tbuf + (uint32_t)(c2 * kCtChunk)) >> 4) & 0x3FFFu);
+                        const uint64_t da = kGtDesc | (uint64_t)(((tbuf + b * tbytes + (uint32_t)(c2 * kCtChunk)) >> 4) & 0x3FFFu);
                         const uint64_t db = kGtDesc | (uint64_t)(a16 & 0x3FFFu);
                         gt_issue_stage<false>(BSP_BF16, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
                         if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                     }
-                    if (ok) gt_commit_elected<false>(sm32(&s_acc2_full[buf]));
+                    gt_commit_elected<false>(sm32(&s_acc2_full[buf]));
                 }
-                // all MMAs that read the tensor have been issued: their completion frees it for the next tile
-                if (ok) gt_commit_elected<false>(sm32(&s_t_empty));
+                // all MMAs that read the tensor have been issued: their completion frees its buffer
+                gt_commit_elected<false>(sm32(&s_t_empty[b]));
+            };
+            if (p.db && t_first < t_count) layer_one(0u);
+            for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
+                if (p.db) { if (tile + t_step < t_count) layer_one(tile_i + 1u); }
+                else layer_one(tile_i);
+                if (ok) layer_two(tile_i);
             }
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
@@ -228,7 +253,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             bool ok = true;
             // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
             const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
-            const uint32_t trow = tbuf + (uint32_t)r * 128u;     // this lane's row of a chunk of T
+            const uint32_t trow = tbuf + (uint32_t)r * 128u;     // this lane's row of a chunk of T (first buffer)
             for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 int in0, y0, x0;
                 ct_tile_origin(p, tile, in0, y0, x0);
@@ -237,18 +262,20 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 const unsigned long long row_off = (unsigned long long)pos * (unsigned long long)(p.O2 * ey);
                 // ---- first epilogue: accumulator one -> + b1 -> activation -> bfloat16 -> T in shared memory ----
                 // (T may be overwritten once the MMAs of the previous tile's second layer have read it)
-                if (!gt_wait(sm32(&s_acc1_full), tile_i & 1u) || !gt_wait(sm32(&s_t_empty), (tile_i & 1u) ^ 1u)) ok = false;
+                const uint32_t b1 = p.db ? (tile_i & 1u) : 0u, u1 = p.db ? (tile_i >> 1) : tile_i;
+                if (!gt_wait(sm32(&s_acc1_full[b1]), u1 & 1u) || !gt_wait(sm32(&s_t_empty[b1]), (u1 & 1u) ^ 1u)) ok = false;
                 if (s_fail) ok = false;
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t t1 = tmem + ((uint32_t)(q * 32) << 16);
+                const uint32_t a1 = t1 + b1 * 128u;                  // this tile's accumulator one
                 for (int c2 = grp; c2 < p.n_c2; c2 += 2) {
                     uint32_t out[32];                            // 64 channels of this lane's row of T
 #pragma unroll
                     for (int sub = 0; sub < 2; ++sub) {
                         uint32_t v[32];
-                        gt_load32(t1 + (uint32_t)(c2 * 64 + sub * 32), v);
+                        gt_load32(a1 + (uint32_t)(c2 * 64 + sub * 32), v);
                         const int ch = c2 * 64 + sub * 32 + lane;
                         const float bl = (p.bias1 != nullptr && ch < p.O1) ? __ldg(p.bias1 + ch) : 0.f;     // lane e: bias of channel .. + e
 #pragma unroll
@@ -261,7 +288,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         }
                     }
                     // K-major rows of 128 bytes under the 128-byte swizzle: the 16-byte piece j of row r sits at piece j ^ (r % 8)
-                    const uint32_t dst = trow + (uint32_t)(c2 * kCtChunk);
+                    const uint32_t dst = trow + b1 * tbytes + (uint32_t)(c2 * kCtChunk);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
@@ -272,8 +299,8 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc1_empty)) : "memory");
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_t_full)) : "memory");
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc1_empty[b1])) : "memory");
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_t_full[b1])) : "memory");
                 }
                 // ---- second epilogue, per tile of 128 output channels: + b2 -> convert -> Y ----
                 for (int t2 = 0; t2 < p.n_t2 && ok; ++t2, ++u2) {
@@ -397,7 +424,8 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
     p.n_c2 = p.O1p / 64;
     p.n_t2 = (wd2.O + kCtBN2 - 1) / kCtBN2;
     p.stage_bytes = kGtABytes + p.O1p * 128;
-    const int fixed = 1024 + p.n_c2 * kCtChunk + 8 * kGtStagingBytes;
+    p.db = p.O1p <= 128 ? 1 : 0;
+    const int fixed = 1024 + (p.db ? 2 : 1) * p.n_c2 * kCtChunk + 8 * kGtStagingBytes;
     int stages = (kGtMaxSmem - fixed) / p.stage_bytes;
     if (stages > kGtMaxStages) stages = kGtMaxStages;
     if (stages < 2) return BSP_ERR_SHAPE;
