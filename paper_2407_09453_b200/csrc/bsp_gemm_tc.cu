@@ -32,7 +32,7 @@ namespace {
 struct GtParams {
     CUtensorMap tmx;          // X as bytes: (I * esz, J, L, N), box 128 bytes x Wt x Ht x Nt positions (in steps of the strides), 128-byte swizzle
     CUtensorMap tmw;          // Gamma (.) W as bytes: (I * esz, H K, O), box 128 bytes x 1 tap x BN channels, 128-byte swizzle
-    CUtensorMap tmy;          // Y as bytes: (O * ey, P), box 128 bytes x 32 positions, 128-byte swizzle (store_tma only)
+    CUtensorMap tmy;          // Y as bytes: (O * ey, N_w, M, N), box 128 bytes x Wt x Ht x Nt positions (a tile), 128-byte swizzle
     const void *bias;         // float32 or int32 [O], may be NULL
     const int32_t *shift;     // int8 output only: right shift per output channel, 0..31
     const uint8_t *packed;
@@ -44,7 +44,6 @@ struct GtParams {
     int N, M, Nw, Wt, Ht, Nt, tiles_x, tiles_y, rows_tile;
     int sh, sw, ph, pw, cpt;          // strides, padding, 128-byte channel chunks per tap
     int a_bytes;                      // bytes of one activation box
-    int store_tma;                    // a tile is 128 consecutive rows of Y: the epilogue stores by TMA
     uint8_t *Y;
     int ey;
     uint32_t m_ntn, m_tx, m_ty;       // floor(2^32 / d) of n_tiles_n, tiles_x, tiles_y (division by multiplication)
@@ -243,11 +242,11 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             const int ew = warp - 2, grp = ew >> 2;
             const int ey = p.ey;
             const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
-            const uint32_t sb = staging + (uint32_t)(ew * kGtStagingBytes);      // this warp's staging buffer
+            // the group's staging buffer: 128 rows of 128 bytes, this warp's 32 rows at its quarter
+            const uint32_t sg = staging + (uint32_t)(grp * 4 * kGtStagingBytes), sb = sg + (uint32_t)(q * kGtStagingBytes);
+            const bool issuer = q == 0 && lane == 0;             // one thread of the group issues its stores
             uint32_t tile_i = (uint32_t)grp;
             bool ok = true;
-            // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
-            const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
             for (int tile = t_first + grp * t_step; tile < t_count && ok; tile += 2 * t_step, tile_i += 2) {
                 const uint32_t buf = tile_i & 1u, use = tile_i >> 1;
                 int mt, tn;
@@ -255,14 +254,9 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                 const int n0 = tn * BN;
                 int in0, y0, x0;
                 gt_tile_origin(p, kPair ? 2 * mt + (int)rank : mt, in0, y0, x0);
-                const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
-                // byte offset of the row in Y (rows of O * ey bytes); m0: the tile's first row when rows are consecutive
-                const long long pos = ((long long)(in0 + ri) * p.M + (y0 + rh)) * p.Nw + (x0 + rw);
-                const unsigned long long row_off = (unsigned long long)pos * (unsigned long long)(p.O * ey);
-                const int m0 = (int)(((long long)in0 * p.M + y0) * p.Nw + x0);
                 if (!gt_wait(sm32(&s_acc_full[buf]), use & 1u)) ok = false;
                 if (s_fail) ok = false;
-                ok = __all_sync(0xFFFFFFFFu, ok);             // the warp goes on or gives up as one (aligned tcgen05.ld below)
+                ok = gt_group_all(1 + grp, ok);                // the four warps go on or give up as one (they meet at barriers below)
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16) + buf * 256u;
@@ -313,42 +307,23 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                             }
                         }
                     }
-                    // the staging buffer was handed to a TMA store in the previous round: wait until it has been read (the
-                    // loads and the arithmetic of this round ran meanwhile)
-                    if (lane == 0 && p.store_tma) asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
-                    __syncwarp();
+                    // the staging buffer was handed to a TMA store in the previous round: the issuing thread waits until it
+                    // has been read (the loads and the arithmetic of this round ran meanwhile), then the group may write
+                    if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
+                    gt_group_sync(1 + grp);
                     const uint32_t srow = sb + (uint32_t)lane * 128u;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
                                      ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
-                    if (p.store_tma) {
-                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-                        __syncwarp();
-                        // (a box that starts past the last channel or position is not stored; one that straddles the end is clipped)
-                        if (lane == 0 && n0 + c0 < p.O && m0 + q * 32 < p.P) {
-                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];\n"
-                                         ::"l"(&p.tmy), "r"(sb), "r"((n0 + c0) * ey), "r"(m0 + q * 32) : "memory");
-                            asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
-                        }
-                    } else {
-                        // rows of the tile are scattered over Y (a box of positions): the warp reads the staged rows back
-                        // four at a time, eight lanes per row, and writes whole 128-byte pieces of rows
-                        __syncwarp();
-                        const int chunk = lane & 7;
-                        const bool ch_ok = (n0 + c0) * ey + chunk * 16 < p.O * ey;
-#pragma unroll
-                        for (int it = 0; it < 8; ++it) {
-                            const int row = it * 4 + (lane >> 3);
-                            const unsigned long long off = __shfl_sync(0xFFFFFFFFu, row_off, row);
-                            const int okr = __shfl_sync(0xFFFFFFFFu, (int)row_ok, row);
-                            uint32_t a0, a1, a2, a3;
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];\n"
-                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(sb + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4)) : "memory");
-                            if (okr && ch_ok)
-                                *(uint4 *)(p.Y + off + (unsigned long long)((n0 + c0) * ey + chunk * 16)) = make_uint4(a0, a1, a2, a3);
-                        }
-                        __syncwarp();
+                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    gt_group_sync(1 + grp);
+                    // one store of the tile's box: 128 bytes of every row; what lies past the last channel, column, row or image
+                    // of Y is clipped (rows of the buffer beyond the box are not part of the store)
+                    if (issuer && n0 + c0 < p.O) {
+                        asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];\n"
+                                     ::"l"(&p.tmy), "r"(sg), "r"((n0 + c0) * ey), "r"(x0), "r"(y0), "r"(in0) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
                     }
                 }
                 // the accumulator buffer has been read: hand it back to the MMA issuer
@@ -361,7 +336,7 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc_empty[buf])) : "memory");
                 }
             }
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
+            if (issuer) asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
     }
@@ -420,8 +395,6 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     p.Wt = T.Wt; p.Ht = T.Ht; p.Nt = T.Nt; p.rows_tile = T.Wt * T.Ht * T.Nt;
     p.tiles_x = (p.Nw + T.Wt - 1) / T.Wt; p.tiles_y = (p.M + T.Ht - 1) / T.Ht;
     p.a_bytes = p.rows_tile * 128;
-    // a tile of 128 rows that are consecutive in Y (whole images, or the positions of a matrix product) is stored by TMA
-    p.store_tma = (T.Wt == p.Nw && T.Ht == p.M && p.rows_tile == kGtBM) ? 1 : 0;
     static bool opted[kGtMaxDevices] = {};
     static int n_sm[kGtMaxDevices] = {};
     int dev = 0;
@@ -492,11 +465,12 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
             return BSP_ERR_CUDA;
     }
     {
-        const cuuint64_t gdim[2] = {(cuuint64_t)wd.O * ey, (cuuint64_t)P};
-        const cuuint64_t gstr[1] = {(cuuint64_t)wd.O * ey};
-        const cuuint32_t box[2] = {128, (cuuint32_t)kGtStageRows};
-        const cuuint32_t estr[2] = {1, 1};
-        if (enc(&p.tmy, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, Y, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        const cuuint64_t row = (cuuint64_t)wd.O * ey;
+        const cuuint64_t gdim[4] = {row, (cuuint64_t)p.Nw, (cuuint64_t)p.M, (cuuint64_t)xd.N};
+        const cuuint64_t gstr[3] = {row, row * p.Nw, row * p.Nw * p.M};
+        const cuuint32_t box[4] = {128, (cuuint32_t)T.Wt, (cuuint32_t)T.Ht, (cuuint32_t)T.Nt};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(&p.tmy, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, Y, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
     }

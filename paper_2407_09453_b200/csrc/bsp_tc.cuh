@@ -113,6 +113,16 @@ __device__ __forceinline__ void gt_divmod(int n, int d, uint32_t m, int &q, int 
     if (r >= d) { ++q; r -= d; }
 }
 
+// Barrier `id` (1..15) over the 128 threads of a group of four warps, and the same with the AND of a flag.
+__device__ __forceinline__ void gt_group_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
+__device__ __forceinline__ bool gt_group_all(int id, bool flag)
+{
+    uint32_t r;
+    asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %1, 0;\n bar.red.and.pred q, %2, 128, p;\n selp.b32 %0, 1, 0, q;\n}\n"
+                 : "=r"(r) : "r"((uint32_t)flag), "r"(id) : "memory");
+    return r != 0u;
+}
+
 // 32 consecutive accumulator columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void gt_load32(uint32_t taddr, uint32_t (&v)[32])
 {
