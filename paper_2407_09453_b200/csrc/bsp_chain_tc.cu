@@ -28,6 +28,7 @@ struct CtParams {
     CUtensorMap tmx;          // X as bytes: (I1 * 2, J, L, N), box 128 bytes x Wt x Ht x Nt positions
     CUtensorMap tmw1;         // Gamma1 (.) W1 as bytes: (I1 * 2, H K, O1), box 128 bytes x 1 tap x O1p channels
     CUtensorMap tmw2;         // Gamma2 (.) W2 as bytes: (O1 * 2, 1, O2), box 128 bytes x 1 x 128 channels
+    CUtensorMap tmy;          // Y as bytes: (O2 * ey, N_w, M, N), box 128 bytes x Wt x Ht x Nt positions (a tile)
     const float *bias1, *bias2;
     const uint8_t *packed1, *packed2;
     int *status;
@@ -96,6 +97,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmx) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmw1) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmw2) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&p.tmy) : "memory");
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(sm32(&s_tmem)), "r"(kGtTmemCols) : "memory");
@@ -248,24 +250,22 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
             const int grp = (warp - 2) >> 2;
             const int ey = p.ey;
             const int cpr = 128 / ey;                            // output channels per staging round (128 bytes of a row)
-            const uint32_t sb = staging + (uint32_t)((warp - 2) * kGtStagingBytes);
+            // the group's staging buffer: 128 rows of 128 bytes, this warp's 32 rows at its quarter
+            const uint32_t sg = staging + (uint32_t)(grp * 4 * kGtStagingBytes), sb = sg + (uint32_t)(q * kGtStagingBytes);
+            const bool issuer = q == 0 && lane == 0;             // one thread of the group issues its stores
             uint32_t tile_i = 0, u2 = 0;
             bool ok = true;
-            // this lane's row of a tile: position (w, h, image i) of the tile's box, w fastest
-            const int r = q * 32 + lane, rw = r % p.Wt, rh = (r / p.Wt) % p.Ht, ri = r / (p.Wt * p.Ht);
+            const int r = q * 32 + lane;                         // this lane's row of a tile
             const uint32_t trow = tbuf + (uint32_t)r * 128u;     // this lane's row of a chunk of T (first buffer)
             for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
                 int in0, y0, x0;
                 ct_tile_origin(p, tile, in0, y0, x0);
-                const bool row_ok = r < p.rows_tile && x0 + rw < p.Nw && y0 + rh < p.M && in0 + ri < p.N;
-                const long long pos = ((long long)(in0 + ri) * p.M + (y0 + rh)) * p.Nw + (x0 + rw);
-                const unsigned long long row_off = (unsigned long long)pos * (unsigned long long)(p.O2 * ey);
                 // ---- first epilogue: accumulator one -> + b1 -> activation -> bfloat16 -> T in shared memory ----
                 // (T may be overwritten once the MMAs of the previous tile's second layer have read it)
                 const uint32_t b1 = p.db ? (tile_i & 1u) : 0u, u1 = p.db ? (tile_i >> 1) : tile_i;
                 if (!gt_wait(sm32(&s_acc1_full[b1]), u1 & 1u) || !gt_wait(sm32(&s_t_empty[b1]), (u1 & 1u) ^ 1u)) ok = false;
                 if (s_fail) ok = false;
-                ok = __all_sync(0xFFFFFFFFu, ok);
+                ok = gt_group_all(1 + grp, ok);                  // the four warps of a group go on or give up as one
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const uint32_t t1 = tmem + ((uint32_t)(q * 32) << 16);
@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     const int n0 = t2 * kCtBN2;
                     if (!gt_wait(sm32(&s_acc2_full[buf]), use & 1u)) ok = false;
                     if (s_fail) ok = false;
-                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    ok = gt_group_all(1 + grp, ok);              // the four warps go on or give up as one (they meet at barriers below)
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint32_t t2base = t1 + 256u + buf * (uint32_t)kCtBN2;
@@ -337,26 +337,21 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                                 }
                             }
                         }
-                        // staged in shared memory, read back four rows at a time, eight lanes per row: whole 128-byte pieces of rows of Y
-                        __syncwarp();
+                        // staged under the 128-byte swizzle and stored as the tile's box of positions by one TMA store; what lies
+                        // past the last channel, column, row or image of Y is clipped
+                        if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
+                        gt_group_sync(1 + grp);
                         const uint32_t srow = sb + (uint32_t)lane * 128u;
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
                                          ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(out[4 * j]), "r"(out[4 * j + 1]), "r"(out[4 * j + 2]), "r"(out[4 * j + 3]) : "memory");
-                        __syncwarp();
-                        const int chunk = lane & 7;
-                        const bool ch_ok = (n0 + c0) * ey + chunk * 16 < p.O2 * ey;
-#pragma unroll
-                        for (int it = 0; it < 8; ++it) {
-                            const int row = it * 4 + (lane >> 3);
-                            const unsigned long long off = __shfl_sync(0xFFFFFFFFu, row_off, row);
-                            const int okr = __shfl_sync(0xFFFFFFFFu, (int)row_ok, row);
-                            uint32_t a0, a1, a2, a3;
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];\n"
-                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(sb + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4)) : "memory");
-                            if (okr && ch_ok)
-                                *(uint4 *)(p.Y + off + (unsigned long long)((n0 + c0) * ey + chunk * 16)) = make_uint4(a0, a1, a2, a3);
+                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                        gt_group_sync(1 + grp);
+                        if (issuer && n0 + c0 < p.O2) {
+                            asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];\n"
+                                         ::"l"(&p.tmy), "r"(sg), "r"((n0 + c0) * ey), "r"(x0), "r"(y0), "r"(in0) : "memory");
+                            asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
                         }
                     }
                     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -364,6 +359,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(sm32(&s_acc2_empty[buf])) : "memory");
                 }
             }
+            if (issuer) asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
             if (!ok && lane == 0) atomicExch((uint32_t *)&s_fail, 1u);
         }
     }
@@ -474,6 +470,16 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
         if (enc(&p.tmw2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed2 + L2.off_payload), gdim, gstr, box,
                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return BSP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t row = (cuuint64_t)wd2.O * ey;
+        const cuuint64_t gdim[4] = {row, (cuuint64_t)p.Nw, (cuuint64_t)p.M, (cuuint64_t)xd.N};
+        const cuuint64_t gstr[3] = {row, row * p.Nw, row * p.Nw * p.M};
+        const cuuint32_t box[4] = {128, (cuuint32_t)T.Wt, (cuuint32_t)T.Ht, (cuuint32_t)T.Nt};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(&p.tmy, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, Y, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
     }
     const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
