@@ -215,6 +215,19 @@ def chain2(w1shape, bo1, bi1, c1, X, b1, relu, O2, bo2, bi2, c2, b2, stride=(1, 
     return gemm(O2, O1, bo2, bi2, c2[0], c2[1], np.asarray(c2[2]).reshape(-1, bo2, bi2), Tb, b2)
 
 
+def chain2_q8(w1shape, bo1, bi1, c1, X, b1, shift1, relu, O2, bo2, bi2, c2, b2, shift2=None, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
+    """The 8-bit chain (Section "Depth-wise Tiling" with the tensors of Section "Compiler and its Code generation"): the
+    tensor between the layers is the requantised int8 output of layer one, T = act(requant(W1 * X + b1, shift1)); Y is
+    the int32 result W2 * T + b2 of the 1x1 second layer, or its requantised int8 form when shift2 is given."""
+    T32 = conv2d(w1shape, bo1, bi1, c1[0], c1[1], c1[2], X, b1, stride, pad)
+    T8 = requant_i8(T32, shift1)
+    if relu:
+        T8 = np.maximum(T8, 0).astype(np.int8)
+    O1 = w1shape[0]
+    Y32 = gemm(O2, O1, bo2, bi2, c2[0], c2[1], np.asarray(c2[2]).reshape(-1, bo2, bi2), T8, b2)
+    return Y32 if shift2 is None else requant_i8(Y32, shift2)
+
+
 def spgemm(kb, a, b) -> np.ndarray:
     """C = (Gamma . A)(Omega . B)^t from two compact forms (row_ptr, col_idx, payload [nnz][kb][kb]) with kb x kb blocks;
     dense float64 [NBa*kb][NBb*kb]."""

@@ -74,3 +74,40 @@ def test_chain_with_an_identity_second_layer_returns_the_rounded_tensor():
     T = np.maximum(ref.conv2d(W1.shape, 8, 8, *ref.compact(W1, g1, 8, 8), X, b1, (1, 1), (1, 1)), 0.0)
     assert np.array_equal(got, ref.round_bf16(T).astype(np.float64))
     assert np.all(got >= 0.0)
+
+
+@pytest.mark.parametrize("relu,with_shift2", [(0, False), (1, False), (1, True)])
+def test_int8_chain_equals_integer_numpy_layers(relu, with_shift2):
+    """The 8-bit chain against plain integer numpy: dense masked layer one (the pinned dense reference), the
+    rounding shift written out with exact rationals, max(., 0), an int64 matrix product for layer two."""
+    from fractions import Fraction
+    N, L, J, I, O1, O2 = 2, 7, 6, 16, 16, 24
+    W1 = synth.uniform_int(831, (O1, 3, 3, I), -127, 127).astype(np.int8)
+    W2 = synth.uniform_int(832, (O2, 1, 1, O1), -127, 127).astype(np.int8)
+    X = synth.uniform_int(833, (N, L, J, I), -127, 127).astype(np.int8)
+    b1 = synth.uniform_int(834, (O1,), -(1 << 15), 1 << 15).astype(np.int32)
+    b2 = synth.uniform_int(835, (O2,), -(1 << 15), 1 << 15).astype(np.int32)
+    s1 = synth.uniform_int(836, (O1,), 9, 13).astype(np.int32)
+    s2 = synth.uniform_int(837, (O2,), 8, 12).astype(np.int32) if with_shift2 else None
+    g1 = synth.random_gamma(838, O1 // 8, I // 8, 2)
+    g2 = synth.random_gamma(839, O2 // 8, O1 // 8, 3)
+    got = ref.chain2_q8(W1.shape, 8, 8, ref.compact(W1, g1, 8, 8), X, b1, s1, relu, O2, 8, 8, ref.compact(W2, g2, 8, 8), b2, s2, (1, 1), (1, 1))
+
+    def rq(v, sh):                                        # nearest integer of v / 2^sh, halves away from zero, saturated
+        out = np.empty(v.shape, dtype=np.int64)
+        for idx in np.ndindex(*v.shape):
+            f = Fraction(int(v[idx]), 1 << int(sh[idx[-1]]))
+            q = int(abs(f) + Fraction(1, 2))               # floor(|f| + 1/2)
+            out[idx] = max(-128, min(127, q if f >= 0 else -q))
+        return out
+
+    T = ref.dense_conv2d(ref.apply_mask(W1, g1, 8, 8), X, b1, (1, 1), (1, 1)).astype(np.int64).reshape(-1, O1)
+    T8 = rq(T, s1)
+    if relu:
+        T8 = np.maximum(T8, 0)
+    Y = T8 @ ref.apply_mask(W2, g2, 8, 8)[:, 0, 0, :].astype(np.int64).T + b2.astype(np.int64)
+    want = rq(Y, s2) if with_shift2 else Y
+    assert np.array_equal(got.astype(np.int64), want)
+    assert got.dtype == (np.int8 if with_shift2 else np.int32)
+    if not with_shift2:
+        assert np.abs(T8).max() == 127 or np.abs(T8).max() > 20          # the shifts leave a tensor that uses the int8 range
