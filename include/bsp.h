@@ -208,6 +208,17 @@ bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc
 bsp_status bsp_conv2d_chain(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
                             const bsp_xdesc *xd, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
                             bsp_dtype ytype, void *ws, void *stream);
+/* bsp_conv2d_chain_q8: the same chain on I8 layers with the 8-bit tensors of Section "Compiler and its Code generation":
+ *             T = act(saturate_int8(round((W1 * X + bias1) / 2^shift1[o]))) is the requantised int8 output of layer one
+ *             (the rounding of bsp_conv2d_q8; act = max(., 0) if relu != 0), Y = W2 * T + bias2 as int32, or, when
+ *             shift2 is not NULL, requantised to int8 in the same way.  bias1 / bias2 int32 (device, may be NULL),
+ *             shift1 [O1] required, shift2 [O2] optional, entries 0..31.  I1 and O1 multiples of 16, O2 a multiple of
+ *             16 for an int8 Y.  Exact integer arithmetic: bit-identical to bsp_conv2d_q8 followed by bsp_conv2d
+ *             (or bsp_conv2d_q8).
+ * Errors: as bsp_conv2d_chain; NULL shift1; DTYPE if the layers are not I8. */
+bsp_status bsp_conv2d_chain_q8(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
+                               const bsp_xdesc *xd, const void *X, const int32_t *bias1, const int32_t *shift1, int relu,
+                               const int32_t *bias2, const int32_t *shift2, void *Y, void *ws, void *stream);
 
 /* ---- Block-sparse x block-sparse product (Section "Block-Sparse Matrix-Matrix Multiplication") and the relative column
  * index (Section "Block Sparsity in a Matrix": "a relative row/col index") ------------------------------------------

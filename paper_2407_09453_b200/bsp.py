@@ -22,7 +22,7 @@ SCOPE_LAYER, SCOPE_ROW = 0, 1
 
 EXPORTS = ["bsp_mask_workspace_bytes", "bsp_mask", "bsp_mask_static", "bsp_packed_bytes",
            "bsp_compact_workspace_bytes", "bsp_compact_nnz", "bsp_compact", "bsp_conv_workspace_bytes", "bsp_gemm",
-           "bsp_conv2d", "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv2d_chain", "bsp_conv_kernel_name", "bsp_spgemm",
+           "bsp_conv2d", "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv2d_chain", "bsp_conv2d_chain_q8", "bsp_conv_kernel_name", "bsp_spgemm",
            "bsp_index_to_relative", "bsp_index_from_relative", "bsp_check", "bsp_status_string"]
 
 
@@ -63,7 +63,7 @@ def lib():
         L.bsp_status_string.restype = C.c_char_p
         L.bsp_conv_kernel_name.restype = C.c_char_p
         for n in ("bsp_mask", "bsp_mask_static", "bsp_compact_nnz", "bsp_compact", "bsp_gemm", "bsp_conv2d",
-                  "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv2d_chain", "bsp_spgemm", "bsp_index_to_relative", "bsp_index_from_relative", "bsp_check"):
+                  "bsp_gemm_q8", "bsp_conv2d_q8", "bsp_conv2d_chain", "bsp_conv2d_chain_q8", "bsp_spgemm", "bsp_index_to_relative", "bsp_index_from_relative", "bsp_check"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -164,6 +164,12 @@ def bsp_conv2d_chain(wd1: WDesc, w1: Bcsr, wd2: WDesc, w2: Bcsr, xd: XDesc, X, b
     _raise(lib().bsp_conv2d_chain(C.byref(wd1), C.byref(w1), C.byref(wd2), C.byref(w2), C.byref(xd), _ptr(X), _ptr(bias1),
                                   C.c_int(1 if relu else 0), _ptr(bias2), _ptr(Y), C.c_int(ytype), _ptr(ws), _stream(stream)),
            "bsp_conv2d_chain")
+
+
+def bsp_conv2d_chain_q8(wd1: WDesc, w1: Bcsr, wd2: WDesc, w2: Bcsr, xd: XDesc, X, bias1, shift1, relu, bias2, shift2, Y, ws, stream=None):
+    _raise(lib().bsp_conv2d_chain_q8(C.byref(wd1), C.byref(w1), C.byref(wd2), C.byref(w2), C.byref(xd), _ptr(X), _ptr(bias1),
+                                     _ptr(shift1), C.c_int(1 if relu else 0), _ptr(bias2), _ptr(shift2), _ptr(Y), _ptr(ws),
+                                     _stream(stream)), "bsp_conv2d_chain_q8")
 
 
 def bsp_spgemm(wa: WDesc, a: Bcsr, wb: WDesc, b: Bcsr, Cm, ws, stream=None):

@@ -166,9 +166,9 @@ bsp_status bsp_conv2d_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const bsp_xdesc
     return conv2d_any(wd, w, xd, X, bias, shift, Y, BSP_I8, ws, stream);
 }
 
-bsp_status bsp_conv2d_chain(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
-                            const bsp_xdesc *xd, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
-                            bsp_dtype ytype, void *ws, void *stream)
+static bsp_status chain_any(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2, const bsp_xdesc *xd,
+                            const void *X, const void *bias1, const int32_t *shift1, int relu, const void *bias2,
+                            const int32_t *shift2, void *Y, bsp_dtype ytype, void *ws, void *stream)
 {
     bsp_status rc = check_wdesc(wd1);
     if (rc != BSP_OK) return rc;
@@ -178,15 +178,33 @@ bsp_status bsp_conv2d_chain(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_
     if (xd->N <= 0 || xd->L <= 0 || xd->J <= 0 || xd->stride_h <= 0 || xd->stride_w <= 0 || xd->pad_h < 0 || xd->pad_w < 0)
         return BSP_ERR_SHAPE;
     if (xd->L + 2 * xd->pad_h < wd1->H || xd->J + 2 * xd->pad_w < wd1->K) return BSP_ERR_SHAPE;
-    if (wd1->wtype != BSP_BF16 || wd2->wtype != BSP_BF16) return BSP_ERR_DTYPE;
-    if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
     if (wd2->H != 1 || wd2->K != 1 || wd2->I != wd1->O || wd1->O > 256) return BSP_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(Y) || !aligned16(w1->packed) || !aligned16(w2->packed)) return BSP_ERR_SHAPE;
-    if ((bias1 && !aligned4(bias1)) || (bias2 && !aligned4(bias2))) return BSP_ERR_SHAPE;
+    if ((bias1 && !aligned4(bias1)) || (bias2 && !aligned4(bias2)) || (shift1 && !aligned4(shift1)) || (shift2 && !aligned4(shift2)))
+        return BSP_ERR_SHAPE;
     const int64_t NB1 = (int64_t)(wd1->O / wd1->bo) * (wd1->I / wd1->bi), NB2 = (int64_t)(wd2->O / wd2->bo) * (wd2->I / wd2->bi);
     if (w1->nnz < 0 || w1->nnz > NB1 || w2->nnz < 0 || w2->nnz > NB2) return BSP_ERR_INDEX;
     if (!chain_tc_eligible(*wd1, *wd2, *xd, ytype)) return BSP_ERR_SHAPE;
-    return launch_chain_tc(*wd1, w1->packed, *wd2, w2->packed, *xd, X, bias1, relu, bias2, Y, ytype, ws, (cudaStream_t)stream);
+    return launch_chain_tc(*wd1, w1->packed, *wd2, w2->packed, *xd, X, bias1, shift1, relu, bias2, shift2, Y, ytype, ws,
+                           (cudaStream_t)stream);
+}
+
+bsp_status bsp_conv2d_chain(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
+                            const bsp_xdesc *xd, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
+                            bsp_dtype ytype, void *ws, void *stream)
+{
+    if (wd1 && wd2 && (wd1->wtype != BSP_BF16 || wd2->wtype != BSP_BF16)) return BSP_ERR_DTYPE;
+    if (ytype != BSP_F32 && ytype != BSP_BF16) return BSP_ERR_DTYPE;
+    return chain_any(wd1, w1, wd2, w2, xd, X, bias1, nullptr, relu, bias2, nullptr, Y, ytype, ws, stream);
+}
+
+bsp_status bsp_conv2d_chain_q8(const bsp_wdesc *wd1, const bsp_bcsr *w1, const bsp_wdesc *wd2, const bsp_bcsr *w2,
+                               const bsp_xdesc *xd, const void *X, const int32_t *bias1, const int32_t *shift1, int relu,
+                               const int32_t *bias2, const int32_t *shift2, void *Y, void *ws, void *stream)
+{
+    if (wd1 && wd2 && (wd1->wtype != BSP_I8 || wd2->wtype != BSP_I8)) return BSP_ERR_DTYPE;
+    if (!shift1) return BSP_ERR_NULL;
+    return chain_any(wd1, w1, wd2, w2, xd, X, bias1, shift1, relu, bias2, shift2, Y, shift2 ? BSP_I8 : BSP_I32, ws, stream);
 }
 
 bsp_status bsp_gemm_q8(const bsp_wdesc *wd, const bsp_bcsr *w, const void *X, int64_t P, const int32_t *bias,

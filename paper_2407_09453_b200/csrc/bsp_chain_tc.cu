@@ -1,5 +1,6 @@
 // Two consecutive block-sparse layers in one kernel: T = act(W1 * X + b1) stored as bfloat16, Y = W2 * T + b2 with a 1x1
-// second layer.  Section "Depth-wise Tiling" of the paper: the output is cut into tiles, every tile is carried through
+// second layer; or the 8-bit chain, where T is the requantised int8 output of layer one (Section "Compiler and its Code
+// generation": power-of-two scales) and Y is int32 or requantised int8.  Section "Depth-wise Tiling" of the paper: the output is cut into tiles, every tile is carried through
 // the whole chain, and the tensor between the layers never goes to external memory.  A 1x1 second layer needs no
 // overlap between tiles (its projection of one output position is one position of T), so the tiles are those of the
 // first layer.
@@ -7,8 +8,9 @@
 // Per tile of up to 128 output positions a persistent CTA runs
 //   1. the first layer as an implicit GEMM over taps x 128-byte channel chunks (activation box + weight tile per
 //      K-stage, both by tiled TMA loads) into accumulator one, all O1 <= 256 channels in tensor memory;
-//   2. its epilogue: tensor memory -> registers -> + b1 -> max(., 0) if asked -> bfloat16 -> shared memory, written in
-//      the K-major 128-byte-swizzled layout that an MMA reads as its A operand (64 channels per 16 KB chunk);
+//   2. its epilogue: tensor memory -> registers -> + b1 -> max(., 0) if asked -> bfloat16 (int8: rounding shift, then
+//      max(., 0)) -> shared memory, written in the K-major 128-byte-swizzled layout that an MMA reads as its A operand
+//      (128 bytes of channels, that is 64 bfloat16 or 128 int8, per 16 KB chunk);
 //   3. the second layer: for every tile of 128 output channels, MMAs of that tensor against weight chunks that arrive
 //      through the same ring of stages, into one of two 128-column accumulators;
 //   4. its epilogue: + b2 -> convert -> global memory, overlapping the MMAs of the next 128 channels.
@@ -22,18 +24,20 @@ namespace {
 
 constexpr int kCtThreads = 320;                    // producer warp, MMA warp, two groups of four epilogue warps
 constexpr int kCtBN2 = 128;                        // channels of layer two per accumulator buffer
-constexpr int kCtChunk = kGtBM * 128;              // bytes of one 64-channel chunk of the tensor between the layers
+constexpr int kCtChunk = kGtBM * 128;              // bytes of one chunk (128 bytes of channels) of the tensor between the layers
 
 struct CtParams {
     CUtensorMap tmx;          // X as bytes: (I1 * 2, J, L, N), box 128 bytes x Wt x Ht x Nt positions
     CUtensorMap tmw1;         // Gamma1 (.) W1 as bytes: (I1 * 2, H K, O1), box 128 bytes x 1 tap x O1p channels
     CUtensorMap tmw2;         // Gamma2 (.) W2 as bytes: (O1 * 2, 1, O2), box 128 bytes x 1 x 128 channels
     CUtensorMap tmy;          // Y as bytes: (O2 * ey, N_w, M, N), box 128 bytes x Wt x Ht x Nt positions (a tile)
-    const float *bias1, *bias2;
+    const void *bias1, *bias2;        // float32, or int32 for the 8-bit chain
+    const int32_t *shift1, *shift2;   // 8-bit chain: rounding shifts of T (required) and of an int8 Y
     const uint8_t *packed1, *packed2;
     int *status;
-    int O1, I1, H, K, bo1, bi1, O2, bo2, bi2, relu, ytype, ey;
-    int O1p;                  // O1 rounded up to 64: columns of accumulator one
+    int O1, I1, H, K, bo1, bi1, O2, bo2, bi2, relu, wtype, ytype, ey;
+    int O1p;                  // O1 rounded up to a whole chunk of T (64 or 128 channels): columns of accumulator one
+    int tcc;                  // channels per chunk of T: 64 (bfloat16) or 128 (int8)
     int n_ks1, cpt1, n_c2, n_t2;      // K-stages of layer one, its channel chunks per tap; chunks of T; channel tiles of layer two
     int stages, stage_bytes, n_tiles;
     int db;                   // O1p <= 128: accumulator one and the tensor between the layers are double-buffered
@@ -51,10 +55,10 @@ __device__ __forceinline__ void ct_tile_origin(const CtParams &p, int mt, int &n
     x0 = tx * p.Wt; y0 = ty * p.Ht; n0 = ni * p.Nt;
 }
 
-__device__ __forceinline__ bool ct_header_ok(const uint8_t *packed, int O, int I, int H, int K, int bo, int bi)
+__device__ __forceinline__ bool ct_header_ok(const uint8_t *packed, int wtype, int O, int I, int H, int K, int bo, int bi)
 {
     const PackedHeader *h = (const PackedHeader *)packed;
-    return h->magic == kPackedMagic && h->dtype == BSP_BF16 && h->O == O && h->I == I && h->H == H && h->K == K && h->bo == bo &&
+    return h->magic == kPackedMagic && h->dtype == wtype && h->O == O && h->I == I && h->H == H && h->K == K && h->bo == bo &&
            h->bi == bi && (h->forms & kFormDense) != 0;
 }
 
@@ -76,7 +80,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
     const int t_first = (int)blockIdx.x, t_step = (int)gridDim.x, t_count = p.n_tiles;
 
     if (tid == 0) {
-        const bool ok = ct_header_ok(p.packed1, p.O1, p.I1, p.H, p.K, p.bo1, p.bi1) && ct_header_ok(p.packed2, p.O2, p.O1, 1, 1, p.bo2, p.bi2);
+        const bool ok = ct_header_ok(p.packed1, p.wtype, p.O1, p.I1, p.H, p.K, p.bo1, p.bi1) && ct_header_ok(p.packed2, p.wtype, p.O2, p.O1, 1, 1, p.bo2, p.bi2);
         s_fail = ok ? 0u : 2u;
         if (!ok) atomicMax(p.status, (int)BSP_ERR_INDEX);
         for (int s = 0; s < S; ++s) {
@@ -180,9 +184,10 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (run) {
-            // instruction descriptors: D fp32, A and B bf16, K-major both, M = 128; N = O1p for layer one, 128 for layer two
-            const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.O1p >> 3) << 17) | ((128u >> 4) << 24);
-            const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCtBN2 >> 3) << 17) | ((128u >> 4) << 24);
+            // instruction descriptors: A and B bf16 (signed int8), K-major both, M = 128; N = O1p for layer one, 128 for layer two
+            const uint32_t dfmt = p.wtype == BSP_I8 ? 2u : 1u;      // D int32 for int8 operands, fp32 otherwise
+            const uint32_t idesc1 = (dfmt << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.O1p >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc2 = (dfmt << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCtBN2 >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
             uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0, u2 = 0;
             bool ok = true;
@@ -201,7 +206,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     if (!got) { ok = false; return; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
-                    gt_issue_stage<false>(BSP_BF16, d, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    gt_issue_stage<false>(p.wtype, d, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
                     if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                 }
                 gt_commit_elected<false>(sm32(&s_acc1_full[b]));
@@ -227,7 +232,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                         const uint64_t da = kGtDesc | (uint64_t)(((tbuf + b * tbytes + (uint32_t)(c2 * kCtChunk)) >> 4) & 0x3FFFu);
                         const uint64_t db = kGtDesc | (uint64_t)(a16 & 0x3FFFu);
-                        gt_issue_stage<false>(BSP_BF16, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
+                        gt_issue_stage<false>(p.wtype, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
                         if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                     }
                     gt_commit_elected<false>(sm32(&s_acc2_full[buf]));
@@ -271,13 +276,35 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 const uint32_t t1 = tmem + ((uint32_t)(q * 32) << 16);
                 const uint32_t a1 = t1 + b1 * 128u;                  // this tile's accumulator one
                 for (int c2 = grp; c2 < p.n_c2; c2 += 2) {
-                    uint32_t out[32];                            // 64 channels of this lane's row of T
+                    uint32_t out[32];                            // one chunk (128 bytes of channels) of this lane's row of T
+                    if (p.wtype == BSP_I8) {                     // 128 channels: + b1, rounding shift, activation, int8
+#pragma unroll
+                        for (int sub = 0; sub < 4; ++sub) {
+                            uint32_t v[32];
+                            gt_load32(a1 + (uint32_t)(c2 * 128 + sub * 32), v);
+                            const int ch = c2 * 128 + sub * 32 + lane;
+                            const int bl = (p.bias1 != nullptr && ch < p.O1) ? __ldg((const int *)p.bias1 + ch) : 0;   // lane e: channel .. + e
+                            const uint32_t sl = ch < p.O1 ? (uint32_t)__ldg(p.shift1 + ch) & 31u : 0u;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                uint32_t w = 0u;
+#pragma unroll
+                                for (int b = 0; b < 4; ++b) {
+                                    uint32_t qv = gt_requant((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
+                                                             __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b));
+                                    if (p.relu && (qv & 0x80u)) qv = 0u;
+                                    w |= qv << (8 * b);
+                                }
+                                out[sub * 8 + e] = w;
+                            }
+                        }
+                    } else {
 #pragma unroll
                     for (int sub = 0; sub < 2; ++sub) {
                         uint32_t v[32];
                         gt_load32(a1 + (uint32_t)(c2 * 64 + sub * 32), v);
                         const int ch = c2 * 64 + sub * 32 + lane;
-                        const float bl = (p.bias1 != nullptr && ch < p.O1) ? __ldg(p.bias1 + ch) : 0.f;     // lane e: bias of channel .. + e
+                        const float bl = (p.bias1 != nullptr && ch < p.O1) ? __ldg((const float *)p.bias1 + ch) : 0.f;     // lane e: bias of channel .. + e
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
                             float a = __uint_as_float(v[2 * e]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e);
@@ -286,6 +313,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                             const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
                             out[sub * 16 + e] = *(const uint32_t *)&h;
                         }
+                    }
                     }
                     // K-major rows of 128 bytes under the 128-byte swizzle: the 16-byte piece j of row r sits at piece j ^ (r % 8)
                     const uint32_t dst = trow + b1 * tbytes + (uint32_t)(c2 * kCtChunk);
@@ -315,20 +343,42 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     const uint32_t t2base = t1 + 256u + buf * (uint32_t)kCtBN2;
                     for (int c0 = 0; c0 < kCtBN2; c0 += cpr) {
                         uint32_t out[32];                        // 128 bytes of this lane's row of Y
-                        if (ey == 4) {
+                        if (ey == 4) {                           // float32 or int32 output: 32 channels
                             uint32_t v[32];
                             gt_load32(t2base + (uint32_t)c0, v);
                             const int ch = n0 + c0 + lane;
-                            const float bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg(p.bias2 + ch) : 0.f;
+                            const uint32_t bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg((const uint32_t *)p.bias2 + ch) : 0u;
+                            if (p.wtype == BSP_I8) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) out[e] = __float_as_uint(__uint_as_float(v[e]) + __shfl_sync(0xFFFFFFFFu, bl, e));
-                        } else {
+                                for (int e = 0; e < 32; ++e) out[e] = (uint32_t)((int)v[e] + (int)__shfl_sync(0xFFFFFFFFu, bl, e));
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 32; ++e) out[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, e)));
+                            }
+                        } else if (ey == 1) {                    // int8 output: 128 channels, requantised after the bias
+#pragma unroll
+                            for (int sub = 0; sub < 4; ++sub) {
+                                uint32_t v[32];
+                                gt_load32(t2base + (uint32_t)(c0 + sub * 32), v);
+                                const int ch = n0 + c0 + sub * 32 + lane;
+                                const int bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg((const int *)p.bias2 + ch) : 0;
+                                const uint32_t sl = ch < p.O2 ? (uint32_t)__ldg(p.shift2 + ch) & 31u : 0u;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    uint32_t w = 0u;
+#pragma unroll
+                                    for (int b = 0; b < 4; ++b)
+                                        w |= gt_requant((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b), __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b)) << (8 * b);
+                                    out[sub * 8 + e] = w;
+                                }
+                            }
+                        } else {                                 // bfloat16 output: 64 channels
 #pragma unroll
                             for (int sub = 0; sub < 2; ++sub) {
                                 uint32_t v[32];
                                 gt_load32(t2base + (uint32_t)(c0 + sub * 32), v);
                                 const int ch = n0 + c0 + sub * 32 + lane;
-                                const float bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg(p.bias2 + ch) : 0.f;
+                                const float bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg((const float *)p.bias2 + ch) : 0.f;
 #pragma unroll
                                 for (int e = 0; e < 16; ++e) {
                                     const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * e]) + __shfl_sync(0xFFFFFFFFu, bl, 2 * e),
@@ -373,14 +423,19 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
 
 }  // namespace
 
-// True if the fused kernel can run this pair: bfloat16 layers, a 1x1 second layer on the first one's output channels,
-// at most 256 of them (accumulator one holds them all), rows of X, of both weights and of Y that are multiples of 16 bytes.
+// True if the fused kernel can run this pair: two bfloat16 or two int8 layers, a 1x1 second layer on the first one's
+// output channels, at most 256 of them (accumulator one holds them all), rows of X, of both weights and of Y that are
+// multiples of 16 bytes.
 bool chain_tc_eligible(const bsp_wdesc &wd1, const bsp_wdesc &wd2, const bsp_xdesc &xd0, bsp_dtype ytype)
 {
-    if (wd1.wtype != BSP_BF16 || wd2.wtype != BSP_BF16) return false;
+    if (wd1.wtype != wd2.wtype || (wd1.wtype != BSP_BF16 && wd1.wtype != BSP_I8)) return false;
     if (wd2.H != 1 || wd2.K != 1 || wd2.I != wd1.O) return false;
     if (wd1.O > 256 || wd1.O % 8 != 0 || wd1.I % 8 != 0 || wd2.O % 8 != 0) return false;
-    if (ytype != BSP_F32 && ytype != BSP_BF16) return false;
+    const int esz = elem_bytes(wd1.wtype);
+    if (wd1.wtype == BSP_I8) { if (ytype != BSP_I32 && ytype != BSP_I8) return false; }
+    else if (ytype != BSP_F32 && ytype != BSP_BF16) return false;
+    const int ey = ytype == BSP_BF16 ? 2 : (ytype == BSP_I8 ? 1 : 4);
+    if ((wd1.I * esz) % 16 != 0 || (wd1.O * esz) % 16 != 0 || (wd2.O * ey) % 16 != 0) return false;
     if (!packed_layout(wd1).enabled || !packed_layout(wd2).enabled) return false;
     const bsp_xdesc xd = gt_flatten(wd1, xd0);
     const int M = (xd.L + 2 * xd.pad_h - wd1.H) / xd.stride_h + 1, Nw = (xd.J + 2 * xd.pad_w - wd1.K) / xd.stride_w + 1;
@@ -390,19 +445,22 @@ bool chain_tc_eligible(const bsp_wdesc &wd1, const bsp_wdesc &wd2, const bsp_xde
 }
 
 bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_wdesc &wd2, const void *packed2,
-                           const bsp_xdesc &xd0, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
-                           bsp_dtype ytype, void *ws, cudaStream_t st)
+                           const bsp_xdesc &xd0, const void *X, const void *bias1, const int32_t *shift1, int relu,
+                           const void *bias2, const int32_t *shift2, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st)
 {
     const bsp_xdesc xd = gt_flatten(wd1, xd0);
     const PackedLayout L1 = packed_layout(wd1), L2 = packed_layout(wd2);
     if (!L1.enabled || !L2.enabled) return BSP_ERR_SHAPE;
-    const int ey = ytype == BSP_BF16 ? 2 : 4;
+    const int ey = ytype == BSP_BF16 ? 2 : (ytype == BSP_I8 ? 1 : 4);
+    const int esz = elem_bytes(wd1.wtype);
+    if (wd1.wtype == BSP_I8 && (shift1 == nullptr || (ytype == BSP_I8 && shift2 == nullptr))) return BSP_ERR_NULL;
     CtParams p = {};
-    p.bias1 = bias1; p.bias2 = bias2; p.packed1 = (const uint8_t *)packed1; p.packed2 = (const uint8_t *)packed2;
+    p.bias1 = bias1; p.bias2 = bias2; p.shift1 = shift1; p.shift2 = shift2; p.wtype = wd1.wtype; p.packed1 = (const uint8_t *)packed1; p.packed2 = (const uint8_t *)packed2;
     p.status = (int *)ws;
     p.O1 = wd1.O; p.I1 = wd1.I; p.H = wd1.H; p.K = wd1.K; p.bo1 = wd1.bo; p.bi1 = wd1.bi;
     p.O2 = wd2.O; p.bo2 = wd2.bo; p.bi2 = wd2.bi; p.relu = relu ? 1 : 0; p.ytype = ytype; p.ey = ey; p.Y = (uint8_t *)Y;
-    p.O1p = (wd1.O + 63) / 64 * 64;
+    p.tcc = 128 / esz;
+    p.O1p = (wd1.O + p.tcc - 1) / p.tcc * p.tcc;
     p.N = xd.N; p.sh = xd.stride_h; p.sw = xd.stride_w; p.ph = xd.pad_h; p.pw = xd.pad_w;
     p.M = (xd.L + 2 * xd.pad_h - wd1.H) / xd.stride_h + 1;
     p.Nw = (xd.J + 2 * xd.pad_w - wd1.K) / xd.stride_w + 1;
@@ -415,9 +473,9 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
     p.m_tx = gt_magic(p.tiles_x); p.m_ty = gt_magic(p.tiles_y);
     p.a_bytes = p.rows_tile * 128;
     p.n_tiles = (int)T.tiles;
-    p.cpt1 = (wd1.I * 2 + 127) / 128;
+    p.cpt1 = (wd1.I * esz + 127) / 128;
     p.n_ks1 = wd1.H * wd1.K * p.cpt1;
-    p.n_c2 = p.O1p / 64;
+    p.n_c2 = p.O1p / p.tcc;
     p.n_t2 = (wd2.O + kCtBN2 - 1) / kCtBN2;
     p.stage_bytes = kGtABytes + p.O1p * 128;
     p.db = p.O1p <= 128 ? 1 : 0;
@@ -441,7 +499,7 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
     GtEncodeFn enc = gt_encode();
     if (!enc) return BSP_ERR_CUDA;
     {
-        const cuuint64_t row = (cuuint64_t)wd1.I * 2;
+        const cuuint64_t row = (cuuint64_t)wd1.I * esz;
         const cuuint64_t gdim[4] = {row, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N};
         const cuuint64_t gstr[3] = {row, row * xd.J, row * xd.J * xd.L};
         const cuuint32_t box[4] = {128, (cuuint32_t)(T.Wt * p.sw), (cuuint32_t)(T.Ht * p.sh), (cuuint32_t)T.Nt};
@@ -451,7 +509,7 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
             return BSP_ERR_CUDA;
     }
     {
-        const cuuint64_t row = (cuuint64_t)wd1.I * 2;
+        const cuuint64_t row = (cuuint64_t)wd1.I * esz;
         const cuuint64_t gdim[3] = {row, (cuuint64_t)(wd1.H * wd1.K), (cuuint64_t)wd1.O};
         const cuuint64_t gstr[2] = {row, row * wd1.H * wd1.K};
         const cuuint32_t box[3] = {128, 1, (cuuint32_t)p.O1p};
@@ -462,7 +520,7 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
             return BSP_ERR_CUDA;
     }
     {
-        const cuuint64_t row = (cuuint64_t)wd2.I * 2;
+        const cuuint64_t row = (cuuint64_t)wd2.I * esz;
         const cuuint64_t gdim[3] = {row, 1, (cuuint64_t)wd2.O};
         const cuuint64_t gstr[2] = {row, row};
         const cuuint32_t box[3] = {128, 1, (cuuint32_t)kCtBN2};

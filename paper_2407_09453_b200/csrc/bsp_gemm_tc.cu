@@ -49,16 +49,6 @@ struct GtParams {
     uint32_t m_ntn, m_tx, m_ty;       // floor(2^32 / d) of n_tiles_n, tiles_x, tiles_y (division by multiplication)
 };
 
-// Requantisation of the 8-bit path (Section "Compiler and its Code generation", Eq. (quant)): v / 2^s rounded to the
-// nearest integer, halves away from zero, saturated to int8.
-__device__ __forceinline__ uint32_t gt_requant(int v, uint32_t s)
-{
-    const uint32_t mag = v < 0 ? 0u - (uint32_t)v : (uint32_t)v;        // at most 2^31
-    const uint32_t r = s ? (mag + (1u << (s - 1u))) >> s : mag;          // no overflow: mag + 2^30 < 2^32
-    const int q = v < 0 ? -(int)min(r, 128u) : (int)min(r, 127u);
-    return (uint32_t)q & 0xFFu;
-}
-
 // First output position (image, row, column) of position tile mt.
 __device__ __forceinline__ void gt_tile_origin(const GtParams &p, int mt, int &n0, int &y0, int &x0)
 {

@@ -60,8 +60,8 @@ void report_cuda_error(cudaError_t e, const char *expr, const char *file, int li
 bool gemm_tc_eligible(const bsp_wdesc &wd, const bsp_xdesc &xd, bsp_dtype ytype);
 bool chain_tc_eligible(const bsp_wdesc &wd1, const bsp_wdesc &wd2, const bsp_xdesc &xd, bsp_dtype ytype);
 bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_wdesc &wd2, const void *packed2,
-                           const bsp_xdesc &xd, const void *X, const float *bias1, int relu, const float *bias2, void *Y,
-                           bsp_dtype ytype, void *ws, cudaStream_t st);
+                           const bsp_xdesc &xd, const void *X, const void *bias1, const int32_t *shift1, int relu,
+                           const void *bias2, const int32_t *shift2, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
 bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd, const void *packed, const void *X,
                           const void *bias, const int32_t *shift, void *Y, bsp_dtype ytype, void *ws, cudaStream_t st);
 // Output channels per CTA tile of the product kernel (a multiple of 64, at most 256).

@@ -113,6 +113,16 @@ __device__ __forceinline__ void gt_divmod(int n, int d, uint32_t m, int &q, int 
     if (r >= d) { ++q; r -= d; }
 }
 
+// Requantisation of the 8-bit path (Section "Compiler and its Code generation", Eq. (quant)): v / 2^s rounded to the
+// nearest integer, halves away from zero, saturated to int8.
+__device__ __forceinline__ uint32_t gt_requant(int v, uint32_t s)
+{
+    const uint32_t mag = v < 0 ? 0u - (uint32_t)v : (uint32_t)v;        // at most 2^31
+    const uint32_t r = s ? (mag + (1u << (s - 1u))) >> s : mag;          // no overflow: mag + 2^30 < 2^32
+    const int q = v < 0 ? -(int)min(r, 128u) : (int)min(r, 127u);
+    return (uint32_t)q & 0xFFu;
+}
+
 // Barrier `id` (1..15) over the 128 threads of a group of four warps, and the same with the AND of a flag.
 __device__ __forceinline__ void gt_group_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
 __device__ __forceinline__ bool gt_group_all(int id, bool flag)

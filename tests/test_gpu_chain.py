@@ -100,6 +100,54 @@ def test_equals_the_two_separate_calls_bit_for_bit(N, L, J, I, O1, O2, relu):
     assert torch.equal(Ya, Yb)
 
 
+def run_chain_q8(seed, N, L, J, I, O1, O2, H, K, stride, pad, relu, int8_out):
+    W1 = make_case(seed, O1, I, H, K, "i8")
+    W2 = make_case(seed + 1, O2, O1, 1, 1, "i8")
+    g1 = synth.random_gamma(seed + 2, O1 // 8, I // 8, (O1 // 8) * (I // 8) // 2)
+    g2 = synth.random_gamma(seed + 3, O2 // 8, O1 // 8, (O2 // 8) * (O1 // 8) // 2)
+    X = make_x(seed + 4, (N, L, J, I), "i8")
+    b1, b2 = make_bias(seed + 5, O1, "i8"), make_bias(seed + 6, O2, "i8")
+    # shifts that leave tensors which use the int8 range (sums of H K I / 2 products of magnitude ~ 64^2)
+    base1 = int(np.log2(np.sqrt(H * K * I / 2.0) * 5500 / 40))
+    s1 = (base1 + synth.uniform_int(seed + 7, (O1,), -1, 1)).astype(np.int32)
+    base2 = int(np.log2(np.sqrt(O1 / 2.0) * 64 * 40 / 40))
+    s2 = (base2 + synth.uniform_int(seed + 8, (O2,), -1, 1)).astype(np.int32)
+    l1, l2 = gpu_layer(W1, g1, 8, 8, "i8"), gpu_layer(W2, g2, 8, 8, "i8")
+    M = (L + 2 * pad[0] - H) // stride[0] + 1
+    Nw = (J + 2 * pad[1] - K) // stride[1] + 1
+    Y = torch.full((N, M, Nw, O2), -7, dtype=torch.int8 if int8_out else torch.int32, device="cuda")
+    xd = bsp.XDesc(N, L, J, stride[0], stride[1], pad[0], pad[1])
+    dev = lambda a: torch.from_numpy(a).cuda()
+    bsp.bsp_conv2d_chain_q8(l1.wd, l1.handle(), l2.wd, l2.handle(), xd, dev(X), dev(b1), dev(s1), relu, dev(b2),
+                            dev(s2) if int8_out else None, Y, l1.ws)
+    l1.check()
+    got = Y.cpu().numpy().reshape(-1, O2)
+    want = ref.chain2_q8(W1.shape, 8, 8, ref.compact(W1, g1, 8, 8), X, b1, s1, relu, O2, 8, 8, ref.compact(W2, g2, 8, 8), b2,
+                         s2 if int8_out else None, stride, pad)
+    assert got.dtype == want.dtype and np.array_equal(got, want)
+    T8 = ref.requant_i8(ref.conv2d(W1.shape, 8, 8, *ref.compact(W1, g1, 8, 8), X, b1, stride, pad), s1)
+    assert 16 < np.abs(T8).max() and (np.abs(T8) == 127).mean() < 0.2         # the tensor between the layers is neither tiny nor all saturated
+    return got
+
+
+@pytest.mark.parametrize("relu", [0, 1])
+@pytest.mark.parametrize("int8_out", [False, True])
+def test_int8_chain_bit_exact(relu, int8_out):
+    run_chain_q8(1101, 3, 14, 14, 64, 64, 256, 3, 3, (1, 1), (1, 1), relu, int8_out)
+
+
+@pytest.mark.parametrize("O1,O2,I", [(128, 512, 128), (256, 128, 64), (16, 16, 16), (144, 208, 48)])
+def test_int8_chain_channel_counts(O1, O2, I):
+    run_chain_q8(1111, 2, 9, 11, I, O1, O2, 3, 3, (1, 1), (1, 1), 1, True)
+
+
+def test_int8_chain_many_tiles_strides_and_taps():
+    run_chain_q8(1121, 8, 56, 56, 64, 64, 128, 3, 3, (1, 1), (1, 1), 1, False)
+    run_chain_q8(1123, 2, 35, 35, 32, 96, 64, 3, 3, (2, 2), (0, 0), 0, True)
+    run_chain_q8(1125, 2, 17, 17, 128, 128, 192, 1, 7, (1, 1), (0, 3), 1, True)
+    run_chain_q8(1127, 4, 28, 28, 256, 64, 256, 1, 1, (1, 1), (0, 0), 1, True)
+
+
 def test_argument_errors():
     l1 = bsp.SparseLayer(64, 64, 3, 3, 8, 8, torch.bfloat16)
     l3 = bsp.SparseLayer(128, 64, 3, 3, 8, 8, torch.bfloat16)          # not 1x1
