@@ -436,6 +436,40 @@ def pass_chain(gpu, bsp, torch, pk, reps=10):
                     "bit_identical": bool(torch.equal(Ya, Yb)), "effective_tflops": useful / (tf["ms"] * 1e-3) / 1e12,
                     "algorithmic_bytes": hbm, "bytes_saved_vs_separate": 2 * T.numel() * 2, "roofline_ms": t_roof,
                     "frac": t_roof / tf["ms"]})
+    # the same tail on 8-bit tensors (int8 between the layers and out, power-of-two scales): exact, so the comparison is bit for bit
+    N, L, I, O1, O2 = 64, 56, 64, 64, 256
+    W1 = torch.randint(-127, 128, (O1, 3, 3, I), device="cuda", dtype=torch.int8, generator=g)
+    W2 = torch.randint(-127, 128, (O2, 1, 1, O1), device="cuda", dtype=torch.int8, generator=g)
+    X = torch.randint(-127, 128, (N, L, L, I), device="cuda", dtype=torch.int8, generator=g)
+    b1 = torch.randint(-(1 << 15), 1 << 15, (O1,), device="cuda", dtype=torch.int32, generator=g)
+    b2 = torch.randint(-(1 << 15), 1 << 15, (O2,), device="cuda", dtype=torch.int32, generator=g)
+    s1 = torch.full((O1,), 11, device="cuda", dtype=torch.int32)
+    s2 = torch.full((O2,), 9, device="cuda", dtype=torch.int32)
+    l1 = bsp.SparseLayer(O1, I, 3, 3, 8, 8, torch.int8, canonical=False)
+    l2 = bsp.SparseLayer(O2, O1, 1, 1, 8, 8, torch.int8, canonical=False)
+    for lay, W in ((l1, W1), (l2, W2)):
+        lay.mask(W, lay.NBo * lay.NBi // 2)
+        lay.compact(W)
+    T = torch.empty((N, L, L, O1), dtype=torch.int8, device="cuda")
+    Ya = torch.empty((N, L, L, O2), dtype=torch.int8, device="cuda")
+    Yb = torch.empty_like(Ya)
+    xd = bsp.XDesc(N, L, L, 1, 1, 1, 1)
+
+    def separate8():
+        l1.conv2d_q8(X, b1, s1, T, (1, 1), (1, 1))
+        l2.conv2d_q8(T, b2, s2, Ya)
+
+    def fused8():
+        bsp.bsp_conv2d_chain_q8(l1.wd, l1.handle(), l2.wd, l2.handle(), xd, X, b1, s1, 0, b2, s2, Yb, l1.ws)
+
+    ts = stats(gpu.timed(separate8, reps, 2))
+    tf = stats(gpu.timed(fused8, reps, 1))
+    l1.check()
+    l2.check()
+    hbm = X.numel() + Yb.numel() + (W1.numel() + W2.numel()) // 2
+    out.append({"pair": "c2.3x3.64-64+1x1.64-256 int8 -> int8", "separate_ms": ts["ms"], "fused_ms": tf["ms"], "speedup": ts["ms"] / tf["ms"],
+                "bit_identical": bool(torch.equal(Ya, Yb)), "algorithmic_bytes": hbm, "bytes_saved_vs_separate": 2 * T.numel(),
+                "roofline_ms": hbm / (pk["hbm_gbs"] * 1e9) * 1e3, "frac": hbm / (pk["hbm_gbs"] * 1e9) * 1e3 / tf["ms"]})
     return out
 
 
