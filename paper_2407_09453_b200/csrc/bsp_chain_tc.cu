@@ -62,8 +62,11 @@ __device__ __forceinline__ bool ct_header_ok(const uint8_t *packed, int wtype, i
            h->bi == bi && (h->forms & kFormDense) != 0;
 }
 
+// kI8: the 8-bit chain (compiled apart, so that neither form carries the other's epilogue code and registers).
+template <bool kI8>
 __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_constant__ CtParams p)
 {
+    constexpr int kWt = kI8 ? BSP_I8 : BSP_BF16;
     extern __shared__ __align__(16) uint8_t ct_smem_raw[];
     uint8_t *smem = ct_smem_raw + ((1024u - (sm32(ct_smem_raw) & 1023u)) & 1023u);
     __shared__ __align__(8) uint64_t s_full[kGtMaxStages], s_empty[kGtMaxStages];
@@ -185,7 +188,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
         // ================= MMA issuer =================
         if (run) {
             // instruction descriptors: A and B bf16 (signed int8), K-major both, M = 128; N = O1p for layer one, 128 for layer two
-            const uint32_t dfmt = p.wtype == BSP_I8 ? 2u : 1u;      // D int32 for int8 operands, fp32 otherwise
+            const uint32_t dfmt = kI8 ? 2u : 1u;      // D int32 for int8 operands, fp32 otherwise
             const uint32_t idesc1 = (dfmt << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.O1p >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc2 = (dfmt << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCtBN2 >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
@@ -206,7 +209,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     if (!got) { ok = false; return; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
-                    gt_issue_stage<false>(p.wtype, d, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    gt_issue_stage<false>(kWt, d, da, db, idesc1, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
                     if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                 }
                 gt_commit_elected<false>(sm32(&s_acc1_full[b]));
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                         const uint64_t da = kGtDesc | (uint64_t)(((tbuf + b * tbytes + (uint32_t)(c2 * kCtChunk)) >> 4) & 0x3FFFu);
                         const uint64_t db = kGtDesc | (uint64_t)(a16 & 0x3FFFu);
-                        gt_issue_stage<false>(p.wtype, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
+                        gt_issue_stage<false>(kWt, d, da, db, idesc2, empty0 + slot * 8u, c2 != 0 ? 1u : 0u);
                         if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                     }
                     gt_commit_elected<false>(sm32(&s_acc2_full[buf]));
@@ -277,7 +280,7 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                 const uint32_t a1 = t1 + b1 * 128u;                  // this tile's accumulator one
                 for (int c2 = grp; c2 < p.n_c2; c2 += 2) {
                     uint32_t out[32];                            // one chunk (128 bytes of channels) of this lane's row of T
-                    if (p.wtype == BSP_I8) {                     // 128 channels: + b1, rounding shift, activation, int8
+                    if constexpr (kI8) {                         // 128 channels: + b1, rounding shift, activation, int8
 #pragma unroll
                         for (int sub = 0; sub < 4; ++sub) {
                             uint32_t v[32];
@@ -348,14 +351,14 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                             gt_load32(t2base + (uint32_t)c0, v);
                             const int ch = n0 + c0 + lane;
                             const uint32_t bl = (p.bias2 != nullptr && ch < p.O2) ? __ldg((const uint32_t *)p.bias2 + ch) : 0u;
-                            if (p.wtype == BSP_I8) {
+                            if constexpr (kI8) {
 #pragma unroll
                                 for (int e = 0; e < 32; ++e) out[e] = (uint32_t)((int)v[e] + (int)__shfl_sync(0xFFFFFFFFu, bl, e));
                             } else {
 #pragma unroll
                                 for (int e = 0; e < 32; ++e) out[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(__shfl_sync(0xFFFFFFFFu, bl, e)));
                             }
-                        } else if (ey == 1) {                    // int8 output: 128 channels, requantised after the bias
+                        } else if (kI8 && ey == 1) {             // int8 output: 128 channels, requantised after the bias
 #pragma unroll
                             for (int sub = 0; sub < 4; ++sub) {
                                 uint32_t v[32];
@@ -492,7 +495,8 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
     BSP_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kGtMaxDevices) return BSP_ERR_CUDA;
     if (!opted[dev]) {
-        BSP_CUDA_OK(cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(chain_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
+        BSP_CUDA_OK(cudaFuncSetAttribute(chain_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGtMaxSmem));
         BSP_CUDA_OK(cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev));
         opted[dev] = true;
     }
@@ -541,7 +545,8 @@ bsp_status launch_chain_tc(const bsp_wdesc &wd1, const void *packed1, const bsp_
             return BSP_ERR_CUDA;
     }
     const int grid = p.n_tiles < n_sm[dev] ? p.n_tiles : n_sm[dev];
-    chain_tc_kernel<<<grid, kCtThreads, smem, st>>>(p);
+    if (wd1.wtype == BSP_I8) chain_tc_kernel<true><<<grid, kCtThreads, smem, st>>>(p);
+    else chain_tc_kernel<false><<<grid, kCtThreads, smem, st>>>(p);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }
