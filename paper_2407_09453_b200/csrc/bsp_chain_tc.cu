@@ -283,6 +283,11 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                     if constexpr (kI8) {                         // 128 channels: + b1, rounding shift, activation, int8
 #pragma unroll
                         for (int sub = 0; sub < 4; ++sub) {
+                            if (c2 * 128 + sub * 32 >= p.O1) {       // (past the last channel of T: zeros, as the weights of layer two there)
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) out[sub * 8 + e] = 0u;
+                                continue;
+                            }
                             uint32_t v[32];
                             gt_load32(a1 + (uint32_t)(c2 * 128 + sub * 32), v);
                             const int ch = c2 * 128 + sub * 32 + lane;
@@ -361,6 +366,11 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                         } else if (kI8 && ey == 1) {             // int8 output: 128 channels, requantised after the bias
 #pragma unroll
                             for (int sub = 0; sub < 4; ++sub) {
+                                if (n0 + c0 + sub * 32 >= p.O2) {    // (past the last channel: clipped by the store)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) out[sub * 8 + e] = 0u;
+                                    continue;
+                                }
                                 uint32_t v[32];
                                 gt_load32(t2base + (uint32_t)(c0 + sub * 32), v);
                                 const int ch = n0 + c0 + sub * 32 + lane;

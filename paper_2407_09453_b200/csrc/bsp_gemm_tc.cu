@@ -267,6 +267,12 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                     } else if (ey == 1) {                        // int8 output: 128 channels, requantised after the bias
 #pragma unroll
                         for (int sub = 0; sub < 4; ++sub) {
+                            // (32-channel pieces past the tile or past the last channel are not computed: their bytes are clipped by the store)
+                            if (c0 + sub * 32 >= BN || n0 + c0 + sub * 32 >= p.O) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) out[sub * 8 + e] = 0u;
+                                continue;
+                            }
                             uint32_t v[32];
                             gt_load32(tbase + (uint32_t)(c0 + sub * 32), v);
                             const int ch = n0 + c0 + sub * 32 + lane;
@@ -398,14 +404,15 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     }
     // Channels per tile: the widest tile keeps the tensor pipe busiest (a stage costs about 256 + 2 BN cycles of operand
     // fetch from shared memory), but a layer with few position tiles fills more SMs with narrower ones: the width with
-    // the lowest waves x stage cost wins.  (A staging round of the int8 output covers 128 channels, so those tiles are
-    // multiples of 128 channels.)
+    // the lowest waves x stage cost wins.
     {
-        const int step = ytype == BSP_I8 ? 128 : 64;
+        const int step = 64;
         const int widest = (gemm_tile_n(wd.O) + step - 1) / step * step;
         long long best_cost = -1;
         for (int bn = widest; bn >= step; bn -= step) {
             if (bn != widest && bn != 128 && bn != 64) continue;
+            // (a round of the int8 output stores 128 channels: a tile that is not a multiple of that must be the only one)
+            if (ytype == BSP_I8 && bn % 128 != 0 && bn < wd.O) continue;
             const long long tiles = T.tiles * ((wd.O + bn - 1) / bn);
             const long long cost = ((tiles + n_sm[dev] - 1) / n_sm[dev]) * (256 + 2 * bn);
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.BN = bn; }
