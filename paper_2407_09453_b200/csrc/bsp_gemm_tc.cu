@@ -47,6 +47,7 @@ struct GtParams {
     uint8_t *Y;
     int ey;
     uint32_t m_ntn, m_tx, m_ty;       // floor(2^32 / d) of n_tiles_n, tiles_x, tiles_y (division by multiplication)
+    int kbytes, a_stride;             // bytes of K per row of a stage: 128, or 64 for layers with at most 64 bytes of input channels; bytes of the activation part of a stage
 };
 
 // First output position (image, row, column) of position tile mt.
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             // (a pair: each CTA loads its own activation box and its half of the weight tile, all four loads announce their
             // bytes on the leader's barrier, which the leader arms with the total)
             const uint32_t stage_bytes = (uint32_t)p.stage_bytes;
-            const uint32_t tx = (uint32_t)(p.a_bytes + (BN >> (kPair ? 1 : 0)) * 128) * (kPair ? 2u : 1u);
+            const uint32_t tx = (uint32_t)(p.a_bytes + (BN >> (kPair ? 1 : 0)) * p.kbytes) * (kPair ? 2u : 1u);
             const int cpt128 = p.cpt * 128, Kw = p.K, ntn = p.n_tiles_n;
             // (a fresh barrier counts as released: the wait on parity 1 of the first round returns at once)
             uint32_t slot = 0, epar = 1, issued = 0, dst = ring;
@@ -160,14 +161,14 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                                      " @e cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%13];\n"
                                      " @e cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%4, %10, %11}], [%13];\n}\n"
                                      ::"r"(full0 + slot * 8u), "r"(tx), "r"(dst), "l"(&p.tmx), "r"(c128), "r"(kx), "r"(hy), "r"(n0),
-                                       "r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(tap), "r"(ch0), "r"(rank), "r"(lead_full0 + slot * 8u) : "memory");
+                                       "r"(dst + (uint32_t)p.a_stride), "l"(&p.tmw), "r"(tap), "r"(ch0), "r"(rank), "r"(lead_full0 + slot * 8u) : "memory");
                     } else {
                         asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xFFFFFFFF;\n"
                                      " @e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
                                      " @e cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%3, {%4, %5, %6, %7}], [%0];\n"
                                      " @e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%4, %10, %11}], [%0];\n}\n"
                                      ::"r"(full0 + slot * 8u), "r"(tx), "r"(dst), "l"(&p.tmx), "r"(c128), "r"(kx), "r"(hy), "r"(n0),
-                                       "r"(dst + (uint32_t)kGtABytes), "l"(&p.tmw), "r"(tap), "r"(ch0) : "memory");
+                                       "r"(dst + (uint32_t)p.a_stride), "l"(&p.tmw), "r"(tap), "r"(ch0) : "memory");
                     }
                     ++issued;
                     if (++slot == (uint32_t)S) { slot = 0; epar ^= 1u; dst = ring; } else dst += stage_bytes;
@@ -200,7 +201,9 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
             const uint32_t dfmt = p.wtype == BSP_I8 ? 2u : 1u, abfmt = p.wtype == BSP_F32 ? 2u : 1u;
             const uint32_t idesc = (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(BN >> 3) << 17) | (((kPair ? 256u : 128u) >> 4) << 24);
             const uint32_t full0 = sm32(&s_full[0]), empty0 = sm32(&s_empty[0]);
-            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
+            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, astride16 = (uint32_t)p.a_stride >> 4;
+            const uint64_t desc0 = p.kbytes == 64 ? kGtDesc64 : kGtDesc;
+            const uint32_t nk = (uint32_t)p.kbytes >> 5;            // MMAs per stage: 32 bytes of K each
             uint32_t slot = 0, par = 0, a16 = ring >> 4, tile_i = 0;
             bool ok = true;
             for (int tile = t_first; tile < t_count && ok; tile += t_step, ++tile_i) {
@@ -215,8 +218,8 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                     got = __all_sync(0xFFFFFFFFu, got);
                     if (!got) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                    const uint64_t da = kGtDesc | (uint64_t)(a16 & 0x3FFFu), db = kGtDesc | (uint64_t)((a16 + (kGtABytes >> 4)) & 0x3FFFu);
-                    gt_issue_stage<kPair>(p.wtype, d, da, db, idesc, empty0 + slot * 8u, ks != 0 ? 1u : 0u);
+                    const uint64_t da = desc0 | (uint64_t)(a16 & 0x3FFFu), db = desc0 | (uint64_t)((a16 + astride16) & 0x3FFFu);
+                    gt_issue_stage<kPair>(p.wtype, d, da, db, idesc, empty0 + slot * 8u, ks != 0 ? 1u : 0u, nk);
                     if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; a16 = ring >> 4; } else a16 += stage16;
                 }
                 if (ok) gt_commit_elected<kPair>(sm32(&s_acc_full[buf]));
@@ -390,7 +393,10 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     if (T.tiles <= 0) return BSP_ERR_SHAPE;
     p.Wt = T.Wt; p.Ht = T.Ht; p.Nt = T.Nt; p.rows_tile = T.Wt * T.Ht * T.Nt;
     p.tiles_x = (p.Nw + T.Wt - 1) / T.Wt; p.tiles_y = (p.M + T.Ht - 1) / T.Ht;
-    p.a_bytes = p.rows_tile * 128;
+    // layers with at most 64 bytes of input channels per position stage 64-byte rows (64-byte swizzle, two MMAs a stage)
+    p.kbytes = (long long)wd.I * esz <= 64 ? 64 : 128;
+    p.a_stride = kGtBM * p.kbytes;
+    p.a_bytes = p.rows_tile * p.kbytes;
     static bool opted[kGtMaxDevices] = {};
     static int n_sm[kGtMaxDevices] = {};
     int dev = 0;
@@ -426,10 +432,10 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
     // (Tiles of a few K-stages are bound by their epilogue, and there the pair's cross-CTA hand-shakes only cost.)
     p.cpt = (int)(((long long)wd.I * esz + 127) / 128);
     p.n_ks = HK * p.cpt;
-    const bool pair = p.BN == 256 && p.n_ks >= 8 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
+    const bool pair = p.kbytes == 128 && p.BN == 256 && p.n_ks >= 8 && (long long)p.n_tiles >= 4LL * n_sm[dev] && n_sm[dev] >= 2;
     p.n_tile_pairs = (int)(((T.tiles + 1) / 2) * p.n_tiles_n);
     p.m_ntn = gt_magic(p.n_tiles_n); p.m_tx = gt_magic(p.tiles_x); p.m_ty = gt_magic(p.tiles_y);
-    p.stage_bytes = kGtABytes + (pair ? p.BN / 2 : p.BN) * 128;
+    p.stage_bytes = p.a_stride + (pair ? p.BN / 2 : p.BN) * p.kbytes;
     const int staging = 8 * kGtStagingBytes;
     int stages = (kGtMaxSmem - 1024 - staging) / p.stage_bytes;
     if (stages > kGtMaxStages) stages = kGtMaxStages;
@@ -444,20 +450,20 @@ bsp_status launch_gemm_tc(const bsp_wdesc &wd, const bsp_xdesc &xd0, const void 
         const cuuint64_t gdim[4] = {row, (cuuint64_t)xd.J, (cuuint64_t)xd.L, (cuuint64_t)xd.N};
         const cuuint64_t gstr[3] = {row, row * xd.J, row * xd.J * xd.L};
         // a box spans Wt * s_w x Ht * s_h input positions in steps of the strides: Wt x Ht positions arrive
-        const cuuint32_t box[4] = {128, (cuuint32_t)(T.Wt * p.sw), (cuuint32_t)(T.Ht * p.sh), (cuuint32_t)T.Nt};
+        const cuuint32_t box[4] = {(cuuint32_t)p.kbytes, (cuuint32_t)(T.Wt * p.sw), (cuuint32_t)(T.Ht * p.sh), (cuuint32_t)T.Nt};
         const cuuint32_t estr[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
         if (enc(&p.tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(X), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                p.kbytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
     }
     {
         const cuuint64_t row = (cuuint64_t)wd.I * esz;
         const cuuint64_t gdim[3] = {row, (cuuint64_t)HK, (cuuint64_t)wd.O};
         const cuuint64_t gstr[2] = {row, row * HK};
-        const cuuint32_t box[3] = {128, 1, (cuuint32_t)(pair ? p.BN / 2 : p.BN)};
+        const cuuint32_t box[3] = {(cuuint32_t)p.kbytes, 1, (cuuint32_t)(pair ? p.BN / 2 : p.BN)};
         const cuuint32_t estr[3] = {1, 1, 1};
         if (enc(&p.tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>((const uint8_t *)packed + L.off_payload), gdim, gstr, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, p.kbytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return BSP_ERR_CUDA;
     }

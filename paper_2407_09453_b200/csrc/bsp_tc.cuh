@@ -48,27 +48,31 @@ __device__ __forceinline__ bool gt_wait(uint32_t bar, uint32_t parity)
 // the low 14 bits): rows of 128 bytes, 8-row groups 1024 bytes apart; a K-step of 32 bytes inside the swizzle span is
 // an advance of the start address by 2.
 constexpr uint64_t kGtDesc = (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+// The same for rows of 64 bytes under the 64-byte swizzle (layers with at most 64 bytes of input channels): 8-row
+// groups 512 bytes apart, two K-steps of 32 bytes.
+constexpr uint64_t kGtDesc64 = (1ull << 16) | ((uint64_t)(512u >> 4) << 32) | (1ull << 46) | (4ull << 61);
 
-// The four MMAs of one stage and the commit that releases the stage, issued by one elected lane of a converged warp.
-// All lanes execute this statement with the same operands; the MMA of the first K-step overwrites the accumulator
-// when `acc` is 0.
+// The four MMAs of one stage (two when the stage holds 64 bytes of K: `nk`) and the commit that releases the stage,
+// issued by one elected lane of a converged warp.  All lanes execute this statement with the same operands; the MMA of
+// the first K-step overwrites the accumulator when `acc` is 0.
 #define GT_ISSUE_STAGE(KIND, CG, COMMIT_TAIL)                                                                       \
-    asm volatile("{\n .reg .pred e, p, t;\n .reg .b64 a1, a2, a3, b1, b2, b3;\n"                                     \
+    asm volatile("{\n .reg .pred e, e3, p, t;\n .reg .b64 a1, a2, a3, b1, b2, b3;\n"                                 \
                  " elect.sync _|e, 0xFFFFFFFF;\n setp.ne.b32 p, %5, 0;\n setp.eq.b32 t, %5, %5;\n"                    \
+                 " setp.gt.u32 e3, %7, 2;\n and.pred e3, e3, e;\n"                                                    \
                  " add.u64 a1, %1, 2;\n add.u64 a2, %1, 4;\n add.u64 a3, %1, 6;\n"                                    \
                  " add.u64 b1, %2, 2;\n add.u64 b2, %2, 4;\n add.u64 b3, %2, 6;\n"                                    \
                  " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], %1, %2, %3, p;\n"                                 \
                  " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a1, b1, %3, t;\n"                                 \
-                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a2, b2, %3, t;\n"                                 \
-                 " @e tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a3, b3, %3, t;\n"                                 \
+                 " @e3 tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a2, b2, %3, t;\n"                                \
+                 " @e3 tcgen05.mma.cta_group::" CG ".kind::" KIND " [%0], a3, b3, %3, t;\n"                                \
                  " @e tcgen05.commit.cta_group::" CG ".mbarrier::arrive::one.shared::cluster" COMMIT_TAIL ";\n}\n"        \
-                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(bar_empty), "r"(acc), "h"((unsigned short)3) : "memory")
+                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(bar_empty), "r"(acc), "h"((unsigned short)3), "r"(nk) : "memory")
 
 // kPair: the MMAs span a pair of CTAs (cta_group::2, M = 256: each CTA its own 128 positions and half of the weight
 // tile); the commits then arrive on the barrier at the same shared-memory offset in both CTAs.
 template <bool kPair>
 __device__ __forceinline__ void gt_issue_stage(int wtype, uint32_t d, uint64_t da, uint64_t db, uint32_t idesc,
-                                               uint32_t bar_empty, uint32_t acc)
+                                               uint32_t bar_empty, uint32_t acc, uint32_t nk = 4u)
 {
     if constexpr (kPair) {
         if (wtype == BSP_BF16) GT_ISSUE_STAGE("f16", "2", ".multicast::cluster.b64 [%4], %6");
