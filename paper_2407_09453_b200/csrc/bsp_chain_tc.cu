@@ -295,14 +295,13 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                             const uint32_t sl = ch < p.O1 ? (uint32_t)__ldg(p.shift1 + ch) & 31u : 0u;
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
-                                uint32_t w = 0u;
+                                int r4[4];
 #pragma unroll
-                                for (int b = 0; b < 4; ++b) {
-                                    uint32_t qv = gt_requant((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
-                                                             __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b));
-                                    if (p.relu && (qv & 0x80u)) qv = 0u;
-                                    w |= qv << (8 * b);
-                                }
+                                for (int b = 0; b < 4; ++b)
+                                    r4[b] = gt_round_shift((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
+                                                           __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b));
+                                uint32_t w = gt_pack_s8x4(r4[0], r4[1], r4[2], r4[3]);
+                                if (p.relu) w = __vmaxs4(w, 0u);
                                 out[sub * 8 + e] = w;
                             }
                         }
@@ -378,10 +377,11 @@ __global__ void __launch_bounds__(kCtThreads, 1) chain_tc_kernel(const __grid_co
                                 const uint32_t sl = ch < p.O2 ? (uint32_t)__ldg(p.shift2 + ch) & 31u : 0u;
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) {
-                                    uint32_t w = 0u;
+                                    int r4[4];
 #pragma unroll
                                     for (int b = 0; b < 4; ++b)
-                                        w |= gt_requant((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b), __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b)) << (8 * b);
+                                        r4[b] = gt_round_shift((int)v[4 * e + b] + __shfl_sync(0xFFFFFFFFu, bl, 4 * e + b), __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b));
+                                    const uint32_t w = gt_pack_s8x4(r4[0], r4[1], r4[2], r4[3]);
                                     out[sub * 8 + e] = w;
                                 }
                             }

@@ -283,12 +283,12 @@ __global__ void __launch_bounds__(kGtThreads, 1) gemm_tc_kernel(const __grid_con
                             const uint32_t sl = ch < p.O ? (uint32_t)__ldg(p.shift + ch) & 31u : 0u;
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
-                                uint32_t w = 0u;
+                                int r4[4];
 #pragma unroll
                                 for (int b = 0; b < 4; ++b)
-                                    w |= gt_requant((int)v[4 * e + b] + (int)__shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
-                                                    __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b)) << (8 * b);
-                                out[sub * 8 + e] = w;
+                                    r4[b] = gt_round_shift((int)v[4 * e + b] + (int)__shfl_sync(0xFFFFFFFFu, bl, 4 * e + b),
+                                                           __shfl_sync(0xFFFFFFFFu, sl, 4 * e + b));
+                                out[sub * 8 + e] = gt_pack_s8x4(r4[0], r4[1], r4[2], r4[3]);
                             }
                         }
                     } else {                                     // bf16 output: 64 channels, rounded to nearest even after the bias

@@ -118,13 +118,23 @@ __device__ __forceinline__ void gt_divmod(int n, int d, uint32_t m, int &q, int 
 }
 
 // Requantisation of the 8-bit path (Section "Compiler and its Code generation", Eq. (quant)): v / 2^s rounded to the
-// nearest integer, halves away from zero, saturated to int8.
-__device__ __forceinline__ uint32_t gt_requant(int v, uint32_t s)
+// nearest integer, halves away from zero, as a 32-bit value that is not yet saturated (|v| + 2^(s-1) < 2^32, so the
+// magnitude is formed without overflow; -2^31 with s = 0 comes back as itself) ...
+__device__ __forceinline__ int gt_round_shift(int v, uint32_t s)
 {
-    const uint32_t mag = v < 0 ? 0u - (uint32_t)v : (uint32_t)v;        // at most 2^31
-    const uint32_t r = s ? (mag + (1u << (s - 1u))) >> s : mag;          // no overflow: mag + 2^30 < 2^32
-    const int q = v < 0 ? -(int)min(r, 128u) : (int)min(r, 127u);
-    return (uint32_t)q & 0xFFu;
+    const uint32_t sg = (uint32_t)(v >> 31);                              // 0 or all ones
+    const uint32_t mag = ((uint32_t)v ^ sg) - sg;                        // |v|, at most 2^31
+    const uint32_t r = (mag + ((1u << s) >> 1)) >> s;
+    return (int)((r ^ sg) - sg);
+}
+// ... and four such values saturated to int8 and packed, the first in the lowest byte (cvt.pack saturates two 32-bit
+// values to bytes, its first source above its second, and shifts the third operand up by 16 bits).
+__device__ __forceinline__ uint32_t gt_pack_s8x4(int v0, int v1, int v2, int v3)
+{
+    uint32_t hi, out;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;\n" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0u));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;\n" : "=r"(out) : "r"(v1), "r"(v0), "r"(hi));
+    return out;
 }
 
 // Barrier `id` (1..15) over the 128 threads of a group of four warps, and the same with the AND of a flag.
