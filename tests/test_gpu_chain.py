@@ -62,6 +62,13 @@ def test_first_layer_taps_strides_padding(H, K, stride, pad):
     run_chain(1021, 2, 17, 17, 48, 64, 128, H, K, stride, pad, 1)
 
 
+def test_tiles_that_hold_several_small_images():
+    """7x7 and 4x4 images: a tile is a box of whole images (two, eight), the last one ragged in the image count."""
+    run_chain(1025, 5, 7, 7, 64, 128, 256, 3, 3, (1, 1), (1, 1), 1)
+    run_chain(1027, 11, 4, 4, 32, 64, 72, 1, 1, (1, 1), (0, 0), 0)
+    run_chain_q8(1029, 5, 7, 7, 64, 128, 256, 3, 3, (1, 1), (1, 1), 1, True)
+
+
 def test_many_tiles_per_cta_and_long_k():
     """More position tiles than SMs (every CTA takes several: both second accumulators, the tensor buffer and all stages
     are reused) and a first layer of 9 x 4 K-stages."""
