@@ -203,11 +203,10 @@ def conv_kernel_name(wd: WDesc, xd: XDesc) -> str:
 
 
 def launches_per_step(wd: WDesc) -> int:
-    """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass.  General path: score, select;
-    row counts with their scan, fill; the product kernel.  Small layers take one launch for the mask (up to 4096 blocks) and
-    one for the compaction (up to 4096 blocks)."""
+    """Kernel launches of one bsp_mask + bsp_compact + bsp_conv2d/bsp_gemm pass.  General path: score, select; the
+    compaction; the product kernel.  Small layers take one launch for the mask (up to 4096 blocks)."""
     nb = (wd.O // wd.bo) * (wd.I // wd.bi)
-    return (1 if nb <= 4096 else 2) + (1 if nb <= 4096 else 2) + 1
+    return (1 if nb <= 4096 else 2) + 1 + 1
 
 
 class SparseLayer:

@@ -184,6 +184,32 @@ __device__ __forceinline__ int ones_share(const uint8_t *g, int n)
     return c;
 }
 
+// The same count over the first n bytes of Gamma in global memory (layers whose Gamma does not fit shared memory): 16-byte
+// loads, eight in flight per thread, when the addresses allow.
+__device__ __forceinline__ int ones_share_global(const uint8_t *__restrict__ g, int n)
+{
+    int c = 0;
+    if ((((uintptr_t)g) & 15u) == 0) {
+        const uint4 *g4 = (const uint4 *)g;
+        const int n4 = n >> 4;
+        for (int i0 = threadIdx.x; i0 < n4; i0 += 8 * kThreads) {
+            uint4 q[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * kThreads;
+                q[u] = i < n4 ? __ldg(g4 + i) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                c += __popc(__vsetne4(q[u].x, 0u)) + __popc(__vsetne4(q[u].y, 0u)) + __popc(__vsetne4(q[u].z, 0u)) + __popc(__vsetne4(q[u].w, 0u));
+        }
+        for (int i = (n4 << 4) + threadIdx.x; i < n; i += kThreads) c += g[i] ? 1 : 0;
+    } else {
+        for (int i = threadIdx.x; i < n; i += kThreads) c += g[i] ? 1 : 0;
+    }
+    return c;
+}
+
 // The packed form: Gamma (.) W in the layout of W, [O][H][K][I], the channels of zeroed blocks cleared.  CTA `idx` of
 // `n_ctas` takes every n_ctas-th stretch of 16-byte chunks, one chunk of input channels per thread and step, four loads
 // in flight per thread.  A "row" below is one (o, tap).
@@ -244,81 +270,17 @@ struct CompactArgs {
     int *status;
 };
 
-// Larger layers, first launch: CTA l counts the kept blocks of row l of Gamma; the CTA that finishes last (a ticket in
-// the workspace header, which it hands back as zero) turns the counts into row_ptr, checks the capacity and writes the
-// header of the packed buffer.  Nobody waits for anybody.
-__global__ void __launch_bounds__(kThreads)
-count_scan_kernel(const uint8_t *__restrict__ gamma, int NBi, int NBo, int *row_cnt, int32_t *__restrict__ row_ptr,
-                  PackedHeader *__restrict__ hdr, PackedHeader hdr_init, long long capacity_blocks, int *__restrict__ status,
-                  unsigned *ticket)
-{
-    __shared__ int warp_sums[kThreads / 32];
-    __shared__ int s_run;
-    __shared__ bool s_last;
-    const uint8_t *g = gamma + (size_t)blockIdx.x * NBi;
-    int c = 0;
-    if ((NBi & 15) == 0 && (((uintptr_t)gamma) & 15u) == 0) {
-        for (int i = threadIdx.x; i < (NBi >> 4); i += kThreads) {
-            const uint4 q = __ldg((const uint4 *)g + i);
-            c += __popc(__vsetne4(q.x, 0u)) + __popc(__vsetne4(q.y, 0u)) + __popc(__vsetne4(q.z, 0u)) + __popc(__vsetne4(q.w, 0u));
-        }
-    } else {
-        for (int i = threadIdx.x; i < NBi; i += kThreads) c += g[i] ? 1 : 0;
-    }
-    int tot;
-    block_exclusive_scan(c, warp_sums, tot);
-    if (threadIdx.x == 0) {
-        row_cnt[blockIdx.x] = tot;
-        __threadfence();
-        s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
-        s_run = 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    for (int base = 0; base < NBo; base += kThreads) {
-        const int i = base + threadIdx.x;
-        const int v = (i < NBo) ? __ldcg(row_cnt + i) : 0;
-        int all;
-        const int before = block_exclusive_scan(v, warp_sums, all);
-        if (i < NBo) row_ptr[i] = s_run + before;
-        __syncthreads();
-        if (threadIdx.x == 0) s_run += all;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        row_ptr[NBo] = s_run;
-        if ((long long)s_run > capacity_blocks) atomicMax(status, (int)BSP_ERR_CAPACITY);
-        if (hdr != nullptr) *hdr = hdr_init;
-        *ticket = 0u;
-    }
-}
-
-// Launch 3: CTAs [0, NBo * fill_parts) write col_idx and the canonical payload, the rest write the packed form.
+// The whole compaction in ONE launch: CTAs [0, NBo * fill_parts) write col_idx and the canonical payload, one row of
+// Gamma each, the rest write the packed form.  Every CTA of the first part counts for itself the stored blocks that
+// precede its row (no scan launch, nobody waits): from a copy of Gamma in shared memory for layers of up to
+// kSmallBlocks blocks, from global memory (through L2, while the other CTAs write the packed form) for larger ones.
 // T is the storage type of a weight.
-template <typename T>
-__global__ void __launch_bounds__(kThreads) fill_dense_kernel(const CompactArgs a)
-{
-    const int n_fill = a.NBo * a.fill_parts;
-    if ((int)blockIdx.x < n_fill) {
-        const int l = (int)blockIdx.x / a.fill_parts;
-        csr_fill_body<T>(l, (int)blockIdx.x % a.fill_parts, a.fill_parts, (const T *)a.W, a.gamma, a.NBi, a.I, a.HK, a.bo,
-                         a.bi, a.row_ptr[l], a.col_idx, (T *)a.payload, a.capacity_blocks);
-    } else {
-        if (a.dense != nullptr)
-            dense_body<(int)sizeof(T)>((int)blockIdx.x - n_fill, a.dense_ctas, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.dense);
-    }
-}
-
-// Layers of up to kSmallBlocks blocks: the whole compaction in ONE launch.  Gamma fits in shared memory, so every
-// CTA of the first part counts for itself the stored blocks that precede its row (what the count and scan launches
-// hand over through memory in the general path).
 constexpr int kSmallBlocks = 4096;
 
-template <typename T>
-__global__ void __launch_bounds__(kThreads) compact_small_kernel(const CompactArgs a)
+template <typename T, bool kBig>
+__global__ void __launch_bounds__(kThreads) compact_kernel(const CompactArgs a)
 {
-    __shared__ __align__(16) uint8_t s_gamma[kSmallBlocks];
+    __shared__ __align__(16) uint8_t s_gamma[kBig ? 16 : kSmallBlocks];
     __shared__ int s_sum[kThreads / 32];
     const int n_fill = a.NBo * a.fill_parts;
     if ((int)blockIdx.x >= n_fill) {
@@ -327,15 +289,20 @@ __global__ void __launch_bounds__(kThreads) compact_small_kernel(const CompactAr
             dense_body<(int)sizeof(T)>((int)blockIdx.x - n_fill, a.dense_ctas, a.W, a.gamma, a.O, a.I, a.HK, a.bo, a.bi, a.NBi, a.dense);
         return;
     }
-    const int NB = a.NBo * a.NBi;
-    const bool word_ok = (((uintptr_t)a.gamma) & 3u) == 0;
-    for (int i = threadIdx.x * 4; i < NB; i += kThreads * 4) {
-        if (i + 4 <= NB && word_ok) *(uint32_t *)(s_gamma + i) = *(const uint32_t *)(a.gamma + i);
-        else for (int q = i; q < min(NB, i + 4); ++q) s_gamma[q] = a.gamma[q];
-    }
-    __syncthreads();
     const int l = (int)blockIdx.x / a.fill_parts, part = (int)blockIdx.x % a.fill_parts;
-    const int first = block_sum(ones_share(s_gamma, l * a.NBi), s_sum);
+    int first;
+    if constexpr (kBig) {
+        first = block_sum(ones_share_global(a.gamma, l * a.NBi), s_sum);      // (NB_o NB_i < 2^31: checked by the host)
+    } else {
+        const int NB = a.NBo * a.NBi;
+        const bool word_ok = (((uintptr_t)a.gamma) & 3u) == 0;
+        for (int i = threadIdx.x * 4; i < NB; i += kThreads * 4) {
+            if (i + 4 <= NB && word_ok) *(uint32_t *)(s_gamma + i) = *(const uint32_t *)(a.gamma + i);
+            else for (int q = i; q < min(NB, i + 4); ++q) s_gamma[q] = a.gamma[q];
+        }
+        __syncthreads();
+        first = block_sum(ones_share(s_gamma, l * a.NBi), s_sum);
+    }
     const int cnt = csr_fill_body<T>(l, part, a.fill_parts, (const T *)a.W, a.gamma, a.NBi, a.I, a.HK, a.bo, a.bi, first,
                                      a.col_idx, (T *)a.payload, a.capacity_blocks);
     if (part == 0 && threadIdx.x == 0) {
@@ -376,7 +343,6 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
     const int NBo = wd.O / wd.bo, NBi = wd.I / wd.bi, HK = wd.H * wd.K;
     const PackedLayout L = packed_layout(wd);
     int *status = (int *)ws;
-    int *row_cnt = (int *)((char *)ws + kWsHeader);
     uint8_t *pk = (uint8_t *)packed;
     const bool dense_on = pk != nullptr && L.enabled;
     const int esz = elem_bytes(wd.wtype);
@@ -405,24 +371,21 @@ bsp_status launch_compact(const bsp_wdesc &wd, const void *W, const uint8_t *gam
             a.fill_parts = (int)(p < 1 ? 1 : (p > 8 ? 8 : p));
         }
         const unsigned grid = (unsigned)(NBo * a.fill_parts + a.dense_ctas);
-        if (wd.wtype == BSP_I8) compact_small_kernel<uint8_t><<<grid, kThreads, smem, st>>>(a);
-        else if (wd.wtype == BSP_BF16) compact_small_kernel<uint16_t><<<grid, kThreads, smem, st>>>(a);
-        else compact_small_kernel<uint32_t><<<grid, kThreads, smem, st>>>(a);
+        if (wd.wtype == BSP_I8) compact_kernel<uint8_t, false><<<grid, kThreads, smem, st>>>(a);
+        else if (wd.wtype == BSP_BF16) compact_kernel<uint16_t, false><<<grid, kThreads, smem, st>>>(a);
+        else compact_kernel<uint32_t, false><<<grid, kThreads, smem, st>>>(a);
         BSP_CUDA_OK(cudaGetLastError());
         return BSP_OK;
     }
-    count_scan_kernel<<<NBo, kThreads, 0, st>>>(gamma, NBi, NBo, row_cnt, row_ptr, (PackedHeader *)pk, a.hdr_init, (long long)capacity_blocks,
-                                                status, (unsigned *)ws + kWsTicketWord);
-    BSP_CUDA_OK(cudaGetLastError());
+    if ((long long)NBo * NBi > 0x7FFFFFFF) return BSP_ERR_SHAPE;
     // enough CTAs per row to give every SM some of the payload copy
     a.fill_parts = payload ? (296 + NBo - 1) / NBo : 1;
     if (a.fill_parts > 16) a.fill_parts = 16;
     if (a.fill_parts < 1) a.fill_parts = 1;
-    if (!dense_on) a.dense_ctas = 0;
     const unsigned grid = (unsigned)(NBo * a.fill_parts + a.dense_ctas);
-    if (wd.wtype == BSP_I8) fill_dense_kernel<uint8_t><<<grid, kThreads, smem, st>>>(a);
-    else if (wd.wtype == BSP_BF16) fill_dense_kernel<uint16_t><<<grid, kThreads, smem, st>>>(a);
-    else fill_dense_kernel<uint32_t><<<grid, kThreads, smem, st>>>(a);
+    if (wd.wtype == BSP_I8) compact_kernel<uint8_t, true><<<grid, kThreads, smem, st>>>(a);
+    else if (wd.wtype == BSP_BF16) compact_kernel<uint16_t, true><<<grid, kThreads, smem, st>>>(a);
+    else compact_kernel<uint32_t, true><<<grid, kThreads, smem, st>>>(a);
     BSP_CUDA_OK(cudaGetLastError());
     return BSP_OK;
 }

@@ -38,7 +38,6 @@ PackedLayout packed_layout(const bsp_wdesc &wd);
 // barrier of the single-launch kernels (words kWsSyncWord, kWsSyncWord + 1); scratch starts after them.
 constexpr size_t kWsHeader = 256;
 constexpr int kWsSyncWord = 2;
-constexpr int kWsTicketWord = 4;          // count of finished CTAs of the row-count launch (left at zero)
 // Scratch of the cooperative select after the scores in the mask workspace: 8 x 256 histogram words, 8 counter and key-span words,
 // one word per CTA and a list of up to 8192 candidate keys.
 constexpr int kSelectMaxCtas = 1024;
