@@ -374,7 +374,8 @@ def pass_layers(gpu, bsp, torch, layers, dtype, sparsities, pk, ydt, with_setup,
 def pass_spgemm(gpu, bsp, torch, reps=5):
     """Block-sparse x block-sparse product C = (Gamma . A)(Omega . B)^t, 2048 x 4096 times (2048 x 4096)^t, bf16 8x8 blocks,
     magnitude masks at 50 % and 75 %: useful FLOPs are those of the block pairs that both masks keep.  The kernel runs on
-    the fp32 pipes (8 x 8 x 8 products), so its roofline is the fp32 FMA rate: 148 SMs x 128 lanes x 2 x 1.965 GHz."""
+    the general-purpose pipes (index look-ups, ballots; the 8 x 8 x 8 products of bf16 blocks go two at a time through one
+    m16n8k16 tensor-core instruction of the warp), so its yardstick is the fp32 FMA rate: 148 SMs x 128 lanes x 2 x 1.965 GHz."""
     peak = 148 * 128 * 2 * 1.965e9 / 1e12
     out = []
     g = torch.Generator(device="cuda")

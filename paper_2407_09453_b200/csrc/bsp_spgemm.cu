@@ -6,7 +6,8 @@
 // A CTA owns one row i of A: the positions of its kept blocks are spread into a table over the block columns in shared
 // memory (the table replaces one side of the paper's merge of two sorted lists), and every warp takes rows j of B in
 // turn: 32 entries of B's column list are looked up at once, a ballot gives the common columns in ascending order, and
-// for each of them the warp adds the 8 x 8 x 8 product, lane (r, c) holding C[r][2c], C[r][2c + 1] in fp32.  Work and
+// for each of them the warp adds the 8 x 8 x 8 product, lane (r, c) holding C[r][2c], C[r][2c + 1] in fp32 (fp32 blocks:
+// fused multiply-adds; bfloat16 blocks: one m16n8k16 tensor-core instruction per two common columns).  Work and
 // traffic follow the kept blocks only: nothing is read or multiplied where either mask has a zero.
 #include "bsp_internal.cuh"
 
@@ -63,6 +64,27 @@ spgemm_kernel(const int32_t *__restrict__ a_row_ptr, const int32_t *__restrict__
                 else atomicMax(status, (int)BSP_ERR_INDEX);
             }
             unsigned both = __ballot_sync(0xFFFFFFFFu, pa >= 0);
+            if constexpr (sizeof(T) == 2) {
+                // bfloat16 blocks: two common columns per tensor-core instruction (m16n8k16: the 8 x 8 block of C sits in
+                // rows 0-7 of the 16 x 8 result, K = the eight channels of the first column followed by those of the
+                // second).  Lane (r, c) holds exactly the words it needs: entries (r, 2c), (r, 2c + 1) of each block of A
+                // and of B, so a warp reads each 128-byte block once, four bytes per lane.
+                while (both) {
+                    const int s1 = __ffs(both) - 1;
+                    both &= both - 1;
+                    const int s2 = both ? __ffs(both) - 1 : -1;
+                    both &= both - 1;                         // (0 & -1 stays 0)
+                    const int na1 = __shfl_sync(0xFFFFFFFFu, pa, s1);
+                    const int na2 = __shfl_sync(0xFFFFFFFFu, pa, s2 < 0 ? s1 : s2);
+                    const uint32_t *Aw = (const uint32_t *)a_payload, *Bw = (const uint32_t *)b_payload;
+                    const uint32_t a0 = __ldg(Aw + (size_t)na1 * 32 + lane), b0 = __ldg(Bw + (size_t)(base + s1) * 32 + lane);
+                    uint32_t a2 = 0u, b1 = 0u;
+                    if (s2 >= 0) { a2 = __ldg(Aw + (size_t)na2 * 32 + lane); b1 = __ldg(Bw + (size_t)(base + s2) * 32 + lane); }
+                    float d2 = 0.f, d3 = 0.f;
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};\n"
+                                 : "+f"(acc0), "+f"(acc1), "+f"(d2), "+f"(d3) : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+                }
+            } else
             while (both) {                                    // common columns, ascending
                 const int src = __ffs(both) - 1;
                 both &= both - 1;
