@@ -93,3 +93,19 @@ def test_gemm_4096_every_block_shape_and_sparsity(gemm_4096, bo, bi, frac):
     want = ref.gemm(O, O, bo, bi, rp, ci, pl.reshape(-1, bo, bi), X, b, pix=pix)
     check(got[pix], want, "bf16")
     assert np.isfinite(got).all()
+
+
+FULL_BF16 = {l.name: l for l in synth.resnet50_layers(batch=64)}
+FULL_I8 = {l.name: l for l in synth.vgg16_layers(batch=32) + synth.inception_v3_layers(batch=32)}
+
+
+@pytest.mark.parametrize("name", ["c2.3x3.64-64", "c3.1x1.256-512.s2", "c5.1x1.512-2048"])
+def test_resnet50_layers_at_the_batch_the_benchmark_times(name):
+    """Batch 64, as in the benchmark's layer pass: thousands of tiles per launch, every CTA takes many."""
+    run_layer(FULL_BF16[name], "bf16", 0.5, 4, 900 + len(name))
+
+
+@pytest.mark.parametrize("name", ["vgg.64-64@224", "vgg.256-256@56", "inc17.1x7.128-128"])
+def test_int8_layers_at_the_batch_the_benchmark_times(name):
+    """Batch 32: the 224 x 224 layer is 1.6 million positions (64-byte rows of input channels), bit exact on the samples."""
+    run_layer(FULL_I8[name], "i8", 0.5, 5, 950 + len(name))
