@@ -278,7 +278,7 @@ struct CompactArgs {
 constexpr int kSmallBlocks = 4096;
 
 template <typename T, bool kBig>
-__global__ void __launch_bounds__(kThreads) compact_kernel(const CompactArgs a)
+__global__ void __launch_bounds__(kThreads, 5) compact_kernel(const CompactArgs a)
 {
     __shared__ __align__(16) uint8_t s_gamma[kBig ? 16 : kSmallBlocks];
     __shared__ int s_sum[kThreads / 32];
